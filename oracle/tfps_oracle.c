@@ -1,0 +1,249 @@
+/*
+ * TEST INFRASTRUCTURE -- NOT PART OF THE PRODUCT PATH.
+ *
+ * Plain, slow, single-threaded CPU oracle for critical-path evaluation of one
+ * data-flow graph under one partition, written from the paper's definitions.
+ * It shares no code, headers, tables or constants with the CUDA library; only
+ * tests, the smoke check and the benchmark's CPU-baseline leg may call it.
+ *
+ * Model (Section 2): G=(V,E), vertex cost c_i, edge size t_i; device speed s,
+ * capacity C, bandwidth matrix B.  Execution time of a vertex on its device is
+ * c/s (Section 2, the c_1/s_1 example); the transfer time of an edge is 0 when
+ * both end points sit on the same device, else tensor size over the transfer
+ * rate between the two devices (Section 4.1, text before Eq. 12).
+ *
+ * Integer reading: time is counted in ticks, S ticks per paper time unit, and
+ * every real quotient is rounded up once:
+ *      rt(v)   = ceil(c_v * S / s_{p(v)})
+ *      w(u->v) = 0 if p(u)==p(v), else ceil(t_uv * S / B[p(u)][p(v)])
+ * with B indexed [device of the edge's source][device of its target].
+ *
+ * Parity pins (tests/test_oracle_*.py): hand-computed worked DAGs stored under
+ * tests/golden/, brute-force enumeration of all paths on graphs of <= 12
+ * vertices, single-device reduction against networkx/scipy longest path, the
+ * unit-cost setting of the NP-completeness reduction (Lemma 1), exact-rational
+ * error bound against the real-valued model, and the invariants listed there.
+ * No function here is "parity unpinned".
+ *
+ * All arithmetic is int64; every product and sum is checked in __int128 and
+ * reported as ORACLE_OVERFLOW instead of wrapping.
+ */
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define ORACLE_OK 0
+#define ORACLE_BAD_ARG -1
+#define ORACLE_CYCLE -2
+#define ORACLE_OVERFLOW -3
+#define ORACLE_BAD_PARTITION -4
+
+typedef __int128 i128;
+
+static int fits(i128 x) { return x >= 0 && x <= (i128)INT64_MAX; }
+
+/* ceil(a*S/b) for a>=0, S>=1, b>=1 by plain integer division. */
+static int ceil_scaled(int64_t a, int64_t S, int64_t b, int64_t *out)
+{
+    i128 num = (i128)a * (i128)S;
+    i128 q = num / b;
+    if (num % b != 0) q += 1;
+    if (!fits(q)) return ORACLE_OVERFLOW;
+    *out = (int64_t)q;
+    return ORACLE_OK;
+}
+
+/*
+ * Topological structure.  A vertex is schedulable once data on all incoming
+ * edges is available (Section 2); Kahn's algorithm with a FIFO queue emits
+ * vertices in such an order.  level(v) = 0 for sources, else 1 + the largest
+ * level of a predecessor.  `order` lists vertices by level, ascending id
+ * inside a level; level_ptr[l]..level_ptr[l+1] delimits level l.
+ * level_ptr must have room for n+1 entries.  topo (may be NULL) receives the
+ * raw Kahn order.
+ */
+int oracle_topo_levels(int64_t n, const int64_t *in_ptr, const int32_t *in_src,
+                       const int64_t *out_ptr, const int32_t *out_dst,
+                       int32_t *level, int32_t *order, int64_t *level_ptr,
+                       int32_t *num_levels, int32_t *topo)
+{
+    if (n < 0) return ORACLE_BAD_ARG;
+    int64_t *indeg = (int64_t *)malloc(sizeof(int64_t) * (size_t)(n + 1));
+    int32_t *queue = (int32_t *)malloc(sizeof(int32_t) * (size_t)(n + 1));
+    if (!indeg || !queue) { free(indeg); free(queue); return ORACLE_BAD_ARG; }
+    int64_t head = 0, tail = 0;
+    for (int64_t v = 0; v < n; ++v) {
+        indeg[v] = in_ptr[v + 1] - in_ptr[v];
+        if (indeg[v] == 0) queue[tail++] = (int32_t)v;
+    }
+    while (head < tail) {
+        int32_t u = queue[head++];
+        for (int64_t e = out_ptr[u]; e < out_ptr[u + 1]; ++e) {
+            int32_t x = out_dst[e];
+            if (--indeg[x] == 0) queue[tail++] = x;
+        }
+    }
+    if (tail != n) { free(indeg); free(queue); return ORACLE_CYCLE; }
+    int32_t L = 0;
+    for (int64_t i = 0; i < n; ++i) {
+        int32_t v = queue[i];
+        int32_t lv = 0;
+        for (int64_t e = in_ptr[v]; e < in_ptr[v + 1]; ++e) {
+            int32_t cand = level[in_src[e]] + 1;
+            if (cand > lv) lv = cand;
+        }
+        level[v] = lv;
+        if (lv + 1 > L) L = lv + 1;
+    }
+    if (n == 0) L = 0;
+    for (int32_t l = 0; l <= L; ++l) level_ptr[l] = 0;
+    for (int64_t v = 0; v < n; ++v) level_ptr[level[v] + 1] += 1;
+    for (int32_t l = 0; l < L; ++l) level_ptr[l + 1] += level_ptr[l];
+    int64_t *fill = indeg; /* reuse */
+    for (int32_t l = 0; l < L; ++l) fill[l] = level_ptr[l];
+    for (int64_t v = 0; v < n; ++v) order[fill[level[v]]++] = (int32_t)v;
+    if (topo) memcpy(topo, queue, sizeof(int32_t) * (size_t)n);
+    *num_levels = L;
+    free(indeg); free(queue);
+    return ORACLE_OK;
+}
+
+/*
+ * Default per-vertex memory: data leaving the source vertex of an edge
+ * consumes memory of that vertex's device (Section 2), so mem_v = sum of the
+ * sizes of v's outgoing edges.
+ */
+int oracle_default_mem(int64_t n, const int64_t *out_ptr, const int64_t *out_t, int64_t *mem)
+{
+    for (int64_t v = 0; v < n; ++v) {
+        i128 acc = 0;
+        for (int64_t e = out_ptr[v]; e < out_ptr[v + 1]; ++e) acc += out_t[e];
+        if (!fits(acc)) return ORACLE_OVERFLOW;
+        mem[v] = (int64_t)acc;
+    }
+    return ORACLE_OK;
+}
+
+/*
+ * One candidate partition p (uint8 per vertex, element stride p_stride).
+ * topo: any topological order of the graph (oracle_topo_levels gives one).
+ *
+ * tlevel(v): earliest start = max over in-edges (u->v) of
+ *            tlevel(u) + rt(u) + w(u->v); 0 for sources.  This is the
+ *            downward recursion of Eq. 6 carried out with execution times and
+ *            transfer times and without the vertex's own term, i.e. the start
+ *            time that the schedule function f returns (Section 2).
+ * blevel(v): Eq. 12 (path computation time): rt(v) + max over out-edges
+ *            (v->x) of ( blevel(x) + w(v->x) ); rt(v) for sinks.
+ * cp:        start time of the artificial zero-cost sink joined to every sink
+ *            by a zero-cost edge (Section 2, after Eq. 1) = max_v tlevel+rt.
+ * load[d]:   sum of rt(v) over vertices on d (the sum inside Eq. 7).
+ * memload[d]: sum of mem_v over vertices on d; Eq. 2 demands usage < C_d, so
+ *            bit d of *viol is set iff memload[d] >= C[d].
+ * Any of tlevel, blevel, load, memload, viol may be NULL.
+ */
+int oracle_eval_partition(int64_t n,
+                          const int64_t *in_ptr, const int32_t *in_src, const int64_t *in_t,
+                          const int64_t *out_ptr, const int32_t *out_dst, const int64_t *out_t,
+                          const int32_t *c, const int64_t *mem,
+                          int32_t k, const int32_t *s, const int64_t *C, const int64_t *B, int64_t S,
+                          const int32_t *topo,
+                          const uint8_t *p, int64_t p_stride,
+                          int64_t *tlevel, int64_t *blevel, int64_t *cp,
+                          int64_t *load, int64_t *memload, uint64_t *viol)
+{
+    if (n < 0 || k < 1 || k > 64 || S < 1) return ORACLE_BAD_ARG;
+    int rc = ORACLE_OK;
+    int64_t *rt = (int64_t *)malloc(sizeof(int64_t) * (size_t)(n + 1));
+    int64_t *tl = (int64_t *)malloc(sizeof(int64_t) * (size_t)(n + 1));
+    int64_t *bl = (int64_t *)malloc(sizeof(int64_t) * (size_t)(n + 1));
+    if (!rt || !tl || !bl) { rc = ORACLE_BAD_ARG; goto done; }
+
+    for (int64_t v = 0; v < n; ++v) {
+        int d = p[v * p_stride];
+        if (d >= k) { rc = ORACLE_BAD_PARTITION; goto done; }
+        if (c[v] < 0 || s[d] < 1) { rc = ORACLE_BAD_ARG; goto done; }
+        rc = ceil_scaled(c[v], S, s[d], &rt[v]);
+        if (rc) goto done;
+    }
+
+    /* forward: earliest start times */
+    for (int64_t i = 0; i < n; ++i) {
+        int32_t v = topo[i];
+        int dv = p[v * p_stride];
+        i128 best = 0;
+        for (int64_t e = in_ptr[v]; e < in_ptr[v + 1]; ++e) {
+            int32_t u = in_src[e];
+            int du = p[u * p_stride];
+            int64_t w = 0;
+            if (du != dv) {
+                if (in_t[e] < 0 || B[du * k + dv] < 1) { rc = ORACLE_BAD_ARG; goto done; }
+                rc = ceil_scaled(in_t[e], S, B[du * k + dv], &w);
+                if (rc) goto done;
+            }
+            i128 cand = (i128)tl[u] + rt[u] + w;
+            if (cand > best) best = cand;
+        }
+        if (!fits(best)) { rc = ORACLE_OVERFLOW; goto done; }
+        tl[v] = (int64_t)best;
+    }
+
+    /* backward: Eq. 12 */
+    for (int64_t i = n - 1; i >= 0; --i) {
+        int32_t v = topo[i];
+        int dv = p[v * p_stride];
+        i128 best = 0;
+        for (int64_t e = out_ptr[v]; e < out_ptr[v + 1]; ++e) {
+            int32_t x = out_dst[e];
+            int dx = p[x * p_stride];
+            int64_t w = 0;
+            if (dx != dv) {
+                if (out_t[e] < 0 || B[dv * k + dx] < 1) { rc = ORACLE_BAD_ARG; goto done; }
+                rc = ceil_scaled(out_t[e], S, B[dv * k + dx], &w);
+                if (rc) goto done;
+            }
+            i128 cand = (i128)bl[x] + w;
+            if (cand > best) best = cand;
+        }
+        best += rt[v];
+        if (!fits(best)) { rc = ORACLE_OVERFLOW; goto done; }
+        bl[v] = (int64_t)best;
+    }
+
+    {
+        i128 mx = 0;
+        for (int64_t v = 0; v < n; ++v) {
+            i128 f = (i128)tl[v] + rt[v];
+            if (f > mx) mx = f;
+        }
+        if (!fits(mx)) { rc = ORACLE_OVERFLOW; goto done; }
+        if (cp) *cp = (int64_t)mx;
+    }
+
+    {
+        i128 ld[64], ml[64];
+        for (int d = 0; d < k; ++d) { ld[d] = 0; ml[d] = 0; }
+        for (int64_t v = 0; v < n; ++v) {
+            int d = p[v * p_stride];
+            ld[d] += rt[v];
+            if (mem) {
+                if (mem[v] < 0) { rc = ORACLE_BAD_ARG; goto done; }
+                ml[d] += mem[v];
+            }
+        }
+        uint64_t bits = 0;
+        for (int d = 0; d < k; ++d) {
+            if (!fits(ld[d]) || !fits(ml[d])) { rc = ORACLE_OVERFLOW; goto done; }
+            if (load) load[d] = (int64_t)ld[d];
+            if (memload) memload[d] = (int64_t)ml[d];
+            if (mem && C && ml[d] >= (i128)C[d]) bits |= (uint64_t)1 << d;
+        }
+        if (viol) *viol = bits;
+    }
+
+    if (tlevel) memcpy(tlevel, tl, sizeof(int64_t) * (size_t)n);
+    if (blevel) memcpy(blevel, bl, sizeof(int64_t) * (size_t)n);
+done:
+    free(rt); free(tl); free(bl);
+    return rc;
+}
