@@ -1,0 +1,188 @@
+/*
+ * tfps -- batched critical-path evaluation of one data-flow graph under many
+ * candidate partitions (sm_100a CUDA library, C ABI).
+ *
+ * Problem tuple (paper, Section 2): DAG G=(V,E) with vertex cost c_v and edge
+ * size t_e; k devices with speed s_d and capacity C_d; bandwidth matrix B.
+ * A partition p: V -> D places every vertex on a device.
+ *
+ * Cost model in integer ticks (S = `scale` ticks per paper time unit):
+ *   rt(v)   = ceil(c_v * S / s_p(v))                       execution time c/s, Section 2
+ *   w(u->v) = 0 if p(u)==p(v)                              Section 4.1 (text before Eq. 12)
+ *             else ceil(t_uv * S / B[p(u)][p(v)])          B indexed [source device][target device]
+ *   tlevel(v) = max over in-edges (u->v) of tlevel(u)+rt(u)+w(u->v); 0 for sources
+ *               (earliest start; recursion of Eq. 6 with execution and transfer times)
+ *   blevel(v) = rt(v) + max over out-edges (v->x) of w(v->x)+blevel(x); rt(v) for sinks
+ *               (path computation time, Eq. 12)
+ *   CP        = max_v tlevel(v)+rt(v)                      start of the artificial sink, Section 2 after Eq. 1
+ *   load[d]   = sum of rt(v) over vertices on d            the sum inside Eq. 7
+ *   memload[d]= sum of mem_v over vertices on d; bit d of viol set iff memload[d] >= C_d
+ *               (Eq. 2 is a strict inequality)
+ *
+ * Conventions common to all calls
+ *   - Every function returns TFPS_OK (0) or a negative tfps_status.  Nothing
+ *     throws, aborts or traps.  tfps_last_error() gives a thread-local message.
+ *   - "dev" pointers are CUDA device pointers on the handle's device, "host"
+ *     pointers are ordinary host memory.  The caller owns every buffer it
+ *     passes; the handle owns private device copies of graph and tables and
+ *     keeps no reference to caller memory after a call returns (asynchronous
+ *     calls read/write caller buffers until the stream reaches their end).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *   - Vertex ids are 0..n-1 in any order.  Parallel edges are legal (max
+ *     semantics).  A self loop or cycle gives TFPS_ERR_CYCLE.
+ *   - Candidate matrices are vertex-major: element (v, j) of a matrix with
+ *     leading dimension ldp lives at index v*ldp + j; ldp >= P and ldp % 16 == 0.
+ *     Columns P..ldp-1 are padding: read but never written.
+ */
+#ifndef TFPS_H
+#define TFPS_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct tfps_graph tfps_graph;
+
+typedef enum tfps_status {
+    TFPS_OK = 0,
+    TFPS_ERR_INVALID_ARG = -1,   /* NULL where data is required, negative size, bad enum, bad ldp */
+    TFPS_ERR_BAD_CSR = -2,       /* ptr not monotone / wrong end, index out of range, in/out edge multisets differ, negative c/t/mem */
+    TFPS_ERR_CYCLE = -3,         /* graph is not acyclic */
+    TFPS_ERR_BAD_DEVICES = -4,   /* k outside 1..TFPS_K_MAX, s_d < 1, off-diagonal B < 1, C_d < 0, scale < 1 */
+    TFPS_ERR_BAD_PARTITION = -5, /* a partition id >= k (reported through the status word) */
+    TFPS_ERR_OVERFLOW = -6,      /* a path length or load could reach 2^62 ticks */
+    TFPS_ERR_WORKSPACE = -7,     /* workspace NULL or too small */
+    TFPS_ERR_UNSUPPORTED = -8,   /* size beyond an implementation limit */
+    TFPS_ERR_CUDA = -9,          /* a CUDA runtime call failed (message in tfps_last_error) */
+    TFPS_ERR_TIMEOUT = -10,      /* a bounded device-side wait ran out */
+    TFPS_ERR_STATE = -11         /* call order: devices not set, levels not built */
+} tfps_status;
+
+enum { TFPS_K_MAX = 64 };
+enum { TFPS_I32 = 0, TFPS_I64 = 1 };          /* dtype selectors for t and mem */
+enum { TFPS_HOST = 0, TFPS_DEVICE = 1 };      /* where the arrays given to tfps_graph_create live */
+
+/* flags of tfps_eval_batch / tfps_eval_workspace_bytes */
+enum {
+    TFPS_EVAL_AUTO = 0,
+    TFPS_EVAL_LEVEL_SYNC = 1 << 0,   /* one launch per topological level, thread = (vertex, candidates) */
+    TFPS_EVAL_SLICED = 1 << 1,       /* one persistent block per candidate slice walks all levels */
+    TFPS_EVAL_NO_VALIDATE = 1 << 4,  /* caller guarantees every id < k; skips the id check */
+    TFPS_EVAL_SCRATCH_LEVELS = 1 << 5 /* workspace query: caller will pass tlevel == NULL and blevel == NULL */
+};
+
+const char* tfps_strerror(int status);
+const char* tfps_last_error(void);
+
+/*
+ * Build a graph handle (Section 2: G, c, t; optional per-vertex memory).
+ *   n, m         vertices, edges (n < 2^31, m < 2^31)
+ *   in_ptr[n+1], in_src[m], in_t[m]     in-edge CSR: row v lists the sources u of edges u->v and their sizes
+ *   out_ptr[n+1], out_dst[m], out_t[m]  out-edge CSR; pass all three NULL to have it built by transposing.
+ *                                       When given, it must hold the same multiset of (u, v, t) edges.
+ *   t_dtype      TFPS_I32 or TFPS_I64 (element type of in_t/out_t), t >= 0
+ *   c[n]         int32 vertex cost, c >= 0
+ *   mem, mem_dtype  per-vertex memory >= 0, or NULL: mem_v = total size of v's out-edges
+ *                (Section 2: data leaving the source vertex of an edge consumes device memory)
+ *   ptr_space    TFPS_HOST or TFPS_DEVICE: where all of the above arrays live
+ * The arrays are copied; the CSR is validated on the host (device arrays are
+ * fetched first).  Synchronises `stream`.  On error *out is NULL.
+ */
+int tfps_graph_create(tfps_graph** out, int64_t n, int64_t m,
+                      const int64_t* in_ptr, const int32_t* in_src, const void* in_t,
+                      const int64_t* out_ptr, const int32_t* out_dst, const void* out_t,
+                      int t_dtype, const int32_t* c, const void* mem, int mem_dtype,
+                      int ptr_space, void* stream);
+
+/* Free the handle and everything it owns (device memory included).  NULL is allowed. */
+int tfps_graph_destroy(tfps_graph* g);
+
+/* n, m, number of topological levels (0 until built), k (0 until devices are set). host outputs, any may be NULL */
+int tfps_graph_info(const tfps_graph* g, int64_t* n, int64_t* m, int32_t* num_levels, int32_t* k);
+
+/*
+ * Set the device tables (Section 2: speeds s, capacities C, bandwidth matrix B).
+ *   k            1..TFPS_K_MAX
+ *   s[k]         host int32, s_d >= 1
+ *   C[k]         host int64, C_d >= 0, INT64_MAX = unbounded
+ *   B[k*k]       host int64 row-major [source device][target device]; off-diagonal >= 1 and < 2^62, diagonal ignored
+ *   scale        S >= 1, ticks per paper time unit
+ * Builds the per-device and per-device-pair exact-division constants and the
+ * per-vertex / per-edge scaled numerators.  Requires max c*S and max t*S below
+ * 2^62 and the bound  sum_v ceil(c_v S / min s) + sum_e ceil(t_e S / min B)  < 2^62,
+ * else TFPS_ERR_OVERFLOW.  Synchronous (default stream).
+ */
+int tfps_devices_set(tfps_graph* g, int k, const int32_t* s, const int64_t* C, const int64_t* B, int64_t scale);
+
+/*
+ * Topological levels by a Kahn frontier on the GPU (a vertex is schedulable
+ * once all incoming data is available, Section 2).
+ *   level[n]     dev int32 or NULL: 0 for sources, else 1 + max level of a predecessor
+ *   order[n]     dev int32 or NULL: vertices grouped by level, ascending id inside a level
+ *   level_ptr    host int64[cap] or NULL: level l is order[level_ptr[l] .. level_ptr[l+1])
+ *   cap          entries available in level_ptr; TFPS_ERR_INVALID_ARG if cap < num_levels+1
+ *   num_levels   host int32 or NULL
+ * The structure is built on the first call (also implicitly by tfps_eval_batch)
+ * and cached.  Synchronises `stream`.  A cyclic graph gives TFPS_ERR_CYCLE.
+ */
+int tfps_topo_levels(tfps_graph* g, int32_t* level, int32_t* order,
+                     int64_t* level_ptr, int64_t cap, int32_t* num_levels, void* stream);
+
+/*
+ * Bytes of caller workspace tfps_eval_batch needs.  0 unless flags contains
+ * TFPS_EVAL_SCRATCH_LEVELS (critical-path length wanted without either level
+ * matrix), in which case one int64 [n][ldp] matrix is needed.
+ */
+size_t tfps_eval_workspace_bytes(const tfps_graph* g, int64_t P, int64_t ldp, int flags);
+
+/*
+ * Evaluate P candidate partitions.  Asynchronous on `stream`.
+ *   part         dev uint8 [n][ldp], part[v*ldp+j] = device of vertex v under candidate j (< k)
+ *   tlevel       dev int64 [n][ldp] or NULL
+ *   blevel       dev int64 [n][ldp] or NULL     (the PCT priority of Eq. 12)
+ *   cp           dev int64 [P] or NULL
+ *   load         dev int64 [k][ldp] or NULL
+ *   memload      dev int64 [k][ldp] or NULL
+ *   viol         dev uint64 [P] or NULL; bit d = capacity of device d violated
+ *   workspace    dev, 256-byte aligned, workspace_bytes >= tfps_eval_workspace_bytes(...); may be NULL when that is 0
+ *   flags        TFPS_EVAL_* (kernel variant; validation)
+ * The forward pass runs when tlevel is wanted, or when cp is wanted and blevel
+ * is not; the backward pass runs when blevel is wanted.  P == 0 or n == 0:
+ * TFPS_OK, nothing written.  Host-detectable errors are returned at once and
+ * nothing is launched.  An id >= k is found on the device: every later kernel
+ * of the call then returns without touching memory, outputs are unspecified,
+ * and tfps_get_status reports TFPS_ERR_BAD_PARTITION.
+ */
+int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp,
+                    const uint8_t* part, int64_t* tlevel, int64_t* blevel,
+                    int64_t* cp, int64_t* load, int64_t* memload, uint64_t* viol,
+                    void* workspace, size_t workspace_bytes, int flags, void* stream);
+
+/*
+ * Same evaluation from HOST buffers: part is host uint8 [n][ldp]; cp[P],
+ * load[k*ldp], memload[k*ldp], viol[P] are host outputs (any may be NULL).
+ * Copies the ids to the device, runs the forward pass (and the load kernel),
+ * copies the results back and synchronises `stream`.  Staging and scratch
+ * buffers are owned by the handle and grow on demand.  Returns the device
+ * status as tfps_get_status would.
+ */
+int tfps_eval_batch_host(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part,
+                         int64_t* cp, int64_t* load, int64_t* memload, uint64_t* viol,
+                         int flags, void* stream);
+
+/* Synchronise `stream`, return the sticky device-side status of the handle and clear it. */
+int tfps_get_status(tfps_graph* g, void* stream);
+
+/*
+ * Layout helper: src dev uint8 [P][n] (candidate-major) -> dst dev uint8 [n][ldp]
+ * (vertex-major).  Padding columns of dst are not written.  Asynchronous.
+ */
+int tfps_transpose_u8(const uint8_t* src, uint8_t* dst, int64_t P, int64_t n, int64_t ldp, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TFPS_H */

@@ -1,0 +1,670 @@
+// Host runtime and C ABI of libtfps: graph handle, CSR validation, device
+// tables (exact-division constants), topological structure, launch logic.
+#include <algorithm>
+#include <cstdarg>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <utility>
+
+#include "common.cuh"
+
+using namespace tfps;
+
+namespace {
+
+thread_local std::string g_last_error;
+
+int fail(int code, const char* fmt, ...)
+{
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof buf, fmt, ap);
+    va_end(ap);
+    g_last_error = buf;
+    return code;
+}
+
+int fail_cuda(cudaError_t e, const char* what)
+{
+    return fail(TFPS_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+#define CUDA_TRY(expr)                                              \
+    do {                                                            \
+        cudaError_t e__ = (expr);                                   \
+        if (e__ != cudaSuccess) return fail_cuda(e__, #expr);       \
+    } while (0)
+
+#define TFPS_TRY(expr)                   \
+    do {                                 \
+        int rc__ = (expr);               \
+        if (rc__ != TFPS_OK) return rc__; \
+    } while (0)
+
+struct DBuf {
+    void* p = nullptr;
+    size_t bytes = 0;
+    DBuf() = default;
+    DBuf(const DBuf&) = delete;
+    DBuf& operator=(const DBuf&) = delete;
+    ~DBuf() { release(); }
+    void release() { if (p) cudaFree(p); p = nullptr; bytes = 0; }
+    // (re)allocate exactly `b` bytes (at least 16 so that empty graphs still get a pointer)
+    cudaError_t alloc(size_t b)
+    {
+        release();
+        if (b < 16) b = 16;
+        cudaError_t e = cudaMalloc(&p, b);
+        if (e == cudaSuccess) bytes = b; else p = nullptr;
+        return e;
+    }
+    cudaError_t reserve(size_t b) { return b <= bytes ? cudaSuccess : alloc(b); }
+    template <typename T> T* as() const { return static_cast<T*>(p); }
+};
+
+typedef unsigned __int128 u128;
+typedef __int128 i128;
+
+DivConst make_div(unsigned long long d)
+{
+    unsigned sh = 0;
+    while (((u128)1 << sh) < (u128)d) ++sh;  // ceil(log2 d)
+    u128 num = (u128)1 << (62 + sh);
+    u128 mul = (num + d - 1) / d;
+    DivConst dc;
+    dc.mul = (unsigned long long)mul;
+    dc.sh = sh;
+    dc.pad = 0;
+    return dc;
+}
+
+constexpr long long LIMIT62 = (long long)1 << 62;
+
+}  // namespace
+
+struct tfps_graph {
+    int device = 0;
+    int sm_count = 1;
+    long long n = 0, m = 0;
+    // statistics of the inputs kept for the overflow bound
+    long long max_c = 0, max_t = 0;
+    u128 sum_c = 0, sum_t = 0;
+    // graph (device)
+    DBuf in_ptr, in_src, in_t, out_ptr, out_dst, out_t, c, mem;
+    // topological structure
+    bool topo_built = false;
+    int num_levels = 0;
+    std::vector<long long> h_level_ptr;
+    DBuf level, order, level_ptr_d, sink_flag, sink_list;
+    int sink_count = 0;
+    DBuf f_eptr, f_nbr, f_t, b_eptr, b_nbr, b_t;
+    // device tables
+    bool dev_set = false;
+    int k = 0;
+    long long S = 0;
+    DBuf rt_div, w_div, cap, xvert, xw_f, xnbr_f, xw_b;
+    DBuf status;
+    // scratch owned by the handle
+    DBuf scr_memload;
+    DBuf st_part, st_lev, st_cp, st_load, st_mem, st_viol;
+};
+
+namespace {
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev)
+    {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    }
+    ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+template <typename T>
+int fetch(std::vector<T>& dst, const void* src, size_t count, int space, cudaStream_t st)
+{
+    dst.resize(count);
+    if (count == 0) return TFPS_OK;
+    if (space == TFPS_HOST) {
+        memcpy(dst.data(), src, count * sizeof(T));
+    } else {
+        CUDA_TRY(cudaMemcpyAsync(dst.data(), src, count * sizeof(T), cudaMemcpyDeviceToHost, st));
+        CUDA_TRY(cudaStreamSynchronize(st));
+    }
+    return TFPS_OK;
+}
+
+int fetch_wide(std::vector<long long>& dst, const void* src, size_t count, int dtype, int space, cudaStream_t st)
+{
+    if (dtype == TFPS_I64) return fetch(dst, src, count, space, st);
+    std::vector<int> tmp;
+    TFPS_TRY(fetch(tmp, src, count, space, st));
+    dst.assign(tmp.begin(), tmp.end());
+    return TFPS_OK;
+}
+
+int check_csr(const char* name, long long n, long long m, const std::vector<long long>& ptr, const std::vector<int>& idx)
+{
+    if (ptr[0] != 0) return fail(TFPS_ERR_BAD_CSR, "%s_ptr[0] != 0", name);
+    for (long long v = 0; v < n; ++v)
+        if (ptr[v + 1] < ptr[v]) return fail(TFPS_ERR_BAD_CSR, "%s_ptr decreases at %lld", name, v);
+    if (ptr[n] != m) return fail(TFPS_ERR_BAD_CSR, "%s_ptr[n] = %lld, expected m = %lld", name, ptr[n], m);
+    for (long long e = 0; e < m; ++e)
+        if (idx[e] < 0 || idx[e] >= n) return fail(TFPS_ERR_BAD_CSR, "%s index %d out of range at edge %lld", name, idx[e], e);
+    return TFPS_OK;
+}
+
+template <typename T>
+int upload(DBuf& buf, const std::vector<T>& v, cudaStream_t st)
+{
+    CUDA_TRY(buf.alloc(v.size() * sizeof(T)));
+    if (!v.empty()) CUDA_TRY(cudaMemcpyAsync(buf.p, v.data(), v.size() * sizeof(T), cudaMemcpyHostToDevice, st));
+    return TFPS_OK;
+}
+
+int build_topo(tfps_graph* g, cudaStream_t st)
+{
+    if (g->topo_built) return TFPS_OK;
+    const int n = (int)g->n;
+    const int m = (int)g->m;
+    if (n == 0) {
+        g->num_levels = 0;
+        g->h_level_ptr.assign(1, 0);
+        g->topo_built = true;
+        return TFPS_OK;
+    }
+    DBuf indeg, queue, level_cnt, result, keys;
+    CUDA_TRY(indeg.alloc(sizeof(int) * (size_t)n));
+    CUDA_TRY(queue.alloc(sizeof(int) * (size_t)n));
+    CUDA_TRY(level_cnt.alloc(sizeof(int) * ((size_t)n + 2)));
+    CUDA_TRY(result.alloc(sizeof(long long) * 2));
+    CUDA_TRY(g->level.alloc(sizeof(int) * (size_t)n));
+    CUDA_TRY(g->order.alloc(sizeof(int) * (size_t)n));
+    CUDA_TRY(g->level_ptr_d.alloc(sizeof(long long) * ((size_t)n + 2)));
+    CUDA_TRY(cudaMemsetAsync(level_cnt.p, 0, level_cnt.bytes, st));
+    CUDA_TRY(cudaMemsetAsync(result.p, 0, result.bytes, st));
+    CUDA_TRY(launch_kahn(n, g->in_ptr.as<long long>(), g->out_ptr.as<long long>(), g->out_dst.as<int>(),
+                         indeg.as<int>(), g->level.as<int>(), queue.as<int>(), g->level_ptr_d.as<long long>(),
+                         level_cnt.as<int>(), result.as<long long>(), g->sm_count, st));
+    long long res[2] = {0, 0};
+    CUDA_TRY(cudaMemcpyAsync(res, result.p, sizeof res, cudaMemcpyDeviceToHost, st));
+    CUDA_TRY(cudaStreamSynchronize(st));
+    if (res[1] != n) return fail(TFPS_ERR_CYCLE, "graph has a cycle: only %lld of %d vertices are reachable in topological order", res[1], n);
+    g->num_levels = (int)res[0];
+    g->h_level_ptr.resize((size_t)g->num_levels + 1);
+    CUDA_TRY(cudaMemcpyAsync(g->h_level_ptr.data(), g->level_ptr_d.p, sizeof(long long) * g->h_level_ptr.size(),
+                             cudaMemcpyDeviceToHost, st));
+
+    int npad = 1024;
+    while (npad < n) npad <<= 1;
+    CUDA_TRY(keys.alloc(sizeof(unsigned long long) * (size_t)npad));
+    CUDA_TRY(launch_sort_order(n, g->level.as<int>(), keys.as<unsigned long long>(), npad, g->order.as<int>(), st));
+
+    CUDA_TRY(g->f_eptr.alloc(sizeof(int) * ((size_t)n + 1)));
+    CUDA_TRY(g->b_eptr.alloc(sizeof(int) * ((size_t)n + 1)));
+    CUDA_TRY(g->f_nbr.alloc(sizeof(int) * (size_t)m));
+    CUDA_TRY(g->b_nbr.alloc(sizeof(int) * (size_t)m));
+    CUDA_TRY(g->f_t.alloc(sizeof(long long) * (size_t)m));
+    CUDA_TRY(g->b_t.alloc(sizeof(long long) * (size_t)m));
+    CUDA_TRY(launch_build_adj(n, g->order.as<int>(), g->in_ptr.as<long long>(), g->in_src.as<int>(),
+                              g->in_t.as<long long>(), g->f_eptr.as<int>(), g->f_nbr.as<int>(), g->f_t.as<long long>(), st));
+    CUDA_TRY(launch_build_adj(n, g->order.as<int>(), g->out_ptr.as<long long>(), g->out_dst.as<int>(),
+                              g->out_t.as<long long>(), g->b_eptr.as<int>(), g->b_nbr.as<int>(), g->b_t.as<long long>(), st));
+    CUDA_TRY(g->sink_flag.alloc((size_t)n));
+    CUDA_TRY(launch_sink_flags(n, g->order.as<int>(), g->out_ptr.as<long long>(), g->sink_flag.as<uint8_t>(), st));
+    std::vector<uint8_t> flags((size_t)n);
+    CUDA_TRY(cudaMemcpyAsync(flags.data(), g->sink_flag.p, (size_t)n, cudaMemcpyDeviceToHost, st));
+    CUDA_TRY(cudaStreamSynchronize(st));
+    std::vector<int> sinks;
+    for (int i = 0; i < n; ++i)
+        if (flags[i]) sinks.push_back(i);
+    g->sink_count = (int)sinks.size();
+    TFPS_TRY(upload(g->sink_list, sinks, st));
+    CUDA_TRY(cudaStreamSynchronize(st));
+    g->topo_built = true;
+    return TFPS_OK;
+}
+
+PassArgs make_args(const tfps_graph* g, bool fwd, long long P, long long ldp, const uint8_t* part, long long* lev,
+                   long long* cp)
+{
+    PassArgs a;
+    a.adj.vert = g->order.as<int>();
+    a.adj.eptr = fwd ? g->f_eptr.as<int>() : g->b_eptr.as<int>();
+    a.adj.nbr = fwd ? g->f_nbr.as<int>() : g->b_nbr.as<int>();
+    a.adj.xw = fwd ? g->xw_f.as<unsigned long long>() : g->xw_b.as<unsigned long long>();
+    a.adj.xnbr = fwd ? g->xnbr_f.as<unsigned long long>() : nullptr;
+    a.adj.xvert = g->xvert.as<unsigned long long>();
+    a.tab.k = g->k;
+    a.tab.rt_div = g->rt_div.as<DivConst>();
+    a.tab.w_div = g->w_div.as<DivConst>();
+    a.tab.cap = g->cap.as<long long>();
+    a.level_ptr = g->level_ptr_d.as<long long>();
+    a.num_levels = g->num_levels;
+    a.n = (int)g->n;
+    a.P = P;
+    a.ldp = ldp;
+    a.part = part;
+    a.lev = lev;
+    a.cp = cp;
+    a.status = g->status.as<int>();
+    return a;
+}
+
+int env_int(const char* name, int dflt)
+{
+    const char* s = getenv(name);
+    if (!s || !*s) return dflt;
+    return atoi(s);
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* tfps_strerror(int status)
+{
+    switch (status) {
+        case TFPS_OK: return "ok";
+        case TFPS_ERR_INVALID_ARG: return "invalid argument";
+        case TFPS_ERR_BAD_CSR: return "malformed CSR";
+        case TFPS_ERR_CYCLE: return "graph has a cycle";
+        case TFPS_ERR_BAD_DEVICES: return "bad device tables";
+        case TFPS_ERR_BAD_PARTITION: return "partition id out of range";
+        case TFPS_ERR_OVERFLOW: return "possible 64-bit overflow";
+        case TFPS_ERR_WORKSPACE: return "workspace missing or too small";
+        case TFPS_ERR_UNSUPPORTED: return "size beyond implementation limit";
+        case TFPS_ERR_CUDA: return "CUDA runtime error";
+        case TFPS_ERR_TIMEOUT: return "device-side wait timed out";
+        case TFPS_ERR_STATE: return "call order violated";
+        default: return "unknown status";
+    }
+}
+
+const char* tfps_last_error(void) { return g_last_error.c_str(); }
+
+int tfps_graph_create(tfps_graph** out, int64_t n, int64_t m,
+                      const int64_t* in_ptr, const int32_t* in_src, const void* in_t,
+                      const int64_t* out_ptr, const int32_t* out_dst, const void* out_t,
+                      int t_dtype, const int32_t* c, const void* mem, int mem_dtype,
+                      int ptr_space, void* stream)
+{
+    if (!out) return fail(TFPS_ERR_INVALID_ARG, "out is NULL");
+    *out = nullptr;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (n < 0 || m < 0) return fail(TFPS_ERR_INVALID_ARG, "negative size");
+    if (n >= ((int64_t)1 << 26) || m >= ((int64_t)1 << 31) - 64)
+        return fail(TFPS_ERR_UNSUPPORTED, "n must be below 2^26 and m below 2^31");
+    if (!in_ptr || (n > 0 && !c) || (m > 0 && (!in_src || !in_t)))
+        return fail(TFPS_ERR_INVALID_ARG, "in_ptr, in_src, in_t and c are required");
+    const bool have_out = out_ptr || out_dst || out_t;
+    if (have_out && (!out_ptr || (m > 0 && (!out_dst || !out_t))))
+        return fail(TFPS_ERR_INVALID_ARG, "pass all of out_ptr, out_dst, out_t or none");
+    if ((t_dtype != TFPS_I32 && t_dtype != TFPS_I64) || (mem && mem_dtype != TFPS_I32 && mem_dtype != TFPS_I64))
+        return fail(TFPS_ERR_INVALID_ARG, "bad dtype selector");
+    if (ptr_space != TFPS_HOST && ptr_space != TFPS_DEVICE) return fail(TFPS_ERR_INVALID_ARG, "bad ptr_space");
+
+    std::vector<long long> h_in_ptr, h_out_ptr, h_in_t, h_out_t, h_mem;
+    std::vector<int> h_in_src, h_out_dst, h_c;
+    TFPS_TRY(fetch(h_in_ptr, in_ptr, (size_t)n + 1, ptr_space, st));
+    TFPS_TRY(fetch(h_in_src, in_src, (size_t)m, ptr_space, st));
+    TFPS_TRY(fetch_wide(h_in_t, in_t, (size_t)m, t_dtype, ptr_space, st));
+    TFPS_TRY(fetch(h_c, c, (size_t)n, ptr_space, st));
+    TFPS_TRY(check_csr("in", n, m, h_in_ptr, h_in_src));
+
+    tfps_graph* g = new (std::nothrow) tfps_graph();
+    if (!g) return fail(TFPS_ERR_INVALID_ARG, "out of host memory");
+    struct Holder { tfps_graph* g; ~Holder() { delete g; } } holder{g};
+
+    for (long long v = 0; v < n; ++v) {
+        if (h_c[v] < 0) return fail(TFPS_ERR_BAD_CSR, "negative cost c[%lld]", v);
+        g->sum_c += (u128)h_c[v];
+        g->max_c = std::max<long long>(g->max_c, h_c[v]);
+    }
+    for (long long e = 0; e < m; ++e) {
+        if (h_in_t[e] < 0) return fail(TFPS_ERR_BAD_CSR, "negative edge size at in-edge %lld", e);
+        g->sum_t += (u128)h_in_t[e];
+        g->max_t = std::max(g->max_t, h_in_t[e]);
+    }
+    for (long long v = 0; v < n; ++v)
+        for (long long e = h_in_ptr[v]; e < h_in_ptr[v + 1]; ++e)
+            if (h_in_src[e] == v) return fail(TFPS_ERR_CYCLE, "self loop at vertex %lld", v);
+
+    // out-CSR by transposing the in-CSR (rows come out sorted by target, then by in-row order)
+    std::vector<long long> t_ptr((size_t)n + 1, 0), t_t((size_t)m);
+    std::vector<int> t_dst((size_t)m);
+    for (long long e = 0; e < m; ++e) t_ptr[(size_t)h_in_src[e] + 1]++;
+    for (long long v = 0; v < n; ++v) t_ptr[v + 1] += t_ptr[v];
+    {
+        std::vector<long long> fill(t_ptr.begin(), t_ptr.end() - 1);
+        for (long long v = 0; v < n; ++v)
+            for (long long e = h_in_ptr[v]; e < h_in_ptr[v + 1]; ++e) {
+                long long o = fill[h_in_src[e]]++;
+                t_dst[o] = (int)v;
+                t_t[o] = h_in_t[e];
+            }
+    }
+    if (have_out) {
+        TFPS_TRY(fetch(h_out_ptr, out_ptr, (size_t)n + 1, ptr_space, st));
+        TFPS_TRY(fetch(h_out_dst, out_dst, (size_t)m, ptr_space, st));
+        TFPS_TRY(fetch_wide(h_out_t, out_t, (size_t)m, t_dtype, ptr_space, st));
+        TFPS_TRY(check_csr("out", n, m, h_out_ptr, h_out_dst));
+        // both directions must describe the same multiset of (u, v, t)
+        std::vector<std::pair<int, long long>> ra, rb;
+        for (long long v = 0; v < n; ++v) {
+            if (h_out_ptr[v + 1] - h_out_ptr[v] != t_ptr[v + 1] - t_ptr[v])
+                return fail(TFPS_ERR_BAD_CSR, "out-degree of vertex %lld disagrees with the in-edge lists", v);
+            ra.clear(); rb.clear();
+            for (long long e = h_out_ptr[v]; e < h_out_ptr[v + 1]; ++e) ra.emplace_back(h_out_dst[e], h_out_t[e]);
+            for (long long e = t_ptr[v]; e < t_ptr[v + 1]; ++e) rb.emplace_back(t_dst[e], t_t[e]);
+            std::sort(ra.begin(), ra.end());
+            std::sort(rb.begin(), rb.end());
+            if (ra != rb) return fail(TFPS_ERR_BAD_CSR, "out-edges of vertex %lld disagree with the in-edge lists", v);
+        }
+    } else {
+        h_out_ptr.swap(t_ptr);
+        h_out_dst.swap(t_dst);
+        h_out_t.swap(t_t);
+    }
+    if (mem) {
+        TFPS_TRY(fetch_wide(h_mem, mem, (size_t)n, mem_dtype, ptr_space, st));
+        u128 tot = 0;
+        for (long long v = 0; v < n; ++v) {
+            if (h_mem[v] < 0) return fail(TFPS_ERR_BAD_CSR, "negative memory at vertex %lld", v);
+            tot += (u128)h_mem[v];
+        }
+        if (tot >= (u128)LIMIT62) return fail(TFPS_ERR_OVERFLOW, "sum of vertex memory reaches 2^62");
+    } else if (g->sum_t >= (u128)LIMIT62) {
+        return fail(TFPS_ERR_OVERFLOW, "sum of edge sizes reaches 2^62");
+    }
+
+    CUDA_TRY(cudaGetDevice(&g->device));
+    CUDA_TRY(cudaDeviceGetAttribute(&g->sm_count, cudaDevAttrMultiProcessorCount, g->device));
+    g->n = n;
+    g->m = m;
+    TFPS_TRY(upload(g->in_ptr, h_in_ptr, st));
+    TFPS_TRY(upload(g->in_src, h_in_src, st));
+    TFPS_TRY(upload(g->in_t, h_in_t, st));
+    TFPS_TRY(upload(g->out_ptr, h_out_ptr, st));
+    TFPS_TRY(upload(g->out_dst, h_out_dst, st));
+    TFPS_TRY(upload(g->out_t, h_out_t, st));
+    TFPS_TRY(upload(g->c, h_c, st));
+    if (mem) {
+        TFPS_TRY(upload(g->mem, h_mem, st));
+    } else {
+        CUDA_TRY(g->mem.alloc(sizeof(long long) * (size_t)n));
+        CUDA_TRY(launch_default_mem((int)n, g->out_ptr.as<long long>(), g->out_t.as<long long>(), g->mem.as<long long>(), st));
+    }
+    CUDA_TRY(g->status.alloc(sizeof(int)));
+    CUDA_TRY(cudaMemsetAsync(g->status.p, 0, sizeof(int), st));
+    CUDA_TRY(cudaStreamSynchronize(st));  // host vectors go out of scope
+    holder.g = nullptr;
+    *out = g;
+    return TFPS_OK;
+}
+
+int tfps_graph_destroy(tfps_graph* g)
+{
+    if (!g) return TFPS_OK;
+    {
+        DeviceGuard guard(g->device);
+        delete g;
+    }
+    return TFPS_OK;
+}
+
+int tfps_graph_info(const tfps_graph* g, int64_t* n, int64_t* m, int32_t* num_levels, int32_t* k)
+{
+    if (!g) return fail(TFPS_ERR_INVALID_ARG, "graph is NULL");
+    if (n) *n = g->n;
+    if (m) *m = g->m;
+    if (num_levels) *num_levels = g->topo_built ? g->num_levels : 0;
+    if (k) *k = g->dev_set ? g->k : 0;
+    return TFPS_OK;
+}
+
+int tfps_devices_set(tfps_graph* g, int k, const int32_t* s, const int64_t* C, const int64_t* B, int64_t scale)
+{
+    if (!g) return fail(TFPS_ERR_INVALID_ARG, "graph is NULL");
+    if (k < 1 || k > TFPS_K_MAX) return fail(TFPS_ERR_BAD_DEVICES, "k = %d outside 1..%d", k, (int)TFPS_K_MAX);
+    if (!s || !C || !B) return fail(TFPS_ERR_INVALID_ARG, "s, C and B are required");
+    if (scale < 1) return fail(TFPS_ERR_BAD_DEVICES, "scale must be >= 1");
+    long long s_min = INT64_MAX, b_min = INT64_MAX;
+    for (int d = 0; d < k; ++d) {
+        if (s[d] < 1) return fail(TFPS_ERR_BAD_DEVICES, "speed s[%d] = %d < 1", d, s[d]);
+        if (C[d] < 0) return fail(TFPS_ERR_BAD_DEVICES, "capacity C[%d] < 0", d);
+        s_min = std::min<long long>(s_min, s[d]);
+        for (int e = 0; e < k; ++e) {
+            if (d == e) continue;
+            long long b = B[d * k + e];
+            if (b < 1) return fail(TFPS_ERR_BAD_DEVICES, "bandwidth B[%d][%d] = %lld < 1", d, e, b);
+            if (b >= LIMIT62) return fail(TFPS_ERR_BAD_DEVICES, "bandwidth B[%d][%d] too large", d, e);
+            b_min = std::min(b_min, b);
+        }
+    }
+    // numerators c*S and t*S must stay below 2^62; so must every path length and load
+    if ((u128)g->max_c * (u128)scale >= (u128)LIMIT62 || (u128)g->max_t * (u128)scale >= (u128)LIMIT62)
+        return fail(TFPS_ERR_OVERFLOW, "c*scale or t*scale reaches 2^62");
+    u128 bound = g->sum_c * (u128)scale / (u128)s_min + (u128)g->n;
+    if (k > 1) bound += g->sum_t * (u128)scale / (u128)b_min + (u128)g->m;
+    if (bound >= (u128)LIMIT62) return fail(TFPS_ERR_OVERFLOW, "a path length or load could reach 2^62 ticks");
+
+    DeviceGuard guard(g->device);
+    if (!guard.ok) return fail(TFPS_ERR_CUDA, "cannot select the handle's device");
+    cudaStream_t st = 0;
+    TFPS_TRY(build_topo(g, st));
+
+    std::vector<DivConst> rt((size_t)k), w((size_t)k * k);
+    for (int d = 0; d < k; ++d) rt[d] = make_div((unsigned long long)s[d]);
+    for (int a = 0; a < k; ++a)
+        for (int b = 0; b < k; ++b) {
+            if (a == b) { w[a * k + b] = DivConst{0ull, 0u, 0u}; continue; }
+            w[a * k + b] = make_div((unsigned long long)B[a * k + b]);
+        }
+    std::vector<long long> cap(C, C + k);
+    g->dev_set = false;
+    TFPS_TRY(upload(g->rt_div, rt, st));
+    TFPS_TRY(upload(g->w_div, w, st));
+    TFPS_TRY(upload(g->cap, cap, st));
+    const int n = (int)g->n, m = (int)g->m;
+    CUDA_TRY(g->xvert.reserve(sizeof(unsigned long long) * (size_t)n));
+    CUDA_TRY(g->xw_f.reserve(sizeof(unsigned long long) * (size_t)m));
+    CUDA_TRY(g->xnbr_f.reserve(sizeof(unsigned long long) * (size_t)m));
+    CUDA_TRY(g->xw_b.reserve(sizeof(unsigned long long) * (size_t)m));
+    if (n > 0)
+        CUDA_TRY(launch_numerators(n, m, scale, g->order.as<int>(), g->c.as<int>(), g->f_nbr.as<int>(),
+                                   g->f_t.as<long long>(), g->b_nbr.as<int>(), g->b_t.as<long long>(),
+                                   g->xvert.as<unsigned long long>(), g->xw_f.as<unsigned long long>(),
+                                   g->xnbr_f.as<unsigned long long>(), g->xw_b.as<unsigned long long>(), st));
+    CUDA_TRY(cudaStreamSynchronize(st));
+    g->k = k;
+    g->S = scale;
+    g->dev_set = true;
+    return TFPS_OK;
+}
+
+int tfps_topo_levels(tfps_graph* g, int32_t* level, int32_t* order, int64_t* level_ptr, int64_t cap,
+                     int32_t* num_levels, void* stream)
+{
+    if (!g) return fail(TFPS_ERR_INVALID_ARG, "graph is NULL");
+    DeviceGuard guard(g->device);
+    if (!guard.ok) return fail(TFPS_ERR_CUDA, "cannot select the handle's device");
+    cudaStream_t st = (cudaStream_t)stream;
+    TFPS_TRY(build_topo(g, st));
+    if (num_levels) *num_levels = g->num_levels;
+    if (level_ptr) {
+        if (cap < (int64_t)g->num_levels + 1)
+            return fail(TFPS_ERR_INVALID_ARG, "level_ptr has room for %lld entries, %d needed", (long long)cap, g->num_levels + 1);
+        for (int l = 0; l <= g->num_levels; ++l) level_ptr[l] = g->h_level_ptr[l];
+    }
+    if (g->n > 0) {
+        if (level) CUDA_TRY(cudaMemcpyAsync(level, g->level.p, sizeof(int) * (size_t)g->n, cudaMemcpyDeviceToDevice, st));
+        if (order) CUDA_TRY(cudaMemcpyAsync(order, g->order.p, sizeof(int) * (size_t)g->n, cudaMemcpyDeviceToDevice, st));
+    }
+    CUDA_TRY(cudaStreamSynchronize(st));
+    return TFPS_OK;
+}
+
+size_t tfps_eval_workspace_bytes(const tfps_graph* g, int64_t P, int64_t ldp, int flags)
+{
+    if (!g || P <= 0 || ldp < P) return 0;
+    if (flags & TFPS_EVAL_SCRATCH_LEVELS) return sizeof(long long) * (size_t)g->n * (size_t)ldp;
+    return 0;
+}
+
+int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, int64_t* tlevel, int64_t* blevel,
+                    int64_t* cp, int64_t* load, int64_t* memload, uint64_t* viol, void* workspace,
+                    size_t workspace_bytes, int flags, void* stream)
+{
+    if (!g) return fail(TFPS_ERR_INVALID_ARG, "graph is NULL");
+    if (P < 0 || ldp < P || (ldp % 16) != 0) return fail(TFPS_ERR_INVALID_ARG, "need 0 <= P <= ldp and ldp %% 16 == 0");
+    if ((flags & TFPS_EVAL_LEVEL_SYNC) && (flags & TFPS_EVAL_SLICED))
+        return fail(TFPS_ERR_INVALID_ARG, "choose one kernel variant");
+    if (!g->dev_set) return fail(TFPS_ERR_STATE, "tfps_devices_set has not been called");
+    if (P == 0 || g->n == 0) return TFPS_OK;
+    if (!part) return fail(TFPS_ERR_INVALID_ARG, "part is NULL");
+    if (P > ((int64_t)1 << 31)) return fail(TFPS_ERR_UNSUPPORTED, "P above 2^31");
+
+    DeviceGuard guard(g->device);
+    if (!guard.ok) return fail(TFPS_ERR_CUDA, "cannot select the handle's device");
+    cudaStream_t st = (cudaStream_t)stream;
+    TFPS_TRY(build_topo(g, st));
+
+    const bool need_bwd = blevel != nullptr;
+    const bool need_fwd = tlevel != nullptr || (cp != nullptr && !need_bwd);
+    long long* fwd_lev = (long long*)tlevel;
+    if (need_fwd && !tlevel) {
+        const size_t need = sizeof(long long) * (size_t)g->n * (size_t)ldp;
+        if (!workspace || workspace_bytes < need)
+            return fail(TFPS_ERR_WORKSPACE, "workspace of %zu bytes needed for the level scratch, %zu given", need, workspace_bytes);
+        if (((uintptr_t)workspace & 255u) != 0) return fail(TFPS_ERR_WORKSPACE, "workspace must be 256-byte aligned");
+        fwd_lev = (long long*)workspace;
+    }
+    const bool validate = !(flags & TFPS_EVAL_NO_VALIDATE);
+    const int n = (int)g->n;
+    const int k = g->k;
+    DevTables tab;
+    tab.k = k;
+    tab.rt_div = g->rt_div.as<DivConst>();
+    tab.w_div = g->w_div.as<DivConst>();
+    tab.cap = g->cap.as<long long>();
+    int* status = g->status.as<int>();
+
+    // loads first: the same kernel checks the ids, and a bad id stops everything after it
+    long long* ml = (long long*)memload;
+    if (viol && !ml) {
+        CUDA_TRY(g->scr_memload.reserve(sizeof(long long) * (size_t)k * (size_t)ldp));
+        ml = g->scr_memload.as<long long>();
+    }
+    if (load || ml) {
+        if (load) CUDA_TRY(cudaMemset2DAsync(load, sizeof(long long) * (size_t)ldp, 0, sizeof(long long) * (size_t)P, (size_t)k, st));
+        if (ml) CUDA_TRY(cudaMemset2DAsync(ml, sizeof(long long) * (size_t)ldp, 0, sizeof(long long) * (size_t)P, (size_t)k, st));
+        CUDA_TRY(launch_loads(n, P, ldp, part, g->order.as<int>(), g->xvert.as<unsigned long long>(), g->mem.as<long long>(),
+                              tab, (long long*)load, ml, status, validate, g->sm_count, st));
+        if (viol) CUDA_TRY(launch_viol(P, ldp, k, ml, tab.cap, (unsigned long long*)viol, status, st));
+    } else if (validate) {
+        CUDA_TRY(launch_validate(n, P, ldp, part, k, status, g->sm_count, st));
+    }
+
+    // kernel variant
+    bool sliced;
+    if (flags & TFPS_EVAL_SLICED) sliced = true;
+    else if (flags & TFPS_EVAL_LEVEL_SYNC) sliced = false;
+    else {
+        // enough candidate slices to occupy the machine, or levels too narrow to be worth a launch each
+        const long long avg_width = g->num_levels > 0 ? g->n / g->num_levels : g->n;
+        sliced = (P >= 32LL * g->sm_count) || (avg_width * P < (1LL << 18));
+    }
+    int cpt = env_int("TFPS_SLICED_CPT", 0);
+    if (cpt != 1 && cpt != 2 && cpt != 4) cpt = (P >= 64LL * 4 * g->sm_count) ? 2 : 1;
+    int warps = env_int("TFPS_SLICED_WARPS", 0);
+    if (warps < 1 || warps > 8) {
+        const long long avg_width = g->num_levels > 0 ? g->n / g->num_levels : g->n;
+        warps = 1;
+        while (warps < 8 && warps * 2 <= avg_width) warps <<= 1;
+    }
+
+    for (int pass = 0; pass < 2; ++pass) {
+        const bool fwd = pass == 0;
+        if (fwd ? !need_fwd : !need_bwd) continue;
+        long long* lev = fwd ? fwd_lev : (long long*)blevel;
+        long long* cp_here = (cp && (fwd || !need_fwd)) ? (long long*)cp : nullptr;
+        PassArgs a = make_args(g, fwd, P, ldp, part, lev, cp_here);
+        if (sliced) {
+            CUDA_TRY(launch_pass_sliced(a, fwd, g->sink_flag.as<uint8_t>(), cpt, warps, st));
+        } else {
+            CUDA_TRY(launch_pass_level_sync(a, fwd, g->h_level_ptr, st));
+            if (cp_here) {
+                CUDA_TRY(cudaMemsetAsync(cp_here, 0, sizeof(long long) * (size_t)P, st));
+                if (fwd) CUDA_TRY(launch_cp_reduce(a, true, g->sink_list.as<int>(), g->sink_count, st));
+                else CUDA_TRY(launch_cp_reduce(a, false, nullptr, (int)g->h_level_ptr[1], st));
+            }
+        }
+    }
+    return TFPS_OK;
+}
+
+int tfps_get_status(tfps_graph* g, void* stream)
+{
+    if (!g) return fail(TFPS_ERR_INVALID_ARG, "graph is NULL");
+    DeviceGuard guard(g->device);
+    if (!guard.ok) return fail(TFPS_ERR_CUDA, "cannot select the handle's device");
+    cudaStream_t st = (cudaStream_t)stream;
+    int h = 0;
+    CUDA_TRY(cudaMemcpyAsync(&h, g->status.p, sizeof(int), cudaMemcpyDeviceToHost, st));
+    CUDA_TRY(cudaStreamSynchronize(st));
+    if (h != 0) {
+        CUDA_TRY(cudaMemsetAsync(g->status.p, 0, sizeof(int), st));
+        CUDA_TRY(cudaStreamSynchronize(st));
+        return fail(h, "device-side status: %s", tfps_strerror(h));
+    }
+    return TFPS_OK;
+}
+
+int tfps_eval_batch_host(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, int64_t* cp, int64_t* load,
+                         int64_t* memload, uint64_t* viol, int flags, void* stream)
+{
+    if (!g) return fail(TFPS_ERR_INVALID_ARG, "graph is NULL");
+    if (P < 0 || ldp < P || (ldp % 16) != 0) return fail(TFPS_ERR_INVALID_ARG, "need 0 <= P <= ldp and ldp %% 16 == 0");
+    if (!g->dev_set) return fail(TFPS_ERR_STATE, "tfps_devices_set has not been called");
+    if (P == 0 || g->n == 0) return TFPS_OK;
+    if (!part) return fail(TFPS_ERR_INVALID_ARG, "part is NULL");
+    DeviceGuard guard(g->device);
+    if (!guard.ok) return fail(TFPS_ERR_CUDA, "cannot select the handle's device");
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t cells = (size_t)g->n * (size_t)ldp;
+    const size_t kcells = (size_t)g->k * (size_t)ldp;
+    CUDA_TRY(g->st_part.reserve(cells));
+    if (cp) { CUDA_TRY(g->st_lev.reserve(cells * 8)); CUDA_TRY(g->st_cp.reserve((size_t)P * 8)); }
+    if (load) CUDA_TRY(g->st_load.reserve(kcells * 8));
+    if (memload || viol) CUDA_TRY(g->st_mem.reserve(kcells * 8));
+    if (viol) CUDA_TRY(g->st_viol.reserve((size_t)P * 8));
+    CUDA_TRY(cudaMemcpyAsync(g->st_part.p, part, cells, cudaMemcpyHostToDevice, st));
+    TFPS_TRY(tfps_eval_batch(g, P, ldp, g->st_part.as<uint8_t>(), nullptr, nullptr,
+                             cp ? g->st_cp.as<int64_t>() : nullptr, load ? g->st_load.as<int64_t>() : nullptr,
+                             (memload || viol) ? g->st_mem.as<int64_t>() : nullptr,
+                             viol ? g->st_viol.as<uint64_t>() : nullptr, g->st_lev.p, g->st_lev.bytes,
+                             flags | TFPS_EVAL_SCRATCH_LEVELS, st));
+    if (cp) CUDA_TRY(cudaMemcpyAsync(cp, g->st_cp.p, (size_t)P * 8, cudaMemcpyDeviceToHost, st));
+    if (load) CUDA_TRY(cudaMemcpyAsync(load, g->st_load.p, kcells * 8, cudaMemcpyDeviceToHost, st));
+    if (memload) CUDA_TRY(cudaMemcpyAsync(memload, g->st_mem.p, kcells * 8, cudaMemcpyDeviceToHost, st));
+    if (viol) CUDA_TRY(cudaMemcpyAsync(viol, g->st_viol.p, (size_t)P * 8, cudaMemcpyDeviceToHost, st));
+    return tfps_get_status(g, stream);
+}
+
+int tfps_transpose_u8(const uint8_t* src, uint8_t* dst, int64_t P, int64_t n, int64_t ldp, void* stream)
+{
+    if (P < 0 || n < 0 || ldp < P) return fail(TFPS_ERR_INVALID_ARG, "need 0 <= P <= ldp, n >= 0");
+    if (P == 0 || n == 0) return TFPS_OK;
+    if (!src || !dst) return fail(TFPS_ERR_INVALID_ARG, "src and dst are required");
+    if ((P + 63) / 64 > 65535) return fail(TFPS_ERR_UNSUPPORTED, "P above 64*65535");
+    CUDA_TRY(launch_transpose_u8(src, dst, P, n, ldp, (cudaStream_t)stream));
+    return TFPS_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,93 @@
+// Internal declarations shared by the translation units of libtfps.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <string>
+#include <vector>
+
+#include "tfps.h"
+
+namespace tfps {
+
+// ---------------------------------------------------------------------------
+// Exact division by an invariant divisor d >= 1 for numerators x < 2^62:
+//   floor(x / d) == umul64hi(mul, x << 2) >> sh
+// with  sh = ceil(log2 d)  and  mul = ceil(2^(62+sh) / d)   (mul <= 2^63).
+// Proof sketch: mul*d = 2^(62+sh) + e with 0 <= e < d <= 2^sh, so
+// mul*x / 2^(62+sh) = x/d + x*e/(d*2^(62+sh)) and the excess is < 1/d, too
+// small to carry the quotient over the next integer.
+//
+// A ceiling quotient of a positive numerator a is taken as 1 + floor((a-1)/d);
+// the library stores numerators already in the form X = (a-1) << 2, with the
+// reserved value NUM_ZERO standing for a == 0 (quotient 0).
+// ---------------------------------------------------------------------------
+struct DivConst {
+    unsigned long long mul;
+    unsigned int sh;
+    unsigned int pad;
+};
+static_assert(sizeof(DivConst) == 16, "DivConst is loaded as one 16-byte word");
+
+constexpr unsigned long long NUM_ZERO = ~0ull;
+
+// Device tables set by tfps_devices_set (global memory; kernels stage them in
+// shared memory).  rt_div[d] divides by s_d, w_div[a*k+b] by B[a][b].
+struct DevTables {
+    int k;
+    const DivConst* rt_div;  // [k]
+    const DivConst* w_div;   // [k*k]
+    const long long* cap;    // [k]
+};
+
+// Level-ordered adjacency of one direction.  Position i runs over vertices
+// sorted by (level, id); FWD lists in-edges, BWD out-edges.
+struct LevelAdj {
+    const int* vert;                 // [n]   vertex at position i
+    const int* eptr;                 // [n+1] edge offsets by position
+    const int* nbr;                  // [m]   neighbour vertex id
+    const unsigned long long* xw;    // [m]   transfer numerator ((t*S-1)<<2 or NUM_ZERO)
+    const unsigned long long* xnbr;  // [m]   neighbour's runtime numerator ((c*S-1)<<2 or NUM_ZERO)
+    const unsigned long long* xvert; // [n]   own runtime numerator by position
+};
+
+struct PassArgs {
+    LevelAdj adj;
+    DevTables tab;
+    const long long* level_ptr;  // [L+1] device copy
+    int num_levels;
+    int n;
+    long long P, ldp;
+    const uint8_t* part;
+    long long* lev;       // [n][ldp] levels written by this pass
+    long long* cp;        // [P] or NULL
+    int* status;          // sticky status word
+};
+
+// ---- launch wrappers (host side, implemented in the .cu files) -------------
+cudaError_t launch_kahn(int n, const long long* in_ptr, const long long* out_ptr, const int* out_dst,
+                        int* indeg, int* level, int* queue, long long* level_ptr_dev, int* level_cnt,
+                        long long* result, int sm_count, cudaStream_t st);
+cudaError_t launch_sort_order(int n, const int* level, unsigned long long* keys, int npad, int* order, cudaStream_t st);
+cudaError_t launch_build_adj(int n, const int* order, const long long* ptr, const int* idx, const long long* t,
+                             int* eptr, int* nbr, long long* tperm, cudaStream_t st);
+cudaError_t launch_sink_flags(int n, const int* order, const long long* out_ptr, uint8_t* flag, cudaStream_t st);
+cudaError_t launch_numerators(int n, int m, long long S, const int* order, const int* c,
+                              const int* nbr_f, const long long* t_f, const int* nbr_b, const long long* t_b,
+                              unsigned long long* xvert, unsigned long long* xw_f, unsigned long long* xnbr_f,
+                              unsigned long long* xw_b, cudaStream_t st);
+cudaError_t launch_default_mem(int n, const long long* out_ptr, const long long* out_t, long long* mem, cudaStream_t st);
+
+int pick_cpt(long long P);
+cudaError_t launch_pass_level_sync(const PassArgs& a, bool fwd, const std::vector<long long>& level_ptr_host, cudaStream_t st);
+cudaError_t launch_pass_sliced(const PassArgs& a, bool fwd, const uint8_t* cp_flag, int cpt, int warps, cudaStream_t st);
+cudaError_t launch_cp_reduce(const PassArgs& a, bool from_tlevel, const int* list, int list_len, cudaStream_t st);
+cudaError_t launch_loads(int n, long long P, long long ldp, const uint8_t* part, const int* vert,
+                         const unsigned long long* xvert, const long long* mem, DevTables tab, long long* load,
+                         long long* memload, int* status, bool validate, int sm_count, cudaStream_t st);
+cudaError_t launch_validate(long long n, long long P, long long ldp, const uint8_t* part, int k, int* status,
+                            int sm_count, cudaStream_t st);
+cudaError_t launch_viol(long long P, long long ldp, int k, const long long* memload, const long long* cap,
+                        unsigned long long* viol, const int* status, cudaStream_t st);
+cudaError_t launch_transpose_u8(const uint8_t* src, uint8_t* dst, long long P, long long n, long long ldp, cudaStream_t st);
+
+}  // namespace tfps

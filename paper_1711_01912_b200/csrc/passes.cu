@@ -1,0 +1,512 @@
+// Forward (tlevel) and backward (blevel = PCT, Eq. 12) longest-path passes over
+// the vertex-major [n][ldp] candidate layout, critical-path reduction, per-
+// device load / memory reduction, id validation and the uint8 transpose.
+//
+// Lane = candidate(s): a warp covers 32*CPT contiguous candidates of one
+// vertex, so every neighbour-level read is one contiguous 256*CPT-byte row
+// segment and every id read a contiguous 32*CPT-byte one.
+#include "common.cuh"
+
+namespace tfps {
+
+namespace {
+
+// ---- small vector helpers ----------------------------------------------------
+template <int CPT> struct IdVec;
+template <> struct IdVec<1> {
+    static __device__ __forceinline__ unsigned load(const uint8_t* p) { return *p; }
+};
+template <> struct IdVec<2> {
+    static __device__ __forceinline__ unsigned load(const uint8_t* p) { return *reinterpret_cast<const unsigned short*>(p); }
+};
+template <> struct IdVec<4> {
+    static __device__ __forceinline__ unsigned load(const uint8_t* p) { return *reinterpret_cast<const unsigned*>(p); }
+};
+
+template <int CPT>
+__device__ __forceinline__ void load_levels(const long long* p, long long (&out)[CPT])
+{
+    if constexpr (CPT == 1) {
+        out[0] = *p;
+    } else {
+#pragma unroll
+        for (int i = 0; i < CPT; i += 2) {
+            longlong2 v = *reinterpret_cast<const longlong2*>(p + i);
+            out[i] = v.x;
+            out[i + 1] = v.y;
+        }
+    }
+}
+
+template <int CPT>
+__device__ __forceinline__ void store_levels(long long* p, const long long (&v)[CPT], int nvalid)
+{
+    if (nvalid >= CPT) {
+        if constexpr (CPT == 1) {
+            *p = v[0];
+        } else {
+#pragma unroll
+            for (int i = 0; i < CPT; i += 2) *reinterpret_cast<longlong2*>(p + i) = make_longlong2(v[i], v[i + 1]);
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < CPT; ++i)
+            if (i < nvalid) p[i] = v[i];
+    }
+}
+
+__device__ __forceinline__ long long ceil_quot(unsigned long long X, const DivConst& dc)
+{
+    return 1 + (long long)(__umul64hi(dc.mul, X) >> dc.sh);
+}
+
+// Shared-memory copy of the division constants: [k*k] pair table then [k] speed table.
+__device__ __forceinline__ void stage_tables(const DevTables& tab, DivConst* s_w, DivConst* s_rt)
+{
+    const int k = tab.k;
+    for (int i = threadIdx.x; i < k * k; i += blockDim.x) s_w[i] = tab.w_div[i];
+    for (int i = threadIdx.x; i < k; i += blockDim.x) s_rt[i] = tab.rt_div[i];
+    __syncthreads();
+}
+
+// ---- one vertex, 32*CPT candidates --------------------------------------------
+// FWD: best = max over in-edges of tlevel(u) + rt(u) + w(u->v); writes tlevel(v).
+// BWD: best = max over out-edges of blevel(x) + w(v->x); writes blevel(v) = best + rt(v).
+// cpmax (may be unused) accumulates tlevel+rt over sinks (FWD) or blevel over sources (BWD).
+template <int CPT, bool FWD>
+__device__ __forceinline__ void relax_vertex(const PassArgs& a, const DivConst* __restrict__ s_w,
+                                             const DivConst* __restrict__ s_rt, int pos, long long jl,
+                                             unsigned idmask, int nvalid, bool cp_vertex,
+                                             long long (&cpmax)[CPT])
+{
+    const int k = a.tab.k;
+    const int v = a.adj.vert[pos];
+    const int e0 = a.adj.eptr[pos];
+    const int e1 = a.adj.eptr[pos + 1];
+    const long long ldp = a.ldp;
+    const unsigned pv = IdVec<CPT>::load(a.part + (long long)v * ldp + jl) & idmask;
+    unsigned idv[CPT];
+#pragma unroll
+    for (int c = 0; c < CPT; ++c) idv[c] = (pv >> (8 * c)) & 0xffu;
+
+    long long best[CPT];
+#pragma unroll
+    for (int c = 0; c < CPT; ++c) best[c] = 0;
+
+    constexpr int UNR = (CPT >= 4) ? 2 : 4;
+    for (int e = e0; e < e1; e += UNR) {
+        long long lu[UNR][CPT];
+        unsigned pu[UNR];
+        unsigned long long X[UNR], Xn[UNR];
+#pragma unroll
+        for (int q = 0; q < UNR; ++q) {
+            if (e + q < e1) {
+                const int u = a.adj.nbr[e + q];
+                X[q] = a.adj.xw[e + q];
+                if (FWD) Xn[q] = a.adj.xnbr[e + q];
+                const long long off = (long long)u * ldp + jl;
+                pu[q] = IdVec<CPT>::load(a.part + off) & idmask;
+                load_levels<CPT>(a.lev + off, lu[q]);
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < UNR; ++q) {
+            if (e + q < e1) {
+#pragma unroll
+                for (int c = 0; c < CPT; ++c) {
+                    const unsigned idu = (pu[q] >> (8 * c)) & 0xffu;
+                    long long val = lu[q][c];
+                    if (X[q] != NUM_ZERO) {
+                        const DivConst dc = s_w[FWD ? idu * k + idv[c] : idv[c] * k + idu];
+                        const long long w = ceil_quot(X[q], dc);
+                        val += (idu != idv[c]) ? w : 0;
+                    }
+                    if (FWD) {
+                        if (Xn[q] != NUM_ZERO) val += ceil_quot(Xn[q], s_rt[idu]);
+                    }
+                    best[c] = val > best[c] ? val : best[c];
+                }
+            }
+        }
+    }
+
+    if (FWD) {
+        store_levels<CPT>(a.lev + (long long)v * ldp + jl, best, nvalid);
+        if (cp_vertex) {
+            const unsigned long long Xv = a.adj.xvert[pos];
+#pragma unroll
+            for (int c = 0; c < CPT; ++c) {
+                long long fin = best[c];
+                if (Xv != NUM_ZERO) fin += ceil_quot(Xv, s_rt[idv[c]]);
+                cpmax[c] = fin > cpmax[c] ? fin : cpmax[c];
+            }
+        }
+    } else {
+        const unsigned long long Xv = a.adj.xvert[pos];
+#pragma unroll
+        for (int c = 0; c < CPT; ++c) {
+            if (Xv != NUM_ZERO) best[c] += ceil_quot(Xv, s_rt[idv[c]]);
+            if (cp_vertex) cpmax[c] = best[c] > cpmax[c] ? best[c] : cpmax[c];
+        }
+        store_levels<CPT>(a.lev + (long long)v * ldp + jl, best, nvalid);
+    }
+}
+
+// Lane bookkeeping shared by both pass kernels: first candidate of the lane,
+// how many of its CPT candidates are real, the mask that zeroes padding ids and
+// the (always in-bounds) column the lane loads from.
+template <int CPT>
+__device__ __forceinline__ void lane_setup(long long slice0, long long P, int lane, long long& jl, int& nvalid,
+                                           unsigned& idmask)
+{
+    const long long j0 = slice0 + (long long)lane * CPT;
+    long long rem = P - j0;
+    nvalid = rem >= CPT ? CPT : (rem > 0 ? (int)rem : 0);
+    jl = nvalid > 0 ? j0 : slice0;  // idle lanes shadow the slice's first lane and never store
+    idmask = nvalid >= 4 ? 0xffffffffu : ((1u << (8 * nvalid)) - 1u);
+    if (nvalid == 0) idmask = 0;
+}
+
+// ---- level-synchronous variant: one launch per level ----------------------------
+template <int CPT, bool FWD>
+__global__ void __launch_bounds__(128)
+pass_level_kernel(PassArgs a, int pos0, int count)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    DivConst* s_w = reinterpret_cast<DivConst*>(smem_raw);
+    DivConst* s_rt = s_w + a.tab.k * a.tab.k;
+    if (*a.status != 0) return;
+    stage_tables(a.tab, s_w, s_rt);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, wpb = blockDim.x >> 5;
+    const long long slice0 = (long long)blockIdx.x * 32 * CPT;
+    long long jl; int nvalid; unsigned idmask;
+    lane_setup<CPT>(slice0, a.P, lane, jl, nvalid, idmask);
+    long long unused[CPT];
+#pragma unroll
+    for (int c = 0; c < CPT; ++c) unused[c] = 0;
+    for (int i = blockIdx.y * wpb + warp; i < count; i += gridDim.y * wpb)
+        relax_vertex<CPT, FWD>(a, s_w, s_rt, pos0 + i, jl, idmask, nvalid, false, unused);
+}
+
+// ---- candidate-sliced persistent variant ---------------------------------------------
+// One block owns 32*CPT candidates and walks every level; its warps share the
+// vertices of a level and meet at a block barrier between levels.  Candidates
+// are independent, so no block ever waits for another one.
+template <int CPT, bool FWD>
+__global__ void __launch_bounds__(256)
+pass_sliced_kernel(PassArgs a, const uint8_t* __restrict__ cp_flag)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    DivConst* s_w = reinterpret_cast<DivConst*>(smem_raw);
+    DivConst* s_rt = s_w + a.tab.k * a.tab.k;
+    long long* s_cp = reinterpret_cast<long long*>(s_rt + a.tab.k);  // [warps][32*CPT]
+    if (*a.status != 0) return;
+    stage_tables(a.tab, s_w, s_rt);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, wpb = blockDim.x >> 5;
+    const long long slice0 = (long long)blockIdx.x * 32 * CPT;
+    long long jl; int nvalid; unsigned idmask;
+    lane_setup<CPT>(slice0, a.P, lane, jl, nvalid, idmask);
+    const bool want_cp = a.cp != nullptr;
+    long long cpmax[CPT];
+#pragma unroll
+    for (int c = 0; c < CPT; ++c) cpmax[c] = 0;
+
+    const int L = a.num_levels;
+    for (int step = 0; step < L; ++step) {
+        const int l = FWD ? step : L - 1 - step;
+        const int p0 = (int)a.level_ptr[l];
+        const int p1 = (int)a.level_ptr[l + 1];
+        for (int pos = p0 + warp; pos < p1; pos += wpb) {
+            bool cpv = false;
+            if (want_cp) cpv = FWD ? (cp_flag[pos] != 0) : (l == 0);
+            relax_vertex<CPT, FWD>(a, s_w, s_rt, pos, jl, idmask, nvalid, cpv, cpmax);
+        }
+        __syncthreads();
+    }
+
+    if (want_cp) {
+#pragma unroll
+        for (int c = 0; c < CPT; ++c) s_cp[(warp * 32 + lane) * CPT + c] = cpmax[c];
+        __syncthreads();
+        if (warp == 0) {
+#pragma unroll
+            for (int c = 0; c < CPT; ++c) {
+                long long m = cpmax[c];
+                for (int w = 1; w < wpb; ++w) {
+                    long long o = s_cp[(w * 32 + lane) * CPT + c];
+                    m = o > m ? o : m;
+                }
+                if (c < nvalid) a.cp[slice0 + (long long)lane * CPT + c] = m;
+            }
+        }
+    }
+}
+
+// ---- critical-path length for the level-synchronous variant -----------------------
+// cp[j] = max over the listed positions of lev (+ rt when reducing tlevel).  cp is
+// zeroed by the host; partial maxima are merged with atomicMax (order independent).
+template <bool FROM_TLEVEL>
+__global__ void __launch_bounds__(128)
+cp_reduce_kernel(PassArgs a, const int* __restrict__ list, int list_len, int per_block)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    DivConst* s_rt = reinterpret_cast<DivConst*>(smem_raw);
+    if (*a.status != 0) return;
+    for (int i = threadIdx.x; i < a.tab.k; i += blockDim.x) s_rt[i] = a.tab.rt_div[i];
+    __syncthreads();
+    const long long j = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= a.P) return;
+    int i0 = blockIdx.y * per_block;
+    int i1 = i0 + per_block < list_len ? i0 + per_block : list_len;
+    long long m = 0;
+    for (int i = i0; i < i1; ++i) {
+        const int pos = list ? list[i] : i;
+        const int v = a.adj.vert[pos];
+        long long val = a.lev[(long long)v * a.ldp + j];
+        if (FROM_TLEVEL) {
+            const unsigned long long Xv = a.adj.xvert[pos];
+            const unsigned id = a.part[(long long)v * a.ldp + j];
+            if (Xv != NUM_ZERO) val += ceil_quot(Xv, s_rt[id]);
+        }
+        m = val > m ? val : m;
+    }
+    atomicMax(&a.cp[j], m);
+}
+
+// ---- per-device load and memory ----------------------------------------------------------
+// Thread = 4 candidates; a block keeps [k][candidates] accumulators for load
+// and memory in shared memory (each thread touches only its own columns, so no
+// shared-memory atomics), walks a chunk of vertices and merges into global
+// memory with 64-bit atomic adds (integer, order independent).  Doubles as the
+// id validator: an id >= k raises BAD_PARTITION and is counted on device 0.
+__global__ void loads_kernel(int n, long long P, long long ldp, const uint8_t* __restrict__ part,
+                             const int* __restrict__ vert, const unsigned long long* __restrict__ xvert,
+                             const long long* __restrict__ mem, DevTables tab, long long* load,
+                             long long* memload, int* status, int validate, int rows_per_block)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int k = tab.k;
+    const int bc = blockDim.x * 4;
+    DivConst* s_rt = reinterpret_cast<DivConst*>(smem_raw);
+    long long* acc_l = reinterpret_cast<long long*>(s_rt + k);
+    long long* acc_m = acc_l + (size_t)k * bc;
+    for (int i = threadIdx.x; i < k; i += blockDim.x) s_rt[i] = tab.rt_div[i];
+    for (int i = threadIdx.x; i < k * bc; i += blockDim.x) { acc_l[i] = 0; acc_m[i] = 0; }
+    __syncthreads();
+
+    const long long slice0 = (long long)blockIdx.x * bc;
+    const long long j0 = slice0 + (long long)threadIdx.x * 4;
+    const long long rem = P - j0;
+    const int nvalid = rem >= 4 ? 4 : (rem > 0 ? (int)rem : 0);
+    if (nvalid == 0) return;
+    const int col = threadIdx.x * 4;
+    const int r0 = blockIdx.y * rows_per_block;
+    const int r1 = r0 + rows_per_block < n ? r0 + rows_per_block : n;
+    bool bad = false;
+    for (int pos = r0; pos < r1; ++pos) {
+        const int v = vert[pos];
+        const unsigned long long Xv = xvert[pos];
+        const long long mv = mem[v];
+        const unsigned packed = *reinterpret_cast<const unsigned*>(part + (long long)v * ldp + j0);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            if (c < nvalid) {
+                unsigned id = (packed >> (8 * c)) & 0xffu;
+                if (id >= (unsigned)k) { bad = true; id = 0; }
+                const long long rt = Xv != NUM_ZERO ? ceil_quot(Xv, s_rt[id]) : 0;
+                acc_l[id * bc + col + c] += rt;
+                acc_m[id * bc + col + c] += mv;
+            }
+        }
+    }
+    if (bad && validate) atomicCAS(status, 0, (int)TFPS_ERR_BAD_PARTITION);
+    for (int d = 0; d < k; ++d) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            if (c < nvalid) {
+                if (load) atomicAdd(reinterpret_cast<unsigned long long*>(load + d * ldp + j0 + c),
+                                    (unsigned long long)acc_l[d * bc + col + c]);
+                if (memload) atomicAdd(reinterpret_cast<unsigned long long*>(memload + d * ldp + j0 + c),
+                                       (unsigned long long)acc_m[d * bc + col + c]);
+            }
+        }
+    }
+}
+
+// id check alone (no load outputs wanted): 16 ids per thread
+__global__ void validate_kernel(long long n, long long P, long long ldp, const uint8_t* __restrict__ part, int k,
+                                int* status)
+{
+    const long long vecs_per_row = (P + 15) / 16;
+    const long long total = n * vecs_per_row;
+    bool bad = false;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+         i += (long long)gridDim.x * blockDim.x) {
+        const long long v = i / vecs_per_row;
+        const long long j = (i - v * vecs_per_row) * 16;
+        const uint4 q = *reinterpret_cast<const uint4*>(part + v * ldp + j);
+        const unsigned w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+        for (int b = 0; b < 16; ++b) {
+            const unsigned id = (w[b >> 2] >> (8 * (b & 3))) & 0xffu;
+            if (j + b < P && id >= (unsigned)k) bad = true;
+        }
+    }
+    if (bad) atomicCAS(status, 0, (int)TFPS_ERR_BAD_PARTITION);
+}
+
+__global__ void viol_kernel(long long P, long long ldp, int k, const long long* __restrict__ memload,
+                            const long long* __restrict__ cap, unsigned long long* viol, const int* status)
+{
+    if (*status != 0) return;
+    const long long j = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= P) return;
+    unsigned long long bits = 0;
+    for (int d = 0; d < k; ++d)
+        if (memload[d * ldp + j] >= cap[d]) bits |= 1ull << d;
+    viol[j] = bits;
+}
+
+// ---- [P][n] -> [n][ldp] byte transpose ------------------------------------------------------
+__global__ void __launch_bounds__(256)
+transpose_u8_kernel(const uint8_t* __restrict__ src, uint8_t* __restrict__ dst, long long P, long long n, long long ldp)
+{
+    __shared__ uint8_t tile[64][65];
+    const long long v0 = (long long)blockIdx.x * 64;  // along n (contiguous in src)
+    const long long j0 = (long long)blockIdx.y * 64;  // along P (contiguous in dst)
+    const int tx = threadIdx.x & 63, ty = threadIdx.x >> 6;
+    for (int r = ty; r < 64; r += 4) {
+        const long long j = j0 + r, v = v0 + tx;
+        if (j < P && v < n) tile[r][tx] = src[j * n + v];
+    }
+    __syncthreads();
+    for (int r = ty; r < 64; r += 4) {
+        const long long v = v0 + r, j = j0 + tx;
+        if (v < n && j < P) dst[v * ldp + j] = tile[tx][r];
+    }
+}
+
+inline unsigned cdivu(long long a, long long b) { return (unsigned)((a + b - 1) / b); }
+
+size_t table_smem(int k) { return sizeof(DivConst) * (size_t)(k * k + k); }
+
+template <typename K>
+cudaError_t allow_smem(K kernel, size_t bytes)
+{
+    if (bytes <= 48 * 1024) return cudaSuccess;
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+}
+
+}  // namespace
+
+int pick_cpt(long long P)
+{
+    return P >= 64 * 148 ? 2 : 1;
+}
+
+template <int CPT, bool FWD>
+static cudaError_t level_sync_impl(const PassArgs& a, const std::vector<long long>& lp, cudaStream_t st)
+{
+    const size_t smem = table_smem(a.tab.k);
+    cudaError_t e = allow_smem(pass_level_kernel<CPT, FWD>, smem);
+    if (e != cudaSuccess) return e;
+    const unsigned gx = cdivu(a.P, 32 * CPT);
+    const int L = a.num_levels;
+    for (int step = 0; step < L; ++step) {
+        const int l = FWD ? step : L - 1 - step;
+        const int pos0 = (int)lp[l];
+        const int count = (int)(lp[l + 1] - lp[l]);
+        if (FWD && l == 0 && false) continue;
+        unsigned gy = cdivu(count, 4);
+        if (gy > 65535u) gy = 65535u;
+        pass_level_kernel<CPT, FWD><<<dim3(gx, gy), 128, smem, st>>>(a, pos0, count);
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_pass_level_sync(const PassArgs& a, bool fwd, const std::vector<long long>& lp, cudaStream_t st)
+{
+    const int cpt = pick_cpt(a.P);
+    if (cpt == 2) return fwd ? level_sync_impl<2, true>(a, lp, st) : level_sync_impl<2, false>(a, lp, st);
+    return fwd ? level_sync_impl<1, true>(a, lp, st) : level_sync_impl<1, false>(a, lp, st);
+}
+
+template <int CPT, bool FWD>
+static cudaError_t sliced_impl(const PassArgs& a, const uint8_t* cp_flag, int warps, cudaStream_t st)
+{
+    const size_t smem = table_smem(a.tab.k) + sizeof(long long) * (size_t)warps * 32 * CPT;
+    cudaError_t e = allow_smem(pass_sliced_kernel<CPT, FWD>, smem);
+    if (e != cudaSuccess) return e;
+    const unsigned gx = cdivu(a.P, 32 * CPT);
+    pass_sliced_kernel<CPT, FWD><<<gx, warps * 32, smem, st>>>(a, cp_flag);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_pass_sliced(const PassArgs& a, bool fwd, const uint8_t* cp_flag, int cpt, int warps, cudaStream_t st)
+{
+    if (cpt == 4) return fwd ? sliced_impl<4, true>(a, cp_flag, warps, st) : sliced_impl<4, false>(a, cp_flag, warps, st);
+    if (cpt == 2) return fwd ? sliced_impl<2, true>(a, cp_flag, warps, st) : sliced_impl<2, false>(a, cp_flag, warps, st);
+    return fwd ? sliced_impl<1, true>(a, cp_flag, warps, st) : sliced_impl<1, false>(a, cp_flag, warps, st);
+}
+
+cudaError_t launch_cp_reduce(const PassArgs& a, bool from_tlevel, const int* list, int list_len, cudaStream_t st)
+{
+    if (list_len <= 0) return cudaSuccess;
+    const size_t smem = sizeof(DivConst) * (size_t)a.tab.k;
+    const unsigned gx = cdivu(a.P, 128);
+    int per_block = 256;
+    unsigned gy = cdivu(list_len, per_block);
+    if (gy > 65535u) { per_block = (int)cdivu(list_len, 65535); gy = cdivu(list_len, per_block); }
+    if (from_tlevel)
+        cp_reduce_kernel<true><<<dim3(gx, gy), 128, smem, st>>>(a, list, list_len, per_block);
+    else
+        cp_reduce_kernel<false><<<dim3(gx, gy), 128, smem, st>>>(a, list, list_len, per_block);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_loads(int n, long long P, long long ldp, const uint8_t* part, const int* vert,
+                         const unsigned long long* xvert, const long long* mem, DevTables tab, long long* load,
+                         long long* memload, int* status, bool validate, int sm_count, cudaStream_t st)
+{
+    const int k = tab.k;
+    // threads per block sized so that 2*k*(4*threads) int64 accumulators fit in shared memory
+    int threads = 64;
+    while (threads > 32 && sizeof(DivConst) * k + (size_t)2 * k * threads * 4 * 8 > 96 * 1024) threads >>= 1;
+    const size_t smem = sizeof(DivConst) * k + (size_t)2 * k * threads * 4 * 8;
+    cudaError_t e = allow_smem(loads_kernel, smem);
+    if (e != cudaSuccess) return e;
+    const unsigned gx = cdivu(P, threads * 4);
+    long long want_blocks = (long long)sm_count * 8;
+    long long gy = (want_blocks + gx - 1) / gx;
+    if (gy < 1) gy = 1;
+    if (gy > n) gy = n;
+    if (gy > 65535) gy = 65535;
+    int rows = (int)((n + gy - 1) / gy);
+    gy = (n + rows - 1) / rows;
+    loads_kernel<<<dim3(gx, (unsigned)gy), threads, smem, st>>>(n, P, ldp, part, vert, xvert, mem, tab, load, memload,
+                                                                status, validate ? 1 : 0, rows);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_validate(long long n, long long P, long long ldp, const uint8_t* part, int k, int* status,
+                            int sm_count, cudaStream_t st)
+{
+    validate_kernel<<<sm_count * 8, 256, 0, st>>>(n, P, ldp, part, k, status);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_viol(long long P, long long ldp, int k, const long long* memload, const long long* cap,
+                        unsigned long long* viol, const int* status, cudaStream_t st)
+{
+    viol_kernel<<<cdivu(P, 256), 256, 0, st>>>(P, ldp, k, memload, cap, viol, status);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_transpose_u8(const uint8_t* src, uint8_t* dst, long long P, long long n, long long ldp, cudaStream_t st)
+{
+    dim3 grid(cdivu(n, 64), cdivu(P, 64));
+    transpose_u8_kernel<<<grid, 256, 0, st>>>(src, dst, P, n, ldp);
+    return cudaGetLastError();
+}
+
+}  // namespace tfps

@@ -266,13 +266,17 @@ def _random_layered(rng, n: int, m: int, layers: int):
     the remaining edges connect random earlier -> later layer pairs."""
     layer_of = np.sort(rng.integers(0, layers, size=n))
     layer_of[0] = 0
+    if n >= 2 and layer_of[-1] == 0:
+        layer_of[-1] = 1
     first_of = np.searchsorted(layer_of, np.arange(layers + 1))
     non_src = np.nonzero(layer_of > 0)[0]
     hi = first_of[layer_of[non_src]]  # vertices of earlier layers are [0, hi)
     non_src = non_src[hi > 0]; hi = hi[hi > 0]
     src = (rng.random(non_src.shape[0]) * hi).astype(np.int64)
     dst = non_src.astype(np.int64)
-    while src.shape[0] < m:
+    for _attempt in range(64):  # dense requests may not be satisfiable: give up and return fewer edges
+        if src.shape[0] >= m:
+            break
         need = (m - src.shape[0]) * 2 + 8
         d = rng.integers(0, n, size=need)
         h = first_of[layer_of[d]]

@@ -1,0 +1,294 @@
+"""ctypes binding of libtfps.so (argument marshalling only).
+
+Module-level ``tfps_*`` functions mirror the C ABI of ``include/tfps.h`` one to
+one and take raw addresses/ints.  ``Graph`` wraps them for callers that hold
+numpy arrays (host) and torch CUDA tensors (device memory and streams only --
+every step of the evaluation runs in the library's kernels).
+
+There is no CPU fallback: if the shared library is missing or cannot be loaded
+an ImportError is raised at first use.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Dict, Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libtfps.so")
+
+OK = 0
+ERR_INVALID_ARG, ERR_BAD_CSR, ERR_CYCLE, ERR_BAD_DEVICES, ERR_BAD_PARTITION = -1, -2, -3, -4, -5
+ERR_OVERFLOW, ERR_WORKSPACE, ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT, ERR_STATE = -6, -7, -8, -9, -10, -11
+K_MAX = 64
+I32, I64 = 0, 1
+HOST, DEVICE = 0, 1
+EVAL_AUTO, EVAL_LEVEL_SYNC, EVAL_SLICED, EVAL_NO_VALIDATE, EVAL_SCRATCH_LEVELS = 0, 1, 2, 16, 32
+
+EXPORTS = [
+    "tfps_strerror", "tfps_last_error", "tfps_graph_create", "tfps_graph_destroy", "tfps_graph_info",
+    "tfps_devices_set", "tfps_topo_levels", "tfps_eval_workspace_bytes", "tfps_eval_batch",
+    "tfps_eval_batch_host", "tfps_get_status", "tfps_transpose_u8",
+]
+
+
+class TfpsError(RuntimeError):
+    def __init__(self, code: int, message: str):
+        super().__init__(f"tfps error {code}: {message}")
+        self.code = code
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load libtfps.so (built by ``paper_1711_01912_b200.build``); never falls back to anything else."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_1711_01912_b200.build` "
+                          "(or __graft_entry__.build()); there is no CPU fallback")
+    L = ctypes.CDLL(LIB_PATH)
+    vp, i64, i32, ci, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_int, ctypes.c_size_t
+    L.tfps_strerror.restype = ctypes.c_char_p
+    L.tfps_strerror.argtypes = [ci]
+    L.tfps_last_error.restype = ctypes.c_char_p
+    L.tfps_last_error.argtypes = []
+    L.tfps_graph_create.restype = ci
+    L.tfps_graph_create.argtypes = [ctypes.POINTER(vp), i64, i64, vp, vp, vp, vp, vp, vp, ci, vp, vp, ci, ci, vp]
+    L.tfps_graph_destroy.restype = ci
+    L.tfps_graph_destroy.argtypes = [vp]
+    L.tfps_graph_info.restype = ci
+    L.tfps_graph_info.argtypes = [vp, ctypes.POINTER(i64), ctypes.POINTER(i64), ctypes.POINTER(i32), ctypes.POINTER(i32)]
+    L.tfps_devices_set.restype = ci
+    L.tfps_devices_set.argtypes = [vp, ci, vp, vp, vp, i64]
+    L.tfps_topo_levels.restype = ci
+    L.tfps_topo_levels.argtypes = [vp, vp, vp, vp, i64, ctypes.POINTER(i32), vp]
+    L.tfps_eval_workspace_bytes.restype = sz
+    L.tfps_eval_workspace_bytes.argtypes = [vp, i64, i64, ci]
+    L.tfps_eval_batch.restype = ci
+    L.tfps_eval_batch.argtypes = [vp, i64, i64, vp, vp, vp, vp, vp, vp, vp, vp, sz, ci, vp]
+    L.tfps_eval_batch_host.restype = ci
+    L.tfps_eval_batch_host.argtypes = [vp, i64, i64, vp, vp, vp, vp, vp, ci, vp]
+    L.tfps_get_status.restype = ci
+    L.tfps_get_status.argtypes = [vp, vp]
+    L.tfps_transpose_u8.restype = ci
+    L.tfps_transpose_u8.argtypes = [vp, vp, i64, i64, i64, vp]
+    _lib = L
+    return L
+
+
+def _check(rc: int) -> None:
+    if rc != OK:
+        raise TfpsError(rc, lib().tfps_last_error().decode() or lib().tfps_strerror(rc).decode())
+
+
+# ---- one-to-one wrappers (raw addresses in, status checked) ---------------------------------
+def tfps_strerror(status: int) -> str:
+    return lib().tfps_strerror(status).decode()
+
+
+def tfps_last_error() -> str:
+    return lib().tfps_last_error().decode()
+
+
+def tfps_graph_create(n, m, in_ptr, in_src, in_t, out_ptr, out_dst, out_t, t_dtype, c, mem, mem_dtype, ptr_space,
+                      stream=0) -> int:
+    h = ctypes.c_void_p()
+    _check(lib().tfps_graph_create(ctypes.byref(h), n, m, in_ptr, in_src, in_t, out_ptr, out_dst, out_t, t_dtype, c,
+                                   mem, mem_dtype, ptr_space, stream))
+    return h.value
+
+
+def tfps_graph_destroy(g) -> None:
+    _check(lib().tfps_graph_destroy(g))
+
+
+def tfps_graph_info(g):
+    n, m, L, k = ctypes.c_int64(), ctypes.c_int64(), ctypes.c_int32(), ctypes.c_int32()
+    _check(lib().tfps_graph_info(g, ctypes.byref(n), ctypes.byref(m), ctypes.byref(L), ctypes.byref(k)))
+    return n.value, m.value, L.value, k.value
+
+
+def tfps_devices_set(g, k, s, C, B, scale) -> None:
+    _check(lib().tfps_devices_set(g, k, s, C, B, scale))
+
+
+def tfps_topo_levels(g, level, order, level_ptr, cap, stream=0) -> int:
+    L = ctypes.c_int32()
+    _check(lib().tfps_topo_levels(g, level, order, level_ptr, cap, ctypes.byref(L), stream))
+    return L.value
+
+
+def tfps_eval_workspace_bytes(g, P, ldp, flags) -> int:
+    return int(lib().tfps_eval_workspace_bytes(g, P, ldp, flags))
+
+
+def tfps_eval_batch(g, P, ldp, part, tlevel, blevel, cp, load, memload, viol, workspace, workspace_bytes, flags,
+                    stream=0) -> None:
+    _check(lib().tfps_eval_batch(g, P, ldp, part, tlevel, blevel, cp, load, memload, viol, workspace, workspace_bytes,
+                                 flags, stream))
+
+
+def tfps_eval_batch_host(g, P, ldp, part, cp, load, memload, viol, flags, stream=0) -> None:
+    _check(lib().tfps_eval_batch_host(g, P, ldp, part, cp, load, memload, viol, flags, stream))
+
+
+def tfps_get_status(g, stream=0) -> None:
+    _check(lib().tfps_get_status(g, stream))
+
+
+def tfps_transpose_u8(src, dst, P, n, ldp, stream=0) -> None:
+    _check(lib().tfps_transpose_u8(src, dst, P, n, ldp, stream))
+
+
+# ---- convenience layer ------------------------------------------------------------------------
+def _np(a, dtype):
+    return np.ascontiguousarray(np.asarray(a), dtype=dtype)
+
+
+def _addr(a) -> Optional[int]:
+    if a is None:
+        return None
+    if isinstance(a, np.ndarray):
+        return a.ctypes.data
+    return a.data_ptr()  # torch tensor
+
+
+def _stream() -> int:
+    import torch
+    return torch.cuda.current_stream().cuda_stream
+
+
+def round_up_ldp(P: int) -> int:
+    return max(16, (P + 15) // 16 * 16)
+
+
+class Graph:
+    """Owns a tfps_graph handle built from host numpy CSR arrays."""
+
+    def __init__(self, n, in_ptr, in_src, in_t, c, out_ptr=None, out_dst=None, out_t=None, mem=None):
+        import torch
+        if not torch.cuda.is_available():
+            raise RuntimeError("tfps needs a CUDA device; there is no CPU fallback")
+        in_t = np.asarray(in_t)
+        t_np = np.int32 if in_t.dtype == np.int32 else np.int64
+        self._keep = [_np(in_ptr, np.int64), _np(in_src, np.int32), _np(in_t, t_np), _np(c, np.int32)]
+        outs = [None, None, None]
+        if out_ptr is not None:
+            outs = [_np(out_ptr, np.int64), _np(out_dst, np.int32), _np(out_t, t_np)]
+        mem_a, mem_dt = None, I64
+        if mem is not None:
+            mem = np.asarray(mem)
+            mem_dt = I32 if mem.dtype == np.int32 else I64
+            mem_a = _np(mem, np.int32 if mem_dt == I32 else np.int64)
+        self.n = int(n)
+        self.m = int(self._keep[1].shape[0])
+        self.handle = tfps_graph_create(self.n, self.m, _addr(self._keep[0]), _addr(self._keep[1]),
+                                        _addr(self._keep[2]), _addr(outs[0]), _addr(outs[1]), _addr(outs[2]),
+                                        I32 if t_np == np.int32 else I64, _addr(self._keep[3]), _addr(mem_a), mem_dt,
+                                        HOST, _stream())
+        self._keep = None
+        self.k = 0
+
+    def close(self):
+        if getattr(self, "handle", None):
+            tfps_graph_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def devices_set(self, k, s, C, B, scale):
+        s = _np(s, np.int32); C = _np(C, np.int64); B = _np(B, np.int64)
+        tfps_devices_set(self.handle, int(k), _addr(s), _addr(C), _addr(B), int(scale))
+        self.k = int(k)
+
+    def topo_levels(self):
+        import torch
+        level = torch.empty(max(self.n, 1), dtype=torch.int32, device="cuda")
+        order = torch.empty(max(self.n, 1), dtype=torch.int32, device="cuda")
+        lp = np.zeros(self.n + 2, np.int64)
+        L = tfps_topo_levels(self.handle, _addr(level), _addr(order), _addr(lp), lp.shape[0], _stream())
+        return level[: self.n], order[: self.n], lp[: L + 1].copy(), L
+
+    def eval_batch(self, part, P=None, want=("tlevel", "blevel", "cp", "load", "memload", "viol"), flags=EVAL_AUTO,
+                   out: Optional[Dict] = None, check=True) -> Dict:
+        """part: torch uint8 CUDA tensor [n][ldp].  Returns a dict of torch CUDA tensors."""
+        import torch
+        assert part.is_cuda and part.dtype == torch.uint8 and part.dim() == 2 and part.is_contiguous()
+        n, ldp = part.shape
+        assert n == self.n
+        P = ldp if P is None else int(P)
+        out = {} if out is None else out
+        dev = part.device
+
+        def buf(name, shape, dtype):
+            if name not in want:
+                return None
+            if name not in out:
+                out[name] = torch.empty(shape, dtype=dtype, device=dev)
+            return out[name]
+
+        tl = buf("tlevel", (n, ldp), torch.int64)
+        bl = buf("blevel", (n, ldp), torch.int64)
+        cp = buf("cp", (max(P, 1),), torch.int64)
+        ld = buf("load", (self.k, ldp), torch.int64)
+        ml = buf("memload", (self.k, ldp), torch.int64)
+        vi = buf("viol", (max(P, 1),), torch.int64)  # bit pattern of uint64
+        ws, ws_bytes = None, 0
+        if cp is not None and tl is None and bl is None:
+            ws_bytes = tfps_eval_workspace_bytes(self.handle, P, ldp, flags | EVAL_SCRATCH_LEVELS)
+            if "workspace" not in out or out["workspace"].numel() < ws_bytes:
+                out["workspace"] = torch.empty(max(ws_bytes, 256), dtype=torch.uint8, device=dev)
+            ws = out["workspace"]
+        tfps_eval_batch(self.handle, P, ldp, _addr(part), _addr(tl), _addr(bl), _addr(cp), _addr(ld), _addr(ml),
+                        _addr(vi), _addr(ws), ws_bytes, flags, _stream())
+        if check:
+            self.status()
+        return out
+
+    def eval_batch_host(self, part: np.ndarray, P=None, want=("cp", "load", "memload", "viol"), flags=EVAL_AUTO) -> Dict:
+        """part: host uint8 [n][ldp] (numpy, or a pinned torch CPU tensor).  Returns numpy arrays."""
+        n, ldp = part.shape
+        P = ldp if P is None else int(P)
+        res = {}
+        cp = np.zeros(max(P, 1), np.int64) if "cp" in want else None
+        ld = np.zeros((self.k, ldp), np.int64) if "load" in want else None
+        ml = np.zeros((self.k, ldp), np.int64) if "memload" in want else None
+        vi = np.zeros(max(P, 1), np.uint64) if "viol" in want else None
+        tfps_eval_batch_host(self.handle, P, ldp, _addr(part), _addr(cp), _addr(ld), _addr(ml), _addr(vi), flags,
+                             _stream())
+        for name, a in (("cp", cp), ("load", ld), ("memload", ml), ("viol", vi)):
+            if a is not None:
+                res[name] = a
+        return res
+
+    def status(self):
+        tfps_get_status(self.handle, _stream())
+
+
+def transpose_u8(src, ldp: Optional[int] = None):
+    """src: torch uint8 CUDA tensor [P][n] -> [n][ldp] (padding columns zero-initialised by torch)."""
+    import torch
+    P, n = src.shape
+    ldp = round_up_ldp(P) if ldp is None else ldp
+    dst = torch.zeros((n, ldp), dtype=torch.uint8, device=src.device)
+    tfps_transpose_u8(_addr(src), _addr(dst), P, n, ldp, _stream())
+    return dst
+
+
+def graph_from_workload(w) -> "Graph":
+    """Build a Graph (and set its device tables) from an ``inputs.Workload``."""
+    from . import inputs
+    c = inputs.to_csr(w.graph)
+    g = Graph(w.graph.n, c.in_ptr, c.in_src, c.in_t, w.graph.c, c.out_ptr, c.out_dst, c.out_t, w.graph.mem)
+    d = w.devices
+    g.devices_set(d.k, d.s, d.C, d.B, d.scale)
+    return g

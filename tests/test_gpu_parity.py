@@ -1,0 +1,331 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU
+oracle on the same seeded inputs.  Everything is integer, so the bar is
+bit-exact equality of every output."""
+from __future__ import annotations
+
+import numpy as np
+import pytest
+
+from paper_1711_01912_b200 import inputs as I
+from helpers import graph_from_edges, load_golden, oracle_graph
+
+pytestmark = pytest.mark.gpu
+
+INF = np.iinfo(np.int64).max
+SENTINEL = -0x0123456789ABCDEF
+
+
+def _torch():
+    import torch
+    return torch
+
+
+def gpu_graph(g, dev=None):
+    from paper_1711_01912_b200 import tfps
+    c = I.to_csr(g)
+    G = tfps.Graph(g.n, c.in_ptr, c.in_src, c.in_t, g.c, c.out_ptr, c.out_dst, c.out_t, g.mem)
+    if dev is not None:
+        G.devices_set(dev.k, dev.s, dev.C, dev.B, dev.scale)
+    return G
+
+
+def padded(part: np.ndarray, ldp=None, fill=0):
+    torch = _torch()
+    n, P = part.shape
+    ldp = max(16, (P + 15) // 16 * 16) if ldp is None else ldp
+    buf = np.full((n, ldp), fill, np.uint8)
+    buf[:, :P] = part
+    return torch.from_numpy(buf).cuda(), P, ldp
+
+
+def run_and_compare(g, dev, part, flags, cols=None, pad_fill=0, check_padding=True):
+    """Evaluate all P candidates on the GPU, compare the listed columns (default
+    all) with the oracle, and check that padding columns keep their sentinel."""
+    import oracle
+    from paper_1711_01912_b200 import tfps
+    torch = _torch()
+    G = gpu_graph(g, dev)
+    dpart, P, ldp = padded(part, fill=pad_fill)
+    n, k = g.n, dev.k
+    out = {
+        "tlevel": torch.full((n, ldp), SENTINEL, dtype=torch.int64, device="cuda"),
+        "blevel": torch.full((n, ldp), SENTINEL, dtype=torch.int64, device="cuda"),
+        "cp": torch.full((max(P, 1),), SENTINEL, dtype=torch.int64, device="cuda"),
+        "load": torch.full((k, ldp), SENTINEL, dtype=torch.int64, device="cuda"),
+        "memload": torch.full((k, ldp), SENTINEL, dtype=torch.int64, device="cuda"),
+        "viol": torch.full((max(P, 1),), SENTINEL, dtype=torch.int64, device="cuda"),
+    }
+    G.eval_batch(dpart, P, flags=flags, out=out)
+    og = oracle_graph(g)
+    cols = list(range(P)) if cols is None else list(cols)
+    ref = oracle.eval_batch(og, k, dev.s, dev.C, dev.B, dev.scale, part, cols)
+    tl = out["tlevel"].cpu().numpy(); bl = out["blevel"].cpu().numpy()
+    assert np.array_equal(tl[:, cols], ref.tlevel)
+    assert np.array_equal(bl[:, cols], ref.blevel)
+    assert np.array_equal(out["cp"].cpu().numpy()[cols], ref.cp)
+    assert np.array_equal(out["load"].cpu().numpy()[:, cols], ref.load)
+    assert np.array_equal(out["memload"].cpu().numpy()[:, cols], ref.memload)
+    assert np.array_equal(out["viol"].cpu().numpy().view(np.uint64)[cols], ref.viol)
+    if check_padding and ldp > P:
+        for name in ("tlevel", "blevel", "load", "memload"):
+            assert (out[name][:, P:] == SENTINEL).all(), f"{name}: padding columns were written"
+    G.close()
+    return out
+
+
+VARIANTS = [1, 2]  # TFPS_EVAL_LEVEL_SYNC, TFPS_EVAL_SLICED
+
+
+# -------------------------------------------------------------------- worked DAGs
+@pytest.mark.parametrize("flags", VARIANTS)
+@pytest.mark.parametrize("fname", ["w1_diamond.json", "w2_two_sinks.json"])
+def test_worked_examples_on_gpu(fname, flags):
+    from paper_1711_01912_b200 import tfps
+    w = load_golden(fname)
+    g = graph_from_edges(w["n"], w["edges"], w["c"])
+    for case in w["cases"]:
+        k = w["k"]
+        dev = I.Devices(k, np.array(w["s"], np.int32), np.array(case.get("C", [INF] * k), np.int64),
+                        np.array(case["B"], np.int64), scale=w["S"])
+        G = gpu_graph(g, dev)
+        part, P, ldp = padded(np.array(case["p"], np.uint8)[:, None])
+        out = G.eval_batch(part, P, flags=flags)
+        assert out["tlevel"][:, 0].tolist() == case["tlevel"]
+        assert out["blevel"][:, 0].tolist() == case["blevel"]
+        assert out["cp"][0].item() == case["cp"]
+        assert out["load"][:, 0].tolist() == case["load"]
+        if "memload" in case:
+            assert out["memload"][:, 0].tolist() == case["memload"]
+            assert out["viol"][0].item() == case["viol"]
+        level, order, lp, L = G.topo_levels()
+        assert level.tolist() == w["level"]
+        G.close()
+
+
+# ------------------------------------------------------------------ configs 1 and 2
+@pytest.mark.parametrize("flags", VARIANTS + [0])
+def test_config1_every_candidate(flags):
+    w = I.config1()
+    run_and_compare(w.graph, w.devices, w.part_full(), flags)
+
+
+@pytest.mark.parametrize("flags", VARIANTS)
+def test_config2_every_candidate(flags):
+    w = I.config2()
+    run_and_compare(w.graph, w.devices, w.part_full(), flags)
+
+
+def test_config1_relabelled():
+    w = I.config1()
+    g2, perm = I.relabel(w.graph, 5)
+    part = w.part_full()
+    part2 = np.empty_like(part)
+    part2[perm] = part
+    run_and_compare(g2, w.devices, part2, 2)
+    run_and_compare(g2, w.devices, part2, 1)
+
+
+# ----------------------------------------------------------------- topological levels
+@pytest.mark.parametrize("maker", [I.config1, I.config2, I.config3, I.config4])
+def test_topo_levels_match_oracle(maker):
+    w = maker()
+    g, _ = I.relabel(w.graph, 9)
+    og = oracle_graph(g)
+    G = gpu_graph(g)
+    level, order, lp, L = G.topo_levels()
+    assert L == og.num_levels
+    assert np.array_equal(lp, og.level_ptr)
+    assert np.array_equal(level.cpu().numpy(), og.level)
+    assert np.array_equal(order.cpu().numpy(), og.order)
+    G.close()
+
+
+# ------------------------------------------------------------------- awkward shapes
+@pytest.mark.parametrize("flags", VARIANTS)
+@pytest.mark.parametrize("n,m,k,P,tdt", [
+    (1, 0, 1, 1, np.int64), (2, 1, 2, 3, np.int32), (37, 90, 3, 17, np.int64), (300, 900, 5, 33, np.int32),
+    (513, 2000, 8, 70, np.int64), (1000, 2500, 64, 48, np.int64), (257, 700, 16, 129, np.int32),
+    (64, 0, 4, 40, np.int64), (700, 3000, 2, 1000, np.int64),
+])
+def test_random_small_graphs(n, m, k, P, tdt, flags):
+    w = I.small_random(1000 + n + P, n, m, k, P, t_dtype=tdt, with_mem=(n % 2 == 1))
+    part = w.part_full()
+    # garbage in the padding columns must be ignored (and must not be validated)
+    run_and_compare(w.graph, w.devices, part, flags, pad_fill=255)
+
+
+@pytest.mark.parametrize("which", [0, 1])
+def test_paper_shaped_graphs_k50(which):
+    w = I.paper_shaped(which)
+    run_and_compare(w.graph, w.devices, w.part_full(), 2)
+    run_and_compare(w.graph, w.devices, w.part_full(), 1)
+
+
+def test_parallel_edges_zero_costs_isolated_vertices():
+    edges = [(0, 1, 10), (0, 1, 5000), (1, 2, 0), (0, 2, 7)]
+    g = graph_from_edges(5, edges, [3, 0, 4, 9, 0])
+    dev = I.Devices(3, np.array([1, 2, 5], np.int32), np.array([10, 5000, INF], np.int64),
+                    np.array([[0, 3, 1], [7, 0, 2], [1, 1, 0]], np.int64), scale=5)
+    rng = np.random.default_rng(3)
+    part = rng.integers(0, 3, size=(5, 27), dtype=np.uint8)
+    for flags in VARIANTS:
+        run_and_compare(g, dev, part, flags)
+
+
+def test_extreme_magnitudes_exact_division():
+    # large t, large and tiny bandwidths, large scale: exercises the division constants at the domain's edge
+    rng = np.random.default_rng(17)
+    n = 64
+    w = I.small_random(5, n, 200, 6, 40)
+    g = w.graph
+    t = rng.integers(0, 2 ** 40, size=g.m).astype(np.int64)
+    t[:8] = [0, 1, 2, 2 ** 40, 2 ** 40 - 1, 3, 2 ** 39, 2 ** 20 + 1]
+    g = I.Graph(n=n, src=g.src, dst=g.dst, t=t, c=rng.integers(0, 2 ** 31 - 1, size=n).astype(np.int32), mem=None, layers=0)
+    B = rng.integers(1, 2 ** 40, size=(6, 6)).astype(np.int64)
+    B[0, 1] = 1; B[1, 0] = 2; B[2, 3] = 3; B[3, 2] = 2 ** 40; B[4, 5] = 2 ** 31 - 1; B[5, 4] = 2 ** 31 + 1
+    dev = I.Devices(6, np.array([1, 2, 3, 7, 2 ** 31 - 1, 65536], np.int32), np.full(6, INF, np.int64), B, scale=2 ** 12 - 1)
+    for flags in VARIANTS:
+        run_and_compare(g, dev, w.part_full(), flags)
+
+
+# -------------------------------------------------------------------- option handling
+def test_cp_only_uses_workspace_and_matches():
+    import oracle
+    from paper_1711_01912_b200 import tfps
+    w = I.config2()
+    part = w.part_full()[:, :100]
+    G = gpu_graph(w.graph, w.devices)
+    dpart, P, ldp = padded(part)
+    og = oracle_graph(w.graph)
+    d = w.devices
+    ref = oracle.eval_batch(og, d.k, d.s, d.C, d.B, d.scale, part, want_levels=False)
+    for flags in VARIANTS:
+        out = G.eval_batch(dpart, P, want=("cp",), flags=flags)
+        assert np.array_equal(out["cp"].cpu().numpy(), ref.cp)
+        out = G.eval_batch(dpart, P, want=("cp", "blevel"), flags=flags)  # CP from the backward pass alone
+        assert np.array_equal(out["cp"].cpu().numpy(), ref.cp)
+        out = G.eval_batch(dpart, P, want=("viol",), flags=flags)
+        assert np.array_equal(out["viol"].cpu().numpy().view(np.uint64), ref.viol)
+    G.close()
+
+
+def test_host_entry_point_matches():
+    import oracle
+    w = I.config2()
+    part = w.part_full()[:, :200]
+    G = gpu_graph(w.graph, w.devices)
+    n, P = part.shape
+    ldp = 208
+    buf = np.zeros((n, ldp), np.uint8); buf[:, :P] = part
+    res = G.eval_batch_host(buf, P)
+    og = oracle_graph(w.graph)
+    d = w.devices
+    ref = oracle.eval_batch(og, d.k, d.s, d.C, d.B, d.scale, part, want_levels=False)
+    assert np.array_equal(res["cp"], ref.cp)
+    assert np.array_equal(res["load"][:, :P], ref.load)
+    assert np.array_equal(res["memload"][:, :P], ref.memload)
+    assert np.array_equal(res["viol"], ref.viol)
+    G.close()
+
+
+def test_transpose_u8():
+    from paper_1711_01912_b200 import tfps
+    torch = _torch()
+    rng = np.random.default_rng(0)
+    for P, n in [(1, 1), (70, 130), (64, 64), (333, 1000)]:
+        src = rng.integers(0, 255, size=(P, n), dtype=np.uint8)
+        dst = tfps.transpose_u8(torch.from_numpy(src).cuda())
+        assert np.array_equal(dst.cpu().numpy()[:, :P], src.T)
+        assert (dst[:, P:] == 0).all()
+
+
+def test_deterministic_repeat():
+    torch = _torch()
+    w = I.config2()
+    G = gpu_graph(w.graph, w.devices)
+    dpart, P, ldp = padded(w.part_full())
+    a = G.eval_batch(dpart, P, flags=2)
+    b = G.eval_batch(dpart, P, flags=2, out={})
+    for kname in ("tlevel", "blevel", "cp", "load", "memload", "viol"):
+        assert torch.equal(a[kname], b[kname])
+    G.close()
+
+
+# ------------------------------------------------------------------------- errors
+def test_error_codes():
+    from paper_1711_01912_b200 import tfps
+    torch = _torch()
+    # cycle
+    g = graph_from_edges(3, [(0, 1, 1), (1, 2, 1), (2, 0, 1)], [1, 1, 1])
+    G = gpu_graph(g)
+    with pytest.raises(tfps.TfpsError) as ei:
+        G.topo_levels()
+    assert ei.value.code == tfps.ERR_CYCLE
+    with pytest.raises(tfps.TfpsError) as ei:
+        G.devices_set(1, [1], [INF], [[0]], 1)
+    assert ei.value.code == tfps.ERR_CYCLE
+    G.close()
+    # self loop
+    c = I.to_csr(graph_from_edges(2, [(0, 1, 1)], [1, 1]))
+    bad_src = c.in_src.copy(); bad_src[0] = 1
+    with pytest.raises(tfps.TfpsError) as ei:
+        tfps.Graph(2, c.in_ptr, bad_src, c.in_t, [1, 1])
+    assert ei.value.code == tfps.ERR_CYCLE
+    # malformed CSR
+    w = I.config1()
+    c = I.to_csr(w.graph)
+    p2 = c.in_ptr.copy(); p2[5] = p2[4] - 1
+    with pytest.raises(tfps.TfpsError) as ei:
+        tfps.Graph(w.graph.n, p2, c.in_src, c.in_t, w.graph.c)
+    assert ei.value.code == tfps.ERR_BAD_CSR
+    s2 = c.in_src.copy(); s2[3] = w.graph.n
+    with pytest.raises(tfps.TfpsError) as ei:
+        tfps.Graph(w.graph.n, c.in_ptr, s2, c.in_t, w.graph.c)
+    assert ei.value.code == tfps.ERR_BAD_CSR
+    t2 = c.out_t.copy(); t2[7] += 1  # in/out multisets differ
+    with pytest.raises(tfps.TfpsError) as ei:
+        tfps.Graph(w.graph.n, c.in_ptr, c.in_src, c.in_t, w.graph.c, c.out_ptr, c.out_dst, t2)
+    assert ei.value.code == tfps.ERR_BAD_CSR
+    # devices
+    G = gpu_graph(w.graph)
+    d = w.devices
+    with pytest.raises(tfps.TfpsError) as ei:
+        G.eval_batch(torch.zeros((w.graph.n, 16), dtype=torch.uint8, device="cuda"), 4)
+    assert ei.value.code == tfps.ERR_STATE
+    with pytest.raises(tfps.TfpsError) as ei:
+        G.devices_set(65, np.ones(65), np.ones(65), np.ones((65, 65)), 1)
+    assert ei.value.code == tfps.ERR_BAD_DEVICES
+    with pytest.raises(tfps.TfpsError) as ei:
+        G.devices_set(2, [1, 0], d.C, d.B, 16)
+    assert ei.value.code == tfps.ERR_BAD_DEVICES
+    with pytest.raises(tfps.TfpsError) as ei:
+        G.devices_set(2, d.s, d.C, [[0, 0], [5, 0]], 16)
+    assert ei.value.code == tfps.ERR_BAD_DEVICES
+    with pytest.raises(tfps.TfpsError) as ei:
+        G.devices_set(2, d.s, d.C, d.B, 2 ** 45)
+    assert ei.value.code == tfps.ERR_OVERFLOW
+    G.devices_set(d.k, d.s, d.C, d.B, d.scale)
+    # bad ldp, missing workspace
+    part = torch.zeros((w.graph.n, 16), dtype=torch.uint8, device="cuda")
+    with pytest.raises(tfps.TfpsError) as ei:
+        tfps.tfps_eval_batch(G.handle, 20, 16, part.data_ptr(), None, None, None, None, None, None, None, 0, 0, 0)
+    assert ei.value.code == tfps.ERR_INVALID_ARG
+    cp = torch.zeros(16, dtype=torch.int64, device="cuda")
+    with pytest.raises(tfps.TfpsError) as ei:
+        tfps.tfps_eval_batch(G.handle, 16, 16, part.data_ptr(), None, None, cp.data_ptr(), None, None, None, None, 0, 0, 0)
+    assert ei.value.code == tfps.ERR_WORKSPACE
+    # P == 0: nothing happens
+    tfps.tfps_eval_batch(G.handle, 0, 16, part.data_ptr(), None, None, None, None, None, None, None, 0, 0, 0)
+    # id >= k is reported through the status word and the context stays usable
+    part[5, 3] = 2
+    for flags in VARIANTS:
+        with pytest.raises(tfps.TfpsError) as ei:
+            G.eval_batch(part, 16, flags=flags)
+        assert ei.value.code == tfps.ERR_BAD_PARTITION
+        with pytest.raises(tfps.TfpsError) as ei:
+            G.eval_batch(part, 16, want=("cp",), flags=flags)
+        assert ei.value.code == tfps.ERR_BAD_PARTITION
+    part[5, 3] = 1
+    out = G.eval_batch(part, 16)
+    assert (out["cp"] > 0).all()
+    G.close()
