@@ -71,7 +71,8 @@ enum {
     TFPS_EVAL_LEVEL_SYNC = 1 << 0,   /* one launch per topological level, thread = (vertex, candidates) */
     TFPS_EVAL_SLICED = 1 << 1,       /* one persistent block per candidate slice walks all levels */
     TFPS_EVAL_NO_VALIDATE = 1 << 4,  /* caller guarantees every id < k; skips the id check */
-    TFPS_EVAL_SCRATCH_LEVELS = 1 << 5 /* workspace query: caller will pass tlevel == NULL and blevel == NULL */
+    TFPS_EVAL_SCRATCH_LEVELS = 1 << 5, /* workspace query: caller will pass tlevel == NULL and blevel == NULL */
+    TFPS_EVAL_PROFILE = 1 << 6        /* record CUDA events around the phases, read back with tfps_phase_times */
 };
 
 const char* tfps_strerror(int status);
@@ -162,16 +163,31 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp,
                     void* workspace, size_t workspace_bytes, int flags, void* stream);
 
 /*
- * Same evaluation from HOST buffers: part is host uint8 [n][ldp]; cp[P],
- * load[k*ldp], memload[k*ldp], viol[P] are host outputs (any may be NULL).
- * Copies the ids to the device, runs the forward pass (and the load kernel),
- * copies the results back and synchronises `stream`.  Staging and scratch
- * buffers are owned by the handle and grow on demand.  Returns the device
- * status as tfps_get_status would.
+ * Same evaluation from HOST buffers: part is host uint8 [n][ldp]; tlevel and
+ * blevel (host int64 [n][ldp]), cp[P], load[k*ldp], memload[k*ldp], viol[P] are
+ * host outputs, any of which may be NULL.  Copies the ids to the device, runs
+ * the load kernel and BOTH passes (the level matrices live in scratch owned by
+ * the handle and are copied back only when a host pointer is given), copies
+ * the other results back and synchronises `stream`.  Staging and scratch
+ * buffers grow on demand and stay with the handle.  Pinned host memory makes
+ * the copies asynchronous and fast; pageable memory works too.  Returns the
+ * device status as tfps_get_status would.
  */
 int tfps_eval_batch_host(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part,
+                         int64_t* tlevel, int64_t* blevel,
                          int64_t* cp, int64_t* load, int64_t* memload, uint64_t* viol,
                          int flags, void* stream);
+
+/*
+ * Device time in milliseconds of the phases of the most recent tfps_eval_batch
+ * call that carried TFPS_EVAL_PROFILE: ms[0] = load/validate/violation
+ * kernels, ms[1] = forward pass, ms[2] = backward pass (0 for a phase that did
+ * not run).  Synchronises on the recorded events.
+ */
+int tfps_phase_times(tfps_graph* g, float ms[3]);
+
+/* Number of kernels this library has launched in the calling process so far. */
+int64_t tfps_kernel_launches(void);
 
 /* Synchronise `stream`, return the sticky device-side status of the handle and clear it. */
 int tfps_get_status(tfps_graph* g, void* stream);

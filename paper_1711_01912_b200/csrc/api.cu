@@ -1,6 +1,7 @@
 // Host runtime and C ABI of libtfps: graph handle, CSR validation, device
 // tables (exact-division constants), topological structure, launch logic.
 #include <algorithm>
+#include <atomic>
 #include <cstdarg>
 #include <cstdio>
 #include <cstdlib>
@@ -11,6 +12,11 @@
 #include "common.cuh"
 
 using namespace tfps;
+
+namespace tfps {
+static std::atomic<long long> g_launches{0};
+void count_launches(long long n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+}  // namespace tfps
 
 namespace {
 
@@ -109,7 +115,16 @@ struct tfps_graph {
     DBuf status;
     // scratch owned by the handle
     DBuf scr_memload;
-    DBuf st_part, st_lev, st_cp, st_load, st_mem, st_viol;
+    DBuf st_part, st_lev, st_lev2, st_cp, st_load, st_mem, st_viol;
+    // phase timing (TFPS_EVAL_PROFILE)
+    cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
+    bool ev_valid = false;
+    bool ran_fwd = false, ran_bwd = false;
+    ~tfps_graph()
+    {
+        for (cudaEvent_t e : ev)
+            if (e) cudaEventDestroy(e);
+    }
 };
 
 namespace {
@@ -555,6 +570,14 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
     tab.cap = g->cap.as<long long>();
     int* status = g->status.as<int>();
 
+    const bool profile = (flags & TFPS_EVAL_PROFILE) != 0;
+    if (profile) {
+        for (cudaEvent_t& e : g->ev)
+            if (!e) CUDA_TRY(cudaEventCreate(&e));
+        g->ev_valid = false;
+        CUDA_TRY(cudaEventRecord(g->ev[0], st));
+    }
+
     // loads first: the same kernel checks the ids, and a bad id stops everything after it
     long long* ml = (long long*)memload;
     if (viol && !ml) {
@@ -589,8 +612,10 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
         while (warps < 8 && warps * 2 <= avg_width) warps <<= 1;
     }
 
+    if (profile) CUDA_TRY(cudaEventRecord(g->ev[1], st));
     for (int pass = 0; pass < 2; ++pass) {
         const bool fwd = pass == 0;
+        if (profile && !fwd) CUDA_TRY(cudaEventRecord(g->ev[2], st));
         if (fwd ? !need_fwd : !need_bwd) continue;
         long long* lev = fwd ? fwd_lev : (long long*)blevel;
         long long* cp_here = (cp && (fwd || !need_fwd)) ? (long long*)cp : nullptr;
@@ -606,8 +631,29 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
             }
         }
     }
+    if (profile) {
+        CUDA_TRY(cudaEventRecord(g->ev[3], st));
+        g->ev_valid = true;
+        g->ran_fwd = need_fwd;
+        g->ran_bwd = need_bwd;
+    }
     return TFPS_OK;
 }
+
+int tfps_phase_times(tfps_graph* g, float ms[3])
+{
+    if (!g || !ms) return fail(TFPS_ERR_INVALID_ARG, "graph or ms is NULL");
+    if (!g->ev_valid) return fail(TFPS_ERR_STATE, "no profiled tfps_eval_batch call to report");
+    DeviceGuard guard(g->device);
+    if (!guard.ok) return fail(TFPS_ERR_CUDA, "cannot select the handle's device");
+    CUDA_TRY(cudaEventSynchronize(g->ev[3]));
+    for (int i = 0; i < 3; ++i) CUDA_TRY(cudaEventElapsedTime(&ms[i], g->ev[i], g->ev[i + 1]));
+    if (!g->ran_fwd) ms[1] = 0.f;
+    if (!g->ran_bwd) ms[2] = 0.f;
+    return TFPS_OK;
+}
+
+int64_t tfps_kernel_launches(void) { return (int64_t)tfps::g_launches.load(std::memory_order_relaxed); }
 
 int tfps_get_status(tfps_graph* g, void* stream)
 {
@@ -626,8 +672,9 @@ int tfps_get_status(tfps_graph* g, void* stream)
     return TFPS_OK;
 }
 
-int tfps_eval_batch_host(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, int64_t* cp, int64_t* load,
-                         int64_t* memload, uint64_t* viol, int flags, void* stream)
+int tfps_eval_batch_host(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, int64_t* tlevel,
+                         int64_t* blevel, int64_t* cp, int64_t* load, int64_t* memload, uint64_t* viol, int flags,
+                         void* stream)
 {
     if (!g) return fail(TFPS_ERR_INVALID_ARG, "graph is NULL");
     if (P < 0 || ldp < P || (ldp % 16) != 0) return fail(TFPS_ERR_INVALID_ARG, "need 0 <= P <= ldp and ldp %% 16 == 0");
@@ -640,16 +687,19 @@ int tfps_eval_batch_host(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* p
     const size_t cells = (size_t)g->n * (size_t)ldp;
     const size_t kcells = (size_t)g->k * (size_t)ldp;
     CUDA_TRY(g->st_part.reserve(cells));
-    if (cp) { CUDA_TRY(g->st_lev.reserve(cells * 8)); CUDA_TRY(g->st_cp.reserve((size_t)P * 8)); }
+    CUDA_TRY(g->st_lev.reserve(cells * 8));
+    CUDA_TRY(g->st_lev2.reserve(cells * 8));
+    CUDA_TRY(g->st_cp.reserve((size_t)P * 8));
     if (load) CUDA_TRY(g->st_load.reserve(kcells * 8));
     if (memload || viol) CUDA_TRY(g->st_mem.reserve(kcells * 8));
     if (viol) CUDA_TRY(g->st_viol.reserve((size_t)P * 8));
     CUDA_TRY(cudaMemcpyAsync(g->st_part.p, part, cells, cudaMemcpyHostToDevice, st));
-    TFPS_TRY(tfps_eval_batch(g, P, ldp, g->st_part.as<uint8_t>(), nullptr, nullptr,
-                             cp ? g->st_cp.as<int64_t>() : nullptr, load ? g->st_load.as<int64_t>() : nullptr,
+    TFPS_TRY(tfps_eval_batch(g, P, ldp, g->st_part.as<uint8_t>(), g->st_lev.as<int64_t>(), g->st_lev2.as<int64_t>(),
+                             g->st_cp.as<int64_t>(), load ? g->st_load.as<int64_t>() : nullptr,
                              (memload || viol) ? g->st_mem.as<int64_t>() : nullptr,
-                             viol ? g->st_viol.as<uint64_t>() : nullptr, g->st_lev.p, g->st_lev.bytes,
-                             flags | TFPS_EVAL_SCRATCH_LEVELS, st));
+                             viol ? g->st_viol.as<uint64_t>() : nullptr, nullptr, 0, flags, st));
+    if (tlevel) CUDA_TRY(cudaMemcpyAsync(tlevel, g->st_lev.p, cells * 8, cudaMemcpyDeviceToHost, st));
+    if (blevel) CUDA_TRY(cudaMemcpyAsync(blevel, g->st_lev2.p, cells * 8, cudaMemcpyDeviceToHost, st));
     if (cp) CUDA_TRY(cudaMemcpyAsync(cp, g->st_cp.p, (size_t)P * 8, cudaMemcpyDeviceToHost, st));
     if (load) CUDA_TRY(cudaMemcpyAsync(load, g->st_load.p, kcells * 8, cudaMemcpyDeviceToHost, st));
     if (memload) CUDA_TRY(cudaMemcpyAsync(memload, g->st_mem.p, kcells * 8, cudaMemcpyDeviceToHost, st));

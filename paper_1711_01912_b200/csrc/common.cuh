@@ -63,6 +63,9 @@ struct PassArgs {
     int* status;          // sticky status word
 };
 
+// every kernel launch of the library goes through the wrappers below and is counted here
+void count_launches(long long n);
+
 // ---- launch wrappers (host side, implemented in the .cu files) -------------
 cudaError_t launch_kahn(int n, const long long* in_ptr, const long long* out_ptr, const int* out_dst,
                         int* indeg, int* level, int* queue, long long* level_ptr_dev, int* level_cnt,

@@ -416,11 +416,11 @@ static cudaError_t level_sync_impl(const PassArgs& a, const std::vector<long lon
         const int l = FWD ? step : L - 1 - step;
         const int pos0 = (int)lp[l];
         const int count = (int)(lp[l + 1] - lp[l]);
-        if (FWD && l == 0 && false) continue;
         unsigned gy = cdivu(count, 4);
         if (gy > 65535u) gy = 65535u;
         pass_level_kernel<CPT, FWD><<<dim3(gx, gy), 128, smem, st>>>(a, pos0, count);
     }
+    count_launches(L);
     return cudaGetLastError();
 }
 
@@ -439,6 +439,7 @@ static cudaError_t sliced_impl(const PassArgs& a, const uint8_t* cp_flag, int wa
     if (e != cudaSuccess) return e;
     const unsigned gx = cdivu(a.P, 32 * CPT);
     pass_sliced_kernel<CPT, FWD><<<gx, warps * 32, smem, st>>>(a, cp_flag);
+    count_launches(1);
     return cudaGetLastError();
 }
 
@@ -457,6 +458,7 @@ cudaError_t launch_cp_reduce(const PassArgs& a, bool from_tlevel, const int* lis
     int per_block = 256;
     unsigned gy = cdivu(list_len, per_block);
     if (gy > 65535u) { per_block = (int)cdivu(list_len, 65535); gy = cdivu(list_len, per_block); }
+    count_launches(1);
     if (from_tlevel)
         cp_reduce_kernel<true><<<dim3(gx, gy), 128, smem, st>>>(a, list, list_len, per_block);
     else
@@ -483,6 +485,7 @@ cudaError_t launch_loads(int n, long long P, long long ldp, const uint8_t* part,
     if (gy > 65535) gy = 65535;
     int rows = (int)((n + gy - 1) / gy);
     gy = (n + rows - 1) / rows;
+    count_launches(1);
     loads_kernel<<<dim3(gx, (unsigned)gy), threads, smem, st>>>(n, P, ldp, part, vert, xvert, mem, tab, load, memload,
                                                                 status, validate ? 1 : 0, rows);
     return cudaGetLastError();
@@ -492,6 +495,7 @@ cudaError_t launch_validate(long long n, long long P, long long ldp, const uint8
                             int sm_count, cudaStream_t st)
 {
     validate_kernel<<<sm_count * 8, 256, 0, st>>>(n, P, ldp, part, k, status);
+    count_launches(1);
     return cudaGetLastError();
 }
 
@@ -499,6 +503,7 @@ cudaError_t launch_viol(long long P, long long ldp, int k, const long long* meml
                         unsigned long long* viol, const int* status, cudaStream_t st)
 {
     viol_kernel<<<cdivu(P, 256), 256, 0, st>>>(P, ldp, k, memload, cap, viol, status);
+    count_launches(1);
     return cudaGetLastError();
 }
 
@@ -506,6 +511,7 @@ cudaError_t launch_transpose_u8(const uint8_t* src, uint8_t* dst, long long P, l
 {
     dim3 grid(cdivu(n, 64), cdivu(P, 64));
     transpose_u8_kernel<<<grid, 256, 0, st>>>(src, dst, P, n, ldp);
+    count_launches(1);
     return cudaGetLastError();
 }
 

@@ -255,21 +255,27 @@ cudaError_t launch_kahn(int n, const long long* in_ptr, const long long* out_ptr
     if (blocks > sm_count) blocks = sm_count;
     if (blocks < 1) blocks = 1;
     void* args[] = {&n, &in_ptr, &out_ptr, &out_dst, &indeg, &level, &queue, &level_ptr_dev, &level_cnt, &result};
+    count_launches(1);
     return cudaLaunchCooperativeKernel((void*)kahn_kernel, dim3(blocks), dim3(256), args, 0, st);
 }
 
 cudaError_t launch_sort_order(int n, const int* level, unsigned long long* keys, int npad, int* order, cudaStream_t st)
 {
+    long long launches = 3;
     make_keys<<<cdiv(npad, 256), 256, 0, st>>>(n, npad, level, keys);
     int tiles = npad / SORT_TILE;  // npad is a power of two >= SORT_TILE
     int k_local_max = SORT_TILE;
     bitonic_local<<<tiles, SORT_TILE / 2, 0, st>>>(keys, 2, k_local_max, 0);
     for (int k = SORT_TILE * 2; k <= npad; k <<= 1) {
-        for (int j = k >> 1; j >= SORT_TILE; j >>= 1)
+        for (int j = k >> 1; j >= SORT_TILE; j >>= 1) {
             bitonic_global<<<cdiv(npad / 2, 256), 256, 0, st>>>(keys, npad, k, j);
+            ++launches;
+        }
         bitonic_local<<<tiles, SORT_TILE / 2, 0, st>>>(keys, k, k, SORT_TILE / 2);
+        ++launches;
     }
     keys_to_order<<<cdiv(n, 256), 256, 0, st>>>(n, keys, order);
+    count_launches(launches);
     return cudaGetLastError();
 }
 
@@ -278,12 +284,13 @@ cudaError_t launch_build_adj(int n, const int* order, const long long* ptr, cons
 {
     degree_scan<<<1, 1024, 0, st>>>(n, order, ptr, eptr);
     fill_adj<<<cdiv((long long)n * 32, 256), 256, 0, st>>>(n, order, ptr, idx, t, eptr, nbr, tperm);
+    count_launches(2);
     return cudaGetLastError();
 }
 
 cudaError_t launch_sink_flags(int n, const int* order, const long long* out_ptr, uint8_t* flag, cudaStream_t st)
 {
-    if (n > 0) sink_flags_kernel<<<cdiv(n, 256), 256, 0, st>>>(n, order, out_ptr, flag);
+    if (n > 0) { sink_flags_kernel<<<cdiv(n, 256), 256, 0, st>>>(n, order, out_ptr, flag); count_launches(1); }
     return cudaGetLastError();
 }
 
@@ -292,8 +299,9 @@ cudaError_t launch_numerators(int n, int m, long long S, const int* order, const
                               unsigned long long* xvert, unsigned long long* xw_f, unsigned long long* xnbr_f,
                               unsigned long long* xw_b, cudaStream_t st)
 {
-    if (n > 0) numerators_vertex<<<cdiv(n, 256), 256, 0, st>>>(n, S, order, c, xvert);
+    if (n > 0) { numerators_vertex<<<cdiv(n, 256), 256, 0, st>>>(n, S, order, c, xvert); count_launches(1); }
     if (m > 0) {
+        count_launches(2);
         numerators_edge<<<cdiv(m, 256), 256, 0, st>>>(m, S, t_f, nbr_f, c, xw_f, xnbr_f);
         numerators_edge<<<cdiv(m, 256), 256, 0, st>>>(m, S, t_b, nbr_b, c, xw_b, nullptr);
     }
@@ -302,7 +310,7 @@ cudaError_t launch_numerators(int n, int m, long long S, const int* order, const
 
 cudaError_t launch_default_mem(int n, const long long* out_ptr, const long long* out_t, long long* mem, cudaStream_t st)
 {
-    if (n > 0) default_mem_kernel<<<cdiv(n, 256), 256, 0, st>>>(n, out_ptr, out_t, mem);
+    if (n > 0) { default_mem_kernel<<<cdiv(n, 256), 256, 0, st>>>(n, out_ptr, out_t, mem); count_launches(1); }
     return cudaGetLastError();
 }
 

@@ -25,12 +25,12 @@ ERR_OVERFLOW, ERR_WORKSPACE, ERR_UNSUPPORTED, ERR_CUDA, ERR_TIMEOUT, ERR_STATE =
 K_MAX = 64
 I32, I64 = 0, 1
 HOST, DEVICE = 0, 1
-EVAL_AUTO, EVAL_LEVEL_SYNC, EVAL_SLICED, EVAL_NO_VALIDATE, EVAL_SCRATCH_LEVELS = 0, 1, 2, 16, 32
+EVAL_AUTO, EVAL_LEVEL_SYNC, EVAL_SLICED, EVAL_NO_VALIDATE, EVAL_SCRATCH_LEVELS, EVAL_PROFILE = 0, 1, 2, 16, 32, 64
 
 EXPORTS = [
     "tfps_strerror", "tfps_last_error", "tfps_graph_create", "tfps_graph_destroy", "tfps_graph_info",
     "tfps_devices_set", "tfps_topo_levels", "tfps_eval_workspace_bytes", "tfps_eval_batch",
-    "tfps_eval_batch_host", "tfps_get_status", "tfps_transpose_u8",
+    "tfps_eval_batch_host", "tfps_get_status", "tfps_transpose_u8", "tfps_phase_times", "tfps_kernel_launches",
 ]
 
 
@@ -72,7 +72,11 @@ def lib() -> ctypes.CDLL:
     L.tfps_eval_batch.restype = ci
     L.tfps_eval_batch.argtypes = [vp, i64, i64, vp, vp, vp, vp, vp, vp, vp, vp, sz, ci, vp]
     L.tfps_eval_batch_host.restype = ci
-    L.tfps_eval_batch_host.argtypes = [vp, i64, i64, vp, vp, vp, vp, vp, ci, vp]
+    L.tfps_eval_batch_host.argtypes = [vp, i64, i64, vp, vp, vp, vp, vp, vp, vp, ci, vp]
+    L.tfps_phase_times.restype = ci
+    L.tfps_phase_times.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
+    L.tfps_kernel_launches.restype = i64
+    L.tfps_kernel_launches.argtypes = []
     L.tfps_get_status.restype = ci
     L.tfps_get_status.argtypes = [vp, vp]
     L.tfps_transpose_u8.restype = ci
@@ -133,8 +137,18 @@ def tfps_eval_batch(g, P, ldp, part, tlevel, blevel, cp, load, memload, viol, wo
                                  flags, stream))
 
 
-def tfps_eval_batch_host(g, P, ldp, part, cp, load, memload, viol, flags, stream=0) -> None:
-    _check(lib().tfps_eval_batch_host(g, P, ldp, part, cp, load, memload, viol, flags, stream))
+def tfps_eval_batch_host(g, P, ldp, part, tlevel, blevel, cp, load, memload, viol, flags, stream=0) -> None:
+    _check(lib().tfps_eval_batch_host(g, P, ldp, part, tlevel, blevel, cp, load, memload, viol, flags, stream))
+
+
+def tfps_phase_times(g):
+    ms = (ctypes.c_float * 3)()
+    _check(lib().tfps_phase_times(g, ms))
+    return [float(x) for x in ms]
+
+
+def tfps_kernel_launches() -> int:
+    return int(lib().tfps_kernel_launches())
 
 
 def tfps_get_status(g, stream=0) -> None:
@@ -259,13 +273,15 @@ class Graph:
         n, ldp = part.shape
         P = ldp if P is None else int(P)
         res = {}
+        tl = np.zeros((n, ldp), np.int64) if "tlevel" in want else None
+        bl = np.zeros((n, ldp), np.int64) if "blevel" in want else None
         cp = np.zeros(max(P, 1), np.int64) if "cp" in want else None
         ld = np.zeros((self.k, ldp), np.int64) if "load" in want else None
         ml = np.zeros((self.k, ldp), np.int64) if "memload" in want else None
         vi = np.zeros(max(P, 1), np.uint64) if "viol" in want else None
-        tfps_eval_batch_host(self.handle, P, ldp, _addr(part), _addr(cp), _addr(ld), _addr(ml), _addr(vi), flags,
-                             _stream())
-        for name, a in (("cp", cp), ("load", ld), ("memload", ml), ("viol", vi)):
+        tfps_eval_batch_host(self.handle, P, ldp, _addr(part), _addr(tl), _addr(bl), _addr(cp), _addr(ld), _addr(ml),
+                             _addr(vi), flags, _stream())
+        for name, a in (("tlevel", tl), ("blevel", bl), ("cp", cp), ("load", ld), ("memload", ml), ("viol", vi)):
             if a is not None:
                 res[name] = a
         return res

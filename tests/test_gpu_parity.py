@@ -217,10 +217,12 @@ def test_host_entry_point_matches():
     n, P = part.shape
     ldp = 208
     buf = np.zeros((n, ldp), np.uint8); buf[:, :P] = part
-    res = G.eval_batch_host(buf, P)
+    res = G.eval_batch_host(buf, P, want=("tlevel", "blevel", "cp", "load", "memload", "viol"))
     og = oracle_graph(w.graph)
     d = w.devices
-    ref = oracle.eval_batch(og, d.k, d.s, d.C, d.B, d.scale, part, want_levels=False)
+    ref = oracle.eval_batch(og, d.k, d.s, d.C, d.B, d.scale, part)
+    assert np.array_equal(res["tlevel"][:, :P], ref.tlevel)
+    assert np.array_equal(res["blevel"][:, :P], ref.blevel)
     assert np.array_equal(res["cp"], ref.cp)
     assert np.array_equal(res["load"][:, :P], ref.load)
     assert np.array_equal(res["memload"][:, :P], ref.memload)
