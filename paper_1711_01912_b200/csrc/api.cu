@@ -107,6 +107,9 @@ struct tfps_graph {
     DBuf level, order, level_ptr_d, sink_flag, sink_list;
     int sink_count = 0;
     DBuf f_eptr, f_nbr, f_t, b_eptr, b_nbr, b_t;
+    // chunk tables of the candidate-sliced pass
+    DBuf vertf, f_chunks, b_chunks;
+    int f_num_chunks = 0, b_num_chunks = 0;
     // device tables
     bool dev_set = false;
     int k = 0;
@@ -240,6 +243,32 @@ int build_topo(tfps_graph* g, cudaStream_t st)
         if (flags[i]) sinks.push_back(i);
     g->sink_count = (int)sinks.size();
     TFPS_TRY(upload(g->sink_list, sinks, st));
+    CUDA_TRY(g->vertf.alloc(sizeof(int) * (size_t)n));
+    CUDA_TRY(launch_vertf(n, g->order.as<int>(), g->sink_flag.as<uint8_t>(), g->vertf.as<int>(), st));
+    // chunk tables: runs of positions inside one level, bounded in vertices and edges
+    for (int dir = 0; dir < 2; ++dir) {
+        std::vector<int> eptr((size_t)n + 1);
+        CUDA_TRY(cudaMemcpyAsync(eptr.data(), dir == 0 ? g->f_eptr.p : g->b_eptr.p, sizeof(int) * ((size_t)n + 1),
+                                 cudaMemcpyDeviceToHost, st));
+        CUDA_TRY(cudaStreamSynchronize(st));
+        std::vector<int> chunks;
+        for (int l = 0; l < g->num_levels; ++l) {
+            int p = (int)g->h_level_ptr[l];
+            const int pend = (int)g->h_level_ptr[l + 1];
+            while (p < pend) {
+                int q = p + 1;  // a chunk holds at least one vertex, however many edges it has
+                while (q < pend && q - p < CHUNK_V && eptr[q + 1] - eptr[p] <= CHUNK_E) ++q;
+                chunks.push_back(p);
+                chunks.push_back(q - p);
+                chunks.push_back(eptr[p]);
+                chunks.push_back(eptr[q] - eptr[p]);
+                p = q;
+            }
+        }
+        (dir == 0 ? g->f_num_chunks : g->b_num_chunks) = (int)(chunks.size() / 4);
+        TFPS_TRY(upload(dir == 0 ? g->f_chunks : g->b_chunks, chunks, st));
+        CUDA_TRY(cudaStreamSynchronize(st));
+    }
     CUDA_TRY(cudaStreamSynchronize(st));
     g->topo_built = true;
     return TFPS_OK;
@@ -621,7 +650,12 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
         long long* cp_here = (cp && (fwd || !need_fwd)) ? (long long*)cp : nullptr;
         PassArgs a = make_args(g, fwd, P, ldp, part, lev, cp_here);
         if (sliced) {
-            CUDA_TRY(launch_pass_sliced(a, fwd, g->sink_flag.as<uint8_t>(), cpt, warps, st));
+            SlicedPlan plan;
+            plan.vertf = g->vertf.as<int>();
+            plan.chunks = fwd ? g->f_chunks.as<int>() : g->b_chunks.as<int>();
+            plan.num_chunks = fwd ? g->f_num_chunks : g->b_num_chunks;
+            plan.src_end = (int)g->h_level_ptr[1];
+            CUDA_TRY(launch_pass_sliced(a, fwd, plan, cpt, warps, st));
         } else {
             CUDA_TRY(launch_pass_level_sync(a, fwd, g->h_level_ptr, st));
             if (cp_here) {

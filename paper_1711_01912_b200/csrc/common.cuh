@@ -63,6 +63,19 @@ struct PassArgs {
     int* status;          // sticky status word
 };
 
+// Chunking of the candidate-sliced pass: a chunk is a run of positions inside one
+// level with at most CHUNK_V vertices and CHUNK_E edges (a single vertex with more
+// edges forms a chunk of its own and is read straight from global memory).
+constexpr int CHUNK_V = 128;
+constexpr int CHUNK_E = 512;
+
+struct SlicedPlan {
+    const int* vertf;    // [n] vertex id by position, bit 31 set for sinks
+    const int* chunks;   // [num_chunks][4] = {first position, vertices, first edge, edges}
+    int num_chunks;
+    int src_end;         // positions below this are sources (level 0)
+};
+
 // every kernel launch of the library goes through the wrappers below and is counted here
 void count_launches(long long n);
 
@@ -82,7 +95,8 @@ cudaError_t launch_default_mem(int n, const long long* out_ptr, const long long*
 
 int pick_cpt(long long P);
 cudaError_t launch_pass_level_sync(const PassArgs& a, bool fwd, const std::vector<long long>& level_ptr_host, cudaStream_t st);
-cudaError_t launch_pass_sliced(const PassArgs& a, bool fwd, const uint8_t* cp_flag, int cpt, int warps, cudaStream_t st);
+cudaError_t launch_pass_sliced(const PassArgs& a, bool fwd, const SlicedPlan& plan, int cpt, int warps, cudaStream_t st);
+cudaError_t launch_vertf(int n, const int* order, const uint8_t* sink_flag, int* vertf, cudaStream_t st);
 cudaError_t launch_cp_reduce(const PassArgs& a, bool from_tlevel, const int* list, int list_len, cudaStream_t st);
 cudaError_t launch_loads(int n, long long P, long long ldp, const uint8_t* part, const int* vert,
                          const unsigned long long* xvert, const long long* mem, DevTables tab, long long* load,

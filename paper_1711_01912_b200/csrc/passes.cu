@@ -70,19 +70,30 @@ __device__ __forceinline__ void stage_tables(const DevTables& tab, DivConst* s_w
 }
 
 // ---- one vertex, 32*CPT candidates --------------------------------------------
+// Where the adjacency of the vertex being relaxed comes from: global memory
+// (level-synchronous kernel, oversized chunks) or the staged copy in shared memory.
+struct VertexMeta {
+    int v;                             // vertex id
+    int e0, e1;                        // edge range, as indices into the three arrays below
+    const int* nbr;                    // neighbour vertex ids
+    const unsigned long long* xw;      // transfer numerators
+    const unsigned long long* xnbr;    // neighbour runtime numerators (forward only)
+    unsigned long long xvert;          // own runtime numerator
+};
+
 // FWD: best = max over in-edges of tlevel(u) + rt(u) + w(u->v); writes tlevel(v).
 // BWD: best = max over out-edges of blevel(x) + w(v->x); writes blevel(v) = best + rt(v).
 // cpmax (may be unused) accumulates tlevel+rt over sinks (FWD) or blevel over sources (BWD).
 template <int CPT, bool FWD>
 __device__ __forceinline__ void relax_vertex(const PassArgs& a, const DivConst* __restrict__ s_w,
-                                             const DivConst* __restrict__ s_rt, int pos, long long jl,
+                                             const DivConst* __restrict__ s_rt, const VertexMeta& vm, long long jl,
                                              unsigned idmask, int nvalid, bool cp_vertex,
                                              long long (&cpmax)[CPT])
 {
     const int k = a.tab.k;
-    const int v = a.adj.vert[pos];
-    const int e0 = a.adj.eptr[pos];
-    const int e1 = a.adj.eptr[pos + 1];
+    const int v = vm.v;
+    const int e0 = vm.e0;
+    const int e1 = vm.e1;
     const long long ldp = a.ldp;
     const unsigned pv = IdVec<CPT>::load(a.part + (long long)v * ldp + jl) & idmask;
     unsigned idv[CPT];
@@ -101,9 +112,9 @@ __device__ __forceinline__ void relax_vertex(const PassArgs& a, const DivConst* 
 #pragma unroll
         for (int q = 0; q < UNR; ++q) {
             if (e + q < e1) {
-                const int u = a.adj.nbr[e + q];
-                X[q] = a.adj.xw[e + q];
-                if (FWD) Xn[q] = a.adj.xnbr[e + q];
+                const int u = vm.nbr[e + q];
+                X[q] = vm.xw[e + q];
+                if (FWD) Xn[q] = vm.xnbr[e + q];
                 const long long off = (long long)u * ldp + jl;
                 pu[q] = IdVec<CPT>::load(a.part + off) & idmask;
                 load_levels<CPT>(a.lev + off, lu[q]);
@@ -133,7 +144,7 @@ __device__ __forceinline__ void relax_vertex(const PassArgs& a, const DivConst* 
     if (FWD) {
         store_levels<CPT>(a.lev + (long long)v * ldp + jl, best, nvalid);
         if (cp_vertex) {
-            const unsigned long long Xv = a.adj.xvert[pos];
+            const unsigned long long Xv = vm.xvert;
 #pragma unroll
             for (int c = 0; c < CPT; ++c) {
                 long long fin = best[c];
@@ -142,7 +153,7 @@ __device__ __forceinline__ void relax_vertex(const PassArgs& a, const DivConst* 
             }
         }
     } else {
-        const unsigned long long Xv = a.adj.xvert[pos];
+        const unsigned long long Xv = vm.xvert;
 #pragma unroll
         for (int c = 0; c < CPT; ++c) {
             if (Xv != NUM_ZERO) best[c] += ceil_quot(Xv, s_rt[idv[c]]);
@@ -150,6 +161,19 @@ __device__ __forceinline__ void relax_vertex(const PassArgs& a, const DivConst* 
         }
         store_levels<CPT>(a.lev + (long long)v * ldp + jl, best, nvalid);
     }
+}
+
+__device__ __forceinline__ VertexMeta global_meta(const LevelAdj& adj, int pos)
+{
+    VertexMeta vm;
+    vm.v = adj.vert[pos];
+    vm.e0 = adj.eptr[pos];
+    vm.e1 = adj.eptr[pos + 1];
+    vm.nbr = adj.nbr;
+    vm.xw = adj.xw;
+    vm.xnbr = adj.xnbr;
+    vm.xvert = adj.xvert[pos];
+    return vm;
 }
 
 // Lane bookkeeping shared by both pass kernels: first candidate of the lane,
@@ -185,19 +209,65 @@ pass_level_kernel(PassArgs a, int pos0, int count)
 #pragma unroll
     for (int c = 0; c < CPT; ++c) unused[c] = 0;
     for (int i = blockIdx.y * wpb + warp; i < count; i += gridDim.y * wpb)
-        relax_vertex<CPT, FWD>(a, s_w, s_rt, pos0 + i, jl, idmask, nvalid, false, unused);
+        relax_vertex<CPT, FWD>(a, s_w, s_rt, global_meta(a.adj, pos0 + i), jl, idmask, nvalid, false, unused);
 }
 
 // ---- candidate-sliced persistent variant ---------------------------------------------
-// One block owns 32*CPT candidates and walks every level; its warps share the
-// vertices of a level and meet at a block barrier between levels.  Candidates
-// are independent, so no block ever waits for another one.
+// One block owns 32*CPT candidates and walks the whole graph chunk by chunk; a
+// chunk is a run of at most CHUNK_V positions / CHUNK_E edges inside one level
+// (table built on the host).  Candidates are independent, so no block ever
+// waits for another one; the block's warps share the vertices of a chunk and
+// meet at one block barrier per chunk.  The adjacency of the NEXT chunk is
+// copied into shared memory with cp.async while the current one is processed,
+// so a warp's dependent global-memory chain per vertex is a single hop
+// (neighbour ids and levels).
+__device__ __forceinline__ void cp_async4(void* smem, const void* g)
+{
+    unsigned s = (unsigned)__cvta_generic_to_shared(smem);
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(s), "l"(g));
+}
+__device__ __forceinline__ void cp_async8(void* smem, const void* g)
+{
+    unsigned s = (unsigned)__cvta_generic_to_shared(smem);
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(s), "l"(g));
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+
+struct ChunkBuf {
+    unsigned long long xvert[CHUNK_V];
+    unsigned long long xw[CHUNK_E];
+    unsigned long long xnbr[CHUNK_E];
+    int vertf[CHUNK_V];
+    int eoff[CHUNK_V + 4];
+    int nbr[CHUNK_E];
+};
+
+template <bool FWD>
+__device__ __forceinline__ void stage_chunk(const PassArgs& a, const int* __restrict__ vertf, int4 ent, ChunkBuf& b)
+{
+    const int p0 = ent.x, cnt = ent.y, e0 = ent.z, ecnt = ent.w;
+    for (int i = threadIdx.x; i < cnt; i += blockDim.x) {
+        cp_async4(&b.vertf[i], vertf + p0 + i);
+        cp_async8(&b.xvert[i], a.adj.xvert + p0 + i);
+    }
+    for (int i = threadIdx.x; i <= cnt; i += blockDim.x) cp_async4(&b.eoff[i], a.adj.eptr + p0 + i);
+    if (ecnt <= CHUNK_E) {
+        for (int i = threadIdx.x; i < ecnt; i += blockDim.x) {
+            cp_async4(&b.nbr[i], a.adj.nbr + e0 + i);
+            cp_async8(&b.xw[i], a.adj.xw + e0 + i);
+            if (FWD) cp_async8(&b.xnbr[i], a.adj.xnbr + e0 + i);
+        }
+    }
+}
+
 template <int CPT, bool FWD>
 __global__ void __launch_bounds__(256)
-pass_sliced_kernel(PassArgs a, const uint8_t* __restrict__ cp_flag)
+pass_sliced_kernel(PassArgs a, const int* __restrict__ vertf, const int4* __restrict__ chunks, int num_chunks, int src_end)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    DivConst* s_w = reinterpret_cast<DivConst*>(smem_raw);
+    ChunkBuf* bufs = reinterpret_cast<ChunkBuf*>(smem_raw);
+    DivConst* s_w = reinterpret_cast<DivConst*>(bufs + 2);
     DivConst* s_rt = s_w + a.tab.k * a.tab.k;
     long long* s_cp = reinterpret_cast<long long*>(s_rt + a.tab.k);  // [warps][32*CPT]
     if (*a.status != 0) return;
@@ -211,17 +281,44 @@ pass_sliced_kernel(PassArgs a, const uint8_t* __restrict__ cp_flag)
 #pragma unroll
     for (int c = 0; c < CPT; ++c) cpmax[c] = 0;
 
-    const int L = a.num_levels;
-    for (int step = 0; step < L; ++step) {
-        const int l = FWD ? step : L - 1 - step;
-        const int p0 = (int)a.level_ptr[l];
-        const int p1 = (int)a.level_ptr[l + 1];
-        for (int pos = p0 + warp; pos < p1; pos += wpb) {
-            bool cpv = false;
-            if (want_cp) cpv = FWD ? (cp_flag[pos] != 0) : (l == 0);
-            relax_vertex<CPT, FWD>(a, s_w, s_rt, pos, jl, idmask, nvalid, cpv, cpmax);
+    // chunk ci of this pass is table entry ci (forward) or num_chunks-1-ci (backward)
+    auto entry = [&](int ci) { return chunks[FWD ? ci : num_chunks - 1 - ci]; };
+    int4 cur = entry(0);
+    int4 nxt = num_chunks > 1 ? entry(1) : cur;
+    stage_chunk<FWD>(a, vertf, cur, bufs[0]);
+    cp_async_commit();
+    cp_async_wait_all();
+    __syncthreads();
+    for (int ci = 0; ci < num_chunks; ++ci) {
+        ChunkBuf& b = bufs[ci & 1];
+        int4 nxt2 = nxt;
+        if (ci + 1 < num_chunks) {
+            stage_chunk<FWD>(a, vertf, nxt, bufs[(ci + 1) & 1]);
+            cp_async_commit();
+            if (ci + 2 < num_chunks) nxt2 = entry(ci + 2);
         }
+        const int p0 = cur.x, cnt = cur.y, e0 = cur.z;
+        const bool staged = cur.w <= CHUNK_E;
+        for (int i = warp; i < cnt; i += wpb) {
+            VertexMeta vm;
+            const int vf = b.vertf[i];
+            vm.v = vf & 0x7fffffff;
+            vm.xvert = b.xvert[i];
+            // a vertex whose adjacency did not fit the chunk buffer is read from global memory
+            const int ebase = staged ? e0 : 0;
+            vm.e0 = b.eoff[i] - ebase;
+            vm.e1 = b.eoff[i + 1] - ebase;
+            vm.nbr = staged ? b.nbr : a.adj.nbr;
+            vm.xw = staged ? b.xw : a.adj.xw;
+            vm.xnbr = staged ? b.xnbr : a.adj.xnbr;
+            bool cpv = false;
+            if (want_cp) cpv = FWD ? (vf < 0) : (p0 + i < src_end);
+            relax_vertex<CPT, FWD>(a, s_w, s_rt, vm, jl, idmask, nvalid, cpv, cpmax);
+        }
+        cp_async_wait_all();
         __syncthreads();
+        cur = nxt;
+        nxt = nxt2;
     }
 
     if (want_cp) {
@@ -432,22 +529,24 @@ cudaError_t launch_pass_level_sync(const PassArgs& a, bool fwd, const std::vecto
 }
 
 template <int CPT, bool FWD>
-static cudaError_t sliced_impl(const PassArgs& a, const uint8_t* cp_flag, int warps, cudaStream_t st)
+static cudaError_t sliced_impl(const PassArgs& a, const SlicedPlan& plan, int warps, cudaStream_t st)
 {
-    const size_t smem = table_smem(a.tab.k) + sizeof(long long) * (size_t)warps * 32 * CPT;
+    const size_t smem = 2 * sizeof(ChunkBuf) + table_smem(a.tab.k) + sizeof(long long) * (size_t)warps * 32 * CPT;
     cudaError_t e = allow_smem(pass_sliced_kernel<CPT, FWD>, smem);
     if (e != cudaSuccess) return e;
     const unsigned gx = cdivu(a.P, 32 * CPT);
-    pass_sliced_kernel<CPT, FWD><<<gx, warps * 32, smem, st>>>(a, cp_flag);
+    pass_sliced_kernel<CPT, FWD><<<gx, warps * 32, smem, st>>>(a, plan.vertf, reinterpret_cast<const int4*>(plan.chunks),
+                                                                plan.num_chunks, plan.src_end);
     count_launches(1);
     return cudaGetLastError();
 }
 
-cudaError_t launch_pass_sliced(const PassArgs& a, bool fwd, const uint8_t* cp_flag, int cpt, int warps, cudaStream_t st)
+cudaError_t launch_pass_sliced(const PassArgs& a, bool fwd, const SlicedPlan& plan, int cpt, int warps, cudaStream_t st)
 {
-    if (cpt == 4) return fwd ? sliced_impl<4, true>(a, cp_flag, warps, st) : sliced_impl<4, false>(a, cp_flag, warps, st);
-    if (cpt == 2) return fwd ? sliced_impl<2, true>(a, cp_flag, warps, st) : sliced_impl<2, false>(a, cp_flag, warps, st);
-    return fwd ? sliced_impl<1, true>(a, cp_flag, warps, st) : sliced_impl<1, false>(a, cp_flag, warps, st);
+    if (plan.num_chunks <= 0) return cudaSuccess;
+    if (cpt == 4) return fwd ? sliced_impl<4, true>(a, plan, warps, st) : sliced_impl<4, false>(a, plan, warps, st);
+    if (cpt == 2) return fwd ? sliced_impl<2, true>(a, plan, warps, st) : sliced_impl<2, false>(a, plan, warps, st);
+    return fwd ? sliced_impl<1, true>(a, plan, warps, st) : sliced_impl<1, false>(a, plan, warps, st);
 }
 
 cudaError_t launch_cp_reduce(const PassArgs& a, bool from_tlevel, const int* list, int list_len, cudaStream_t st)

@@ -206,6 +206,12 @@ __global__ void sink_flags_kernel(int n, const int* __restrict__ order, const lo
     if (i < n) { int v = order[i]; flag[i] = out_ptr[v + 1] == out_ptr[v] ? 1 : 0; }
 }
 
+__global__ void vertf_kernel(int n, const int* __restrict__ order, const uint8_t* __restrict__ sink_flag, int* vertf)
+{
+    int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) vertf[i] = order[i] | (sink_flag[i] ? (int)0x80000000 : 0);
+}
+
 __device__ __forceinline__ unsigned long long numerator(long long a)
 {
     return a == 0 ? NUM_ZERO : ((unsigned long long)(a - 1) << 2);
@@ -291,6 +297,12 @@ cudaError_t launch_build_adj(int n, const int* order, const long long* ptr, cons
 cudaError_t launch_sink_flags(int n, const int* order, const long long* out_ptr, uint8_t* flag, cudaStream_t st)
 {
     if (n > 0) { sink_flags_kernel<<<cdiv(n, 256), 256, 0, st>>>(n, order, out_ptr, flag); count_launches(1); }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_vertf(int n, const int* order, const uint8_t* sink_flag, int* vertf, cudaStream_t st)
+{
+    if (n > 0) { vertf_kernel<<<cdiv(n, 256), 256, 0, st>>>(n, order, sink_flag, vertf); count_launches(1); }
     return cudaGetLastError();
 }
 
