@@ -115,6 +115,8 @@ struct tfps_graph {
     int k = 0;
     long long S = 0;
     DBuf rt_div, w_div, cap, xvert, xw_f, xnbr_f, xw_b;
+    DBuf pair_f, pair_b, cls_div, sel_f, sel_b;
+    int npass = 0, use_cls = 0, ncls_w = 0;
     DBuf status;
     // scratch owned by the handle
     DBuf scr_memload;
@@ -274,6 +276,24 @@ int build_topo(tfps_graph* g, cudaStream_t st)
     return TFPS_OK;
 }
 
+DevTables make_tables(const tfps_graph* g)
+{
+    DevTables t;
+    t.k = g->k;
+    t.rt_div = g->rt_div.as<DivConst>();
+    t.w_div = g->w_div.as<DivConst>();
+    t.cap = g->cap.as<long long>();
+    t.npass = g->npass;
+    t.use_cls = g->use_cls;
+    t.ncls_w = g->ncls_w;
+    t.pair_f = g->pair_f.as<DivConst>();
+    t.pair_b = g->pair_b.as<DivConst>();
+    t.cls_div = g->cls_div.as<DivConst>();
+    t.sel_f = g->sel_f.as<unsigned short>();
+    t.sel_b = g->sel_b.as<unsigned short>();
+    return t;
+}
+
 PassArgs make_args(const tfps_graph* g, bool fwd, long long P, long long ldp, const uint8_t* part, long long* lev,
                    long long* cp)
 {
@@ -284,10 +304,7 @@ PassArgs make_args(const tfps_graph* g, bool fwd, long long P, long long ldp, co
     a.adj.xw = fwd ? g->xw_f.as<unsigned long long>() : g->xw_b.as<unsigned long long>();
     a.adj.xnbr = fwd ? g->xnbr_f.as<unsigned long long>() : nullptr;
     a.adj.xvert = g->xvert.as<unsigned long long>();
-    a.tab.k = g->k;
-    a.tab.rt_div = g->rt_div.as<DivConst>();
-    a.tab.w_div = g->w_div.as<DivConst>();
-    a.tab.cap = g->cap.as<long long>();
+    a.tab = make_tables(g);
     a.level_ptr = g->level_ptr_d.as<long long>();
     a.num_levels = g->num_levels;
     a.n = (int)g->n;
@@ -512,6 +529,56 @@ int tfps_devices_set(tfps_graph* g, int k, const int32_t* s, const int64_t* C, c
         }
     std::vector<long long> cap(C, C + k);
     g->dev_set = false;
+    // pair tables and value classes for the per-edge cost table
+    g->npass = k <= TABLE_K_MAX ? (k * k + 31) / 32 : 0;
+    g->use_cls = 0;
+    g->ncls_w = 0;
+    if (g->npass > 0) {
+        const int ent = g->npass * 32;
+        std::vector<DivConst> pf((size_t)ent), pb((size_t)ent), cls(32, DivConst{0ull, 0u, 0u});
+        std::vector<unsigned short> sf((size_t)ent), sb((size_t)ent);
+        std::vector<long long> wvals, svals;  // distinct off-diagonal bandwidths, distinct speeds
+        auto cls_of = [](std::vector<long long>& vals, long long x) {
+            for (size_t i = 0; i < vals.size(); ++i)
+                if (vals[i] == x) return (int)i;
+            vals.push_back(x);
+            return (int)vals.size() - 1;
+        };
+        for (int a = 0; a < k; ++a)
+            for (int b = 0; b < k; ++b)
+                if (a != b) cls_of(wvals, B[a * k + b]);
+        for (int d = 0; d < k; ++d) cls_of(svals, s[d]);
+        const bool use_cls = wvals.size() + svals.size() <= 32;
+        const int ncw = (int)wvals.size();
+        for (int i = 0; i < ent; ++i) {
+            const bool real = i < k * k;
+            const int nb = real ? i / k : 0, vv = real ? i % k : 0;
+            const bool diag = !real || nb == vv;
+            pf[i] = diag ? DivConst{0ull, 0u, 0u} : make_div((unsigned long long)B[nb * k + vv]);
+            pb[i] = diag ? DivConst{0ull, 0u, 0u} : make_div((unsigned long long)B[vv * k + nb]);
+            pf[i].pad = (unsigned)nb | (diag ? 256u : 0u);
+            pb[i].pad = (unsigned)vv | (diag ? 256u : 0u);
+            if (use_cls) {
+                const int cwf = diag ? 255 : cls_of(wvals, B[nb * k + vv]);
+                const int cwb = diag ? 255 : cls_of(wvals, B[vv * k + nb]);
+                sf[i] = (unsigned short)(cwf | ((ncw + cls_of(svals, s[nb])) << 8));
+                sb[i] = (unsigned short)(cwb | ((ncw + cls_of(svals, s[vv])) << 8));
+            } else {
+                sf[i] = sb[i] = 255;
+            }
+        }
+        if (use_cls) {
+            for (int c = 0; c < ncw; ++c) cls[c] = make_div((unsigned long long)wvals[c]);
+            for (size_t c = 0; c < svals.size(); ++c) cls[ncw + c] = make_div((unsigned long long)svals[c]);
+        }
+        g->use_cls = use_cls ? 1 : 0;
+        g->ncls_w = ncw;
+        TFPS_TRY(upload(g->pair_f, pf, st));
+        TFPS_TRY(upload(g->pair_b, pb, st));
+        TFPS_TRY(upload(g->cls_div, cls, st));
+        TFPS_TRY(upload(g->sel_f, sf, st));
+        TFPS_TRY(upload(g->sel_b, sb, st));
+    }
     TFPS_TRY(upload(g->rt_div, rt, st));
     TFPS_TRY(upload(g->w_div, w, st));
     TFPS_TRY(upload(g->cap, cap, st));
@@ -592,11 +659,7 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
     const bool validate = !(flags & TFPS_EVAL_NO_VALIDATE);
     const int n = (int)g->n;
     const int k = g->k;
-    DevTables tab;
-    tab.k = k;
-    tab.rt_div = g->rt_div.as<DivConst>();
-    tab.w_div = g->w_div.as<DivConst>();
-    tab.cap = g->cap.as<long long>();
+    const DevTables tab = make_tables(g);
     int* status = g->status.as<int>();
 
     const bool profile = (flags & TFPS_EVAL_PROFILE) != 0;
@@ -632,13 +695,21 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
         const long long avg_width = g->num_levels > 0 ? g->n / g->num_levels : g->n;
         sliced = (P >= 32LL * g->sm_count) || (avg_width * P < (1LL << 18));
     }
+    // shape of the sliced kernel: candidates per lane and warps per block (overridable for tuning).
+    // Wider lanes amortise the per-edge cost table over more candidates; keep enough slices to fill the SMs.
+    const bool table = env_int("TFPS_SLICED_TABLE", 1) != 0;
     int cpt = env_int("TFPS_SLICED_CPT", 0);
-    if (cpt != 1 && cpt != 2 && cpt != 4) cpt = (P >= 64LL * 4 * g->sm_count) ? 2 : 1;
+    if (cpt != 1 && cpt != 2 && cpt != 4 && cpt != 8) {
+        cpt = 1;
+        if (table && g->npass > 0)
+            for (int c = 4; c > 1; c >>= 1)
+                if ((P + 32 * c - 1) / (32 * c) >= (3LL * g->sm_count) / 4) { cpt = c; break; }
+    }
     int warps = env_int("TFPS_SLICED_WARPS", 0);
-    if (warps < 1 || warps > 8) {
+    if (warps < 1 || warps > 32) {
         const long long avg_width = g->num_levels > 0 ? g->n / g->num_levels : g->n;
-        warps = 1;
-        while (warps < 8 && warps * 2 <= avg_width) warps <<= 1;
+        warps = 4;
+        while (warps < 32 && warps < avg_width) warps <<= 1;
     }
 
     if (profile) CUDA_TRY(cudaEventRecord(g->ev[1], st));
@@ -655,7 +726,7 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
             plan.chunks = fwd ? g->f_chunks.as<int>() : g->b_chunks.as<int>();
             plan.num_chunks = fwd ? g->f_num_chunks : g->b_num_chunks;
             plan.src_end = (int)g->h_level_ptr[1];
-            CUDA_TRY(launch_pass_sliced(a, fwd, plan, cpt, warps, st));
+            CUDA_TRY(launch_pass_sliced(a, fwd, plan, cpt, warps, table, st));
         } else {
             CUDA_TRY(launch_pass_level_sync(a, fwd, g->h_level_ptr, st));
             if (cp_here) {

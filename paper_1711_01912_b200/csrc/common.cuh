@@ -32,11 +32,34 @@ constexpr unsigned long long NUM_ZERO = ~0ull;
 
 // Device tables set by tfps_devices_set (global memory; kernels stage them in
 // shared memory).  rt_div[d] divides by s_d, w_div[a*k+b] by B[a][b].
+//
+// Pair tables for the per-edge cost table of the sliced pass (k <= TABLE_K_MAX):
+// entry i = nb*k + vv pairs the neighbour's device nb with the vertex's device
+// vv.  pair_f[i] divides by B[nb][vv] (forward: edge neighbour -> vertex),
+// pair_b[i] by B[vv][nb] (backward: edge vertex -> neighbour).  Both are padded
+// to npass*32 entries; DivConst::pad holds  dev | diag << 8  where dev is the
+// device whose speed enters the entry (nb forward, vv backward) and diag marks
+// nb == vv or a padding entry (transfer cost 0).
+//
+// When the off-diagonal bandwidths and the speeds take at most 32 distinct
+// values together ("classes"), cls_div[c] holds one divisor per class (transfer
+// classes first, then ncls_w.. the speed classes) and sel_f/sel_b[i] = cw | cr << 8
+// name the transfer class (255 = none) and the speed class lane of entry i.
+constexpr int TABLE_K_MAX = 16;
+
 struct DevTables {
     int k;
     const DivConst* rt_div;  // [k]
     const DivConst* w_div;   // [k*k]
     const long long* cap;    // [k]
+    int npass;               // ceil(k*k/32) when k <= TABLE_K_MAX, else 0
+    int use_cls;             // classes available
+    int ncls_w;              // number of transfer classes
+    const DivConst* pair_f;  // [npass*32]
+    const DivConst* pair_b;  // [npass*32]
+    const DivConst* cls_div; // [32]
+    const unsigned short* sel_f;  // [npass*32]
+    const unsigned short* sel_b;  // [npass*32]
 };
 
 // Level-ordered adjacency of one direction.  Position i runs over vertices
@@ -95,7 +118,8 @@ cudaError_t launch_default_mem(int n, const long long* out_ptr, const long long*
 
 int pick_cpt(long long P);
 cudaError_t launch_pass_level_sync(const PassArgs& a, bool fwd, const std::vector<long long>& level_ptr_host, cudaStream_t st);
-cudaError_t launch_pass_sliced(const PassArgs& a, bool fwd, const SlicedPlan& plan, int cpt, int warps, cudaStream_t st);
+cudaError_t launch_pass_sliced(const PassArgs& a, bool fwd, const SlicedPlan& plan, int cpt, int warps, bool table,
+                               cudaStream_t st);
 cudaError_t launch_vertf(int n, const int* order, const uint8_t* sink_flag, int* vertf, cudaStream_t st);
 cudaError_t launch_cp_reduce(const PassArgs& a, bool from_tlevel, const int* list, int list_len, cudaStream_t st);
 cudaError_t launch_loads(int n, long long P, long long ldp, const uint8_t* part, const int* vert,

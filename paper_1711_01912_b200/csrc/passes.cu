@@ -12,16 +12,30 @@ namespace tfps {
 namespace {
 
 // ---- small vector helpers ----------------------------------------------------
-template <int CPT> struct IdVec;
-template <> struct IdVec<1> {
-    static __device__ __forceinline__ unsigned load(const uint8_t* p) { return *p; }
-};
-template <> struct IdVec<2> {
-    static __device__ __forceinline__ unsigned load(const uint8_t* p) { return *reinterpret_cast<const unsigned short*>(p); }
-};
-template <> struct IdVec<4> {
-    static __device__ __forceinline__ unsigned load(const uint8_t* p) { return *reinterpret_cast<const unsigned*>(p); }
-};
+constexpr unsigned FULL = 0xffffffffu;
+
+template <int CPT> struct IdWords { static constexpr int N = (CPT + 3) / 4; };
+
+// CPT partition ids (one byte each) starting at p, packed little-endian into 32-bit words
+template <int CPT>
+__device__ __forceinline__ void load_ids(const uint8_t* p, unsigned (&w)[IdWords<CPT>::N])
+{
+    if constexpr (CPT == 1) w[0] = *p;
+    else if constexpr (CPT == 2) w[0] = *reinterpret_cast<const unsigned short*>(p);
+    else if constexpr (CPT == 4) w[0] = *reinterpret_cast<const unsigned*>(p);
+    else {
+        static_assert(CPT == 8, "CPT must be 1, 2, 4 or 8");
+        const uint2 v = *reinterpret_cast<const uint2*>(p);
+        w[0] = v.x;
+        w[1] = v.y;
+    }
+}
+
+template <int CPT>
+__device__ __forceinline__ unsigned id_at(const unsigned (&w)[IdWords<CPT>::N], int c)
+{
+    return (w[c >> 2] >> (8 * (c & 3))) & 0xffu;
+}
 
 template <int CPT>
 __device__ __forceinline__ void load_levels(const long long* p, long long (&out)[CPT])
@@ -60,6 +74,13 @@ __device__ __forceinline__ long long ceil_quot(unsigned long long X, const DivCo
     return 1 + (long long)(__umul64hi(dc.mul, X) >> dc.sh);
 }
 
+__device__ __forceinline__ long long shfl64(long long v, int src)
+{
+    int lo = __shfl_sync(FULL, (int)(unsigned)(unsigned long long)v, src);
+    int hi = __shfl_sync(FULL, (int)((unsigned long long)v >> 32), src);
+    return (long long)(((unsigned long long)(unsigned)hi << 32) | (unsigned)lo);
+}
+
 // Shared-memory copy of the division constants: [k*k] pair table then [k] speed table.
 __device__ __forceinline__ void stage_tables(const DevTables& tab, DivConst* s_w, DivConst* s_rt)
 {
@@ -67,6 +88,38 @@ __device__ __forceinline__ void stage_tables(const DevTables& tab, DivConst* s_w
     for (int i = threadIdx.x; i < k * k; i += blockDim.x) s_w[i] = tab.w_div[i];
     for (int i = threadIdx.x; i < k; i += blockDim.x) s_rt[i] = tab.rt_div[i];
     __syncthreads();
+}
+
+// Per-lane candidate bookkeeping shared by the pass kernels.
+template <int CPT>
+struct LaneCtx {
+    long long jl;                         // (always in-bounds) first column the lane loads from
+    int nvalid;                           // how many of the lane's CPT candidates are real
+    unsigned maskw[IdWords<CPT>::N];      // zeroes the ids of padding candidates
+};
+
+template <int CPT>
+__device__ __forceinline__ LaneCtx<CPT> lane_setup(long long slice0, long long P, int lane)
+{
+    LaneCtx<CPT> lc;
+    const long long j0 = slice0 + (long long)lane * CPT;
+    const long long rem = P - j0;
+    lc.nvalid = rem >= CPT ? CPT : (rem > 0 ? (int)rem : 0);
+    lc.jl = lc.nvalid > 0 ? j0 : slice0;  // idle lanes shadow the slice's first lane and never store
+#pragma unroll
+    for (int w = 0; w < IdWords<CPT>::N; ++w) {
+        const int nv = lc.nvalid - 4 * w;  // valid bytes in this word
+        lc.maskw[w] = nv >= 4 ? 0xffffffffu : (nv > 0 ? ((1u << (8 * nv)) - 1u) : 0u);
+    }
+    return lc;
+}
+
+template <int CPT>
+__device__ __forceinline__ void load_ids_masked(const uint8_t* p, const LaneCtx<CPT>& lc, unsigned (&w)[IdWords<CPT>::N])
+{
+    load_ids<CPT>(p, w);
+#pragma unroll
+    for (int i = 0; i < IdWords<CPT>::N; ++i) w[i] &= lc.maskw[i];
 }
 
 // ---- one vertex, 32*CPT candidates --------------------------------------------
@@ -81,24 +134,22 @@ struct VertexMeta {
     unsigned long long xvert;          // own runtime numerator
 };
 
+// Direct form: every relaxation divides on its own (any k).
 // FWD: best = max over in-edges of tlevel(u) + rt(u) + w(u->v); writes tlevel(v).
 // BWD: best = max over out-edges of blevel(x) + w(v->x); writes blevel(v) = best + rt(v).
-// cpmax (may be unused) accumulates tlevel+rt over sinks (FWD) or blevel over sources (BWD).
+// cpmax accumulates tlevel+rt over sinks (FWD) or blevel over sources (BWD).
 template <int CPT, bool FWD>
 __device__ __forceinline__ void relax_vertex(const PassArgs& a, const DivConst* __restrict__ s_w,
-                                             const DivConst* __restrict__ s_rt, const VertexMeta& vm, long long jl,
-                                             unsigned idmask, int nvalid, bool cp_vertex,
-                                             long long (&cpmax)[CPT])
+                                             const DivConst* __restrict__ s_rt, const VertexMeta& vm,
+                                             const LaneCtx<CPT>& lc, bool cp_vertex, long long* cpmax)
 {
     const int k = a.tab.k;
     const int v = vm.v;
     const int e0 = vm.e0;
     const int e1 = vm.e1;
     const long long ldp = a.ldp;
-    const unsigned pv = IdVec<CPT>::load(a.part + (long long)v * ldp + jl) & idmask;
-    unsigned idv[CPT];
-#pragma unroll
-    for (int c = 0; c < CPT; ++c) idv[c] = (pv >> (8 * c)) & 0xffu;
+    unsigned pv[IdWords<CPT>::N];
+    load_ids_masked<CPT>(a.part + (long long)v * ldp + lc.jl, lc, pv);
 
     long long best[CPT];
 #pragma unroll
@@ -107,7 +158,7 @@ __device__ __forceinline__ void relax_vertex(const PassArgs& a, const DivConst* 
     constexpr int UNR = (CPT >= 4) ? 2 : 4;
     for (int e = e0; e < e1; e += UNR) {
         long long lu[UNR][CPT];
-        unsigned pu[UNR];
+        unsigned pu[UNR][IdWords<CPT>::N];
         unsigned long long X[UNR], Xn[UNR];
 #pragma unroll
         for (int q = 0; q < UNR; ++q) {
@@ -115,8 +166,8 @@ __device__ __forceinline__ void relax_vertex(const PassArgs& a, const DivConst* 
                 const int u = vm.nbr[e + q];
                 X[q] = vm.xw[e + q];
                 if (FWD) Xn[q] = vm.xnbr[e + q];
-                const long long off = (long long)u * ldp + jl;
-                pu[q] = IdVec<CPT>::load(a.part + off) & idmask;
+                const long long off = (long long)u * ldp + lc.jl;
+                load_ids_masked<CPT>(a.part + off, lc, pu[q]);
                 load_levels<CPT>(a.lev + off, lu[q]);
             }
         }
@@ -125,12 +176,13 @@ __device__ __forceinline__ void relax_vertex(const PassArgs& a, const DivConst* 
             if (e + q < e1) {
 #pragma unroll
                 for (int c = 0; c < CPT; ++c) {
-                    const unsigned idu = (pu[q] >> (8 * c)) & 0xffu;
+                    const unsigned idu = id_at<CPT>(pu[q], c);
+                    const unsigned idv = id_at<CPT>(pv, c);
                     long long val = lu[q][c];
                     if (X[q] != NUM_ZERO) {
-                        const DivConst dc = s_w[FWD ? idu * k + idv[c] : idv[c] * k + idu];
+                        const DivConst dc = s_w[FWD ? idu * k + idv : idv * k + idu];
                         const long long w = ceil_quot(X[q], dc);
-                        val += (idu != idv[c]) ? w : 0;
+                        val += (idu != idv) ? w : 0;
                     }
                     if (FWD) {
                         if (Xn[q] != NUM_ZERO) val += ceil_quot(Xn[q], s_rt[idu]);
@@ -141,25 +193,118 @@ __device__ __forceinline__ void relax_vertex(const PassArgs& a, const DivConst* 
         }
     }
 
-    if (FWD) {
-        store_levels<CPT>(a.lev + (long long)v * ldp + jl, best, nvalid);
-        if (cp_vertex) {
-            const unsigned long long Xv = vm.xvert;
+    const unsigned long long Xv = vm.xvert;
+    if (!FWD) {
 #pragma unroll
-            for (int c = 0; c < CPT; ++c) {
-                long long fin = best[c];
-                if (Xv != NUM_ZERO) fin += ceil_quot(Xv, s_rt[idv[c]]);
-                cpmax[c] = fin > cpmax[c] ? fin : cpmax[c];
-            }
-        }
-    } else {
-        const unsigned long long Xv = vm.xvert;
+        for (int c = 0; c < CPT; ++c)
+            if (Xv != NUM_ZERO) best[c] += ceil_quot(Xv, s_rt[id_at<CPT>(pv, c)]);
+    }
+    store_levels<CPT>(a.lev + (long long)v * ldp + lc.jl, best, lc.nvalid);
+    if (cp_vertex) {
 #pragma unroll
         for (int c = 0; c < CPT; ++c) {
-            if (Xv != NUM_ZERO) best[c] += ceil_quot(Xv, s_rt[idv[c]]);
-            if (cp_vertex) cpmax[c] = best[c] > cpmax[c] ? best[c] : cpmax[c];
+            long long fin = best[c];
+            if (FWD && Xv != NUM_ZERO) fin += ceil_quot(Xv, s_rt[id_at<CPT>(pv, c)]);
+            cpmax[c] = fin > cpmax[c] ? fin : cpmax[c];
         }
-        store_levels<CPT>(a.lev + (long long)v * ldp + jl, best, nvalid);
+    }
+}
+
+// Table form (k <= TABLE_K_MAX).  The cost of an edge depends on the candidate
+// only through the pair (device of the neighbour nb, device of the vertex vv),
+// so the warp first fills a k*k table for the edge,
+//   FWD: T[nb*k+vv] = rt(u on nb) + w(nb -> vv),   BWD: T[nb*k+vv] = rt(v on vv) + w(vv -> nb),
+// one entry per lane and pass, and every candidate then needs a single
+// shared-memory lookup instead of two 64-bit divisions.  The neighbour's ids
+// and levels are requested before the table is built, so the build overlaps
+// their latency.
+struct TableCtx {
+    const DivConst* s_pair;         // [npass*32] pair divisors of this direction (+ dev | diag << 8)
+    const DivConst* s_rt;           // [k] speed divisors
+    const unsigned short* s_sel;    // [npass*32] class selectors, valid when use_cls
+    long long* T;                   // this warp's table, npass*32 entries
+    DivConst my_cls;                // class divisor of this lane, valid when use_cls
+    int npass;
+    int use_cls;
+    int ncls_w;
+};
+
+template <bool FWD>
+__device__ __forceinline__ void build_edge_table(const TableCtx& tc, unsigned long long X, unsigned long long Xr, int lane)
+{
+    __syncwarp();  // lookups of the previous edge are done
+    if (tc.use_cls) {
+        // one division per distinct bandwidth / speed value, spread to the entries by shuffles
+        const unsigned long long num = lane < tc.ncls_w ? X : Xr;
+        const long long val = num != NUM_ZERO ? ceil_quot(num, tc.my_cls) : 0;
+        for (int p = 0; p < tc.npass; ++p) {
+            const int i = lane + 32 * p;
+            const unsigned sel = tc.s_sel[i];
+            const unsigned cw = sel & 0xffu;
+            long long w = shfl64(val, (int)(cw & 31u));
+            const long long r = shfl64(val, (int)(sel >> 8));
+            if (cw == 255u) w = 0;
+            tc.T[i] = w + r;
+        }
+    } else {
+        for (int p = 0; p < tc.npass; ++p) {
+            const int i = lane + 32 * p;
+            const DivConst dc = tc.s_pair[i];
+            long long t = 0;
+            if (X != NUM_ZERO && (dc.pad & 256u) == 0) t = ceil_quot(X, dc);
+            if (Xr != NUM_ZERO) t += ceil_quot(Xr, tc.s_rt[dc.pad & 0xffu]);
+            tc.T[i] = t;
+        }
+    }
+    __syncwarp();
+}
+
+template <int CPT, bool FWD>
+__device__ __forceinline__ void relax_vertex_table(const PassArgs& a, const TableCtx& tc, const VertexMeta& vm,
+                                                   const LaneCtx<CPT>& lc, int lane, bool cp_vertex, long long* cpmax)
+{
+    const int k = a.tab.k;
+    const int v = vm.v;
+    const long long ldp = a.ldp;
+    unsigned pv[IdWords<CPT>::N];
+    load_ids_masked<CPT>(a.part + (long long)v * ldp + lc.jl, lc, pv);
+    const unsigned long long Xv = vm.xvert;
+
+    long long best[CPT];
+#pragma unroll
+    for (int c = 0; c < CPT; ++c) best[c] = 0;
+
+    for (int e = vm.e0; e < vm.e1; ++e) {
+        const int u = vm.nbr[e];
+        const unsigned long long X = vm.xw[e];
+        const unsigned long long Xr = FWD ? vm.xnbr[e] : Xv;
+        const long long off = (long long)u * ldp + lc.jl;
+        unsigned pu[IdWords<CPT>::N];
+        long long lu[CPT];
+        load_ids_masked<CPT>(a.part + off, lc, pu);
+        load_levels<CPT>(a.lev + off, lu);
+        build_edge_table<FWD>(tc, X, Xr, lane);
+#pragma unroll
+        for (int c = 0; c < CPT; ++c) {
+            const unsigned idx = id_at<CPT>(pu, c) * k + id_at<CPT>(pv, c);
+            const long long val = lu[c] + tc.T[idx];
+            best[c] = val > best[c] ? val : best[c];
+        }
+    }
+
+    if (!FWD && vm.e0 == vm.e1) {  // sink: blevel = own runtime
+#pragma unroll
+        for (int c = 0; c < CPT; ++c)
+            if (Xv != NUM_ZERO) best[c] = ceil_quot(Xv, tc.s_rt[id_at<CPT>(pv, c)]);
+    }
+    store_levels<CPT>(a.lev + (long long)v * ldp + lc.jl, best, lc.nvalid);
+    if (cp_vertex) {
+#pragma unroll
+        for (int c = 0; c < CPT; ++c) {
+            long long fin = best[c];
+            if (FWD && Xv != NUM_ZERO) fin += ceil_quot(Xv, tc.s_rt[id_at<CPT>(pv, c)]);
+            cpmax[c] = fin > cpmax[c] ? fin : cpmax[c];
+        }
     }
 }
 
@@ -176,21 +321,6 @@ __device__ __forceinline__ VertexMeta global_meta(const LevelAdj& adj, int pos)
     return vm;
 }
 
-// Lane bookkeeping shared by both pass kernels: first candidate of the lane,
-// how many of its CPT candidates are real, the mask that zeroes padding ids and
-// the (always in-bounds) column the lane loads from.
-template <int CPT>
-__device__ __forceinline__ void lane_setup(long long slice0, long long P, int lane, long long& jl, int& nvalid,
-                                           unsigned& idmask)
-{
-    const long long j0 = slice0 + (long long)lane * CPT;
-    long long rem = P - j0;
-    nvalid = rem >= CPT ? CPT : (rem > 0 ? (int)rem : 0);
-    jl = nvalid > 0 ? j0 : slice0;  // idle lanes shadow the slice's first lane and never store
-    idmask = nvalid >= 4 ? 0xffffffffu : ((1u << (8 * nvalid)) - 1u);
-    if (nvalid == 0) idmask = 0;
-}
-
 // ---- level-synchronous variant: one launch per level ----------------------------
 template <int CPT, bool FWD>
 __global__ void __launch_bounds__(128)
@@ -203,13 +333,12 @@ pass_level_kernel(PassArgs a, int pos0, int count)
     stage_tables(a.tab, s_w, s_rt);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, wpb = blockDim.x >> 5;
     const long long slice0 = (long long)blockIdx.x * 32 * CPT;
-    long long jl; int nvalid; unsigned idmask;
-    lane_setup<CPT>(slice0, a.P, lane, jl, nvalid, idmask);
+    const LaneCtx<CPT> lc = lane_setup<CPT>(slice0, a.P, lane);
     long long unused[CPT];
 #pragma unroll
     for (int c = 0; c < CPT; ++c) unused[c] = 0;
     for (int i = blockIdx.y * wpb + warp; i < count; i += gridDim.y * wpb)
-        relax_vertex<CPT, FWD>(a, s_w, s_rt, global_meta(a.adj, pos0 + i), jl, idmask, nvalid, false, unused);
+        relax_vertex<CPT, FWD>(a, s_w, s_rt, global_meta(a.adj, pos0 + i), lc, false, unused);
 }
 
 // ---- candidate-sliced persistent variant ---------------------------------------------
@@ -261,23 +390,63 @@ __device__ __forceinline__ void stage_chunk(const PassArgs& a, const int* __rest
     }
 }
 
-template <int CPT, bool FWD>
-__global__ void __launch_bounds__(256)
+// shared-memory bytes of the sliced kernel besides the two chunk buffers
+__host__ __device__ inline size_t sliced_tail_smem(int k, int npass, int warps, int cpt, bool table)
+{
+    size_t b = sizeof(DivConst) * (size_t)k;                       // s_rt
+    b += sizeof(long long) * (size_t)warps * 32 * cpt;             // s_cp
+    if (table) {
+        b += sizeof(DivConst) * (size_t)npass * 32;                // s_pair
+        b += sizeof(long long) * (size_t)warps * npass * 32;       // per-warp tables
+        b += sizeof(unsigned short) * (size_t)npass * 32;          // s_sel
+    } else {
+        b += sizeof(DivConst) * (size_t)k * k;                     // s_w
+    }
+    return b;
+}
+
+// largest block the sliced kernel may be launched with (bounds its registers per thread)
+template <int CPT, bool TABLE> struct SlicedBounds { static constexpr int THREADS = (TABLE && CPT <= 4) ? 1024 : 256; };
+
+template <int CPT, bool FWD, bool TABLE>
+__global__ void __launch_bounds__(SlicedBounds<CPT, TABLE>::THREADS)
 pass_sliced_kernel(PassArgs a, const int* __restrict__ vertf, const int4* __restrict__ chunks, int num_chunks, int src_end)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    ChunkBuf* bufs = reinterpret_cast<ChunkBuf*>(smem_raw);
-    DivConst* s_w = reinterpret_cast<DivConst*>(bufs + 2);
-    DivConst* s_rt = s_w + a.tab.k * a.tab.k;
-    long long* s_cp = reinterpret_cast<long long*>(s_rt + a.tab.k);  // [warps][32*CPT]
-    if (*a.status != 0) return;
-    stage_tables(a.tab, s_w, s_rt);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, wpb = blockDim.x >> 5;
+    const int k = a.tab.k;
+    const int npass = a.tab.npass;
+    ChunkBuf* bufs = reinterpret_cast<ChunkBuf*>(smem_raw);
+    DivConst* s_rt = reinterpret_cast<DivConst*>(bufs + 2);
+    long long* s_cp = reinterpret_cast<long long*>(s_rt + k);  // [warps][32*CPT]
+    unsigned char* tail = reinterpret_cast<unsigned char*>(s_cp + (size_t)wpb * 32 * CPT);
+    DivConst* s_w = reinterpret_cast<DivConst*>(tail);      // direct: [k*k]; table: pair table [npass*32]
+    if (*a.status != 0) return;
+
+    TableCtx tc;
+    if (TABLE) {
+        long long* s_T = reinterpret_cast<long long*>(s_w + npass * 32);
+        unsigned short* s_sel = reinterpret_cast<unsigned short*>(s_T + (size_t)wpb * npass * 32);
+        const DivConst* pair = FWD ? a.tab.pair_f : a.tab.pair_b;
+        const unsigned short* sel = FWD ? a.tab.sel_f : a.tab.sel_b;
+        for (int i = threadIdx.x; i < npass * 32; i += blockDim.x) { s_w[i] = pair[i]; s_sel[i] = sel[i]; }
+        tc.s_pair = s_w;
+        tc.s_rt = s_rt;
+        tc.s_sel = s_sel;
+        tc.T = s_T + (size_t)warp * npass * 32;
+        tc.my_cls = a.tab.cls_div[lane];
+        tc.npass = npass;
+        tc.use_cls = a.tab.use_cls;
+        tc.ncls_w = a.tab.ncls_w;
+    } else {
+        for (int i = threadIdx.x; i < k * k; i += blockDim.x) s_w[i] = a.tab.w_div[i];
+    }
+    for (int i = threadIdx.x; i < k; i += blockDim.x) s_rt[i] = a.tab.rt_div[i];
+
     const long long slice0 = (long long)blockIdx.x * 32 * CPT;
-    long long jl; int nvalid; unsigned idmask;
-    lane_setup<CPT>(slice0, a.P, lane, jl, nvalid, idmask);
+    const LaneCtx<CPT> lc = lane_setup<CPT>(slice0, a.P, lane);
     const bool want_cp = a.cp != nullptr;
-    long long cpmax[CPT];
+    long long* cpmax = s_cp + ((size_t)warp * 32 + lane) * CPT;   // this lane's running maxima
 #pragma unroll
     for (int c = 0; c < CPT; ++c) cpmax[c] = 0;
 
@@ -313,7 +482,8 @@ pass_sliced_kernel(PassArgs a, const int* __restrict__ vertf, const int4* __rest
             vm.xnbr = staged ? b.xnbr : a.adj.xnbr;
             bool cpv = false;
             if (want_cp) cpv = FWD ? (vf < 0) : (p0 + i < src_end);
-            relax_vertex<CPT, FWD>(a, s_w, s_rt, vm, jl, idmask, nvalid, cpv, cpmax);
+            if (TABLE) relax_vertex_table<CPT, FWD>(a, tc, vm, lc, lane, cpv, cpmax);
+            else relax_vertex<CPT, FWD>(a, s_w, s_rt, vm, lc, cpv, cpmax);
         }
         cp_async_wait_all();
         __syncthreads();
@@ -321,20 +491,15 @@ pass_sliced_kernel(PassArgs a, const int* __restrict__ vertf, const int4* __rest
         nxt = nxt2;
     }
 
-    if (want_cp) {
+    if (want_cp && warp == 0) {
 #pragma unroll
-        for (int c = 0; c < CPT; ++c) s_cp[(warp * 32 + lane) * CPT + c] = cpmax[c];
-        __syncthreads();
-        if (warp == 0) {
-#pragma unroll
-            for (int c = 0; c < CPT; ++c) {
-                long long m = cpmax[c];
-                for (int w = 1; w < wpb; ++w) {
-                    long long o = s_cp[(w * 32 + lane) * CPT + c];
-                    m = o > m ? o : m;
-                }
-                if (c < nvalid) a.cp[slice0 + (long long)lane * CPT + c] = m;
+        for (int c = 0; c < CPT; ++c) {
+            long long m = cpmax[c];
+            for (int w = 1; w < wpb; ++w) {
+                long long o = s_cp[((size_t)w * 32 + lane) * CPT + c];
+                m = o > m ? o : m;
             }
+            if (c < lc.nvalid) a.cp[slice0 + (long long)lane * CPT + c] = m;
         }
     }
 }
@@ -528,25 +693,36 @@ cudaError_t launch_pass_level_sync(const PassArgs& a, bool fwd, const std::vecto
     return fwd ? level_sync_impl<1, true>(a, lp, st) : level_sync_impl<1, false>(a, lp, st);
 }
 
-template <int CPT, bool FWD>
+template <int CPT, bool FWD, bool TABLE>
 static cudaError_t sliced_impl(const PassArgs& a, const SlicedPlan& plan, int warps, cudaStream_t st)
 {
-    const size_t smem = 2 * sizeof(ChunkBuf) + table_smem(a.tab.k) + sizeof(long long) * (size_t)warps * 32 * CPT;
-    cudaError_t e = allow_smem(pass_sliced_kernel<CPT, FWD>, smem);
+    if (warps * 32 > SlicedBounds<CPT, TABLE>::THREADS) warps = SlicedBounds<CPT, TABLE>::THREADS / 32;
+    const size_t smem = 2 * sizeof(ChunkBuf) + sliced_tail_smem(a.tab.k, a.tab.npass, warps, CPT, TABLE);
+    cudaError_t e = allow_smem(pass_sliced_kernel<CPT, FWD, TABLE>, smem);
     if (e != cudaSuccess) return e;
     const unsigned gx = cdivu(a.P, 32 * CPT);
-    pass_sliced_kernel<CPT, FWD><<<gx, warps * 32, smem, st>>>(a, plan.vertf, reinterpret_cast<const int4*>(plan.chunks),
-                                                                plan.num_chunks, plan.src_end);
+    pass_sliced_kernel<CPT, FWD, TABLE><<<gx, warps * 32, smem, st>>>(
+        a, plan.vertf, reinterpret_cast<const int4*>(plan.chunks), plan.num_chunks, plan.src_end);
     count_launches(1);
     return cudaGetLastError();
 }
 
-cudaError_t launch_pass_sliced(const PassArgs& a, bool fwd, const SlicedPlan& plan, int cpt, int warps, cudaStream_t st)
+template <int CPT>
+static cudaError_t sliced_dispatch(const PassArgs& a, bool fwd, bool table, const SlicedPlan& plan, int warps, cudaStream_t st)
+{
+    if (table) return fwd ? sliced_impl<CPT, true, true>(a, plan, warps, st) : sliced_impl<CPT, false, true>(a, plan, warps, st);
+    return fwd ? sliced_impl<CPT, true, false>(a, plan, warps, st) : sliced_impl<CPT, false, false>(a, plan, warps, st);
+}
+
+cudaError_t launch_pass_sliced(const PassArgs& a, bool fwd, const SlicedPlan& plan, int cpt, int warps, bool table,
+                               cudaStream_t st)
 {
     if (plan.num_chunks <= 0) return cudaSuccess;
-    if (cpt == 4) return fwd ? sliced_impl<4, true>(a, plan, warps, st) : sliced_impl<4, false>(a, plan, warps, st);
-    if (cpt == 2) return fwd ? sliced_impl<2, true>(a, plan, warps, st) : sliced_impl<2, false>(a, plan, warps, st);
-    return fwd ? sliced_impl<1, true>(a, plan, warps, st) : sliced_impl<1, false>(a, plan, warps, st);
+    if (a.tab.npass <= 0) table = false;
+    if (cpt == 8) return sliced_dispatch<8>(a, fwd, table, plan, warps, st);
+    if (cpt == 4) return sliced_dispatch<4>(a, fwd, table, plan, warps, st);
+    if (cpt == 2) return sliced_dispatch<2>(a, fwd, table, plan, warps, st);
+    return sliced_dispatch<1>(a, fwd, table, plan, warps, st);
 }
 
 cudaError_t launch_cp_reduce(const PassArgs& a, bool from_tlevel, const int* list, int list_len, cudaStream_t st)

@@ -331,3 +331,35 @@ def test_error_codes():
     out = G.eval_batch(part, 16)
     assert (out["cp"] > 0).all()
     G.close()
+
+
+# ------------------------------------------------------ kernel shapes of the sliced pass
+@pytest.mark.parametrize("table", [0, 1])
+@pytest.mark.parametrize("cpt", [1, 2, 4, 8])
+def test_sliced_kernel_shapes(cpt, table, monkeypatch):
+    """Every candidates-per-lane width, with the per-edge cost table on and off,
+    on device tables that exercise each table-building path: few distinct values
+    (classes), many distinct values with k*k <= 64 (per-entry division), k = 16
+    grouped (8 table passes) and k = 50 (no table: direct division)."""
+    monkeypatch.setenv("TFPS_SLICED_CPT", str(cpt))
+    monkeypatch.setenv("TFPS_SLICED_TABLE", str(table))
+    monkeypatch.setenv("TFPS_SLICED_WARPS", "4")
+    rng = np.random.default_rng(cpt * 2 + table)
+    cases = []
+    w = I.small_random(70 + cpt, 300, 900, 3, 77)          # classes, one pass
+    cases.append((w.graph, w.devices, w.part_full()))
+    w = I.small_random(80 + cpt, 400, 1300, 8, 300)        # 56 distinct bandwidths: per-entry division, two passes
+    cases.append((w.graph, w.devices, w.part_full()))
+    w = I.config5(layers=12, width=64, P=100)               # k = 16 grouped: classes, eight passes, fan-in up to 64
+    cases.append((w.graph, w.devices, w.part_full()))
+    w = I.paper_shaped(0)                                   # k = 50
+    cases.append((w.graph, w.devices, w.part_full()))
+    # a vertex with more in-edges than a staged chunk holds
+    n = 700
+    edges = [(u, n - 1, int(rng.integers(0, 10 ** 6))) for u in range(n - 1)] + [(0, u, 5) for u in range(1, 40)]
+    g = graph_from_edges(n, edges, rng.integers(0, 100, size=n))
+    dev = I.Devices(4, np.array([1, 2, 2, 4], np.int32), np.full(4, INF, np.int64),
+                    np.array([[0, 10, 10, 7], [10, 0, 7, 7], [3, 3, 0, 10], [7, 10, 3, 0]], np.int64), scale=3)
+    cases.append((g, dev, rng.integers(0, 4, size=(n, 45), dtype=np.uint8)))
+    for g, dev, part in cases:
+        run_and_compare(g, dev, part, 2, pad_fill=255)
