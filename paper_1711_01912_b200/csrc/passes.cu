@@ -5,6 +5,8 @@
 // Lane = candidate(s): a warp covers 32*CPT contiguous candidates of one
 // vertex, so every neighbour-level read is one contiguous 256*CPT-byte row
 // segment and every id read a contiguous 32*CPT-byte one.
+#include <cstdlib>
+
 #include "common.cuh"
 
 namespace tfps {
@@ -341,6 +343,99 @@ pass_level_kernel(PassArgs a, int pos0, int count)
         relax_vertex<CPT, FWD>(a, s_w, s_rt, global_meta(a.adj, pos0 + i), lc, false, unused);
 }
 
+// ---- level-synchronous tile variant (k <= TABLE_K_MAX) ---------------------------
+// One launch per level.  A block of TILE_WARPS warps takes ONE vertex and
+// TILE_WARPS*32*CPT candidates: the per-edge cost tables are built once per block
+// (warp w builds the table of edge w of the batch) and shared through shared
+// memory, so their cost is spread over the whole candidate tile.
+//
+// Launches are chained with programmatic dependent launch: a block first reads
+// what does not depend on the previous level (adjacency, partition ids) and
+// builds its tables, and only then waits for the previous level's grid before
+// it touches neighbour levels.  Every block executes the wait, so the completion
+// of a level's grid implies the completion of all earlier levels.
+constexpr int TILE_WARPS = 4;
+constexpr int TILE_EB = 4;  // edges per batch = tables resident per block
+
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <int CPT, bool FWD>
+__global__ void __launch_bounds__(TILE_WARPS * 32)
+pass_tile_kernel(PassArgs a, int pos0, int count)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    long long* s_T = reinterpret_cast<long long*>(smem_raw);  // [TILE_EB][npass*32]
+    grid_launch_dependents();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int k = a.tab.k;
+    const int tsz = a.tab.npass * 32;
+    const bool live = *a.status == 0;
+    TableCtx tc;
+    tc.s_pair = FWD ? a.tab.pair_f : a.tab.pair_b;
+    tc.s_rt = a.tab.rt_div;
+    tc.s_sel = FWD ? a.tab.sel_f : a.tab.sel_b;
+    tc.T = s_T + (size_t)warp * tsz;   // table slot this warp fills
+    tc.my_cls = a.tab.cls_div[lane];
+    tc.npass = a.tab.npass;
+    tc.use_cls = a.tab.use_cls;
+    tc.ncls_w = a.tab.ncls_w;
+    const long long slice0 = ((long long)blockIdx.x * TILE_WARPS + warp) * 32 * CPT;
+    const LaneCtx<CPT> lc = lane_setup<CPT>(slice0, a.P, lane);
+    const long long ldp = a.ldp;
+    bool waited = false;
+
+    for (int i = blockIdx.y; i < count && live; i += gridDim.y) {
+        const VertexMeta vm = global_meta(a.adj, pos0 + i);
+        unsigned pv[IdWords<CPT>::N];
+        load_ids_masked<CPT>(a.part + (long long)vm.v * ldp + lc.jl, lc, pv);
+        long long best[CPT];
+#pragma unroll
+        for (int c = 0; c < CPT; ++c) best[c] = 0;
+
+        for (int b0 = vm.e0; b0 < vm.e1; b0 += TILE_EB) {
+            const int nb = vm.e1 - b0 < TILE_EB ? vm.e1 - b0 : TILE_EB;
+            long long off[TILE_EB];
+            unsigned pu[TILE_EB][IdWords<CPT>::N];
+#pragma unroll
+            for (int q = 0; q < TILE_EB; ++q) {
+                if (q < nb) {
+                    off[q] = (long long)vm.nbr[b0 + q] * ldp + lc.jl;
+                    load_ids_masked<CPT>(a.part + off[q], lc, pu[q]);
+                }
+            }
+            if (b0 != vm.e0) __syncthreads();  // lookups of the previous batch are done
+            if (warp < nb) build_edge_table<FWD>(tc, vm.xw[b0 + warp], FWD ? vm.xnbr[b0 + warp] : vm.xvert, lane);
+            if (!waited) { grid_dependency_wait(); waited = true; }
+            long long lu[TILE_EB][CPT];
+#pragma unroll
+            for (int q = 0; q < TILE_EB; ++q)
+                if (q < nb) load_levels<CPT>(a.lev + off[q], lu[q]);
+            __syncthreads();  // tables of this batch are visible
+#pragma unroll
+            for (int q = 0; q < TILE_EB; ++q) {
+                if (q < nb) {
+                    const long long* T = s_T + (size_t)q * tsz;
+#pragma unroll
+                    for (int c = 0; c < CPT; ++c) {
+                        const long long val = lu[q][c] + T[id_at<CPT>(pu[q], c) * k + id_at<CPT>(pv, c)];
+                        best[c] = val > best[c] ? val : best[c];
+                    }
+                }
+            }
+        }
+        if (!FWD && vm.e0 == vm.e1) {  // sink: blevel = own runtime
+#pragma unroll
+            for (int c = 0; c < CPT; ++c)
+                if (vm.xvert != NUM_ZERO) best[c] = ceil_quot(vm.xvert, tc.s_rt[id_at<CPT>(pv, c)]);
+        }
+        if (!waited) { grid_dependency_wait(); waited = true; }
+        store_levels<CPT>(a.lev + (long long)vm.v * ldp + lc.jl, best, lc.nvalid);
+        if (i + (int)gridDim.y < count) __syncthreads();  // tables are reused by the next vertex
+    }
+    if (!waited) grid_dependency_wait();
+}
+
 // ---- candidate-sliced persistent variant ---------------------------------------------
 // One block owns 32*CPT candidates and walks the whole graph chunk by chunk; a
 // chunk is a run of at most CHUNK_V positions / CHUNK_E edges inside one level
@@ -560,24 +655,50 @@ __global__ void loads_kernel(int n, long long P, long long ldp, const uint8_t* _
     const long long j0 = slice0 + (long long)threadIdx.x * 4;
     const long long rem = P - j0;
     const int nvalid = rem >= 4 ? 4 : (rem > 0 ? (int)rem : 0);
-    if (nvalid == 0) return;
-    const int col = threadIdx.x * 4;
+    const long long jl = nvalid > 0 ? j0 : slice0;  // idle lanes keep the warp's shuffles company
+    const int lane = threadIdx.x & 31;
+    const int nthr = blockDim.x;  // accumulators are laid out [device][c][thread]: conflict-free columns
     const int r0 = blockIdx.y * rows_per_block;
     const int r1 = r0 + rows_per_block < n ? r0 + rows_per_block : n;
     bool bad = false;
-    for (int pos = r0; pos < r1; ++pos) {
-        const int v = vert[pos];
-        const unsigned long long Xv = xvert[pos];
-        const long long mv = mem[v];
-        const unsigned packed = *reinterpret_cast<const unsigned*>(part + (long long)v * ldp + j0);
+    constexpr int RB = 4;  // rows in flight
+    for (int pos = r0; pos < r1; pos += RB) {
+        unsigned long long Xv[RB];
+        long long mv[RB];
+        unsigned packed[RB];
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            if (c < nvalid) {
-                unsigned id = (packed >> (8 * c)) & 0xffu;
-                if (id >= (unsigned)k) { bad = true; id = 0; }
-                const long long rt = Xv != NUM_ZERO ? ceil_quot(Xv, s_rt[id]) : 0;
-                acc_l[id * bc + col + c] += rt;
-                acc_m[id * bc + col + c] += mv;
+        for (int q = 0; q < RB; ++q) {
+            if (pos + q < r1) {
+                const int v = vert[pos + q];
+                Xv[q] = xvert[pos + q];
+                mv[q] = mem[v];
+                packed[q] = *reinterpret_cast<const unsigned*>(part + (long long)v * ldp + jl);
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < RB; ++q) {
+            if (pos + q < r1) {
+                // runtime of this vertex on device `lane` (and lane+32): one division per device, not per candidate
+                long long row_lo = 0, row_hi = 0;
+                if (Xv[q] != NUM_ZERO) {
+                    if (lane < k) row_lo = ceil_quot(Xv[q], s_rt[lane]);
+                    if (k > 32 && lane + 32 < k) row_hi = ceil_quot(Xv[q], s_rt[lane + 32]);
+                }
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    unsigned id = (packed[q] >> (8 * c)) & 0xffu;
+                    if (c >= nvalid) id = 0;
+                    if (id >= (unsigned)k) { bad = true; id = 0; }
+                    long long rt = shfl64(row_lo, (int)(id & 31u));
+                    if (k > 32) {
+                        const long long hi = shfl64(row_hi, (int)(id & 31u));
+                        rt = id >= 32u ? hi : rt;
+                    }
+                    if (c < nvalid) {
+                        acc_l[(id * 4 + c) * nthr + threadIdx.x] += rt;
+                        acc_m[(id * 4 + c) * nthr + threadIdx.x] += mv[q];
+                    }
+                }
             }
         }
     }
@@ -587,9 +708,9 @@ __global__ void loads_kernel(int n, long long P, long long ldp, const uint8_t* _
         for (int c = 0; c < 4; ++c) {
             if (c < nvalid) {
                 if (load) atomicAdd(reinterpret_cast<unsigned long long*>(load + d * ldp + j0 + c),
-                                    (unsigned long long)acc_l[d * bc + col + c]);
+                                    (unsigned long long)acc_l[(d * 4 + c) * nthr + threadIdx.x]);
                 if (memload) atomicAdd(reinterpret_cast<unsigned long long*>(memload + d * ldp + j0 + c),
-                                       (unsigned long long)acc_m[d * bc + col + c]);
+                                       (unsigned long long)acc_m[(d * 4 + c) * nthr + threadIdx.x]);
             }
         }
     }
@@ -686,8 +807,51 @@ static cudaError_t level_sync_impl(const PassArgs& a, const std::vector<long lon
     return cudaGetLastError();
 }
 
+template <int CPT, bool FWD>
+static cudaError_t tile_impl(const PassArgs& a, const std::vector<long long>& lp, cudaStream_t st)
+{
+    const size_t smem = sizeof(long long) * (size_t)TILE_EB * a.tab.npass * 32;
+    cudaError_t e = allow_smem(pass_tile_kernel<CPT, FWD>, smem);
+    if (e != cudaSuccess) return e;
+    const unsigned gx = cdivu(a.P, TILE_WARPS * 32 * CPT);
+    const int L = a.num_levels;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    for (int step = 0; step < L; ++step) {
+        const int l = FWD ? step : L - 1 - step;
+        const int pos0 = (int)lp[l];
+        const int count = (int)(lp[l + 1] - lp[l]);
+        unsigned gy = (unsigned)count;
+        if (gy > 65535u) gy = 65535u;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(gx, gy);
+        cfg.blockDim = dim3(TILE_WARPS * 32);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = st;
+        cfg.attrs = attr;
+        cfg.numAttrs = step == 0 ? 0 : 1;  // the first level follows ordinary stream order
+        e = cudaLaunchKernelEx(&cfg, pass_tile_kernel<CPT, FWD>, a, pos0, count);
+        if (e != cudaSuccess) return e;
+    }
+    count_launches(L);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_pass_level_sync(const PassArgs& a, bool fwd, const std::vector<long long>& lp, cudaStream_t st)
 {
+    if (a.tab.npass > 0) {  // block-shared cost tables
+        const char* ov = getenv("TFPS_TILE_CPT");  // tuning override
+        if (ov && *ov == '4') return fwd ? tile_impl<4, true>(a, lp, st) : tile_impl<4, false>(a, lp, st);
+        if (ov && *ov == '2') return fwd ? tile_impl<2, true>(a, lp, st) : tile_impl<2, false>(a, lp, st);
+        if (ov && *ov == '1') return fwd ? tile_impl<1, true>(a, lp, st) : tile_impl<1, false>(a, lp, st);
+        const long long tiles4 = (a.P + TILE_WARPS * 32 * 4 - 1) / (TILE_WARPS * 32 * 4);
+        const long long width = a.num_levels > 0 ? a.n / a.num_levels : a.n;
+        if (tiles4 * width >= 2048 || a.P >= 4096)
+            return fwd ? tile_impl<4, true>(a, lp, st) : tile_impl<4, false>(a, lp, st);
+        if (a.P >= 256) return fwd ? tile_impl<2, true>(a, lp, st) : tile_impl<2, false>(a, lp, st);
+        return fwd ? tile_impl<1, true>(a, lp, st) : tile_impl<1, false>(a, lp, st);
+    }
     const int cpt = pick_cpt(a.P);
     if (cpt == 2) return fwd ? level_sync_impl<2, true>(a, lp, st) : level_sync_impl<2, false>(a, lp, st);
     return fwd ? level_sync_impl<1, true>(a, lp, st) : level_sync_impl<1, false>(a, lp, st);
@@ -753,7 +917,7 @@ cudaError_t launch_loads(int n, long long P, long long ldp, const uint8_t* part,
     cudaError_t e = allow_smem(loads_kernel, smem);
     if (e != cudaSuccess) return e;
     const unsigned gx = cdivu(P, threads * 4);
-    long long want_blocks = (long long)sm_count * 8;
+    long long want_blocks = (long long)sm_count * 32;
     long long gy = (want_blocks + gx - 1) / gx;
     if (gy < 1) gy = 1;
     if (gy > n) gy = n;
