@@ -116,6 +116,9 @@ struct tfps_graph {
     long long S = 0;
     DBuf rt_div, w_div, cap, xvert, xw_f, xnbr_f, xw_b;
     DBuf pair_f, pair_b, cls_div, sel_f, sel_b;
+    // windowed pass: neighbour positions, comb tables, precomputed edge values
+    DBuf pos_of, npos_f, npos_b, cls2_f, cls2_b, comb_f, comb_b, V_f, V_b;
+    int ncomb = 0, maxspan = 0, smem_optin = 0;
     int npass = 0, use_cls = 0, ncls_w = 0;
     DBuf status;
     // scratch owned by the handle
@@ -235,6 +238,18 @@ int build_topo(tfps_graph* g, cudaStream_t st)
                               g->in_t.as<long long>(), g->f_eptr.as<int>(), g->f_nbr.as<int>(), g->f_t.as<long long>(), st));
     CUDA_TRY(launch_build_adj(n, g->order.as<int>(), g->out_ptr.as<long long>(), g->out_dst.as<int>(),
                               g->out_t.as<long long>(), g->b_eptr.as<int>(), g->b_nbr.as<int>(), g->b_t.as<long long>(), st));
+    {
+        DBuf span;
+        CUDA_TRY(span.alloc(sizeof(int)));
+        CUDA_TRY(cudaMemsetAsync(span.p, 0, sizeof(int), st));
+        CUDA_TRY(g->pos_of.alloc(sizeof(int) * (size_t)n));
+        CUDA_TRY(g->npos_f.alloc(sizeof(int) * (size_t)m));
+        CUDA_TRY(g->npos_b.alloc(sizeof(int) * (size_t)m));
+        CUDA_TRY(launch_positions(n, m, g->order.as<int>(), g->pos_of.as<int>(), g->f_nbr.as<int>(), g->b_nbr.as<int>(),
+                                  g->f_eptr.as<int>(), g->npos_f.as<int>(), g->npos_b.as<int>(), span.as<int>(), st));
+        CUDA_TRY(cudaMemcpyAsync(&g->maxspan, span.p, sizeof(int), cudaMemcpyDeviceToHost, st));
+        CUDA_TRY(cudaStreamSynchronize(st));
+    }
     CUDA_TRY(g->sink_flag.alloc((size_t)n));
     CUDA_TRY(launch_sink_flags(n, g->order.as<int>(), g->out_ptr.as<long long>(), g->sink_flag.as<uint8_t>(), st));
     std::vector<uint8_t> flags((size_t)n);
@@ -446,6 +461,7 @@ int tfps_graph_create(tfps_graph** out, int64_t n, int64_t m,
 
     CUDA_TRY(cudaGetDevice(&g->device));
     CUDA_TRY(cudaDeviceGetAttribute(&g->sm_count, cudaDevAttrMultiProcessorCount, g->device));
+    CUDA_TRY(cudaDeviceGetAttribute(&g->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, g->device));
     g->n = n;
     g->m = m;
     TFPS_TRY(upload(g->in_ptr, h_in_ptr, st));
@@ -578,6 +594,46 @@ int tfps_devices_set(tfps_graph* g, int k, const int32_t* s, const int64_t* C, c
         TFPS_TRY(upload(g->cls_div, cls, st));
         TFPS_TRY(upload(g->sel_f, sf, st));
         TFPS_TRY(upload(g->sel_b, sb, st));
+
+        // comb ids for the windowed pass: (transfer class or "same device", speed class), or the pair itself
+        const int ncs = (int)svals.size();
+        int ncomb = 0;
+        const bool by_class = use_cls && (ncw + 1) * ncs <= COMB_MAX;
+        if (by_class) ncomb = (ncw + 1) * ncs;
+        else if (k * k <= COMB_MAX) ncomb = k * k;
+        g->ncomb = ncomb;
+        if (ncomb > 0) {
+            std::vector<uint8_t> c2f((size_t)k * k), c2b((size_t)k * k);
+            std::vector<CombDiv> cf((size_t)COMB_MAX), cb((size_t)COMB_MAX);
+            const DivConst none = DivConst{0ull, 0u, 1u};
+            for (auto& x : cf) { x.w = none; x.s = make_div(1); }
+            for (auto& x : cb) { x.w = none; x.s = make_div(1); }
+            for (int nb = 0; nb < k; ++nb)
+                for (int vv = 0; vv < k; ++vv) {
+                    const int i = nb * k + vv;
+                    const bool same = nb == vv;
+                    const long long bf = same ? 0 : B[nb * k + vv], bb = same ? 0 : B[vv * k + nb];
+                    int idf, idb;
+                    if (by_class) {
+                        idf = (same ? ncw : cls_of(wvals, bf)) * ncs + cls_of(svals, s[nb]);
+                        idb = (same ? ncw : cls_of(wvals, bb)) * ncs + cls_of(svals, s[vv]);
+                    } else {
+                        idf = idb = i;
+                    }
+                    c2f[i] = (uint8_t)idf;
+                    c2b[i] = (uint8_t)idb;
+                    cf[idf].w = same ? none : make_div((unsigned long long)bf);
+                    cf[idf].s = make_div((unsigned long long)s[nb]);
+                    cb[idb].w = same ? none : make_div((unsigned long long)bb);
+                    cb[idb].s = make_div((unsigned long long)s[vv]);
+                }
+            TFPS_TRY(upload(g->cls2_f, c2f, st));
+            TFPS_TRY(upload(g->cls2_b, c2b, st));
+            TFPS_TRY(upload(g->comb_f, cf, st));
+            TFPS_TRY(upload(g->comb_b, cb, st));
+        }
+    } else {
+        g->ncomb = 0;
     }
     TFPS_TRY(upload(g->rt_div, rt, st));
     TFPS_TRY(upload(g->w_div, w, st));
@@ -592,6 +648,16 @@ int tfps_devices_set(tfps_graph* g, int k, const int32_t* s, const int64_t* C, c
                                    g->f_t.as<long long>(), g->b_nbr.as<int>(), g->b_t.as<long long>(),
                                    g->xvert.as<unsigned long long>(), g->xw_f.as<unsigned long long>(),
                                    g->xnbr_f.as<unsigned long long>(), g->xw_b.as<unsigned long long>(), st));
+    if (g->ncomb > 0 && n > 0) {
+        CUDA_TRY(g->V_f.reserve(sizeof(long long) * (size_t)m * g->ncomb + 16));
+        CUDA_TRY(g->V_b.reserve(sizeof(long long) * (size_t)m * g->ncomb + 16));
+        CUDA_TRY(launch_edge_values(n, g->f_eptr.as<int>(), g->xw_f.as<unsigned long long>(),
+                                    g->xnbr_f.as<unsigned long long>(), g->xvert.as<unsigned long long>(),
+                                    g->comb_f.as<CombDiv>(), g->ncomb, g->V_f.as<long long>(), st));
+        CUDA_TRY(launch_edge_values(n, g->b_eptr.as<int>(), g->xw_b.as<unsigned long long>(), nullptr,
+                                    g->xvert.as<unsigned long long>(), g->comb_b.as<CombDiv>(), g->ncomb,
+                                    g->V_b.as<long long>(), st));
+    }
     CUDA_TRY(cudaStreamSynchronize(st));
     g->k = k;
     g->S = scale;
@@ -713,6 +779,34 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
     }
 
     if (profile) CUDA_TRY(cudaEventRecord(g->ev[1], st));
+    // windowed pass: needs the precomputed edge values (simple device tables)
+    bool use_window = sliced && g->ncomb > 0 && env_int("TFPS_WINDOW", 1) != 0;
+    int win_R = 0;
+    if (use_window) {
+        const int r_need = (g->maxspan + CHUNK_V + 31) / 32 * 32;
+        auto r_fit = [&](int c) {
+            const long long avail = (long long)g->smem_optin - 1024 - (long long)window_smem_bytes(k, g->ncomb, 0, c, warps);
+            long long r = avail / (32LL * c * 9) / 32 * 32;
+            if (r > (1 << 13)) r = 1 << 13;
+            return (int)(r < 0 ? 0 : r);
+        };
+        const int forced = env_int("TFPS_SLICED_CPT", 0);
+        int chosen = 0;
+        if (forced == 1 || forced == 2 || forced == 4) chosen = forced;
+        else {
+            const long long want_slices = std::min<long long>((3LL * g->sm_count) / 4, (P + 31) / 32);
+            for (int c = 4; c >= 1 && !chosen; c >>= 1)      // widest lane that still holds the whole window
+                if (r_fit(c) >= r_need && (P + 32 * c - 1) / (32 * c) >= want_slices) chosen = c;
+            if (!chosen) chosen = cpt > 4 ? 4 : cpt;          // partial window at the width the slice count allows
+        }
+        cpt = chosen;
+        win_R = std::min(r_fit(cpt), r_need);
+        const int forced_r = env_int("TFPS_WINDOW_R", -1);
+        if (forced_r >= 0) win_R = std::min(forced_r / 32 * 32, r_fit(cpt));
+        if (win_R < CHUNK_V + 32) win_R = 0;
+        if (window_smem_bytes(k, g->ncomb, win_R, cpt, warps) > (size_t)g->smem_optin) use_window = false;
+    }
+
     for (int pass = 0; pass < 2; ++pass) {
         const bool fwd = pass == 0;
         if (profile && !fwd) CUDA_TRY(cudaEventRecord(g->ev[2], st));
@@ -720,7 +814,20 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
         long long* lev = fwd ? fwd_lev : (long long*)blevel;
         long long* cp_here = (cp && (fwd || !need_fwd)) ? (long long*)cp : nullptr;
         PassArgs a = make_args(g, fwd, P, ldp, part, lev, cp_here);
-        if (sliced) {
+        if (use_window) {
+            WindowPlan wp;
+            wp.vertf = g->vertf.as<int>();
+            wp.chunks = fwd ? g->f_chunks.as<int>() : g->b_chunks.as<int>();
+            wp.num_chunks = fwd ? g->f_num_chunks : g->b_num_chunks;
+            wp.src_end = (int)g->h_level_ptr[1];
+            wp.npos = fwd ? g->npos_f.as<int>() : g->npos_b.as<int>();
+            wp.V = fwd ? g->V_f.as<long long>() : g->V_b.as<long long>();
+            wp.cls2 = fwd ? g->cls2_f.as<uint8_t>() : g->cls2_b.as<uint8_t>();
+            wp.ncomb = g->ncomb;
+            wp.R = win_R;
+            wp.rmagic = win_R > 0 ? (((1ull << 40) + (unsigned long long)win_R - 1) / (unsigned long long)win_R) : 0ull;
+            CUDA_TRY(launch_pass_window(a, fwd, wp, cpt, warps, st));
+        } else if (sliced) {
             SlicedPlan plan;
             plan.vertf = g->vertf.as<int>();
             plan.chunks = fwd ? g->f_chunks.as<int>() : g->b_chunks.as<int>();

@@ -30,6 +30,14 @@ static_assert(sizeof(DivConst) == 16, "DivConst is loaded as one 16-byte word");
 
 constexpr unsigned long long NUM_ZERO = ~0ull;
 
+#ifdef __CUDACC__
+// ceil(a/d) for the stored numerator X = (a-1)<<2 of a positive a
+__device__ __forceinline__ long long ceil_quot(unsigned long long X, const DivConst& dc)
+{
+    return 1 + (long long)(__umul64hi(dc.mul, X) >> dc.sh);
+}
+#endif
+
 // Device tables set by tfps_devices_set (global memory; kernels stage them in
 // shared memory).  rt_div[d] divides by s_d, w_div[a*k+b] by B[a][b].
 //
@@ -90,13 +98,38 @@ struct PassArgs {
 // level with at most CHUNK_V vertices and CHUNK_E edges (a single vertex with more
 // edges forms a chunk of its own and is read straight from global memory).
 constexpr int CHUNK_V = 128;
-constexpr int CHUNK_E = 512;
+constexpr int CHUNK_E = 256;
 
 struct SlicedPlan {
     const int* vertf;    // [n] vertex id by position, bit 31 set for sinks
     const int* chunks;   // [num_chunks][4] = {first position, vertices, first edge, edges}
     int num_chunks;
     int src_end;         // positions below this are sources (level 0)
+};
+
+// Precomputed edge values for the windowed pass.  When the device tables are
+// simple enough the cost of an edge takes at most COMB_MAX distinct values over
+// all (neighbour device, vertex device) pairs: comb id = cls2[nb*k+vv], and
+// V[e*ncomb + c] holds the cost of edge e for comb c (same meaning as the table
+// T of the sliced pass), filled once per tfps_devices_set.
+constexpr int COMB_MAX = 16;
+
+struct CombDiv {
+    DivConst w;   // transfer divisor; w.pad != 0: no transfer term (same device)
+    DivConst s;   // speed divisor
+};
+
+struct WindowPlan {
+    const int* vertf;            // [n] vertex id by position, bit 31 set for sinks
+    const int* chunks;           // [num_chunks][4]
+    int num_chunks;
+    int src_end;
+    const int* npos;             // [m] position of the neighbour (level-ordered adjacency of this direction)
+    const long long* V;          // [m][ncomb]
+    const uint8_t* cls2;         // [k*k] comb id of (nb, vv)
+    int ncomb;
+    int R;                       // window length in positions (0: no window), multiple of 32
+    unsigned long long rmagic;   // floor(x / R) == (x * rmagic) >> 40 for x < 2^26
 };
 
 // every kernel launch of the library goes through the wrappers below and is counted here
@@ -120,6 +153,13 @@ int pick_cpt(long long P);
 cudaError_t launch_pass_level_sync(const PassArgs& a, bool fwd, const std::vector<long long>& level_ptr_host, cudaStream_t st);
 cudaError_t launch_pass_sliced(const PassArgs& a, bool fwd, const SlicedPlan& plan, int cpt, int warps, bool table,
                                cudaStream_t st);
+cudaError_t launch_pass_window(const PassArgs& a, bool fwd, const WindowPlan& plan, int cpt, int warps, cudaStream_t st);
+size_t window_smem_bytes(int k, int ncomb, int R, int cpt, int warps);
+cudaError_t launch_edge_values(int n, const int* eptr, const unsigned long long* xw, const unsigned long long* xnbr,
+                               const unsigned long long* xvert, const CombDiv* comb, int ncomb, long long* V,
+                               cudaStream_t st);
+cudaError_t launch_positions(int n, int m, const int* order, int* pos_of, const int* nbr_f, const int* nbr_b,
+                             const int* eptr_f, int* npos_f, int* npos_b, int* maxspan, cudaStream_t st);
 cudaError_t launch_vertf(int n, const int* order, const uint8_t* sink_flag, int* vertf, cudaStream_t st);
 cudaError_t launch_cp_reduce(const PassArgs& a, bool from_tlevel, const int* list, int list_len, cudaStream_t st);
 cudaError_t launch_loads(int n, long long P, long long ldp, const uint8_t* part, const int* vert,

@@ -71,11 +71,6 @@ __device__ __forceinline__ void store_levels(long long* p, const long long (&v)[
     }
 }
 
-__device__ __forceinline__ long long ceil_quot(unsigned long long X, const DivConst& dc)
-{
-    return 1 + (long long)(__umul64hi(dc.mul, X) >> dc.sh);
-}
-
 __device__ __forceinline__ long long shfl64(long long v, int src)
 {
     int lo = __shfl_sync(FULL, (int)(unsigned)(unsigned long long)v, src);

@@ -1,0 +1,406 @@
+// Windowed candidate-sliced pass.  Like the sliced pass, one block owns 32*CPT
+// candidates and walks the whole graph chunk by chunk with one block barrier
+// per chunk.  In addition the block keeps the levels and ids of the last R
+// positions of ITS OWN candidates in a shared-memory ring: a neighbour that lies
+// within the window is read from shared memory, so the dependent chain of a
+// vertex never leaves the SM and the neighbour never touches L2; only the
+// compulsory traffic (one id read, one level write per vertex-candidate)
+// reaches global memory.  Neighbours outside the window are read from global
+// memory as in the sliced pass.  Edge costs come from the precomputed value
+// array V (see WindowPlan): one shuffle per candidate replaces the per-edge
+// table build.  Adjacency, edge values and the id rows of coming chunks are
+// staged with cp.async one to two chunks ahead.
+#include "common.cuh"
+
+namespace tfps {
+
+namespace {
+
+constexpr unsigned FULL = 0xffffffffu;
+
+__device__ __forceinline__ void cp_async4(void* smem, const void* g)
+{
+    unsigned s = (unsigned)__cvta_generic_to_shared(smem);
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(s), "l"(g));
+}
+__device__ __forceinline__ void cp_async8(void* smem, const void* g)
+{
+    unsigned s = (unsigned)__cvta_generic_to_shared(smem);
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(s), "l"(g));
+}
+__device__ __forceinline__ void cp_async16(void* smem, const void* g)
+{
+    unsigned s = (unsigned)__cvta_generic_to_shared(smem);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(s), "l"(g));
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+
+__device__ __forceinline__ long long shfl64(long long v, int src)
+{
+    int lo = __shfl_sync(FULL, (int)(unsigned)(unsigned long long)v, src);
+    int hi = __shfl_sync(FULL, (int)((unsigned long long)v >> 32), src);
+    return (long long)(((unsigned long long)(unsigned)hi << 32) | (unsigned)lo);
+}
+
+template <int CPT> struct IdWords { static constexpr int N = (CPT + 3) / 4; };
+
+template <int CPT>
+__device__ __forceinline__ void load_ids(const uint8_t* p, unsigned (&w)[IdWords<CPT>::N])
+{
+    if constexpr (CPT == 1) w[0] = *p;
+    else if constexpr (CPT == 2) w[0] = *reinterpret_cast<const unsigned short*>(p);
+    else w[0] = *reinterpret_cast<const unsigned*>(p);
+}
+template <int CPT>
+__device__ __forceinline__ void store_ids(uint8_t* p, const unsigned (&w)[IdWords<CPT>::N])
+{
+    if constexpr (CPT == 1) *p = (uint8_t)w[0];
+    else if constexpr (CPT == 2) *reinterpret_cast<unsigned short*>(p) = (unsigned short)w[0];
+    else *reinterpret_cast<unsigned*>(p) = w[0];
+}
+template <int CPT>
+__device__ __forceinline__ unsigned id_at(const unsigned (&w)[IdWords<CPT>::N], int c)
+{
+    return (w[c >> 2] >> (8 * (c & 3))) & 0xffu;
+}
+template <int CPT>
+__device__ __forceinline__ void load_levels(const long long* p, long long (&out)[CPT])
+{
+    if constexpr (CPT == 1) {
+        out[0] = *p;
+    } else {
+#pragma unroll
+        for (int i = 0; i < CPT; i += 2) {
+            longlong2 v = *reinterpret_cast<const longlong2*>(p + i);
+            out[i] = v.x;
+            out[i + 1] = v.y;
+        }
+    }
+}
+template <int CPT>
+__device__ __forceinline__ void store_levels(long long* p, const long long (&v)[CPT])
+{
+    if constexpr (CPT == 1) {
+        *p = v[0];
+    } else {
+#pragma unroll
+        for (int i = 0; i < CPT; i += 2) *reinterpret_cast<longlong2*>(p + i) = make_longlong2(v[i], v[i + 1]);
+    }
+}
+
+struct HeadBuf {                 // per-vertex metadata of a chunk
+    unsigned long long xvert[CHUNK_V];
+    int vertf[CHUNK_V];
+    int eoff[CHUNK_V + 4];
+};
+
+// shared-memory carve-up (all offsets multiples of 16 bytes)
+struct Carve {
+    size_t head, edge_nbr, edge_npos, edge_V, ids, rt, cls2, cp, win_lev, win_id, total;
+    size_t edge_stride, ids_stride;
+};
+
+__host__ __device__ inline size_t up16(size_t x) { return (x + 15) & ~(size_t)15; }
+
+__host__ __device__ inline Carve carve(int k, int ncomb, int R, int cpt, int warps)
+{
+    Carve c;
+    const size_t slice = 32 * (size_t)cpt;
+    size_t o = 0;
+    c.head = o; o += 3 * up16(sizeof(HeadBuf));
+    c.edge_nbr = o;
+    c.edge_npos = c.edge_nbr + up16(sizeof(int) * CHUNK_E);
+    c.edge_V = c.edge_npos + up16(sizeof(int) * CHUNK_E);
+    c.edge_stride = (c.edge_V - c.edge_nbr) + up16(sizeof(long long) * CHUNK_E * (size_t)ncomb);
+    o += 2 * c.edge_stride;
+    c.ids = o; c.ids_stride = up16(CHUNK_V * slice); o += 2 * c.ids_stride;
+    c.rt = o; o += up16(sizeof(DivConst) * (size_t)k);
+    c.cls2 = o; o += up16((size_t)k * k);
+    c.cp = o; o += up16(sizeof(long long) * (size_t)warps * slice);
+    c.win_lev = o; o += up16(sizeof(long long) * (size_t)R * slice);
+    c.win_id = o; o += up16((size_t)R * slice);
+    c.total = o;
+    return c;
+}
+
+template <int CPT, bool FWD>
+__global__ void __launch_bounds__(1024)
+pass_window_kernel(PassArgs a, WindowPlan wp)
+{
+    extern __shared__ __align__(16) unsigned char smem[];
+    constexpr int SLICE = 32 * CPT;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, wpb = blockDim.x >> 5;
+    const int k = a.tab.k;
+    const int ncomb = wp.ncomb;
+    const int R = wp.R;
+    const Carve cv = carve(k, ncomb, R, CPT, wpb);
+    DivConst* s_rt = reinterpret_cast<DivConst*>(smem + cv.rt);
+    uint8_t* s_cls2 = smem + cv.cls2;
+    long long* s_cp = reinterpret_cast<long long*>(smem + cv.cp);
+    long long* win_lev = reinterpret_cast<long long*>(smem + cv.win_lev);
+    uint8_t* win_id = smem + cv.win_id;
+    if (*a.status != 0) return;
+    for (int i = threadIdx.x; i < k; i += blockDim.x) s_rt[i] = a.tab.rt_div[i];
+    for (int i = threadIdx.x; i < k * k; i += blockDim.x) s_cls2[i] = wp.cls2[i];
+
+    const long long slice0 = (long long)blockIdx.x * SLICE;
+    const long long j0 = slice0 + (long long)lane * CPT;
+    const long long rem = a.P - j0;
+    const int nvalid = rem >= CPT ? CPT : (rem > 0 ? (int)rem : 0);
+    const long long jl = nvalid > 0 ? j0 : slice0;
+    unsigned idmask = nvalid >= 4 ? 0xffffffffu : (nvalid > 0 ? ((1u << (8 * nvalid)) - 1u) : 0u);
+    const long long ldp = a.ldp;
+    // the slice's id bytes that exist in the row: the last slice may reach beyond ldp
+    const int slice_bytes = (int)((ldp - slice0) < SLICE ? (ldp - slice0) : SLICE);
+    const bool want_cp = a.cp != nullptr;
+    long long* cpmax = s_cp + ((size_t)warp * 32 + lane) * CPT;
+#pragma unroll
+    for (int c = 0; c < CPT; ++c) cpmax[c] = 0;
+
+    const int4* chunks = reinterpret_cast<const int4*>(wp.chunks);
+    const int num_chunks = wp.num_chunks;
+    auto entry = [&](int ci) { return chunks[FWD ? ci : num_chunks - 1 - ci]; };
+    auto head = [&](int ci) -> HeadBuf& { return *reinterpret_cast<HeadBuf*>(smem + cv.head + (size_t)(ci % 3) * up16(sizeof(HeadBuf))); };
+    auto stage_head = [&](int4 ent, HeadBuf& h) {
+        const int p0 = ent.x, cnt = ent.y;
+        for (int i = threadIdx.x; i < cnt; i += blockDim.x) {
+            cp_async4(&h.vertf[i], wp.vertf + p0 + i);
+            cp_async8(&h.xvert[i], a.adj.xvert + p0 + i);
+        }
+        for (int i = threadIdx.x; i <= cnt; i += blockDim.x) cp_async4(&h.eoff[i], a.adj.eptr + p0 + i);
+    };
+    auto stage_edges = [&](int4 ent, int slot) {
+        const int e0 = ent.z, ecnt = ent.w;
+        if (ecnt > CHUNK_E) return;  // read from global memory instead
+        unsigned char* base = smem + cv.edge_nbr + (size_t)slot * cv.edge_stride;
+        int* nbr = reinterpret_cast<int*>(base);
+        int* npos = reinterpret_cast<int*>(base + (cv.edge_npos - cv.edge_nbr));
+        long long* V = reinterpret_cast<long long*>(base + (cv.edge_V - cv.edge_nbr));
+        for (int i = threadIdx.x; i < ecnt; i += blockDim.x) {
+            cp_async4(&nbr[i], a.adj.nbr + e0 + i);
+            cp_async4(&npos[i], wp.npos + e0 + i);
+        }
+        const long long* Vg = wp.V + (long long)e0 * ncomb;
+        for (int i = threadIdx.x; i < ecnt * ncomb; i += blockDim.x) cp_async8(&V[i], Vg + i);
+    };
+    auto stage_ids = [&](int4 ent, const HeadBuf& h, int slot) {
+        const int cnt = ent.y;
+        uint8_t* dst = smem + cv.ids + (size_t)slot * cv.ids_stride;
+        const int per_row = slice_bytes / 16;  // ldp and slice0 are multiples of 16
+        for (int i = threadIdx.x; i < cnt * per_row; i += blockDim.x) {
+            const int r = i / per_row, q = i - r * per_row;
+            const int v = h.vertf[r] & 0x7fffffff;
+            cp_async16(dst + (size_t)r * SLICE + 16 * q, a.part + (long long)v * ldp + slice0 + 16 * q);
+        }
+    };
+
+    int4 cur = entry(0);
+    int4 nxt = num_chunks > 1 ? entry(1) : cur;
+    int4 nxt2 = num_chunks > 2 ? entry(2) : cur;
+    stage_head(cur, head(0));
+    if (num_chunks > 1) stage_head(nxt, head(1));
+    stage_edges(cur, 0);
+    cp_async_commit();
+    cp_async_wait_all();
+    __syncthreads();
+    stage_ids(cur, head(0), 0);
+    cp_async_commit();
+    cp_async_wait_all();
+    __syncthreads();
+
+    for (int ci = 0; ci < num_chunks; ++ci) {
+        int4 nxt3 = nxt2;
+        if (ci + 1 < num_chunks) {
+            stage_ids(nxt, head(ci + 1), (ci + 1) & 1);
+            stage_edges(nxt, (ci + 1) & 1);
+            if (ci + 2 < num_chunks) {
+                stage_head(nxt2, head(ci + 2));
+                if (ci + 3 < num_chunks) nxt3 = entry(ci + 3);
+            }
+            cp_async_commit();
+        }
+        const HeadBuf& h = head(ci);
+        const int p0 = cur.x, cnt = cur.y, e0 = cur.z;
+        const bool staged = cur.w <= CHUNK_E;
+        const unsigned char* ebase = smem + cv.edge_nbr + (size_t)(ci & 1) * cv.edge_stride;
+        const int* nbr = staged ? reinterpret_cast<const int*>(ebase) : a.adj.nbr;
+        const int* npos = staged ? reinterpret_cast<const int*>(ebase + (cv.edge_npos - cv.edge_nbr)) : wp.npos;
+        const long long* V = staged ? reinterpret_cast<const long long*>(ebase + (cv.edge_V - cv.edge_nbr)) : wp.V;
+        const int ebias = staged ? e0 : 0;
+        const uint8_t* idrows = smem + cv.ids + (size_t)(ci & 1) * cv.ids_stride;
+
+        for (int i = warp; i < cnt; i += wpb) {
+            const int vf = h.vertf[i];
+            const int v = vf & 0x7fffffff;
+            const int pos = p0 + i;
+            unsigned pv[IdWords<CPT>::N];
+            load_ids<CPT>(idrows + (size_t)i * SLICE + (jl - slice0), pv);
+            pv[0] &= idmask;
+            long long best[CPT];
+#pragma unroll
+            for (int c = 0; c < CPT; ++c) best[c] = 0;
+            const int ea = h.eoff[i] - ebias, eb = h.eoff[i + 1] - ebias;
+            for (int e = ea; e < eb; ++e) {
+                const int np = npos[e];
+                const int span = FWD ? pos - np : np - pos;
+                long long lu[CPT];
+                unsigned pu[IdWords<CPT>::N];
+                if (span <= R - CHUNK_V) {
+                    const int slot = np - R * (int)(((unsigned long long)np * wp.rmagic) >> 40);
+                    load_levels<CPT>(win_lev + (size_t)slot * SLICE + lane * CPT, lu);
+                    load_ids<CPT>(win_id + (size_t)slot * SLICE + lane * CPT, pu);
+                } else {
+                    const long long off = (long long)nbr[e] * ldp + jl;
+                    load_levels<CPT>(a.lev + off, lu);
+                    load_ids<CPT>(a.part + off, pu);
+                    pu[0] &= idmask;
+                }
+                const long long vreg = lane < ncomb ? V[(long long)e * ncomb + lane] : 0;
+#pragma unroll
+                for (int c = 0; c < CPT; ++c) {
+                    const unsigned cls = s_cls2[id_at<CPT>(pu, c) * k + id_at<CPT>(pv, c)];
+                    const long long val = lu[c] + shfl64(vreg, (int)cls);
+                    best[c] = val > best[c] ? val : best[c];
+                }
+            }
+            const unsigned long long Xv = h.xvert[i];
+            if (!FWD && ea == eb) {  // sink: blevel = own runtime
+#pragma unroll
+                for (int c = 0; c < CPT; ++c)
+                    if (Xv != NUM_ZERO) best[c] = ceil_quot(Xv, s_rt[id_at<CPT>(pv, c)]);
+            }
+            // results: global memory (the output) and the window
+            long long* gout = a.lev + (long long)v * ldp + jl;
+            if (nvalid >= CPT) store_levels<CPT>(gout, best);
+            else {
+#pragma unroll
+                for (int c = 0; c < CPT; ++c)
+                    if (c < nvalid) gout[c] = best[c];
+            }
+            if (R > 0) {
+                const int slot = pos - R * (int)(((unsigned long long)pos * wp.rmagic) >> 40);
+                store_levels<CPT>(win_lev + (size_t)slot * SLICE + lane * CPT, best);
+                store_ids<CPT>(win_id + (size_t)slot * SLICE + lane * CPT, pv);
+            }
+            if (want_cp && (FWD ? (vf < 0) : (pos < wp.src_end))) {
+#pragma unroll
+                for (int c = 0; c < CPT; ++c) {
+                    long long fin = best[c];
+                    if (FWD && Xv != NUM_ZERO) fin += ceil_quot(Xv, s_rt[id_at<CPT>(pv, c)]);
+                    cpmax[c] = fin > cpmax[c] ? fin : cpmax[c];
+                }
+            }
+        }
+        cp_async_wait_all();
+        __syncthreads();
+        cur = nxt; nxt = nxt2; nxt2 = nxt3;
+    }
+
+    if (want_cp && warp == 0) {
+#pragma unroll
+        for (int c = 0; c < CPT; ++c) {
+            long long m = cpmax[c];
+            for (int w = 1; w < wpb; ++w) {
+                long long o = s_cp[((size_t)w * 32 + lane) * CPT + c];
+                m = o > m ? o : m;
+            }
+            if (c < nvalid) a.cp[j0 + c] = m;
+        }
+    }
+}
+
+// ---- set-up kernels ---------------------------------------------------------------------
+__global__ void edge_values_kernel(int n, const int* __restrict__ eptr, const unsigned long long* __restrict__ xw,
+                                   const unsigned long long* __restrict__ xnbr, const unsigned long long* __restrict__ xvert,
+                                   const CombDiv* __restrict__ comb, int ncomb, long long* V)
+{
+    const long long gw = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (gw >= n || lane >= ncomb) return;
+    const CombDiv cd = comb[lane];
+    const int e0 = eptr[gw], e1 = eptr[gw + 1];
+    for (int e = e0; e < e1; ++e) {
+        const unsigned long long X = xw[e];
+        const unsigned long long Xr = xnbr ? xnbr[e] : xvert[gw];
+        long long t = 0;
+        if (cd.w.pad == 0 && X != NUM_ZERO) t = ceil_quot(X, cd.w);
+        if (Xr != NUM_ZERO) t += ceil_quot(Xr, cd.s);
+        V[(long long)e * ncomb + lane] = t;
+    }
+}
+
+__global__ void pos_of_kernel(int n, const int* __restrict__ order, int* pos_of)
+{
+    int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) pos_of[order[i]] = i;
+}
+
+// neighbour positions of both directions; the largest forward span |pos(v) - pos(u)| over all edges
+__global__ void npos_kernel(int n, const int* __restrict__ pos_of, const int* __restrict__ eptr_f,
+                            const int* __restrict__ nbr_f, const int* __restrict__ nbr_b, int m, int* npos_f,
+                            int* npos_b, int* maxspan)
+{
+    const int e = blockIdx.x * blockDim.x + threadIdx.x;
+    if (e < m) {
+        npos_f[e] = pos_of[nbr_f[e]];
+        npos_b[e] = pos_of[nbr_b[e]];
+    }
+    // spans: one thread per position walks its in-edges
+    if (e < n) {
+        int mx = 0;
+        for (int q = eptr_f[e]; q < eptr_f[e + 1]; ++q) {
+            const int s = e - pos_of[nbr_f[q]];
+            mx = s > mx ? s : mx;
+        }
+        if (mx > 0) atomicMax(maxspan, mx);
+    }
+}
+
+inline unsigned cdivu(long long a, long long b) { return (unsigned)((a + b - 1) / b); }
+
+template <int CPT, bool FWD>
+cudaError_t window_impl(const PassArgs& a, const WindowPlan& plan, int warps, cudaStream_t st)
+{
+    const size_t smem = carve(a.tab.k, plan.ncomb, plan.R, CPT, warps).total;
+    cudaError_t e = cudaFuncSetAttribute(pass_window_kernel<CPT, FWD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    pass_window_kernel<CPT, FWD><<<cdivu(a.P, 32 * CPT), warps * 32, smem, st>>>(a, plan);
+    count_launches(1);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+size_t window_smem_bytes(int k, int ncomb, int R, int cpt, int warps) { return carve(k, ncomb, R, cpt, warps).total; }
+
+cudaError_t launch_pass_window(const PassArgs& a, bool fwd, const WindowPlan& plan, int cpt, int warps, cudaStream_t st)
+{
+    if (plan.num_chunks <= 0) return cudaSuccess;
+    if (cpt == 4) return fwd ? window_impl<4, true>(a, plan, warps, st) : window_impl<4, false>(a, plan, warps, st);
+    if (cpt == 2) return fwd ? window_impl<2, true>(a, plan, warps, st) : window_impl<2, false>(a, plan, warps, st);
+    return fwd ? window_impl<1, true>(a, plan, warps, st) : window_impl<1, false>(a, plan, warps, st);
+}
+
+cudaError_t launch_edge_values(int n, const int* eptr, const unsigned long long* xw, const unsigned long long* xnbr,
+                               const unsigned long long* xvert, const CombDiv* comb, int ncomb, long long* V,
+                               cudaStream_t st)
+{
+    if (n <= 0) return cudaSuccess;
+    edge_values_kernel<<<cdivu((long long)n * 32, 256), 256, 0, st>>>(n, eptr, xw, xnbr, xvert, comb, ncomb, V);
+    count_launches(1);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_positions(int n, int m, const int* order, int* pos_of, const int* nbr_f, const int* nbr_b,
+                             const int* eptr_f, int* npos_f, int* npos_b, int* maxspan, cudaStream_t st)
+{
+    if (n <= 0) return cudaSuccess;
+    pos_of_kernel<<<cdivu(n, 256), 256, 0, st>>>(n, order, pos_of);
+    const int work = n > m ? n : m;
+    npos_kernel<<<cdivu(work, 256), 256, 0, st>>>(n, pos_of, eptr_f, nbr_f, nbr_b, m, npos_f, npos_b, maxspan);
+    count_launches(2);
+    return cudaGetLastError();
+}
+
+}  // namespace tfps

@@ -344,7 +344,14 @@ def test_sliced_kernel_shapes(cpt, table, monkeypatch):
     monkeypatch.setenv("TFPS_SLICED_CPT", str(cpt))
     monkeypatch.setenv("TFPS_SLICED_TABLE", str(table))
     monkeypatch.setenv("TFPS_SLICED_WARPS", "4")
-    rng = np.random.default_rng(cpt * 2 + table)
+    monkeypatch.setenv("TFPS_WINDOW", "0")
+    for g, dev, part in _shape_cases(cpt * 2 + table):
+        run_and_compare(g, dev, part, 2, pad_fill=255)
+
+
+def _shape_cases(seed):
+    rng = np.random.default_rng(seed)
+    cpt = seed // 2
     cases = []
     w = I.small_random(70 + cpt, 300, 900, 3, 77)          # classes, one pass
     cases.append((w.graph, w.devices, w.part_full()))
@@ -361,5 +368,26 @@ def test_sliced_kernel_shapes(cpt, table, monkeypatch):
     dev = I.Devices(4, np.array([1, 2, 2, 4], np.int32), np.full(4, INF, np.int64),
                     np.array([[0, 10, 10, 7], [10, 0, 7, 7], [3, 3, 0, 10], [7, 10, 3, 0]], np.int64), scale=3)
     cases.append((g, dev, rng.integers(0, 4, size=(n, 45), dtype=np.uint8)))
-    for g, dev, part in cases:
+    return cases
+
+
+@pytest.mark.parametrize("win_r", [-1, 160, 0])
+@pytest.mark.parametrize("cpt", [1, 2, 4])
+def test_windowed_kernel_shapes(cpt, win_r, monkeypatch):
+    """The windowed pass with the whole window resident (-1: automatic), with a
+    window too short for many edges (hits and misses mixed) and with no window at
+    all, for every lane width; the cases with many distinct costs or k > 16 fall
+    back to the sliced kernel and must still agree."""
+    monkeypatch.setenv("TFPS_SLICED_CPT", str(cpt))
+    monkeypatch.setenv("TFPS_SLICED_WARPS", "8")
+    monkeypatch.setenv("TFPS_WINDOW", "1")
+    monkeypatch.setenv("TFPS_WINDOW_R", str(win_r))
+    for g, dev, part in _shape_cases(cpt * 2 + 1):
         run_and_compare(g, dev, part, 2, pad_fill=255)
+    w = I.config2()
+    run_and_compare(w.graph, w.devices, w.part_full()[:, :333], 2, pad_fill=255)
+    w = I.config4()
+    g = w.graph
+    keep = g.dst < 16 * 300  # first 300 layers of the deep narrow graph
+    g2 = I.Graph(n=16 * 300, src=g.src[keep], dst=g.dst[keep], t=g.t[keep], c=g.c[:16 * 300], mem=None, layers=300)
+    run_and_compare(g2, w.devices, w.part_rows(0, 16 * 300)[:, :97], 2, pad_fill=255)
