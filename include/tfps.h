@@ -189,6 +189,39 @@ int tfps_phase_times(tfps_graph* g, float ms[3]);
 /* Number of kernels this library has launched in the calling process so far. */
 int64_t tfps_kernel_launches(void);
 
+/*
+ * Critical-path lengths without any allocation.  (The paper has no counterpart
+ * of this call; it exists for callers of this library that are not allowed to
+ * allocate device memory when they evaluate: code running inside a framework's
+ * allocator-managed region or under a memory budget that must not move, plug-ins
+ * that are handed buffers but no allocator, and real-time loops where a
+ * cudaMalloc -- which may synchronise the whole device -- is unacceptable.)
+ *
+ * Same result as tfps_eval_batch(g, P, ldp, part, NULL, NULL, cp, NULL, NULL,
+ * NULL, workspace, ...): cp[j] for the P candidates of `part` (dev uint8
+ * [n][ldp]) into `cp` (dev int64 [P]).  The forward pass needs one int64
+ * [n][ldp] matrix of scratch; here it lives in a fixed array inside the library
+ * (TFPS_NOALLOC_SCRATCH_BYTES, resident on every GPU that loads the library
+ * until the process exits) instead of a caller workspace.  The call performs no
+ * cudaMalloc/cudaFree and calls no allocating routine.
+ *
+ *   - n*ldp*8 must not exceed TFPS_NOALLOC_SCRATCH_BYTES, else TFPS_ERR_WORKSPACE.
+ *   - tfps_devices_set must have been called (it builds everything the pass
+ *     needs), else TFPS_ERR_STATE.
+ *   - The first call on a device looks up the device address of the scratch
+ *     array; make that first call outside of any stream capture.
+ *   - All calls on a device share the one array.  It keeps whatever the last call
+ *     left in it; nothing in it has to start at zero, because every cell the
+ *     pass reads was written earlier in the same call.  Two calls that overlap
+ *     on the GPU (different streams, different handles, different host threads)
+ *     race on it: serialise them.
+ *   - Asynchronous on `stream` like tfps_eval_batch; id errors are reported
+ *     through tfps_get_status.
+ */
+#define TFPS_NOALLOC_SCRATCH_BYTES ((size_t)32 << 20)
+int tfps_eval_cp_noalloc(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, int64_t* cp,
+                         int flags, void* stream);
+
 /* Synchronise `stream`, return the sticky device-side status of the handle and clear it. */
 int tfps_get_status(tfps_graph* g, void* stream);
 

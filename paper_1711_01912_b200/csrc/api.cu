@@ -6,6 +6,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <utility>
 
@@ -866,6 +867,44 @@ int tfps_phase_times(tfps_graph* g, float ms[3])
 }
 
 int64_t tfps_kernel_launches(void) { return (int64_t)tfps::g_launches.load(std::memory_order_relaxed); }
+
+// Scratch of tfps_eval_cp_noalloc: one int64 level matrix, resident on every device that loads the library.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[TFPS_NOALLOC_SCRATCH_BYTES];
+
+namespace {
+std::mutex g_noalloc_mutex;
+void* g_noalloc_ptr[128] = {};  // device address of g_noalloc_scratch, by device ordinal
+}  // namespace
+
+int tfps_eval_cp_noalloc(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, int64_t* cp, int flags,
+                         void* stream)
+{
+    if (!g) return fail(TFPS_ERR_INVALID_ARG, "graph is NULL");
+    if (P < 0 || ldp < P || (ldp % 16) != 0) return fail(TFPS_ERR_INVALID_ARG, "need 0 <= P <= ldp and ldp %% 16 == 0");
+    if (!g->dev_set) return fail(TFPS_ERR_STATE, "tfps_devices_set has not been called");
+    if (P == 0 || g->n == 0) return TFPS_OK;
+    if (!part || !cp) return fail(TFPS_ERR_INVALID_ARG, "part and cp are required");
+    const unsigned __int128 need = (unsigned __int128)g->n * (unsigned __int128)ldp * 8u;
+    if (need > (unsigned __int128)TFPS_NOALLOC_SCRATCH_BYTES)
+        return fail(TFPS_ERR_WORKSPACE, "n*ldp*8 = %llu bytes of level scratch needed, the built-in array holds %zu; "
+                    "use tfps_eval_batch with a caller workspace", (unsigned long long)need, (size_t)TFPS_NOALLOC_SCRATCH_BYTES);
+    if (g->device < 0 || g->device >= 128) return fail(TFPS_ERR_UNSUPPORTED, "device ordinal %d out of range", g->device);
+    DeviceGuard guard(g->device);
+    if (!guard.ok) return fail(TFPS_ERR_CUDA, "cannot select the handle's device");
+    void* scratch = nullptr;
+    {
+        // the array's name is only a host-side handle: ask the runtime for its address on this device, once
+        std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+        if (!g_noalloc_ptr[g->device]) {
+            void* p = nullptr;
+            CUDA_TRY(cudaGetSymbolAddress(&p, g_noalloc_scratch));
+            g_noalloc_ptr[g->device] = p;
+        }
+        scratch = g_noalloc_ptr[g->device];
+    }
+    return tfps_eval_batch(g, P, ldp, part, nullptr, nullptr, cp, nullptr, nullptr, nullptr, scratch,
+                           TFPS_NOALLOC_SCRATCH_BYTES, flags & ~TFPS_EVAL_PROFILE, stream);
+}
 
 int tfps_get_status(tfps_graph* g, void* stream)
 {

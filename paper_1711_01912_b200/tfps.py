@@ -31,6 +31,7 @@ EXPORTS = [
     "tfps_strerror", "tfps_last_error", "tfps_graph_create", "tfps_graph_destroy", "tfps_graph_info",
     "tfps_devices_set", "tfps_topo_levels", "tfps_eval_workspace_bytes", "tfps_eval_batch",
     "tfps_eval_batch_host", "tfps_get_status", "tfps_transpose_u8", "tfps_phase_times", "tfps_kernel_launches",
+    "tfps_eval_cp_noalloc",
 ]
 
 
@@ -77,6 +78,8 @@ def lib() -> ctypes.CDLL:
     L.tfps_phase_times.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
     L.tfps_kernel_launches.restype = i64
     L.tfps_kernel_launches.argtypes = []
+    L.tfps_eval_cp_noalloc.restype = ci
+    L.tfps_eval_cp_noalloc.argtypes = [vp, i64, i64, vp, vp, ci, vp]
     L.tfps_get_status.restype = ci
     L.tfps_get_status.argtypes = [vp, vp]
     L.tfps_transpose_u8.restype = ci
@@ -149,6 +152,14 @@ def tfps_phase_times(g):
 
 def tfps_kernel_launches() -> int:
     return int(lib().tfps_kernel_launches())
+
+
+NOALLOC_SCRATCH_BYTES = 32 << 20
+
+
+def tfps_eval_cp_noalloc(g, P, ldp, part, cp, flags=0, stream=0) -> None:
+    """Critical-path lengths with the level scratch inside the library: no device allocation happens in this call."""
+    _check(lib().tfps_eval_cp_noalloc(g, P, ldp, part, cp, flags, stream))
 
 
 def tfps_get_status(g, stream=0) -> None:
