@@ -111,6 +111,7 @@ struct tfps_graph {
     // chunk tables of the candidate-sliced pass
     DBuf vertf, f_chunks, b_chunks;
     int f_num_chunks = 0, b_num_chunks = 0;
+    bool f_all_staged = true, b_all_staged = true;
     // device tables
     bool dev_set = false;
     int k = 0;
@@ -280,6 +281,7 @@ int build_topo(tfps_graph* g, cudaStream_t st)
                 chunks.push_back(q - p);
                 chunks.push_back(eptr[p]);
                 chunks.push_back(eptr[q] - eptr[p]);
+                if (eptr[q] - eptr[p] > CHUNK_E) (dir == 0 ? g->f_all_staged : g->b_all_staged) = false;
                 p = q;
             }
         }
@@ -784,12 +786,14 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
     bool use_window = sliced && g->ncomb > 0 && env_int("TFPS_WINDOW", 1) != 0;
     int win_R = 0;
     if (use_window) {
-        const int r_need = (g->maxspan + CHUNK_V + 31) / 32 * 32;
+        int r_need = 32;  // smallest power of two that keeps every edge inside the ring
+        while (r_need < g->maxspan + CHUNK_V) r_need <<= 1;
         auto r_fit = [&](int c) {
             const long long avail = (long long)g->smem_optin - 1024 - (long long)window_smem_bytes(k, g->ncomb, 0, c, warps);
-            long long r = avail / (32LL * c * 9) / 32 * 32;
-            if (r > (1 << 13)) r = 1 << 13;
-            return (int)(r < 0 ? 0 : r);
+            const long long rmax = avail / (32LL * c * 9);
+            int r = 0;
+            for (int q = 32; q <= rmax && q <= (1 << 16); q <<= 1) r = q;
+            return r;
         };
         const int forced = env_int("TFPS_SLICED_CPT", 0);
         int chosen = 0;
@@ -803,7 +807,11 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
         cpt = chosen;
         win_R = std::min(r_fit(cpt), r_need);
         const int forced_r = env_int("TFPS_WINDOW_R", -1);
-        if (forced_r >= 0) win_R = std::min(forced_r / 32 * 32, r_fit(cpt));
+        if (forced_r >= 0) {
+            int q = 0;
+            for (int t = 32; t <= forced_r; t <<= 1) q = t;
+            win_R = std::min(q, r_fit(cpt));
+        }
         if (win_R < CHUNK_V + 32) win_R = 0;
         if (window_smem_bytes(k, g->ncomb, win_R, cpt, warps) > (size_t)g->smem_optin) use_window = false;
     }
@@ -826,7 +834,8 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
             wp.cls2 = fwd ? g->cls2_f.as<uint8_t>() : g->cls2_b.as<uint8_t>();
             wp.ncomb = g->ncomb;
             wp.R = win_R;
-            wp.rmagic = win_R > 0 ? (((1ull << 40) + (unsigned long long)win_R - 1) / (unsigned long long)win_R) : 0ull;
+            wp.maxspan = g->maxspan;
+            wp.all_staged = (fwd ? g->f_all_staged : g->b_all_staged) ? 1 : 0;
             CUDA_TRY(launch_pass_window(a, fwd, wp, cpt, warps, st));
         } else if (sliced) {
             SlicedPlan plan;

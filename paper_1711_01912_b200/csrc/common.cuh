@@ -128,8 +128,9 @@ struct WindowPlan {
     const long long* V;          // [m][ncomb]
     const uint8_t* cls2;         // [k*k] comb id of (nb, vv)
     int ncomb;
-    int R;                       // window length in positions (0: no window), multiple of 32
-    unsigned long long rmagic;   // floor(x / R) == (x * rmagic) >> 40 for x < 2^26
+    int R;                       // window length in positions: a power of two, or 0 for no window
+    int maxspan;                 // largest |pos(v) - pos(u)| over all edges
+    int all_staged;              // no vertex has more than CHUNK_E edges
 };
 
 // every kernel launch of the library goes through the wrappers below and is counted here

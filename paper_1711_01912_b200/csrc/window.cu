@@ -124,45 +124,98 @@ __host__ __device__ inline Carve carve(int k, int ncomb, int R, int cpt, int war
     return c;
 }
 
-template <int CPT, bool FWD>
+// 32-bit shared-state-space accessors (addresses from __cvta_generic_to_shared)
+__device__ __forceinline__ unsigned lds_u8(unsigned a) { unsigned v; asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(a)); return v; }
+__device__ __forceinline__ unsigned lds_u16(unsigned a) { unsigned v; asm volatile("ld.shared.u16 %0, [%1];" : "=r"(v) : "r"(a)); return v; }
+__device__ __forceinline__ unsigned lds_u32(unsigned a) { unsigned v; asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a)); return v; }
+__device__ __forceinline__ long long lds_s64(unsigned a) { long long v; asm volatile("ld.shared.s64 %0, [%1];" : "=l"(v) : "r"(a)); return v; }
+__device__ __forceinline__ void lds_v2s64(unsigned a, long long& x, long long& y) { asm volatile("ld.shared.v2.s64 {%0,%1}, [%2];" : "=l"(x), "=l"(y) : "r"(a)); }
+__device__ __forceinline__ void sts_s64(unsigned a, long long v) { asm volatile("st.shared.s64 [%0], %1;" ::"r"(a), "l"(v) : "memory"); }
+__device__ __forceinline__ void sts_v2s64(unsigned a, long long x, long long y) { asm volatile("st.shared.v2.s64 [%0], {%1,%2};" ::"r"(a), "l"(x), "l"(y) : "memory"); }
+__device__ __forceinline__ void sts_u8(unsigned a, unsigned v) { asm volatile("st.shared.u8 [%0], %1;" ::"r"(a), "r"(v) : "memory"); }
+__device__ __forceinline__ void sts_u16(unsigned a, unsigned v) { asm volatile("st.shared.u16 [%0], %1;" ::"r"(a), "r"(v) : "memory"); }
+__device__ __forceinline__ void sts_u32(unsigned a, unsigned v) { asm volatile("st.shared.u32 [%0], %1;" ::"r"(a), "r"(v) : "memory"); }
+
+template <int CPT> __device__ __forceinline__ unsigned lds_ids(unsigned a)
+{
+    if constexpr (CPT == 1) return lds_u8(a);
+    else if constexpr (CPT == 2) return lds_u16(a);
+    else return lds_u32(a);
+}
+template <int CPT> __device__ __forceinline__ void sts_ids(unsigned a, unsigned v)
+{
+    if constexpr (CPT == 1) sts_u8(a, v);
+    else if constexpr (CPT == 2) sts_u16(a, v);
+    else sts_u32(a, v);
+}
+template <int CPT> __device__ __forceinline__ void lds_levels(unsigned a, long long (&out)[CPT])
+{
+    if constexpr (CPT == 1) out[0] = lds_s64(a);
+    else {
+#pragma unroll
+        for (int i = 0; i < CPT; i += 2) lds_v2s64(a + 8 * i, out[i], out[i + 1]);
+    }
+}
+template <int CPT> __device__ __forceinline__ void sts_levels(unsigned a, const long long (&v)[CPT])
+{
+    if constexpr (CPT == 1) sts_s64(a, v[0]);
+    else {
+#pragma unroll
+        for (int i = 0; i < CPT; i += 2) sts_v2s64(a + 8 * i, v[i], v[i + 1]);
+    }
+}
+
+// Byte offsets of the shared-memory regions, computed on the host and passed as a kernel parameter.
+struct WinLayout {
+    unsigned head, head_stride;
+    unsigned edge_nbr, edge_npos, edge_V, edge_stride;
+    unsigned ids, ids_stride;
+    unsigned rt, cls2, cp, win_lev, win_id;
+};
+
+// ALL_STAGED: every chunk's adjacency fits the staging buffers (no vertex with more than CHUNK_E edges).
+template <int CPT, bool FWD, bool ALL_STAGED>
 __global__ void __launch_bounds__(1024)
-pass_window_kernel(PassArgs a, WindowPlan wp)
+pass_window_kernel(PassArgs a, WindowPlan wp, WinLayout L)
 {
     extern __shared__ __align__(16) unsigned char smem[];
     constexpr int SLICE = 32 * CPT;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, wpb = blockDim.x >> 5;
     const int k = a.tab.k;
     const int ncomb = wp.ncomb;
-    const int R = wp.R;
-    const Carve cv = carve(k, ncomb, R, CPT, wpb);
-    DivConst* s_rt = reinterpret_cast<DivConst*>(smem + cv.rt);
-    uint8_t* s_cls2 = smem + cv.cls2;
-    long long* s_cp = reinterpret_cast<long long*>(smem + cv.cp);
-    long long* win_lev = reinterpret_cast<long long*>(smem + cv.win_lev);
-    uint8_t* win_id = smem + cv.win_id;
+    const int R = wp.R;              // power of two (or 0)
+    const int rmask = R - 1;
+    const int hit_span = R - CHUNK_V;  // a neighbour at most this many positions away is still in the ring
+    const unsigned sbase = (unsigned)__cvta_generic_to_shared(smem);
+    DivConst* s_rt = reinterpret_cast<DivConst*>(smem + L.rt);
+    long long* s_cp = reinterpret_cast<long long*>(smem + L.cp);
     if (*a.status != 0) return;
     for (int i = threadIdx.x; i < k; i += blockDim.x) s_rt[i] = a.tab.rt_div[i];
-    for (int i = threadIdx.x; i < k * k; i += blockDim.x) s_cls2[i] = wp.cls2[i];
+    for (int i = threadIdx.x; i < k * k; i += blockDim.x) smem[L.cls2 + i] = wp.cls2[i];
 
     const long long slice0 = (long long)blockIdx.x * SLICE;
     const long long j0 = slice0 + (long long)lane * CPT;
     const long long rem = a.P - j0;
     const int nvalid = rem >= CPT ? CPT : (rem > 0 ? (int)rem : 0);
-    const long long jl = nvalid > 0 ? j0 : slice0;
-    unsigned idmask = nvalid >= 4 ? 0xffffffffu : (nvalid > 0 ? ((1u << (8 * nvalid)) - 1u) : 0u);
+    const int lane_col = nvalid > 0 ? lane * CPT : 0;      // idle lanes shadow the slice's first lane
+    const long long jl = slice0 + lane_col;
+    const unsigned idmask = nvalid >= 4 ? 0xffffffffu : (nvalid > 0 ? ((1u << (8 * nvalid)) - 1u) : 0u);
     const long long ldp = a.ldp;
-    // the slice's id bytes that exist in the row: the last slice may reach beyond ldp
     const int slice_bytes = (int)((ldp - slice0) < SLICE ? (ldp - slice0) : SLICE);
     const bool want_cp = a.cp != nullptr;
     long long* cpmax = s_cp + ((size_t)warp * 32 + lane) * CPT;
 #pragma unroll
     for (int c = 0; c < CPT; ++c) cpmax[c] = 0;
+    // per-lane shared addresses
+    const unsigned win_lev_lane = sbase + L.win_lev + 8u * (unsigned)(lane * CPT);
+    const unsigned win_id_lane = sbase + L.win_id + (unsigned)(lane * CPT);
+    const unsigned cls2_s = sbase + L.cls2;
 
     const int4* chunks = reinterpret_cast<const int4*>(wp.chunks);
     const int num_chunks = wp.num_chunks;
     auto entry = [&](int ci) { return chunks[FWD ? ci : num_chunks - 1 - ci]; };
-    auto head = [&](int ci) -> HeadBuf& { return *reinterpret_cast<HeadBuf*>(smem + cv.head + (size_t)(ci % 3) * up16(sizeof(HeadBuf))); };
-    auto stage_head = [&](int4 ent, HeadBuf& h) {
+    auto stage_head = [&](int4 ent, int slot) {
+        HeadBuf& h = *reinterpret_cast<HeadBuf*>(smem + L.head + (unsigned)slot * L.head_stride);
         const int p0 = ent.x, cnt = ent.y;
         for (int i = threadIdx.x; i < cnt; i += blockDim.x) {
             cp_async4(&h.vertf[i], wp.vertf + p0 + i);
@@ -172,103 +225,157 @@ pass_window_kernel(PassArgs a, WindowPlan wp)
     };
     auto stage_edges = [&](int4 ent, int slot) {
         const int e0 = ent.z, ecnt = ent.w;
-        if (ecnt > CHUNK_E) return;  // read from global memory instead
-        unsigned char* base = smem + cv.edge_nbr + (size_t)slot * cv.edge_stride;
-        int* nbr = reinterpret_cast<int*>(base);
-        int* npos = reinterpret_cast<int*>(base + (cv.edge_npos - cv.edge_nbr));
-        long long* V = reinterpret_cast<long long*>(base + (cv.edge_V - cv.edge_nbr));
-        for (int i = threadIdx.x; i < ecnt; i += blockDim.x) {
-            cp_async4(&nbr[i], a.adj.nbr + e0 + i);
-            cp_async4(&npos[i], wp.npos + e0 + i);
+        if (!ALL_STAGED && ecnt > CHUNK_E) return;  // read from global memory instead
+        unsigned char* base = smem + (unsigned)slot * L.edge_stride;
+        int* npos = reinterpret_cast<int*>(base + L.edge_npos);
+        long long* V = reinterpret_cast<long long*>(base + L.edge_V);
+        for (int i = threadIdx.x; i < ecnt; i += blockDim.x) cp_async4(&npos[i], wp.npos + e0 + i);
+        if (hit_span < wp.maxspan || !ALL_STAGED) {  // neighbour ids are only needed for window misses
+            int* nbr = reinterpret_cast<int*>(base + L.edge_nbr);
+            for (int i = threadIdx.x; i < ecnt; i += blockDim.x) cp_async4(&nbr[i], a.adj.nbr + e0 + i);
         }
         const long long* Vg = wp.V + (long long)e0 * ncomb;
-        for (int i = threadIdx.x; i < ecnt * ncomb; i += blockDim.x) cp_async8(&V[i], Vg + i);
+        const int nv = ecnt * ncomb;
+        if ((((long long)e0 * ncomb) & 1) == 0) {   // 16-byte aligned source: copy pairs
+            for (int i = threadIdx.x; i < (nv >> 1); i += blockDim.x) cp_async16(&V[2 * i], Vg + 2 * i);
+            if ((nv & 1) && threadIdx.x == 0) cp_async8(&V[nv - 1], Vg + nv - 1);
+        } else {
+            for (int i = threadIdx.x; i < nv; i += blockDim.x) cp_async8(&V[i], Vg + i);
+        }
     };
-    auto stage_ids = [&](int4 ent, const HeadBuf& h, int slot) {
+    auto stage_ids = [&](int4 ent, int head_slot, int slot) {
+        const HeadBuf& h = *reinterpret_cast<const HeadBuf*>(smem + L.head + (unsigned)head_slot * L.head_stride);
         const int cnt = ent.y;
-        uint8_t* dst = smem + cv.ids + (size_t)slot * cv.ids_stride;
-        const int per_row = slice_bytes / 16;  // ldp and slice0 are multiples of 16
+        uint8_t* dst = smem + L.ids + (unsigned)slot * L.ids_stride;
+        const int per_row = slice_bytes >> 4;  // ldp and slice0 are multiples of 16
         for (int i = threadIdx.x; i < cnt * per_row; i += blockDim.x) {
             const int r = i / per_row, q = i - r * per_row;
             const int v = h.vertf[r] & 0x7fffffff;
-            cp_async16(dst + (size_t)r * SLICE + 16 * q, a.part + (long long)v * ldp + slice0 + 16 * q);
+            cp_async16(dst + r * SLICE + 16 * q, a.part + (long long)v * ldp + slice0 + 16 * q);
         }
     };
 
     int4 cur = entry(0);
     int4 nxt = num_chunks > 1 ? entry(1) : cur;
     int4 nxt2 = num_chunks > 2 ? entry(2) : cur;
-    stage_head(cur, head(0));
-    if (num_chunks > 1) stage_head(nxt, head(1));
+    stage_head(cur, 0);
+    if (num_chunks > 1) stage_head(nxt, 1);
     stage_edges(cur, 0);
     cp_async_commit();
     cp_async_wait_all();
     __syncthreads();
-    stage_ids(cur, head(0), 0);
+    stage_ids(cur, 0, 0);
     cp_async_commit();
     cp_async_wait_all();
     __syncthreads();
 
+    int hslot = 0;  // ci % 3
     for (int ci = 0; ci < num_chunks; ++ci) {
+        const int hs1 = hslot == 2 ? 0 : hslot + 1;
+        const int hs2 = hs1 == 2 ? 0 : hs1 + 1;
         int4 nxt3 = nxt2;
         if (ci + 1 < num_chunks) {
-            stage_ids(nxt, head(ci + 1), (ci + 1) & 1);
+            stage_ids(nxt, hs1, (ci + 1) & 1);
             stage_edges(nxt, (ci + 1) & 1);
             if (ci + 2 < num_chunks) {
-                stage_head(nxt2, head(ci + 2));
+                stage_head(nxt2, hs2);
                 if (ci + 3 < num_chunks) nxt3 = entry(ci + 3);
             }
             cp_async_commit();
         }
-        const HeadBuf& h = head(ci);
+        const unsigned head_s = sbase + L.head + (unsigned)hslot * L.head_stride;
+        const unsigned xvert_s = head_s;                                   // HeadBuf::xvert
+        const unsigned vertf_s = head_s + 8u * CHUNK_V;                    // HeadBuf::vertf
+        const unsigned eoff_s = vertf_s + 4u * CHUNK_V;                    // HeadBuf::eoff
         const int p0 = cur.x, cnt = cur.y, e0 = cur.z;
-        const bool staged = cur.w <= CHUNK_E;
-        const unsigned char* ebase = smem + cv.edge_nbr + (size_t)(ci & 1) * cv.edge_stride;
-        const int* nbr = staged ? reinterpret_cast<const int*>(ebase) : a.adj.nbr;
-        const int* npos = staged ? reinterpret_cast<const int*>(ebase + (cv.edge_npos - cv.edge_nbr)) : wp.npos;
-        const long long* V = staged ? reinterpret_cast<const long long*>(ebase + (cv.edge_V - cv.edge_nbr)) : wp.V;
-        const int ebias = staged ? e0 : 0;
-        const uint8_t* idrows = smem + cv.ids + (size_t)(ci & 1) * cv.ids_stride;
+        const bool staged = ALL_STAGED || cur.w <= CHUNK_E;
+        const unsigned ebase_s = sbase + (unsigned)(ci & 1) * L.edge_stride;
+        const unsigned npos_s = ebase_s + L.edge_npos;
+        const unsigned nbr_s = ebase_s + L.edge_nbr;
+        const unsigned V_s = ebase_s + L.edge_V;
+        const unsigned idrow_lane = sbase + L.ids + (unsigned)(ci & 1) * L.ids_stride + (unsigned)lane_col;
 
         for (int i = warp; i < cnt; i += wpb) {
-            const int vf = h.vertf[i];
+            const int vf = (int)lds_u32(vertf_s + 4u * i);
             const int v = vf & 0x7fffffff;
             const int pos = p0 + i;
-            unsigned pv[IdWords<CPT>::N];
-            load_ids<CPT>(idrows + (size_t)i * SLICE + (jl - slice0), pv);
-            pv[0] &= idmask;
+            const unsigned pv = lds_ids<CPT>(idrow_lane + (unsigned)(i * SLICE)) & idmask;
+            unsigned cls_v[CPT];   // shared address of cls2[0*k + idv]
+#pragma unroll
+            for (int c = 0; c < CPT; ++c) cls_v[c] = cls2_s + ((pv >> (8 * c)) & 0xffu);
             long long best[CPT];
 #pragma unroll
             for (int c = 0; c < CPT; ++c) best[c] = 0;
-            const int ea = h.eoff[i] - ebias, eb = h.eoff[i + 1] - ebias;
-            for (int e = ea; e < eb; ++e) {
-                const int np = npos[e];
-                const int span = FWD ? pos - np : np - pos;
-                long long lu[CPT];
-                unsigned pu[IdWords<CPT>::N];
-                if (span <= R - CHUNK_V) {
-                    const int slot = np - R * (int)(((unsigned long long)np * wp.rmagic) >> 40);
-                    load_levels<CPT>(win_lev + (size_t)slot * SLICE + lane * CPT, lu);
-                    load_ids<CPT>(win_id + (size_t)slot * SLICE + lane * CPT, pu);
-                } else {
-                    const long long off = (long long)nbr[e] * ldp + jl;
-                    load_levels<CPT>(a.lev + off, lu);
-                    load_ids<CPT>(a.part + off, pu);
-                    pu[0] &= idmask;
-                }
-                const long long vreg = lane < ncomb ? V[(long long)e * ncomb + lane] : 0;
+            const int ea_abs = (int)lds_u32(eoff_s + 4u * i), eb_abs = (int)lds_u32(eoff_s + 4u * i + 4u);
+            if (staged) {
+                const int ea = ea_abs - e0, eb = eb_abs - e0;
+                for (int e = ea; e < eb; ++e) {
+                    const int np = (int)lds_u32(npos_s + 4u * e);
+                    const int span = FWD ? pos - np : np - pos;
+                    long long lu[CPT];
+                    unsigned pu;
+                    if (span <= hit_span) {
+                        const unsigned slot = (unsigned)(np & rmask);
+                        lds_levels<CPT>(win_lev_lane + slot * (8u * SLICE), lu);
+                        pu = lds_ids<CPT>(win_id_lane + slot * (unsigned)SLICE);
+                    } else {
+                        const long long off = (long long)(int)lds_u32(nbr_s + 4u * e) * ldp + jl;
+                        load_levels<CPT>(a.lev + off, lu);
+                        unsigned w[IdWords<CPT>::N];
+                        load_ids<CPT>(a.part + off, w);
+                        pu = w[0] & idmask;
+                    }
+                    const unsigned vrow = V_s + 8u * (unsigned)(e * ncomb);
 #pragma unroll
-                for (int c = 0; c < CPT; ++c) {
-                    const unsigned cls = s_cls2[id_at<CPT>(pu, c) * k + id_at<CPT>(pv, c)];
-                    const long long val = lu[c] + shfl64(vreg, (int)cls);
-                    best[c] = val > best[c] ? val : best[c];
+                    for (int c = 0; c < CPT; ++c) {
+                        const unsigned cls = lds_u8(cls_v[c] + ((pu >> (8 * c)) & 0xffu) * (unsigned)k);
+                        const long long val = lu[c] + lds_s64(vrow + 8u * cls);
+                        best[c] = val > best[c] ? val : best[c];
+                    }
+                }
+            } else {
+                // a vertex whose adjacency did not fit the staging buffers: everything from global memory
+                for (int e = ea_abs; e < eb_abs; ++e) {
+                    const int np = wp.npos[e];
+                    const int span = FWD ? pos - np : np - pos;
+                    long long lu[CPT];
+                    unsigned pu;
+                    if (span <= hit_span) {
+                        const unsigned slot = (unsigned)(np & rmask);
+                        lds_levels<CPT>(win_lev_lane + slot * (8u * SLICE), lu);
+                        pu = lds_ids<CPT>(win_id_lane + slot * (unsigned)SLICE);
+                    } else {
+                        const long long off = (long long)a.adj.nbr[e] * ldp + jl;
+                        load_levels<CPT>(a.lev + off, lu);
+                        unsigned w[IdWords<CPT>::N];
+                        load_ids<CPT>(a.part + off, w);
+                        pu = w[0] & idmask;
+                    }
+                    const long long* vrow = wp.V + (long long)e * ncomb;
+#pragma unroll
+                    for (int c = 0; c < CPT; ++c) {
+                        const unsigned cls = lds_u8(cls_v[c] + ((pu >> (8 * c)) & 0xffu) * (unsigned)k);
+                        const long long val = lu[c] + vrow[cls];
+                        best[c] = val > best[c] ? val : best[c];
+                    }
                 }
             }
-            const unsigned long long Xv = h.xvert[i];
-            if (!FWD && ea == eb) {  // sink: blevel = own runtime
+            const bool is_cp = want_cp && (FWD ? (vf < 0) : (pos < wp.src_end));
+            if ((!FWD && ea_abs == eb_abs) || is_cp) {
+                const unsigned long long Xv = (unsigned long long)lds_s64(xvert_s + 8u * i);
+                if (!FWD && ea_abs == eb_abs) {  // sink: blevel = own runtime
 #pragma unroll
-                for (int c = 0; c < CPT; ++c)
-                    if (Xv != NUM_ZERO) best[c] = ceil_quot(Xv, s_rt[id_at<CPT>(pv, c)]);
+                    for (int c = 0; c < CPT; ++c)
+                        best[c] = Xv != NUM_ZERO ? ceil_quot(Xv, s_rt[(pv >> (8 * c)) & 0xffu]) : 0;
+                }
+                if (is_cp) {
+#pragma unroll
+                    for (int c = 0; c < CPT; ++c) {
+                        long long fin = best[c];
+                        if (FWD && Xv != NUM_ZERO) fin += ceil_quot(Xv, s_rt[(pv >> (8 * c)) & 0xffu]);
+                        cpmax[c] = fin > cpmax[c] ? fin : cpmax[c];
+                    }
+                }
             }
             // results: global memory (the output) and the window
             long long* gout = a.lev + (long long)v * ldp + jl;
@@ -279,22 +386,15 @@ pass_window_kernel(PassArgs a, WindowPlan wp)
                     if (c < nvalid) gout[c] = best[c];
             }
             if (R > 0) {
-                const int slot = pos - R * (int)(((unsigned long long)pos * wp.rmagic) >> 40);
-                store_levels<CPT>(win_lev + (size_t)slot * SLICE + lane * CPT, best);
-                store_ids<CPT>(win_id + (size_t)slot * SLICE + lane * CPT, pv);
-            }
-            if (want_cp && (FWD ? (vf < 0) : (pos < wp.src_end))) {
-#pragma unroll
-                for (int c = 0; c < CPT; ++c) {
-                    long long fin = best[c];
-                    if (FWD && Xv != NUM_ZERO) fin += ceil_quot(Xv, s_rt[id_at<CPT>(pv, c)]);
-                    cpmax[c] = fin > cpmax[c] ? fin : cpmax[c];
-                }
+                const unsigned slot = (unsigned)(pos & rmask);
+                sts_levels<CPT>(win_lev_lane + slot * (8u * SLICE), best);
+                sts_ids<CPT>(win_id_lane + slot * (unsigned)SLICE, pv);
             }
         }
         cp_async_wait_all();
         __syncthreads();
         cur = nxt; nxt = nxt2; nxt2 = nxt3;
+        hslot = hs1;
     }
 
     if (want_cp && warp == 0) {
@@ -359,15 +459,31 @@ __global__ void npos_kernel(int n, const int* __restrict__ pos_of, const int* __
 
 inline unsigned cdivu(long long a, long long b) { return (unsigned)((a + b - 1) / b); }
 
-template <int CPT, bool FWD>
+template <int CPT, bool FWD, bool ALL_STAGED>
 cudaError_t window_impl(const PassArgs& a, const WindowPlan& plan, int warps, cudaStream_t st)
 {
-    const size_t smem = carve(a.tab.k, plan.ncomb, plan.R, CPT, warps).total;
-    cudaError_t e = cudaFuncSetAttribute(pass_window_kernel<CPT, FWD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    const Carve c = carve(a.tab.k, plan.ncomb, plan.R, CPT, warps);
+    WinLayout L;
+    L.head = (unsigned)c.head; L.head_stride = (unsigned)up16(sizeof(HeadBuf));
+    L.edge_nbr = (unsigned)c.edge_nbr; L.edge_npos = (unsigned)c.edge_npos; L.edge_V = (unsigned)c.edge_V;
+    L.edge_stride = (unsigned)c.edge_stride;
+    L.ids = (unsigned)c.ids; L.ids_stride = (unsigned)c.ids_stride;
+    L.rt = (unsigned)c.rt; L.cls2 = (unsigned)c.cls2; L.cp = (unsigned)c.cp;
+    L.win_lev = (unsigned)c.win_lev; L.win_id = (unsigned)c.win_id;
+    cudaError_t e = cudaFuncSetAttribute(pass_window_kernel<CPT, FWD, ALL_STAGED>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c.total);
     if (e != cudaSuccess) return e;
-    pass_window_kernel<CPT, FWD><<<cdivu(a.P, 32 * CPT), warps * 32, smem, st>>>(a, plan);
+    pass_window_kernel<CPT, FWD, ALL_STAGED><<<cdivu(a.P, 32 * CPT), warps * 32, c.total, st>>>(a, plan, L);
     count_launches(1);
     return cudaGetLastError();
+}
+
+template <int CPT>
+cudaError_t window_dispatch(const PassArgs& a, bool fwd, const WindowPlan& plan, int warps, cudaStream_t st)
+{
+    if (plan.all_staged)
+        return fwd ? window_impl<CPT, true, true>(a, plan, warps, st) : window_impl<CPT, false, true>(a, plan, warps, st);
+    return fwd ? window_impl<CPT, true, false>(a, plan, warps, st) : window_impl<CPT, false, false>(a, plan, warps, st);
 }
 
 }  // namespace
@@ -377,9 +493,9 @@ size_t window_smem_bytes(int k, int ncomb, int R, int cpt, int warps) { return c
 cudaError_t launch_pass_window(const PassArgs& a, bool fwd, const WindowPlan& plan, int cpt, int warps, cudaStream_t st)
 {
     if (plan.num_chunks <= 0) return cudaSuccess;
-    if (cpt == 4) return fwd ? window_impl<4, true>(a, plan, warps, st) : window_impl<4, false>(a, plan, warps, st);
-    if (cpt == 2) return fwd ? window_impl<2, true>(a, plan, warps, st) : window_impl<2, false>(a, plan, warps, st);
-    return fwd ? window_impl<1, true>(a, plan, warps, st) : window_impl<1, false>(a, plan, warps, st);
+    if (cpt == 4) return window_dispatch<4>(a, fwd, plan, warps, st);
+    if (cpt == 2) return window_dispatch<2>(a, fwd, plan, warps, st);
+    return window_dispatch<1>(a, fwd, plan, warps, st);
 }
 
 cudaError_t launch_edge_values(int n, const int* eptr, const unsigned long long* xw, const unsigned long long* xnbr,
