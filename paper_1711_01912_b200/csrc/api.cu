@@ -119,8 +119,12 @@ struct tfps_graph {
     DBuf rt_div, w_div, cap, xvert, xw_f, xnbr_f, xw_b;
     DBuf pair_f, pair_b, cls_div, sel_f, sel_b;
     // windowed pass: neighbour positions, comb tables, precomputed edge values
-    DBuf pos_of, npos_f, npos_b, cls2_f, cls2_b, comb_f, comb_b, V_f, V_b;
+    DBuf pos_of, npos_f, npos_b, cls2_f, cls2_b, comb_f, comb_b, V_f, V_b, V32_f, V32_b;
     int ncomb = 0, maxspan = 0, smem_optin = 0;
+    bool fits32 = false;  // every path length under any partition fits int32
+    // host copies of the in-edge CSR for the worst-case path bound
+    std::vector<long long> h_in_ptr, h_in_t;
+    std::vector<int> h_in_src, h_c;
     int npass = 0, use_cls = 0, ncls_w = 0;
     DBuf status;
     // scratch owned by the handle
@@ -483,6 +487,10 @@ int tfps_graph_create(tfps_graph** out, int64_t n, int64_t m,
     CUDA_TRY(g->status.alloc(sizeof(int)));
     CUDA_TRY(cudaMemsetAsync(g->status.p, 0, sizeof(int), st));
     CUDA_TRY(cudaStreamSynchronize(st));  // host vectors go out of scope
+    g->h_in_ptr.swap(h_in_ptr);
+    g->h_in_src.swap(h_in_src);
+    g->h_in_t.swap(h_in_t);
+    g->h_c.swap(h_c);
     holder.g = nullptr;
     *out = g;
     return TFPS_OK;
@@ -651,15 +659,38 @@ int tfps_devices_set(tfps_graph* g, int k, const int32_t* s, const int64_t* C, c
                                    g->f_t.as<long long>(), g->b_nbr.as<int>(), g->b_t.as<long long>(),
                                    g->xvert.as<unsigned long long>(), g->xw_f.as<unsigned long long>(),
                                    g->xnbr_f.as<unsigned long long>(), g->xw_b.as<unsigned long long>(), st));
+    g->fits32 = false;
     if (g->ncomb > 0 && n > 0) {
+        // worst-case critical path: every vertex on the slowest device, every edge over the slowest link
+        std::vector<int> order((size_t)n);
+        CUDA_TRY(cudaMemcpyAsync(order.data(), g->order.p, sizeof(int) * (size_t)n, cudaMemcpyDeviceToHost, st));
+        CUDA_TRY(cudaStreamSynchronize(st));
+        std::vector<long long> fin((size_t)n);
+        long long worst = 0;
+        for (int i = 0; i < n; ++i) {
+            const int v = order[i];
+            long long start = 0;
+            for (long long e = g->h_in_ptr[v]; e < g->h_in_ptr[v + 1]; ++e) {
+                const long long w = k > 1 ? (long long)(((u128)g->h_in_t[e] * (u128)scale + (u128)b_min - 1) / (u128)b_min) : 0;
+                start = std::max(start, fin[g->h_in_src[e]] + w);
+            }
+            fin[v] = start + (long long)(((u128)g->h_c[v] * (u128)scale + (u128)s_min - 1) / (u128)s_min);
+            worst = std::max(worst, fin[v]);
+        }
+        g->fits32 = worst < (1LL << 31) - 1;
         CUDA_TRY(g->V_f.reserve(sizeof(long long) * (size_t)m * g->ncomb + 16));
         CUDA_TRY(g->V_b.reserve(sizeof(long long) * (size_t)m * g->ncomb + 16));
+        if (g->fits32) {
+            CUDA_TRY(g->V32_f.reserve(sizeof(int) * (size_t)m * g->ncomb + 16));
+            CUDA_TRY(g->V32_b.reserve(sizeof(int) * (size_t)m * g->ncomb + 16));
+        }
         CUDA_TRY(launch_edge_values(n, g->f_eptr.as<int>(), g->xw_f.as<unsigned long long>(),
                                     g->xnbr_f.as<unsigned long long>(), g->xvert.as<unsigned long long>(),
-                                    g->comb_f.as<CombDiv>(), g->ncomb, g->V_f.as<long long>(), st));
+                                    g->comb_f.as<CombDiv>(), g->ncomb, g->V_f.as<long long>(),
+                                    g->fits32 ? g->V32_f.as<int>() : nullptr, st));
         CUDA_TRY(launch_edge_values(n, g->b_eptr.as<int>(), g->xw_b.as<unsigned long long>(), nullptr,
                                     g->xvert.as<unsigned long long>(), g->comb_b.as<CombDiv>(), g->ncomb,
-                                    g->V_b.as<long long>(), st));
+                                    g->V_b.as<long long>(), g->fits32 ? g->V32_b.as<int>() : nullptr, st));
     }
     CUDA_TRY(cudaStreamSynchronize(st));
     g->k = k;
@@ -785,12 +816,13 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
     // windowed pass: needs the precomputed edge values (simple device tables)
     bool use_window = sliced && g->ncomb > 0 && env_int("TFPS_WINDOW", 1) != 0;
     int win_R = 0;
+    const int level_bytes = (g->fits32 && env_int("TFPS_LEVEL32", 1) != 0) ? 4 : 8;
     if (use_window) {
         int r_need = 32;  // smallest power of two that keeps every edge inside the ring
         while (r_need < g->maxspan + CHUNK_V) r_need <<= 1;
         auto r_fit = [&](int c) {
-            const long long avail = (long long)g->smem_optin - 1024 - (long long)window_smem_bytes(k, g->ncomb, 0, c, warps);
-            const long long rmax = avail / (32LL * c * 9);
+            const long long avail = (long long)g->smem_optin - 1024 - (long long)window_smem_bytes(k, g->ncomb, 0, c, warps, level_bytes);
+            const long long rmax = avail / (32LL * c * (level_bytes + 1));
             int r = 0;
             for (int q = 32; q <= rmax && q <= (1 << 16); q <<= 1) r = q;
             return r;
@@ -813,7 +845,7 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
             win_R = std::min(q, r_fit(cpt));
         }
         if (win_R < CHUNK_V + 32) win_R = 0;
-        if (window_smem_bytes(k, g->ncomb, win_R, cpt, warps) > (size_t)g->smem_optin) use_window = false;
+        if (window_smem_bytes(k, g->ncomb, win_R, cpt, warps, level_bytes) > (size_t)g->smem_optin) use_window = false;
     }
 
     for (int pass = 0; pass < 2; ++pass) {
@@ -830,7 +862,8 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
             wp.num_chunks = fwd ? g->f_num_chunks : g->b_num_chunks;
             wp.src_end = (int)g->h_level_ptr[1];
             wp.npos = fwd ? g->npos_f.as<int>() : g->npos_b.as<int>();
-            wp.V = fwd ? g->V_f.as<long long>() : g->V_b.as<long long>();
+            wp.V = level_bytes == 4 ? (fwd ? g->V32_f.p : g->V32_b.p) : (fwd ? g->V_f.p : g->V_b.p);
+            wp.level_bytes = level_bytes;
             wp.cls2 = fwd ? g->cls2_f.as<uint8_t>() : g->cls2_b.as<uint8_t>();
             wp.ncomb = g->ncomb;
             wp.R = win_R;

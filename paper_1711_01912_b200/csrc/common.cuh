@@ -125,7 +125,8 @@ struct WindowPlan {
     int num_chunks;
     int src_end;
     const int* npos;             // [m] position of the neighbour (level-ordered adjacency of this direction)
-    const long long* V;          // [m][ncomb]
+    const void* V;               // [m][ncomb] edge values: int64, or int32 when level_bytes == 4
+    int level_bytes;             // 8, or 4 when every path length is known to fit int32
     const uint8_t* cls2;         // [k*k] comb id of (nb, vv)
     int ncomb;
     int R;                       // window length in positions: a power of two, or 0 for no window
@@ -155,9 +156,9 @@ cudaError_t launch_pass_level_sync(const PassArgs& a, bool fwd, const std::vecto
 cudaError_t launch_pass_sliced(const PassArgs& a, bool fwd, const SlicedPlan& plan, int cpt, int warps, bool table,
                                cudaStream_t st);
 cudaError_t launch_pass_window(const PassArgs& a, bool fwd, const WindowPlan& plan, int cpt, int warps, cudaStream_t st);
-size_t window_smem_bytes(int k, int ncomb, int R, int cpt, int warps);
+size_t window_smem_bytes(int k, int ncomb, int R, int cpt, int warps, int level_bytes);
 cudaError_t launch_edge_values(int n, const int* eptr, const unsigned long long* xw, const unsigned long long* xnbr,
-                               const unsigned long long* xvert, const CombDiv* comb, int ncomb, long long* V,
+                               const unsigned long long* xvert, const CombDiv* comb, int ncomb, long long* V, int* V32,
                                cudaStream_t st);
 cudaError_t launch_positions(int n, int m, const int* order, int* pos_of, const int* nbr_f, const int* nbr_b,
                              const int* eptr_f, int* npos_f, int* npos_b, int* maxspan, cudaStream_t st);

@@ -36,13 +36,6 @@ __device__ __forceinline__ void cp_async16(void* smem, const void* g)
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
 
-__device__ __forceinline__ long long shfl64(long long v, int src)
-{
-    int lo = __shfl_sync(FULL, (int)(unsigned)(unsigned long long)v, src);
-    int hi = __shfl_sync(FULL, (int)((unsigned long long)v >> 32), src);
-    return (long long)(((unsigned long long)(unsigned)hi << 32) | (unsigned)lo);
-}
-
 template <int CPT> struct IdWords { static constexpr int N = (CPT + 3) / 4; };
 
 template <int CPT>
@@ -103,22 +96,23 @@ struct Carve {
 
 __host__ __device__ inline size_t up16(size_t x) { return (x + 15) & ~(size_t)15; }
 
-__host__ __device__ inline Carve carve(int k, int ncomb, int R, int cpt, int warps)
+__host__ __device__ inline Carve carve(int k, int ncomb, int R, int cpt, int warps, int lsize)
 {
     Carve c;
     const size_t slice = 32 * (size_t)cpt;
     size_t o = 0;
     c.head = o; o += 3 * up16(sizeof(HeadBuf));
     c.edge_nbr = o;
-    c.edge_npos = c.edge_nbr + up16(sizeof(int) * CHUNK_E);
-    c.edge_V = c.edge_npos + up16(sizeof(int) * CHUNK_E);
-    c.edge_stride = (c.edge_V - c.edge_nbr) + up16(sizeof(long long) * CHUNK_E * (size_t)ncomb);
+    c.edge_npos = c.edge_nbr + up16(sizeof(int) * CHUNK_E) + 16;
+    c.edge_V = c.edge_npos + up16(sizeof(int) * CHUNK_E) + 16;
+    c.edge_stride = (c.edge_V - c.edge_nbr) + up16((size_t)lsize * CHUNK_E * (size_t)ncomb) + 16;
     o += 2 * c.edge_stride;
     c.ids = o; c.ids_stride = up16(CHUNK_V * slice); o += 2 * c.ids_stride;
     c.rt = o; o += up16(sizeof(DivConst) * (size_t)k);
     c.cls2 = o; o += up16((size_t)k * k);
-    c.cp = o; o += up16(sizeof(long long) * (size_t)warps * slice);
-    c.win_lev = o; o += up16(sizeof(long long) * (size_t)R * slice);
+    c.cp = c.ids;  // the id staging area doubles as the reduction buffer of the CP maxima after the last chunk
+    (void)warps;
+    c.win_lev = o; o += up16((size_t)lsize * (size_t)R * slice);
     c.win_id = o; o += up16((size_t)R * slice);
     c.total = o;
     return c;
@@ -164,6 +158,42 @@ template <int CPT> __device__ __forceinline__ void sts_levels(unsigned a, const 
         for (int i = 0; i < CPT; i += 2) sts_v2s64(a + 8 * i, v[i], v[i + 1]);
     }
 }
+// 32-bit level mode
+template <int CPT> __device__ __forceinline__ void lds_levels(unsigned a, int (&out)[CPT])
+{
+    if constexpr (CPT == 1) out[0] = (int)lds_u32(a);
+    else if constexpr (CPT == 2) asm volatile("ld.shared.v2.s32 {%0,%1}, [%2];" : "=r"(out[0]), "=r"(out[1]) : "r"(a));
+    else asm volatile("ld.shared.v4.s32 {%0,%1,%2,%3}, [%4];" : "=r"(out[0]), "=r"(out[1]), "=r"(out[2]), "=r"(out[3]) : "r"(a));
+}
+template <int CPT> __device__ __forceinline__ void sts_levels(unsigned a, const int (&v)[CPT])
+{
+    if constexpr (CPT == 1) sts_u32(a, (unsigned)v[0]);
+    else if constexpr (CPT == 2) asm volatile("st.shared.v2.s32 [%0], {%1,%2};" ::"r"(a), "r"(v[0]), "r"(v[1]) : "memory");
+    else asm volatile("st.shared.v4.s32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]) : "memory");
+}
+__device__ __forceinline__ long long lds_level1(unsigned a, long long) { return lds_s64(a); }
+__device__ __forceinline__ int lds_level1(unsigned a, int) { return (int)lds_u32(a); }
+// best = max(best, lu + w)
+__device__ __forceinline__ long long add_max(long long lu, long long w, long long best) { const long long v = lu + w; return v > best ? v : best; }
+__device__ __forceinline__ int add_max(int lu, int w, int best) { return __viaddmax_s32(lu, w, best); }
+
+// Copies `bytes` (a multiple of 4) from 4-byte aligned global memory into the staging area `dst_area`, keeping
+// the source's offset inside its 16-byte line so that the body moves as 16-byte cp.async; returns that offset.
+__device__ __forceinline__ unsigned stage_bytes(unsigned char* dst_area, const void* src, int bytes)
+{
+    const unsigned mis = (unsigned)((unsigned long long)src & 15ull);
+    unsigned char* dst = dst_area + mis;
+    const unsigned char* s = reinterpret_cast<const unsigned char*>(src);
+    int head = (int)((16u - mis) & 15u);
+    if (head > bytes) head = bytes;
+    const int body = (bytes - head) & ~15;
+    const int tail = bytes - head - body;
+    for (int i = threadIdx.x * 16; i < body; i += blockDim.x * 16) cp_async16(dst + head + i, s + head + i);
+    const int t4 = threadIdx.x * 4;
+    if (t4 < head) cp_async4(dst + t4, s + t4);
+    if (t4 < tail) cp_async4(dst + head + body + t4, s + head + body + t4);
+    return mis;
+}
 
 // Byte offsets of the shared-memory regions, computed on the host and passed as a kernel parameter.
 struct WinLayout {
@@ -174,12 +204,13 @@ struct WinLayout {
 };
 
 // ALL_STAGED: every chunk's adjacency fits the staging buffers (no vertex with more than CHUNK_E edges).
-template <int CPT, bool FWD, bool ALL_STAGED>
+template <int CPT, bool FWD, bool ALL_STAGED, typename LT>
 __global__ void __launch_bounds__(1024)
 pass_window_kernel(PassArgs a, WindowPlan wp, WinLayout L)
 {
     extern __shared__ __align__(16) unsigned char smem[];
     constexpr int SLICE = 32 * CPT;
+    constexpr unsigned LS = sizeof(LT);   // bytes of a level inside the block: 4 when every path length fits int32
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, wpb = blockDim.x >> 5;
     const int k = a.tab.k;
     const int ncomb = wp.ncomb;
@@ -203,11 +234,11 @@ pass_window_kernel(PassArgs a, WindowPlan wp, WinLayout L)
     const long long ldp = a.ldp;
     const int slice_bytes = (int)((ldp - slice0) < SLICE ? (ldp - slice0) : SLICE);
     const bool want_cp = a.cp != nullptr;
-    long long* cpmax = s_cp + ((size_t)warp * 32 + lane) * CPT;
+    long long cpmax[CPT];
 #pragma unroll
     for (int c = 0; c < CPT; ++c) cpmax[c] = 0;
     // per-lane shared addresses
-    const unsigned win_lev_lane = sbase + L.win_lev + 8u * (unsigned)(lane * CPT);
+    const unsigned win_lev_lane = sbase + L.win_lev + LS * (unsigned)(lane * CPT);
     const unsigned win_id_lane = sbase + L.win_id + (unsigned)(lane * CPT);
     const unsigned cls2_s = sbase + L.cls2;
 
@@ -223,25 +254,17 @@ pass_window_kernel(PassArgs a, WindowPlan wp, WinLayout L)
         }
         for (int i = threadIdx.x; i <= cnt; i += blockDim.x) cp_async4(&h.eoff[i], a.adj.eptr + p0 + i);
     };
-    auto stage_edges = [&](int4 ent, int slot) {
+    // returns the byte offsets at which the staged npos / nbr / V arrays start inside their areas
+    auto stage_edges = [&](int4 ent, int slot, unsigned (&mis)[3]) {
         const int e0 = ent.z, ecnt = ent.w;
+        mis[0] = mis[1] = mis[2] = 0;
         if (!ALL_STAGED && ecnt > CHUNK_E) return;  // read from global memory instead
         unsigned char* base = smem + (unsigned)slot * L.edge_stride;
-        int* npos = reinterpret_cast<int*>(base + L.edge_npos);
-        long long* V = reinterpret_cast<long long*>(base + L.edge_V);
-        for (int i = threadIdx.x; i < ecnt; i += blockDim.x) cp_async4(&npos[i], wp.npos + e0 + i);
-        if (hit_span < wp.maxspan || !ALL_STAGED) {  // neighbour ids are only needed for window misses
-            int* nbr = reinterpret_cast<int*>(base + L.edge_nbr);
-            for (int i = threadIdx.x; i < ecnt; i += blockDim.x) cp_async4(&nbr[i], a.adj.nbr + e0 + i);
-        }
-        const long long* Vg = wp.V + (long long)e0 * ncomb;
-        const int nv = ecnt * ncomb;
-        if ((((long long)e0 * ncomb) & 1) == 0) {   // 16-byte aligned source: copy pairs
-            for (int i = threadIdx.x; i < (nv >> 1); i += blockDim.x) cp_async16(&V[2 * i], Vg + 2 * i);
-            if ((nv & 1) && threadIdx.x == 0) cp_async8(&V[nv - 1], Vg + nv - 1);
-        } else {
-            for (int i = threadIdx.x; i < nv; i += blockDim.x) cp_async8(&V[i], Vg + i);
-        }
+        mis[0] = stage_bytes(base + L.edge_npos, wp.npos + e0, ecnt * 4);
+        if (hit_span < wp.maxspan || !ALL_STAGED)  // neighbour ids are only needed for window misses
+            mis[1] = stage_bytes(base + L.edge_nbr, a.adj.nbr + e0, ecnt * 4);
+        const unsigned char* Vg = reinterpret_cast<const unsigned char*>(wp.V) + (long long)e0 * ncomb * (long long)LS;
+        mis[2] = stage_bytes(base + L.edge_V, Vg, ecnt * ncomb * (int)LS);
     };
     auto stage_ids = [&](int4 ent, int head_slot, int slot) {
         const HeadBuf& h = *reinterpret_cast<const HeadBuf*>(smem + L.head + (unsigned)head_slot * L.head_stride);
@@ -258,9 +281,10 @@ pass_window_kernel(PassArgs a, WindowPlan wp, WinLayout L)
     int4 cur = entry(0);
     int4 nxt = num_chunks > 1 ? entry(1) : cur;
     int4 nxt2 = num_chunks > 2 ? entry(2) : cur;
+    unsigned mis_cur[3], mis_nxt[3] = {0, 0, 0};
     stage_head(cur, 0);
     if (num_chunks > 1) stage_head(nxt, 1);
-    stage_edges(cur, 0);
+    stage_edges(cur, 0, mis_cur);
     cp_async_commit();
     cp_async_wait_all();
     __syncthreads();
@@ -276,7 +300,7 @@ pass_window_kernel(PassArgs a, WindowPlan wp, WinLayout L)
         int4 nxt3 = nxt2;
         if (ci + 1 < num_chunks) {
             stage_ids(nxt, hs1, (ci + 1) & 1);
-            stage_edges(nxt, (ci + 1) & 1);
+            stage_edges(nxt, (ci + 1) & 1, mis_nxt);
             if (ci + 2 < num_chunks) {
                 stage_head(nxt2, hs2);
                 if (ci + 3 < num_chunks) nxt3 = entry(ci + 3);
@@ -290,9 +314,9 @@ pass_window_kernel(PassArgs a, WindowPlan wp, WinLayout L)
         const int p0 = cur.x, cnt = cur.y, e0 = cur.z;
         const bool staged = ALL_STAGED || cur.w <= CHUNK_E;
         const unsigned ebase_s = sbase + (unsigned)(ci & 1) * L.edge_stride;
-        const unsigned npos_s = ebase_s + L.edge_npos;
-        const unsigned nbr_s = ebase_s + L.edge_nbr;
-        const unsigned V_s = ebase_s + L.edge_V;
+        const unsigned npos_s = ebase_s + L.edge_npos + mis_cur[0];
+        const unsigned nbr_s = ebase_s + L.edge_nbr + mis_cur[1];
+        const unsigned V_s = ebase_s + L.edge_V + mis_cur[2];
         const unsigned idrow_lane = sbase + L.ids + (unsigned)(ci & 1) * L.ids_stride + (unsigned)lane_col;
 
         for (int i = warp; i < cnt; i += wpb) {
@@ -303,7 +327,7 @@ pass_window_kernel(PassArgs a, WindowPlan wp, WinLayout L)
             unsigned cls_v[CPT];   // shared address of cls2[0*k + idv]
 #pragma unroll
             for (int c = 0; c < CPT; ++c) cls_v[c] = cls2_s + ((pv >> (8 * c)) & 0xffu);
-            long long best[CPT];
+            LT best[CPT];
 #pragma unroll
             for (int c = 0; c < CPT; ++c) best[c] = 0;
             const int ea_abs = (int)lds_u32(eoff_s + 4u * i), eb_abs = (int)lds_u32(eoff_s + 4u * i + 4u);
@@ -312,25 +336,27 @@ pass_window_kernel(PassArgs a, WindowPlan wp, WinLayout L)
                 for (int e = ea; e < eb; ++e) {
                     const int np = (int)lds_u32(npos_s + 4u * e);
                     const int span = FWD ? pos - np : np - pos;
-                    long long lu[CPT];
+                    LT lu[CPT];
                     unsigned pu;
                     if (span <= hit_span) {
                         const unsigned slot = (unsigned)(np & rmask);
-                        lds_levels<CPT>(win_lev_lane + slot * (8u * SLICE), lu);
+                        lds_levels<CPT>(win_lev_lane + slot * (LS * SLICE), lu);
                         pu = lds_ids<CPT>(win_id_lane + slot * (unsigned)SLICE);
                     } else {
                         const long long off = (long long)(int)lds_u32(nbr_s + 4u * e) * ldp + jl;
-                        load_levels<CPT>(a.lev + off, lu);
+                        long long lg[CPT];
+                        load_levels<CPT>(a.lev + off, lg);
+#pragma unroll
+                        for (int c = 0; c < CPT; ++c) lu[c] = (LT)lg[c];
                         unsigned w[IdWords<CPT>::N];
                         load_ids<CPT>(a.part + off, w);
                         pu = w[0] & idmask;
                     }
-                    const unsigned vrow = V_s + 8u * (unsigned)(e * ncomb);
+                    const unsigned vrow = V_s + LS * (unsigned)(e * ncomb);
 #pragma unroll
                     for (int c = 0; c < CPT; ++c) {
                         const unsigned cls = lds_u8(cls_v[c] + ((pu >> (8 * c)) & 0xffu) * (unsigned)k);
-                        const long long val = lu[c] + lds_s64(vrow + 8u * cls);
-                        best[c] = val > best[c] ? val : best[c];
+                        best[c] = add_max(lu[c], lds_level1(vrow + LS * cls, LT()), best[c]);
                     }
                 }
             } else {
@@ -338,25 +364,27 @@ pass_window_kernel(PassArgs a, WindowPlan wp, WinLayout L)
                 for (int e = ea_abs; e < eb_abs; ++e) {
                     const int np = wp.npos[e];
                     const int span = FWD ? pos - np : np - pos;
-                    long long lu[CPT];
+                    LT lu[CPT];
                     unsigned pu;
                     if (span <= hit_span) {
                         const unsigned slot = (unsigned)(np & rmask);
-                        lds_levels<CPT>(win_lev_lane + slot * (8u * SLICE), lu);
+                        lds_levels<CPT>(win_lev_lane + slot * (LS * SLICE), lu);
                         pu = lds_ids<CPT>(win_id_lane + slot * (unsigned)SLICE);
                     } else {
                         const long long off = (long long)a.adj.nbr[e] * ldp + jl;
-                        load_levels<CPT>(a.lev + off, lu);
+                        long long lg[CPT];
+                        load_levels<CPT>(a.lev + off, lg);
+#pragma unroll
+                        for (int c = 0; c < CPT; ++c) lu[c] = (LT)lg[c];
                         unsigned w[IdWords<CPT>::N];
                         load_ids<CPT>(a.part + off, w);
                         pu = w[0] & idmask;
                     }
-                    const long long* vrow = wp.V + (long long)e * ncomb;
+                    const LT* vrow = reinterpret_cast<const LT*>(wp.V) + (long long)e * ncomb;
 #pragma unroll
                     for (int c = 0; c < CPT; ++c) {
                         const unsigned cls = lds_u8(cls_v[c] + ((pu >> (8 * c)) & 0xffu) * (unsigned)k);
-                        const long long val = lu[c] + vrow[cls];
-                        best[c] = val > best[c] ? val : best[c];
+                        best[c] = add_max(lu[c], vrow[cls], best[c]);
                     }
                 }
             }
@@ -366,12 +394,12 @@ pass_window_kernel(PassArgs a, WindowPlan wp, WinLayout L)
                 if (!FWD && ea_abs == eb_abs) {  // sink: blevel = own runtime
 #pragma unroll
                     for (int c = 0; c < CPT; ++c)
-                        best[c] = Xv != NUM_ZERO ? ceil_quot(Xv, s_rt[(pv >> (8 * c)) & 0xffu]) : 0;
+                        best[c] = Xv != NUM_ZERO ? (LT)ceil_quot(Xv, s_rt[(pv >> (8 * c)) & 0xffu]) : (LT)0;
                 }
                 if (is_cp) {
 #pragma unroll
                     for (int c = 0; c < CPT; ++c) {
-                        long long fin = best[c];
+                        long long fin = (long long)best[c];
                         if (FWD && Xv != NUM_ZERO) fin += ceil_quot(Xv, s_rt[(pv >> (8 * c)) & 0xffu]);
                         cpmax[c] = fin > cpmax[c] ? fin : cpmax[c];
                     }
@@ -379,24 +407,33 @@ pass_window_kernel(PassArgs a, WindowPlan wp, WinLayout L)
             }
             // results: global memory (the output) and the window
             long long* gout = a.lev + (long long)v * ldp + jl;
-            if (nvalid >= CPT) store_levels<CPT>(gout, best);
+            long long wide[CPT];
+#pragma unroll
+            for (int c = 0; c < CPT; ++c) wide[c] = (long long)best[c];
+            if (nvalid >= CPT) store_levels<CPT>(gout, wide);
             else {
 #pragma unroll
                 for (int c = 0; c < CPT; ++c)
-                    if (c < nvalid) gout[c] = best[c];
+                    if (c < nvalid) gout[c] = wide[c];
             }
             if (R > 0) {
                 const unsigned slot = (unsigned)(pos & rmask);
-                sts_levels<CPT>(win_lev_lane + slot * (8u * SLICE), best);
+                sts_levels<CPT>(win_lev_lane + slot * (LS * SLICE), best);
                 sts_ids<CPT>(win_id_lane + slot * (unsigned)SLICE, pv);
             }
         }
         cp_async_wait_all();
         __syncthreads();
         cur = nxt; nxt = nxt2; nxt2 = nxt3;
+        mis_cur[0] = mis_nxt[0]; mis_cur[1] = mis_nxt[1]; mis_cur[2] = mis_nxt[2];
         hslot = hs1;
     }
 
+    if (want_cp) {
+#pragma unroll
+        for (int c = 0; c < CPT; ++c) s_cp[((size_t)warp * 32 + lane) * CPT + c] = cpmax[c];
+        __syncthreads();
+    }
     if (want_cp && warp == 0) {
 #pragma unroll
         for (int c = 0; c < CPT; ++c) {
@@ -413,7 +450,7 @@ pass_window_kernel(PassArgs a, WindowPlan wp, WinLayout L)
 // ---- set-up kernels ---------------------------------------------------------------------
 __global__ void edge_values_kernel(int n, const int* __restrict__ eptr, const unsigned long long* __restrict__ xw,
                                    const unsigned long long* __restrict__ xnbr, const unsigned long long* __restrict__ xvert,
-                                   const CombDiv* __restrict__ comb, int ncomb, long long* V)
+                                   const CombDiv* __restrict__ comb, int ncomb, long long* V, int* V32)
 {
     const long long gw = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
@@ -427,6 +464,7 @@ __global__ void edge_values_kernel(int n, const int* __restrict__ eptr, const un
         if (cd.w.pad == 0 && X != NUM_ZERO) t = ceil_quot(X, cd.w);
         if (Xr != NUM_ZERO) t += ceil_quot(Xr, cd.s);
         V[(long long)e * ncomb + lane] = t;
+        if (V32) V32[(long long)e * ncomb + lane] = (int)t;
     }
 }
 
@@ -459,10 +497,10 @@ __global__ void npos_kernel(int n, const int* __restrict__ pos_of, const int* __
 
 inline unsigned cdivu(long long a, long long b) { return (unsigned)((a + b - 1) / b); }
 
-template <int CPT, bool FWD, bool ALL_STAGED>
+template <int CPT, bool FWD, bool ALL_STAGED, typename LT>
 cudaError_t window_impl(const PassArgs& a, const WindowPlan& plan, int warps, cudaStream_t st)
 {
-    const Carve c = carve(a.tab.k, plan.ncomb, plan.R, CPT, warps);
+    const Carve c = carve(a.tab.k, plan.ncomb, plan.R, CPT, warps, (int)sizeof(LT));
     WinLayout L;
     L.head = (unsigned)c.head; L.head_stride = (unsigned)up16(sizeof(HeadBuf));
     L.edge_nbr = (unsigned)c.edge_nbr; L.edge_npos = (unsigned)c.edge_npos; L.edge_V = (unsigned)c.edge_V;
@@ -470,40 +508,48 @@ cudaError_t window_impl(const PassArgs& a, const WindowPlan& plan, int warps, cu
     L.ids = (unsigned)c.ids; L.ids_stride = (unsigned)c.ids_stride;
     L.rt = (unsigned)c.rt; L.cls2 = (unsigned)c.cls2; L.cp = (unsigned)c.cp;
     L.win_lev = (unsigned)c.win_lev; L.win_id = (unsigned)c.win_id;
-    cudaError_t e = cudaFuncSetAttribute(pass_window_kernel<CPT, FWD, ALL_STAGED>,
+    cudaError_t e = cudaFuncSetAttribute(pass_window_kernel<CPT, FWD, ALL_STAGED, LT>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c.total);
     if (e != cudaSuccess) return e;
-    pass_window_kernel<CPT, FWD, ALL_STAGED><<<cdivu(a.P, 32 * CPT), warps * 32, c.total, st>>>(a, plan, L);
+    pass_window_kernel<CPT, FWD, ALL_STAGED, LT><<<cdivu(a.P, 32 * CPT), warps * 32, c.total, st>>>(a, plan, L);
     count_launches(1);
     return cudaGetLastError();
 }
 
-template <int CPT>
+template <int CPT, typename LT>
 cudaError_t window_dispatch(const PassArgs& a, bool fwd, const WindowPlan& plan, int warps, cudaStream_t st)
 {
     if (plan.all_staged)
-        return fwd ? window_impl<CPT, true, true>(a, plan, warps, st) : window_impl<CPT, false, true>(a, plan, warps, st);
-    return fwd ? window_impl<CPT, true, false>(a, plan, warps, st) : window_impl<CPT, false, false>(a, plan, warps, st);
+        return fwd ? window_impl<CPT, true, true, LT>(a, plan, warps, st) : window_impl<CPT, false, true, LT>(a, plan, warps, st);
+    return fwd ? window_impl<CPT, true, false, LT>(a, plan, warps, st) : window_impl<CPT, false, false, LT>(a, plan, warps, st);
 }
 
 }  // namespace
 
-size_t window_smem_bytes(int k, int ncomb, int R, int cpt, int warps) { return carve(k, ncomb, R, cpt, warps).total; }
+size_t window_smem_bytes(int k, int ncomb, int R, int cpt, int warps, int level_bytes)
+{
+    return carve(k, ncomb, R, cpt, warps, level_bytes).total;
+}
 
 cudaError_t launch_pass_window(const PassArgs& a, bool fwd, const WindowPlan& plan, int cpt, int warps, cudaStream_t st)
 {
     if (plan.num_chunks <= 0) return cudaSuccess;
-    if (cpt == 4) return window_dispatch<4>(a, fwd, plan, warps, st);
-    if (cpt == 2) return window_dispatch<2>(a, fwd, plan, warps, st);
-    return window_dispatch<1>(a, fwd, plan, warps, st);
+    if (plan.level_bytes == 4) {
+        if (cpt == 4) return window_dispatch<4, int>(a, fwd, plan, warps, st);
+        if (cpt == 2) return window_dispatch<2, int>(a, fwd, plan, warps, st);
+        return window_dispatch<1, int>(a, fwd, plan, warps, st);
+    }
+    if (cpt == 4) return window_dispatch<4, long long>(a, fwd, plan, warps, st);
+    if (cpt == 2) return window_dispatch<2, long long>(a, fwd, plan, warps, st);
+    return window_dispatch<1, long long>(a, fwd, plan, warps, st);
 }
 
 cudaError_t launch_edge_values(int n, const int* eptr, const unsigned long long* xw, const unsigned long long* xnbr,
-                               const unsigned long long* xvert, const CombDiv* comb, int ncomb, long long* V,
+                               const unsigned long long* xvert, const CombDiv* comb, int ncomb, long long* V, int* V32,
                                cudaStream_t st)
 {
     if (n <= 0) return cudaSuccess;
-    edge_values_kernel<<<cdivu((long long)n * 32, 256), 256, 0, st>>>(n, eptr, xw, xnbr, xvert, comb, ncomb, V);
+    edge_values_kernel<<<cdivu((long long)n * 32, 256), 256, 0, st>>>(n, eptr, xw, xnbr, xvert, comb, ncomb, V, V32);
     count_launches(1);
     return cudaGetLastError();
 }

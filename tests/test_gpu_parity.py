@@ -371,9 +371,10 @@ def _shape_cases(seed):
     return cases
 
 
+@pytest.mark.parametrize("level32", [0, 1])
 @pytest.mark.parametrize("win_r", [-1, 160, 0])
 @pytest.mark.parametrize("cpt", [1, 2, 4])
-def test_windowed_kernel_shapes(cpt, win_r, monkeypatch):
+def test_windowed_kernel_shapes(cpt, win_r, level32, monkeypatch):
     """The windowed pass with the whole window resident (-1: automatic), with a
     window too short for many edges (hits and misses mixed) and with no window at
     all, for every lane width; the cases with many distinct costs or k > 16 fall
@@ -382,6 +383,7 @@ def test_windowed_kernel_shapes(cpt, win_r, monkeypatch):
     monkeypatch.setenv("TFPS_SLICED_WARPS", "8")
     monkeypatch.setenv("TFPS_WINDOW", "1")
     monkeypatch.setenv("TFPS_WINDOW_R", str(win_r))
+    monkeypatch.setenv("TFPS_LEVEL32", str(level32))  # 32-bit levels inside the block when every path fits int32
     for g, dev, part in _shape_cases(cpt * 2 + 1):
         run_and_compare(g, dev, part, 2, pad_fill=255)
     w = I.config2()
