@@ -112,6 +112,7 @@ struct tfps_graph {
     DBuf vertf, f_chunks, b_chunks;
     int f_num_chunks = 0, b_num_chunks = 0;
     bool f_all_staged = true, b_all_staged = true;
+    int max_chunk_v = 1;
     // device tables
     bool dev_set = false;
     int k = 0;
@@ -122,6 +123,10 @@ struct tfps_graph {
     DBuf pos_of, npos_f, npos_b, cls2_f, cls2_b, comb_f, comb_b, V_f, V_b, V32_f, V32_b;
     int ncomb = 0, maxspan = 0, smem_optin = 0;
     bool fits32 = false;  // every path length under any partition fits int32
+    // packed chunk records of the windowed pass, [direction][0: int64 values, 1: int32 values]
+    DBuf blob[2][2], blob_desc[2][2];
+    int blob_head_max[2][2] = {}, blob_body_max[2][2] = {};
+    std::vector<int> h_chunks[2];
     // host copies of the in-edge CSR for the worst-case path bound
     std::vector<long long> h_in_ptr, h_in_t;
     std::vector<int> h_in_src, h_c;
@@ -286,10 +291,12 @@ int build_topo(tfps_graph* g, cudaStream_t st)
                 chunks.push_back(eptr[p]);
                 chunks.push_back(eptr[q] - eptr[p]);
                 if (eptr[q] - eptr[p] > CHUNK_E) (dir == 0 ? g->f_all_staged : g->b_all_staged) = false;
+                g->max_chunk_v = std::max(g->max_chunk_v, q - p);
                 p = q;
             }
         }
         (dir == 0 ? g->f_num_chunks : g->b_num_chunks) = (int)(chunks.size() / 4);
+        g->h_chunks[dir] = chunks;
         TFPS_TRY(upload(dir == 0 ? g->f_chunks : g->b_chunks, chunks, st));
         CUDA_TRY(cudaStreamSynchronize(st));
     }
@@ -692,6 +699,49 @@ int tfps_devices_set(tfps_graph* g, int k, const int32_t* s, const int64_t* C, c
                                     g->xvert.as<unsigned long long>(), g->comb_b.as<CombDiv>(), g->ncomb,
                                     g->V_b.as<long long>(), g->fits32 ? g->V32_b.as<int>() : nullptr, st));
     }
+    if (g->ncomb > 0 && n > 0) {
+        auto up16 = [](size_t x) { return (x + 15) & ~(size_t)15; };
+        for (int dir = 0; dir < 2; ++dir)
+            for (int narrow = 0; narrow < (g->fits32 ? 2 : 1); ++narrow) {
+                const size_t ls = narrow ? 4 : 8;
+                const std::vector<int>& ch = g->h_chunks[dir];
+                const int nc = (int)(ch.size() / 4);
+                std::vector<int> desc((size_t)nc * 8, 0);
+                size_t off = 0;
+                int head_max = 16, body_max = 16;
+                for (int c = 0; c < nc; ++c) {
+                    const size_t cnt = (size_t)ch[4 * c + 1];
+                    const size_t es = ch[4 * c + 3] <= CHUNK_E ? (size_t)ch[4 * c + 3] : 0;
+                    const size_t head = 16 + up16(4 * cnt);
+                    const size_t nbr_bytes = up16(4 * es);
+                    const size_t body = up16(4 * (cnt + 1)) + up16(8 * cnt) + up16(4 * es) + up16(ls * es * (size_t)g->ncomb) + nbr_bytes;
+                    desc[8 * c + 0] = (int)(off / 16);
+                    desc[8 * c + 1] = (int)head;
+                    off += head;
+                    desc[8 * c + 2] = (int)(off / 16);
+                    desc[8 * c + 3] = (int)body;
+                    off += body;
+                    desc[8 * c + 4] = (int)(body - nbr_bytes);
+                    desc[8 * c + 5] = (int)cnt;
+                    head_max = std::max(head_max, (int)head);
+                    body_max = std::max(body_max, (int)body);
+                }
+                if (off / 16 >= (size_t)1 << 31) return fail(TFPS_ERR_UNSUPPORTED, "chunk records exceed 32 GiB");
+                g->blob_head_max[dir][narrow] = head_max;
+                g->blob_body_max[dir][narrow] = body_max;
+                CUDA_TRY(g->blob[dir][narrow].reserve(off + 16));
+                TFPS_TRY(upload(g->blob_desc[dir][narrow], desc, st));
+                const void* V = narrow ? (dir == 0 ? g->V32_f.p : g->V32_b.p) : (dir == 0 ? g->V_f.p : g->V_b.p);
+                CUDA_TRY(launch_pack_chunks(nc, dir == 0 ? g->f_chunks.as<int>() : g->b_chunks.as<int>(),
+                                            g->blob_desc[dir][narrow].as<int>(), g->vertf.as<int>(),
+                                            dir == 0 ? g->f_eptr.as<int>() : g->b_eptr.as<int>(),
+                                            g->xvert.as<unsigned long long>(),
+                                            dir == 0 ? g->npos_f.as<int>() : g->npos_b.as<int>(),
+                                            dir == 0 ? g->f_nbr.as<int>() : g->b_nbr.as<int>(), V, g->ncomb, (int)ls,
+                                            g->blob[dir][narrow].as<unsigned char>(), st));
+                CUDA_TRY(cudaStreamSynchronize(st));  // desc (host vector) was uploaded asynchronously
+            }
+    }
     CUDA_TRY(cudaStreamSynchronize(st));
     g->k = k;
     g->S = scale;
@@ -814,38 +864,53 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
 
     if (profile) CUDA_TRY(cudaEventRecord(g->ev[1], st));
     // windowed pass: needs the precomputed edge values (simple device tables)
-    bool use_window = sliced && g->ncomb > 0 && env_int("TFPS_WINDOW", 1) != 0;
-    int win_R = 0;
+    // (its bulk copies of id rows need a 16-byte aligned id matrix)
+    bool use_window = sliced && g->ncomb > 0 && env_int("TFPS_WINDOW", 1) != 0 && ((uintptr_t)part & 15u) == 0;
+    int win_R = 0, win_depth = 1;
     const int level_bytes = (g->fits32 && env_int("TFPS_LEVEL32", 1) != 0) ? 4 : 8;
+    const int narrow = level_bytes == 4 ? 1 : 0;
+    const int head_max = std::max(g->blob_head_max[0][narrow], g->blob_head_max[1][narrow]);
+    const int body_max = std::max(g->blob_body_max[0][narrow], g->blob_body_max[1][narrow]);
     if (use_window) {
         int r_need = 32;  // smallest power of two that keeps every edge inside the ring
         while (r_need < g->maxspan + CHUNK_V) r_need <<= 1;
-        auto r_fit = [&](int c) {
-            const long long avail = (long long)g->smem_optin - 1024 - (long long)window_smem_bytes(k, g->ncomb, 0, c, warps, level_bytes);
+        auto r_fit = [&](int c, int d) {
+            const long long avail = (long long)g->smem_optin - 1024 -
+                                    (long long)window_smem_bytes(k, 0, c, warps, level_bytes, g->max_chunk_v, head_max, body_max, d);
             const long long rmax = avail / (32LL * c * (level_bytes + 1));
             int r = 0;
             for (int q = 32; q <= rmax && q <= (1 << 16); q <<= 1) r = q;
             return r;
         };
+        // staging depth: about 256 vertices of adjacency and ids in flight ahead of the chunk being processed
+        int d_want = env_int("TFPS_WINDOW_DEPTH", 0);
+        if (d_want < 1 || d_want > 8) d_want = std::max(2, std::min(8, (256 + g->max_chunk_v - 1) / g->max_chunk_v));
         const int forced = env_int("TFPS_SLICED_CPT", 0);
         int chosen = 0;
         if (forced == 1 || forced == 2 || forced == 4) chosen = forced;
-        else {
-            const long long want_slices = std::min<long long>((3LL * g->sm_count) / 4, (P + 31) / 32);
-            for (int c = 4; c >= 1 && !chosen; c >>= 1)      // widest lane that still holds the whole window
-                if (r_fit(c) >= r_need && (P + 32 * c - 1) / (32 * c) >= want_slices) chosen = c;
-            if (!chosen) chosen = cpt > 4 ? 4 : cpt;          // partial window at the width the slice count allows
+        const long long want_slices = std::min<long long>((3LL * g->sm_count) / 4, (P + 31) / 32);
+        win_depth = 0;
+        for (int c = chosen ? chosen : 4; c >= 1 && !win_depth; c >>= 1) {   // widest lane that holds the whole window
+            if (!chosen && (P + 32 * c - 1) / (32 * c) < want_slices && c > 1) continue;
+            for (int d = d_want; d >= 1 && !win_depth; --d)
+                if (r_fit(c, d) >= r_need) { cpt = c; win_depth = d; }
+            if (chosen) break;
         }
-        cpt = chosen;
-        win_R = std::min(r_fit(cpt), r_need);
+        if (!win_depth) {   // partial window at the width the slice count allows
+            cpt = chosen ? chosen : (cpt > 4 ? 4 : cpt);
+            win_depth = std::min(d_want, 2);
+        }
+        win_R = std::min(r_fit(cpt, win_depth), r_need);
         const int forced_r = env_int("TFPS_WINDOW_R", -1);
         if (forced_r >= 0) {
             int q = 0;
             for (int t = 32; t <= forced_r; t <<= 1) q = t;
-            win_R = std::min(q, r_fit(cpt));
+            win_R = std::min(q, r_fit(cpt, win_depth));
         }
         if (win_R < CHUNK_V + 32) win_R = 0;
-        if (window_smem_bytes(k, g->ncomb, win_R, cpt, warps, level_bytes) > (size_t)g->smem_optin) use_window = false;
+        if (window_smem_bytes(k, win_R, cpt, warps, level_bytes, g->max_chunk_v, head_max, body_max, win_depth) >
+            (size_t)g->smem_optin)
+            use_window = false;
     }
 
     for (int pass = 0; pass < 2; ++pass) {
@@ -864,6 +929,12 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
             wp.npos = fwd ? g->npos_f.as<int>() : g->npos_b.as<int>();
             wp.V = level_bytes == 4 ? (fwd ? g->V32_f.p : g->V32_b.p) : (fwd ? g->V_f.p : g->V_b.p);
             wp.level_bytes = level_bytes;
+            wp.desc = g->blob_desc[fwd ? 0 : 1][narrow].as<int>();
+            wp.blob = g->blob[fwd ? 0 : 1][narrow].as<unsigned char>();
+            wp.max_v = g->max_chunk_v;
+            wp.head_max = head_max;
+            wp.body_max = body_max;
+            wp.depth = win_depth;
             wp.cls2 = fwd ? g->cls2_f.as<uint8_t>() : g->cls2_b.as<uint8_t>();
             wp.ncomb = g->ncomb;
             wp.R = win_R;

@@ -98,7 +98,7 @@ struct PassArgs {
 // level with at most CHUNK_V vertices and CHUNK_E edges (a single vertex with more
 // edges forms a chunk of its own and is read straight from global memory).
 constexpr int CHUNK_V = 128;
-constexpr int CHUNK_E = 256;
+constexpr int CHUNK_E = 320;
 
 struct SlicedPlan {
     const int* vertf;    // [n] vertex id by position, bit 31 set for sinks
@@ -132,6 +132,12 @@ struct WindowPlan {
     int R;                       // window length in positions: a power of two, or 0 for no window
     int maxspan;                 // largest |pos(v) - pos(u)| over all edges
     int all_staged;              // no vertex has more than CHUNK_E edges
+    // packed chunk records staged by bulk copies: desc[2*c] = {head offset/16, head bytes, body offset/16, body bytes},
+    // desc[2*c+1] = {body bytes without the trailing neighbour-id array, vertices, 0, 0}
+    const int* desc;
+    const unsigned char* blob;
+    int max_v, head_max, body_max;  // largest chunk: vertices, head bytes, body bytes
+    int depth;                   // chunks staged ahead
 };
 
 // every kernel launch of the library goes through the wrappers below and is counted here
@@ -156,7 +162,10 @@ cudaError_t launch_pass_level_sync(const PassArgs& a, bool fwd, const std::vecto
 cudaError_t launch_pass_sliced(const PassArgs& a, bool fwd, const SlicedPlan& plan, int cpt, int warps, bool table,
                                cudaStream_t st);
 cudaError_t launch_pass_window(const PassArgs& a, bool fwd, const WindowPlan& plan, int cpt, int warps, cudaStream_t st);
-size_t window_smem_bytes(int k, int ncomb, int R, int cpt, int warps, int level_bytes);
+size_t window_smem_bytes(int k, int R, int cpt, int warps, int level_bytes, int max_v, int head_max, int body_max, int depth);
+cudaError_t launch_pack_chunks(int num_chunks, const int* chunks, const int* desc, const int* vertf, const int* eptr,
+                               const unsigned long long* xvert, const int* npos, const int* nbr, const void* V, int ncomb,
+                               int lsize, unsigned char* blob, cudaStream_t st);
 cudaError_t launch_edge_values(int n, const int* eptr, const unsigned long long* xw, const unsigned long long* xnbr,
                                const unsigned long long* xvert, const CombDiv* comb, int ncomb, long long* V, int* V32,
                                cudaStream_t st);

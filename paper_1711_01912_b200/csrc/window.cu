@@ -16,25 +16,47 @@ namespace tfps {
 
 namespace {
 
-constexpr unsigned FULL = 0xffffffffu;
-
-__device__ __forceinline__ void cp_async4(void* smem, const void* g)
+// ---- TMA bulk copies completing on an mbarrier ---------------------------------------------
+__device__ __forceinline__ void mbar_init(unsigned bar, unsigned count)
 {
-    unsigned s = (unsigned)__cvta_generic_to_shared(smem);
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(s), "l"(g));
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
-__device__ __forceinline__ void cp_async8(void* smem, const void* g)
+__device__ __forceinline__ void mbar_init_fence() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void mbar_expect_tx(unsigned bar, unsigned bytes)
 {
-    unsigned s = (unsigned)__cvta_generic_to_shared(smem);
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(s), "l"(g));
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ void cp_async16(void* smem, const void* g)
+// global -> shared bulk copy; both addresses 16-byte aligned, bytes a multiple of 16
+__device__ __forceinline__ void bulk_g2s(unsigned dst, const void* src, unsigned bytes, unsigned bar)
 {
-    unsigned s = (unsigned)__cvta_generic_to_shared(smem);
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(s), "l"(g));
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity)
+{
+    unsigned ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// 16-byte asynchronous copy through the load/store path, and the hook that makes an mbarrier count the
+// completion of all cp.async issued so far by this thread as one (pre-counted) arrival
+__device__ __forceinline__ void cp_async16(unsigned dst, const void* g)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(g) : "memory");
+}
+__device__ __forceinline__ void cp_async_arrive_on(unsigned bar)
+{
+    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
+}
+// Bounded wait: gives up after WAIT_LIMIT polls (each poll itself blocks for a hardware-defined time slice).
+constexpr int WAIT_LIMIT = 1 << 20;
+__device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity)
+{
+    for (int i = 0; i < WAIT_LIMIT; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
 
 template <int CPT> struct IdWords { static constexpr int N = (CPT + 3) / 4; };
 
@@ -82,128 +104,65 @@ __device__ __forceinline__ void store_levels(long long* p, const long long (&v)[
     }
 }
 
-struct HeadBuf {                 // per-vertex metadata of a chunk
-    unsigned long long xvert[CHUNK_V];
-    int vertf[CHUNK_V];
-    int eoff[CHUNK_V + 4];
-};
-
-// shared-memory carve-up (all offsets multiples of 16 bytes)
+// Shared-memory carve-up (all offsets multiples of 16 bytes).  Rings: chunk heads (2*depth+1 slots: a head
+// must have landed before the id rows of its chunk can be requested), chunk bodies and id rows (depth+1 each).
 struct Carve {
-    size_t head, edge_nbr, edge_npos, edge_V, ids, rt, cls2, cp, win_lev, win_id, total;
-    size_t edge_stride, ids_stride;
+    size_t bars, rt, cls2, cp, head, head_stride, body, body_stride, ids, ids_stride, win_lev, win_id, total;
 };
 
 __host__ __device__ inline size_t up16(size_t x) { return (x + 15) & ~(size_t)15; }
 
-__host__ __device__ inline Carve carve(int k, int ncomb, int R, int cpt, int warps, int lsize)
+__host__ __device__ inline Carve carve(int k, int R, int cpt, int warps, int lsize, int max_v, int head_max, int body_max,
+                                       int depth)
 {
     Carve c;
     const size_t slice = 32 * (size_t)cpt;
     size_t o = 0;
-    c.head = o; o += 3 * up16(sizeof(HeadBuf));
-    c.edge_nbr = o;
-    c.edge_npos = c.edge_nbr + up16(sizeof(int) * CHUNK_E) + 16;
-    c.edge_V = c.edge_npos + up16(sizeof(int) * CHUNK_E) + 16;
-    c.edge_stride = (c.edge_V - c.edge_nbr) + up16((size_t)lsize * CHUNK_E * (size_t)ncomb) + 16;
-    o += 2 * c.edge_stride;
-    c.ids = o; c.ids_stride = up16(CHUNK_V * slice); o += 2 * c.ids_stride;
+    c.bars = o; o += up16(8 * (size_t)(3 * depth + 2) + 8);
     c.rt = o; o += up16(sizeof(DivConst) * (size_t)k);
     c.cls2 = o; o += up16((size_t)k * k);
-    c.cp = c.ids;  // the id staging area doubles as the reduction buffer of the CP maxima after the last chunk
-    (void)warps;
+    c.cp = o;   // the staging rings double as the reduction buffer of the CP maxima after the last chunk
+    c.head = o; c.head_stride = up16((size_t)head_max); o += (size_t)(2 * depth + 1) * c.head_stride;
+    c.body = o; c.body_stride = up16((size_t)body_max); o += (size_t)(depth + 1) * c.body_stride;
+    c.ids = o; c.ids_stride = up16((size_t)max_v * slice); o += (size_t)(depth + 1) * c.ids_stride;
+    if (o < c.cp + sizeof(long long) * (size_t)warps * slice) o = up16(c.cp + sizeof(long long) * (size_t)warps * slice);
     c.win_lev = o; o += up16((size_t)lsize * (size_t)R * slice);
     c.win_id = o; o += up16((size_t)R * slice);
     c.total = o;
     return c;
 }
 
-// 32-bit shared-state-space accessors (addresses from __cvta_generic_to_shared)
-__device__ __forceinline__ unsigned lds_u8(unsigned a) { unsigned v; asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(a)); return v; }
-__device__ __forceinline__ unsigned lds_u16(unsigned a) { unsigned v; asm volatile("ld.shared.u16 %0, [%1];" : "=r"(v) : "r"(a)); return v; }
+// 32-bit shared-state-space load (address from __cvta_generic_to_shared)
 __device__ __forceinline__ unsigned lds_u32(unsigned a) { unsigned v; asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a)); return v; }
-__device__ __forceinline__ long long lds_s64(unsigned a) { long long v; asm volatile("ld.shared.s64 %0, [%1];" : "=l"(v) : "r"(a)); return v; }
-__device__ __forceinline__ void lds_v2s64(unsigned a, long long& x, long long& y) { asm volatile("ld.shared.v2.s64 {%0,%1}, [%2];" : "=l"(x), "=l"(y) : "r"(a)); }
-__device__ __forceinline__ void sts_s64(unsigned a, long long v) { asm volatile("st.shared.s64 [%0], %1;" ::"r"(a), "l"(v) : "memory"); }
-__device__ __forceinline__ void sts_v2s64(unsigned a, long long x, long long y) { asm volatile("st.shared.v2.s64 [%0], {%1,%2};" ::"r"(a), "l"(x), "l"(y) : "memory"); }
-__device__ __forceinline__ void sts_u8(unsigned a, unsigned v) { asm volatile("st.shared.u8 [%0], %1;" ::"r"(a), "r"(v) : "memory"); }
-__device__ __forceinline__ void sts_u16(unsigned a, unsigned v) { asm volatile("st.shared.u16 [%0], %1;" ::"r"(a), "r"(v) : "memory"); }
-__device__ __forceinline__ void sts_u32(unsigned a, unsigned v) { asm volatile("st.shared.u32 [%0], %1;" ::"r"(a), "r"(v) : "memory"); }
 
-template <int CPT> __device__ __forceinline__ unsigned lds_ids(unsigned a)
+// window rows through typed shared-memory pointers (vector width = CPT levels)
+template <int CPT> __device__ __forceinline__ void load_win(const long long* p, long long (&out)[CPT]) { load_levels<CPT>(p, out); }
+template <int CPT> __device__ __forceinline__ void store_win(long long* p, const long long (&v)[CPT]) { store_levels<CPT>(p, v); }
+template <int CPT> __device__ __forceinline__ void load_win(const int* p, int (&out)[CPT])
 {
-    if constexpr (CPT == 1) return lds_u8(a);
-    else if constexpr (CPT == 2) return lds_u16(a);
-    else return lds_u32(a);
+    if constexpr (CPT == 1) out[0] = *p;
+    else if constexpr (CPT == 2) { const int2 v = *reinterpret_cast<const int2*>(p); out[0] = v.x; out[1] = v.y; }
+    else { const int4 v = *reinterpret_cast<const int4*>(p); out[0] = v.x; out[1] = v.y; out[2] = v.z; out[3] = v.w; }
 }
-template <int CPT> __device__ __forceinline__ void sts_ids(unsigned a, unsigned v)
+template <int CPT> __device__ __forceinline__ void store_win(int* p, const int (&v)[CPT])
 {
-    if constexpr (CPT == 1) sts_u8(a, v);
-    else if constexpr (CPT == 2) sts_u16(a, v);
-    else sts_u32(a, v);
+    if constexpr (CPT == 1) *p = v[0];
+    else if constexpr (CPT == 2) *reinterpret_cast<int2*>(p) = make_int2(v[0], v[1]);
+    else *reinterpret_cast<int4*>(p) = make_int4(v[0], v[1], v[2], v[3]);
 }
-template <int CPT> __device__ __forceinline__ void lds_levels(unsigned a, long long (&out)[CPT])
-{
-    if constexpr (CPT == 1) out[0] = lds_s64(a);
-    else {
-#pragma unroll
-        for (int i = 0; i < CPT; i += 2) lds_v2s64(a + 8 * i, out[i], out[i + 1]);
-    }
-}
-template <int CPT> __device__ __forceinline__ void sts_levels(unsigned a, const long long (&v)[CPT])
-{
-    if constexpr (CPT == 1) sts_s64(a, v[0]);
-    else {
-#pragma unroll
-        for (int i = 0; i < CPT; i += 2) sts_v2s64(a + 8 * i, v[i], v[i + 1]);
-    }
-}
-// 32-bit level mode
-template <int CPT> __device__ __forceinline__ void lds_levels(unsigned a, int (&out)[CPT])
-{
-    if constexpr (CPT == 1) out[0] = (int)lds_u32(a);
-    else if constexpr (CPT == 2) asm volatile("ld.shared.v2.s32 {%0,%1}, [%2];" : "=r"(out[0]), "=r"(out[1]) : "r"(a));
-    else asm volatile("ld.shared.v4.s32 {%0,%1,%2,%3}, [%4];" : "=r"(out[0]), "=r"(out[1]), "=r"(out[2]), "=r"(out[3]) : "r"(a));
-}
-template <int CPT> __device__ __forceinline__ void sts_levels(unsigned a, const int (&v)[CPT])
-{
-    if constexpr (CPT == 1) sts_u32(a, (unsigned)v[0]);
-    else if constexpr (CPT == 2) asm volatile("st.shared.v2.s32 [%0], {%1,%2};" ::"r"(a), "r"(v[0]), "r"(v[1]) : "memory");
-    else asm volatile("st.shared.v4.s32 [%0], {%1,%2,%3,%4};" ::"r"(a), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]) : "memory");
-}
-__device__ __forceinline__ long long lds_level1(unsigned a, long long) { return lds_s64(a); }
-__device__ __forceinline__ int lds_level1(unsigned a, int) { return (int)lds_u32(a); }
 // best = max(best, lu + w)
 __device__ __forceinline__ long long add_max(long long lu, long long w, long long best) { const long long v = lu + w; return v > best ? v : best; }
 __device__ __forceinline__ int add_max(int lu, int w, int best) { return __viaddmax_s32(lu, w, best); }
 
-// Copies `bytes` (a multiple of 4) from 4-byte aligned global memory into the staging area `dst_area`, keeping
-// the source's offset inside its 16-byte line so that the body moves as 16-byte cp.async; returns that offset.
-__device__ __forceinline__ unsigned stage_bytes(unsigned char* dst_area, const void* src, int bytes)
-{
-    const unsigned mis = (unsigned)((unsigned long long)src & 15ull);
-    unsigned char* dst = dst_area + mis;
-    const unsigned char* s = reinterpret_cast<const unsigned char*>(src);
-    int head = (int)((16u - mis) & 15u);
-    if (head > bytes) head = bytes;
-    const int body = (bytes - head) & ~15;
-    const int tail = bytes - head - body;
-    for (int i = threadIdx.x * 16; i < body; i += blockDim.x * 16) cp_async16(dst + head + i, s + head + i);
-    const int t4 = threadIdx.x * 4;
-    if (t4 < head) cp_async4(dst + t4, s + t4);
-    if (t4 < tail) cp_async4(dst + head + body + t4, s + head + body + t4);
-    return mis;
-}
-
 // Byte offsets of the shared-memory regions, computed on the host and passed as a kernel parameter.
 struct WinLayout {
-    unsigned head, head_stride;
-    unsigned edge_nbr, edge_npos, edge_V, edge_stride;
-    unsigned ids, ids_stride;
-    unsigned rt, cls2, cp, win_lev, win_id;
+    unsigned bars, rt, cls2, cp, head, head_stride, body, body_stride, ids, ids_stride, win_lev, win_id;
+    int depth;
 };
 
 // ALL_STAGED: every chunk's adjacency fits the staging buffers (no vertex with more than CHUNK_E edges).
+// Warp 0 doubles as the producer: at the top of every chunk it issues the copies for the chunk `depth`
+// ahead (heads 2*depth ahead) before it takes its share of the vertices.
 template <int CPT, bool FWD, bool ALL_STAGED, typename LT>
 __global__ void __launch_bounds__(1024)
 pass_window_kernel(PassArgs a, WindowPlan wp, WinLayout L)
@@ -212,17 +171,31 @@ pass_window_kernel(PassArgs a, WindowPlan wp, WinLayout L)
     constexpr int SLICE = 32 * CPT;
     constexpr unsigned LS = sizeof(LT);   // bytes of a level inside the block: 4 when every path length fits int32
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, wpb = blockDim.x >> 5;
+    const bool producer = warp == 0;
     const int k = a.tab.k;
     const int ncomb = wp.ncomb;
     const int R = wp.R;              // power of two (or 0)
     const int rmask = R - 1;
     const int hit_span = R - CHUNK_V;  // a neighbour at most this many positions away is still in the ring
+    const bool need_nbr = hit_span < wp.maxspan;   // some neighbours are read from global memory
     const unsigned sbase = (unsigned)__cvta_generic_to_shared(smem);
     DivConst* s_rt = reinterpret_cast<DivConst*>(smem + L.rt);
     long long* s_cp = reinterpret_cast<long long*>(smem + L.cp);
+    volatile int* s_abort = reinterpret_cast<volatile int*>(smem + L.bars + 8 * (3 * L.depth + 2));
     if (*a.status != 0) return;
+    const int D = L.depth, NB = 2 * D + 1, NS = D + 1;
+    const unsigned head_bar0 = sbase + L.bars, stage_bar0 = head_bar0 + 8u * NB;
+    if (threadIdx.x == 0) {
+        for (int j = 0; j < NB; ++j) mbar_init(head_bar0 + 8u * j, 1);
+        // a stage completes on the body's bulk copy (one arrival with its byte count) plus one arrival per
+        // producer lane once that lane's id-row copies have landed
+        for (int j = 0; j < NS; ++j) mbar_init(stage_bar0 + 8u * j, 33);
+        *s_abort = 0;
+        mbar_init_fence();
+    }
     for (int i = threadIdx.x; i < k; i += blockDim.x) s_rt[i] = a.tab.rt_div[i];
     for (int i = threadIdx.x; i < k * k; i += blockDim.x) smem[L.cls2 + i] = wp.cls2[i];
+    __syncthreads();
 
     const long long slice0 = (long long)blockIdx.x * SLICE;
     const long long j0 = slice0 + (long long)lane * CPT;
@@ -232,201 +205,250 @@ pass_window_kernel(PassArgs a, WindowPlan wp, WinLayout L)
     const long long jl = slice0 + lane_col;
     const unsigned idmask = nvalid >= 4 ? 0xffffffffu : (nvalid > 0 ? ((1u << (8 * nvalid)) - 1u) : 0u);
     const long long ldp = a.ldp;
-    const int slice_bytes = (int)((ldp - slice0) < SLICE ? (ldp - slice0) : SLICE);
+    const unsigned slice_bytes = (unsigned)((ldp - slice0) < SLICE ? (ldp - slice0) : SLICE);  // multiple of 16
     const bool want_cp = a.cp != nullptr;
     long long cpmax[CPT];
 #pragma unroll
     for (int c = 0; c < CPT; ++c) cpmax[c] = 0;
-    // per-lane shared addresses
-    const unsigned win_lev_lane = sbase + L.win_lev + LS * (unsigned)(lane * CPT);
-    const unsigned win_id_lane = sbase + L.win_id + (unsigned)(lane * CPT);
-    const unsigned cls2_s = sbase + L.cls2;
-
-    const int4* chunks = reinterpret_cast<const int4*>(wp.chunks);
+    LT* win_lev_lane = reinterpret_cast<LT*>(smem + L.win_lev) + lane * CPT;
+    uint8_t* win_id_lane = smem + L.win_id + lane * CPT;
+    const unsigned char* s_cls2 = smem + L.cls2;
     const int num_chunks = wp.num_chunks;
-    auto entry = [&](int ci) { return chunks[FWD ? ci : num_chunks - 1 - ci]; };
-    auto stage_head = [&](int4 ent, int slot) {
-        HeadBuf& h = *reinterpret_cast<HeadBuf*>(smem + L.head + (unsigned)slot * L.head_stride);
-        const int p0 = ent.x, cnt = ent.y;
-        for (int i = threadIdx.x; i < cnt; i += blockDim.x) {
-            cp_async4(&h.vertf[i], wp.vertf + p0 + i);
-            cp_async8(&h.xvert[i], a.adj.xvert + p0 + i);
-        }
-        for (int i = threadIdx.x; i <= cnt; i += blockDim.x) cp_async4(&h.eoff[i], a.adj.eptr + p0 + i);
+    const int4* desc = reinterpret_cast<const int4*>(wp.desc);
+    const unsigned char* blob = reinterpret_cast<const unsigned char*>(wp.blob);
+
+    auto fail_wait = [&]() {
+        atomicCAS(a.status, 0, (int)TFPS_ERR_TIMEOUT);
+        *s_abort = 1;
     };
-    // returns the byte offsets at which the staged npos / nbr / V arrays start inside their areas
-    auto stage_edges = [&](int4 ent, int slot, unsigned (&mis)[3]) {
-        const int e0 = ent.z, ecnt = ent.w;
-        mis[0] = mis[1] = mis[2] = 0;
-        if (!ALL_STAGED && ecnt > CHUNK_E) return;  // read from global memory instead
-        unsigned char* base = smem + (unsigned)slot * L.edge_stride;
-        mis[0] = stage_bytes(base + L.edge_npos, wp.npos + e0, ecnt * 4);
-        if (hit_span < wp.maxspan || !ALL_STAGED)  // neighbour ids are only needed for window misses
-            mis[1] = stage_bytes(base + L.edge_nbr, a.adj.nbr + e0, ecnt * 4);
-        const unsigned char* Vg = reinterpret_cast<const unsigned char*>(wp.V) + (long long)e0 * ncomb * (long long)LS;
-        mis[2] = stage_bytes(base + L.edge_V, Vg, ecnt * ncomb * (int)LS);
-    };
-    auto stage_ids = [&](int4 ent, int head_slot, int slot) {
-        const HeadBuf& h = *reinterpret_cast<const HeadBuf*>(smem + L.head + (unsigned)head_slot * L.head_stride);
-        const int cnt = ent.y;
-        uint8_t* dst = smem + L.ids + (unsigned)slot * L.ids_stride;
-        const int per_row = slice_bytes >> 4;  // ldp and slice0 are multiples of 16
-        for (int i = threadIdx.x; i < cnt * per_row; i += blockDim.x) {
-            const int r = i / per_row, q = i - r * per_row;
-            const int v = h.vertf[r] & 0x7fffffff;
-            cp_async16(dst + r * SLICE + 16 * q, a.part + (long long)v * ldp + slice0 + 16 * q);
+    // ---- producer side -------------------------------------------------------------------------
+    // Descriptors of the coming chunks are fetched 32 at a time (one per lane) and handed out by shuffles, so
+    // the producer does not pay a global-memory round trip per chunk.
+    auto load_desc = [&](int first, int4& d0, int4& d1) {   // lane l gets the descriptor of chunk first+l
+        const int j = first + lane;
+        d0 = make_int4(0, 0, 0, 0); d1 = d0;
+        if (j < num_chunks) {
+            const int idx = FWD ? j : num_chunks - 1 - j;
+            d0 = desc[2 * idx];
+            d1 = desc[2 * idx + 1];
         }
     };
+    auto bcast = [&](const int4& v, int src) {
+        return make_int4(__shfl_sync(0xffffffffu, v.x, src), __shfl_sync(0xffffffffu, v.y, src),
+                         __shfl_sync(0xffffffffu, v.z, src), __shfl_sync(0xffffffffu, v.w, src));
+    };
+    auto issue_head = [&](const int4& d, int slot) {   // chunk -> head ring slot
+        if (lane == 0) {
+            const unsigned bar = head_bar0 + 8u * slot;
+            mbar_expect_tx(bar, (unsigned)d.y);
+            bulk_g2s(sbase + L.head + (unsigned)slot * L.head_stride, blob + 16ll * (unsigned)d.x, (unsigned)d.y, bar);
+        }
+    };
+    auto issue_stage = [&](const int4& d0, const int4& d1, int slot, int hslot, unsigned hpar) {   // body + id rows
+        // warp-uniform outcome: the lanes below meet at a __syncwarp
+        if (!__all_sync(0xffffffffu, mbar_wait(head_bar0 + 8u * hslot, hpar))) { fail_wait(); return; }
+        const int cnt = d1.y;
+        const unsigned body_bytes = (unsigned)((need_nbr || !ALL_STAGED) ? d0.w : d1.x);
+        const unsigned bar = stage_bar0 + 8u * slot;
+        if (lane == 0) {
+            mbar_expect_tx(bar, body_bytes);
+            bulk_g2s(sbase + L.body + (unsigned)slot * L.body_stride, blob + 16ll * (unsigned)d0.z, body_bytes, bar);
+        }
+        // id rows: short scattered pieces, cheaper as 16-byte cp.async than as one bulk copy each
+        const unsigned vertf_s = sbase + L.head + (unsigned)hslot * L.head_stride + 16u;
+        const unsigned ids_s = sbase + L.ids + (unsigned)slot * L.ids_stride;
+        const int sh = slice_bytes >= 128u ? 3 : (slice_bytes >= 64u ? 2 : (slice_bytes >= 32u ? 1 : 0));
+        const int per_row = (int)(slice_bytes >> 4);
+        if ((per_row & (per_row - 1)) == 0) {
+            for (int i = lane; i < (cnt << sh); i += 32) {
+                const int r = i >> sh, q = i & (per_row - 1);
+                const int v = (int)lds_u32(vertf_s + 4u * r) & 0x7fffffff;
+                cp_async16(ids_s + (unsigned)(r * SLICE + 16 * q), a.part + (long long)v * ldp + slice0 + 16 * q);
+            }
+        } else {
+            for (int i = lane; i < cnt * per_row; i += 32) {
+                const int r = i / per_row, q = i - r * per_row;
+                const int v = (int)lds_u32(vertf_s + 4u * r) & 0x7fffffff;
+                cp_async16(ids_s + (unsigned)(r * SLICE + 16 * q), a.part + (long long)v * ldp + slice0 + 16 * q);
+            }
+        }
+        cp_async_arrive_on(bar);
+    };
 
-    int4 cur = entry(0);
-    int4 nxt = num_chunks > 1 ? entry(1) : cur;
-    int4 nxt2 = num_chunks > 2 ? entry(2) : cur;
-    unsigned mis_cur[3], mis_nxt[3] = {0, 0, 0};
-    stage_head(cur, 0);
-    if (num_chunks > 1) stage_head(nxt, 1);
-    stage_edges(cur, 0, mis_cur);
-    cp_async_commit();
-    cp_async_wait_all();
-    __syncthreads();
-    stage_ids(cur, 0, 0);
-    cp_async_commit();
-    cp_async_wait_all();
-    __syncthreads();
+    // register batches of descriptors: hq* for head issue (chunk ci+2D), sq* for stage issue (chunk ci+D)
+    int4 hq0, hq1, sq0, sq1;
+    int hq_first = 0, sq_first = 0;
+    hq0 = hq1 = sq0 = sq1 = make_int4(0, 0, 0, 0);
+    if (producer) {
+        load_desc(0, hq0, hq1);
+        sq0 = hq0; sq1 = hq1;
+        for (int j = 0; j < 2 * D && j < num_chunks; ++j) issue_head(bcast(hq0, j), j);       // 2D <= 16 < 32
+        for (int j = 0; j < D && j < num_chunks; ++j) issue_stage(bcast(sq0, j), bcast(sq1, j), j, j, 0u);
+    }
+    // ring positions: chunk ci (consumers), ci+D (producer: stage), ci+2D (producer: head)
+    int hs = 0, ss = 0;
+    unsigned hp = 0, sp = 0;
+    int hsD = D % NB, ssD = D % NS, hs2D = (2 * D) % NB;
+    unsigned hpD = (unsigned)((D / NB) & 1);
 
-    int hslot = 0;  // ci % 3
     for (int ci = 0; ci < num_chunks; ++ci) {
-        const int hs1 = hslot == 2 ? 0 : hslot + 1;
-        const int hs2 = hs1 == 2 ? 0 : hs1 + 1;
-        int4 nxt3 = nxt2;
-        if (ci + 1 < num_chunks) {
-            stage_ids(nxt, hs1, (ci + 1) & 1);
-            stage_edges(nxt, (ci + 1) & 1, mis_nxt);
-            if (ci + 2 < num_chunks) {
-                stage_head(nxt2, hs2);
-                if (ci + 3 < num_chunks) nxt3 = entry(ci + 3);
+        if (producer) {   // warp-uniform
+            if (ci + 2 * D < num_chunks) {
+                if (ci + 2 * D >= hq_first + 32) { hq_first += 32; load_desc(hq_first, hq0, hq1); }
+                issue_head(bcast(hq0, ci + 2 * D - hq_first), hs2D);
             }
-            cp_async_commit();
+            if (ci + D < num_chunks) {
+                if (ci + D >= sq_first + 32) { sq_first += 32; load_desc(sq_first, sq0, sq1); }
+                const int src = ci + D - sq_first;
+                issue_stage(bcast(sq0, src), bcast(sq1, src), ssD, hsD, hpD);
+            }
         }
-        const unsigned head_s = sbase + L.head + (unsigned)hslot * L.head_stride;
-        const unsigned xvert_s = head_s;                                   // HeadBuf::xvert
-        const unsigned vertf_s = head_s + 8u * CHUNK_V;                    // HeadBuf::vertf
-        const unsigned eoff_s = vertf_s + 4u * CHUNK_V;                    // HeadBuf::eoff
-        const int p0 = cur.x, cnt = cur.y, e0 = cur.z;
-        const bool staged = ALL_STAGED || cur.w <= CHUNK_E;
-        const unsigned ebase_s = sbase + (unsigned)(ci & 1) * L.edge_stride;
-        const unsigned npos_s = ebase_s + L.edge_npos + mis_cur[0];
-        const unsigned nbr_s = ebase_s + L.edge_nbr + mis_cur[1];
-        const unsigned V_s = ebase_s + L.edge_V + mis_cur[2];
-        const unsigned idrow_lane = sbase + L.ids + (unsigned)(ci & 1) * L.ids_stride + (unsigned)lane_col;
+        // A stage is armed only after the producer has seen its head land, so seeing the stage complete
+        // orders this thread after the head's arrival as well: one wait per chunk.
+        if (!mbar_wait(stage_bar0 + 8u * ss, sp)) {
+            fail_wait();
+        } else {
+            const unsigned char* head_p = smem + L.head + (unsigned)hs * L.head_stride;
+            const int4 hdr = *reinterpret_cast<const int4*>(head_p);
+            const int p0 = hdr.x, cnt = hdr.y, e0 = hdr.z, es = hdr.w;  // es: staged edges, -1: edges stay in global memory
+            const bool staged = ALL_STAGED || es >= 0;
+            const unsigned esz = es > 0 ? (unsigned)es : 0u;
+            const int* vertf_p = reinterpret_cast<const int*>(head_p + 16);
+            const unsigned char* body_p = smem + L.body + (unsigned)ss * L.body_stride;
+            const int* eoff_p = reinterpret_cast<const int*>(body_p);
+            const unsigned char* xvert_b = body_p + (((unsigned)(cnt + 1) * 4u + 15u) & ~15u);
+            const unsigned long long* xvert_p = reinterpret_cast<const unsigned long long*>(xvert_b);
+            const unsigned char* npos_b = xvert_b + (((unsigned)cnt * 8u + 15u) & ~15u);
+            const int* npos_p = reinterpret_cast<const int*>(npos_b);
+            const unsigned char* V_b = npos_b + ((esz * 4u + 15u) & ~15u);
+            const LT* V_p = reinterpret_cast<const LT*>(V_b);
+            const int* nbr_p = reinterpret_cast<const int*>(V_b + ((esz * (unsigned)ncomb * LS + 15u) & ~15u));
+            const unsigned char* idrow_p = smem + L.ids + (unsigned)ss * L.ids_stride + (unsigned)lane_col;
 
-        for (int i = warp; i < cnt; i += wpb) {
-            const int vf = (int)lds_u32(vertf_s + 4u * i);
-            const int v = vf & 0x7fffffff;
-            const int pos = p0 + i;
-            const unsigned pv = lds_ids<CPT>(idrow_lane + (unsigned)(i * SLICE)) & idmask;
-            unsigned cls_v[CPT];   // shared address of cls2[0*k + idv]
+            for (int i = warp; i < cnt; i += wpb) {
+                const int vf = vertf_p[i];
+                const int v = vf & 0x7fffffff;
+                const int pos = p0 + i;
+                unsigned pvw[IdWords<CPT>::N];
+                load_ids<CPT>(idrow_p + i * SLICE, pvw);
+                const unsigned pv = pvw[0] & idmask;
+                const unsigned char* cls_v[CPT];   // &cls2[0*k + idv]
 #pragma unroll
-            for (int c = 0; c < CPT; ++c) cls_v[c] = cls2_s + ((pv >> (8 * c)) & 0xffu);
-            LT best[CPT];
+                for (int c = 0; c < CPT; ++c) cls_v[c] = s_cls2 + ((pv >> (8 * c)) & 0xffu);
+                LT best[CPT];
 #pragma unroll
-            for (int c = 0; c < CPT; ++c) best[c] = 0;
-            const int ea_abs = (int)lds_u32(eoff_s + 4u * i), eb_abs = (int)lds_u32(eoff_s + 4u * i + 4u);
-            if (staged) {
-                const int ea = ea_abs - e0, eb = eb_abs - e0;
-                for (int e = ea; e < eb; ++e) {
-                    const int np = (int)lds_u32(npos_s + 4u * e);
-                    const int span = FWD ? pos - np : np - pos;
-                    LT lu[CPT];
-                    unsigned pu;
-                    if (span <= hit_span) {
-                        const unsigned slot = (unsigned)(np & rmask);
-                        lds_levels<CPT>(win_lev_lane + slot * (LS * SLICE), lu);
-                        pu = lds_ids<CPT>(win_id_lane + slot * (unsigned)SLICE);
-                    } else {
-                        const long long off = (long long)(int)lds_u32(nbr_s + 4u * e) * ldp + jl;
-                        long long lg[CPT];
-                        load_levels<CPT>(a.lev + off, lg);
+                for (int c = 0; c < CPT; ++c) best[c] = 0;
+                const int ea_abs = eoff_p[i], eb_abs = eoff_p[i + 1];
+                if (staged) {
+                    const int ea = ea_abs - e0, eb = eb_abs - e0;
+                    for (int e = ea; e < eb; ++e) {
+                        const int np = npos_p[e];
+                        const int span = FWD ? pos - np : np - pos;
+                        LT lu[CPT];
+                        unsigned pu;
+                        if (span <= hit_span) {
+                            const int slot = np & rmask;
+                            load_win<CPT>(win_lev_lane + slot * SLICE, lu);
+                            unsigned w[IdWords<CPT>::N];
+                            load_ids<CPT>(win_id_lane + slot * SLICE, w);
+                            pu = w[0];
+                        } else {
+                            const long long off = (long long)nbr_p[e] * ldp + jl;
+                            long long lg[CPT];
+                            load_levels<CPT>(a.lev + off, lg);
 #pragma unroll
-                        for (int c = 0; c < CPT; ++c) lu[c] = (LT)lg[c];
-                        unsigned w[IdWords<CPT>::N];
-                        load_ids<CPT>(a.part + off, w);
-                        pu = w[0] & idmask;
+                            for (int c = 0; c < CPT; ++c) lu[c] = (LT)lg[c];
+                            unsigned w[IdWords<CPT>::N];
+                            load_ids<CPT>(a.part + off, w);
+                            pu = w[0] & idmask;
+                        }
+                        const LT* vrow = V_p + e * ncomb;
+#pragma unroll
+                        for (int c = 0; c < CPT; ++c) {
+                            const unsigned cls = cls_v[c][((pu >> (8 * c)) & 0xffu) * (unsigned)k];
+                            best[c] = add_max(lu[c], vrow[cls], best[c]);
+                        }
                     }
-                    const unsigned vrow = V_s + LS * (unsigned)(e * ncomb);
+                } else {
+                    // a vertex whose adjacency did not fit the staging buffers: everything from global memory
+                    for (int e = ea_abs; e < eb_abs; ++e) {
+                        const int np = wp.npos[e];
+                        const int span = FWD ? pos - np : np - pos;
+                        LT lu[CPT];
+                        unsigned pu;
+                        if (span <= hit_span) {
+                            const int slot = np & rmask;
+                            load_win<CPT>(win_lev_lane + slot * SLICE, lu);
+                            unsigned w[IdWords<CPT>::N];
+                            load_ids<CPT>(win_id_lane + slot * SLICE, w);
+                            pu = w[0];
+                        } else {
+                            const long long off = (long long)a.adj.nbr[e] * ldp + jl;
+                            long long lg[CPT];
+                            load_levels<CPT>(a.lev + off, lg);
 #pragma unroll
-                    for (int c = 0; c < CPT; ++c) {
-                        const unsigned cls = lds_u8(cls_v[c] + ((pu >> (8 * c)) & 0xffu) * (unsigned)k);
-                        best[c] = add_max(lu[c], lds_level1(vrow + LS * cls, LT()), best[c]);
+                            for (int c = 0; c < CPT; ++c) lu[c] = (LT)lg[c];
+                            unsigned w[IdWords<CPT>::N];
+                            load_ids<CPT>(a.part + off, w);
+                            pu = w[0] & idmask;
+                        }
+                        const LT* vrow = reinterpret_cast<const LT*>(wp.V) + (long long)e * ncomb;
+#pragma unroll
+                        for (int c = 0; c < CPT; ++c) {
+                            const unsigned cls = cls_v[c][((pu >> (8 * c)) & 0xffu) * (unsigned)k];
+                            best[c] = add_max(lu[c], vrow[cls], best[c]);
+                        }
                     }
                 }
-            } else {
-                // a vertex whose adjacency did not fit the staging buffers: everything from global memory
-                for (int e = ea_abs; e < eb_abs; ++e) {
-                    const int np = wp.npos[e];
-                    const int span = FWD ? pos - np : np - pos;
-                    LT lu[CPT];
-                    unsigned pu;
-                    if (span <= hit_span) {
-                        const unsigned slot = (unsigned)(np & rmask);
-                        lds_levels<CPT>(win_lev_lane + slot * (LS * SLICE), lu);
-                        pu = lds_ids<CPT>(win_id_lane + slot * (unsigned)SLICE);
-                    } else {
-                        const long long off = (long long)a.adj.nbr[e] * ldp + jl;
-                        long long lg[CPT];
-                        load_levels<CPT>(a.lev + off, lg);
+                const bool is_cp = want_cp && (FWD ? (vf < 0) : (pos < wp.src_end));
+                if ((!FWD && ea_abs == eb_abs) || is_cp) {
+                    const unsigned long long Xv = xvert_p[i];
+                    if (!FWD && ea_abs == eb_abs) {  // sink: blevel = own runtime
 #pragma unroll
-                        for (int c = 0; c < CPT; ++c) lu[c] = (LT)lg[c];
-                        unsigned w[IdWords<CPT>::N];
-                        load_ids<CPT>(a.part + off, w);
-                        pu = w[0] & idmask;
+                        for (int c = 0; c < CPT; ++c)
+                            best[c] = Xv != NUM_ZERO ? (LT)ceil_quot(Xv, s_rt[(pv >> (8 * c)) & 0xffu]) : (LT)0;
                     }
-                    const LT* vrow = reinterpret_cast<const LT*>(wp.V) + (long long)e * ncomb;
+                    if (is_cp) {
 #pragma unroll
-                    for (int c = 0; c < CPT; ++c) {
-                        const unsigned cls = lds_u8(cls_v[c] + ((pu >> (8 * c)) & 0xffu) * (unsigned)k);
-                        best[c] = add_max(lu[c], vrow[cls], best[c]);
+                        for (int c = 0; c < CPT; ++c) {
+                            long long fin = (long long)best[c];
+                            if (FWD && Xv != NUM_ZERO) fin += ceil_quot(Xv, s_rt[(pv >> (8 * c)) & 0xffu]);
+                            cpmax[c] = fin > cpmax[c] ? fin : cpmax[c];
+                        }
                     }
                 }
-            }
-            const bool is_cp = want_cp && (FWD ? (vf < 0) : (pos < wp.src_end));
-            if ((!FWD && ea_abs == eb_abs) || is_cp) {
-                const unsigned long long Xv = (unsigned long long)lds_s64(xvert_s + 8u * i);
-                if (!FWD && ea_abs == eb_abs) {  // sink: blevel = own runtime
+                // results: global memory (the output) and the window
+                long long* gout = a.lev + (long long)v * ldp + jl;
+                long long wide[CPT];
+#pragma unroll
+                for (int c = 0; c < CPT; ++c) wide[c] = (long long)best[c];
+                if (nvalid >= CPT) store_levels<CPT>(gout, wide);
+                else {
 #pragma unroll
                     for (int c = 0; c < CPT; ++c)
-                        best[c] = Xv != NUM_ZERO ? (LT)ceil_quot(Xv, s_rt[(pv >> (8 * c)) & 0xffu]) : (LT)0;
+                        if (c < nvalid) gout[c] = wide[c];
                 }
-                if (is_cp) {
-#pragma unroll
-                    for (int c = 0; c < CPT; ++c) {
-                        long long fin = (long long)best[c];
-                        if (FWD && Xv != NUM_ZERO) fin += ceil_quot(Xv, s_rt[(pv >> (8 * c)) & 0xffu]);
-                        cpmax[c] = fin > cpmax[c] ? fin : cpmax[c];
-                    }
+                if (R > 0) {
+                    const int slot = pos & rmask;
+                    store_win<CPT>(win_lev_lane + slot * SLICE, best);
+                    pvw[0] = pv;
+                    store_ids<CPT>(win_id_lane + slot * SLICE, pvw);
                 }
-            }
-            // results: global memory (the output) and the window
-            long long* gout = a.lev + (long long)v * ldp + jl;
-            long long wide[CPT];
-#pragma unroll
-            for (int c = 0; c < CPT; ++c) wide[c] = (long long)best[c];
-            if (nvalid >= CPT) store_levels<CPT>(gout, wide);
-            else {
-#pragma unroll
-                for (int c = 0; c < CPT; ++c)
-                    if (c < nvalid) gout[c] = wide[c];
-            }
-            if (R > 0) {
-                const unsigned slot = (unsigned)(pos & rmask);
-                sts_levels<CPT>(win_lev_lane + slot * (LS * SLICE), best);
-                sts_ids<CPT>(win_id_lane + slot * (unsigned)SLICE, pv);
             }
         }
-        cp_async_wait_all();
         __syncthreads();
-        cur = nxt; nxt = nxt2; nxt2 = nxt3;
-        mis_cur[0] = mis_nxt[0]; mis_cur[1] = mis_nxt[1]; mis_cur[2] = mis_nxt[2];
-        hslot = hs1;
+        if (*s_abort) break;
+        if (++hs == NB) { hs = 0; hp ^= 1u; }
+        if (++ss == NS) { ss = 0; sp ^= 1u; }
+        if (++hsD == NB) { hsD = 0; hpD ^= 1u; }
+        if (++ssD == NS) ssD = 0;
+        if (++hs2D == NB) hs2D = 0;
+    }
+    if (*s_abort) {
+        // copies that were already requested may still be landing in this block's shared memory: give them
+        // a bounded time before the block (and its shared memory) goes away
+        for (int i = 0; i < 1000; ++i) __nanosleep(1000);
+        return;
     }
 
     if (want_cp) {
@@ -445,6 +467,39 @@ pass_window_kernel(PassArgs a, WindowPlan wp, WinLayout L)
             if (c < nvalid) a.cp[j0 + c] = m;
         }
     }
+}
+
+// Packs one chunk's record.  head: int4 {p0, cnt, e0, staged edges or -1}, vertf[cnt].
+// body: eoff[cnt+1], xvert[cnt], npos[es], V[es*ncomb] (lsize bytes each), nbr[es]; every array padded to 16 bytes.
+__global__ void pack_chunks_kernel(const int4* __restrict__ chunks, const int4* __restrict__ desc,
+                                   const int* __restrict__ vertf, const int* __restrict__ eptr,
+                                   const unsigned long long* __restrict__ xvert, const int* __restrict__ npos,
+                                   const int* __restrict__ nbr, const void* __restrict__ V, int ncomb, int lsize,
+                                   unsigned char* blob)
+{
+    const int4 ch = chunks[blockIdx.x];
+    const int4 d0 = desc[2 * blockIdx.x];
+    const int p0 = ch.x, cnt = ch.y, e0 = ch.z, ecnt = ch.w;
+    const int es = ecnt <= CHUNK_E ? ecnt : -1;
+    const unsigned esz = es > 0 ? (unsigned)es : 0u;
+    unsigned char* head = blob + 16ll * (unsigned)d0.x;
+    unsigned char* body = blob + 16ll * (unsigned)d0.z;
+    if (threadIdx.x == 0) *reinterpret_cast<int4*>(head) = make_int4(p0, cnt, e0, es);
+    int* o_vertf = reinterpret_cast<int*>(head + 16);
+    int* o_eoff = reinterpret_cast<int*>(body);
+    unsigned long long* o_xvert = reinterpret_cast<unsigned long long*>(body + (((unsigned)(cnt + 1) * 4u + 15u) & ~15u));
+    unsigned char* p_npos = reinterpret_cast<unsigned char*>(o_xvert) + (((unsigned)cnt * 8u + 15u) & ~15u);
+    int* o_npos = reinterpret_cast<int*>(p_npos);
+    unsigned char* p_V = p_npos + ((esz * 4u + 15u) & ~15u);
+    unsigned char* p_nbr = p_V + ((esz * (unsigned)ncomb * (unsigned)lsize + 15u) & ~15u);
+    int* o_nbr = reinterpret_cast<int*>(p_nbr);
+    for (int i = threadIdx.x; i < cnt; i += blockDim.x) { o_vertf[i] = vertf[p0 + i]; o_xvert[i] = xvert[p0 + i]; }
+    for (int i = threadIdx.x; i <= cnt; i += blockDim.x) o_eoff[i] = eptr[p0 + i];
+    for (int i = threadIdx.x; i < (int)esz; i += blockDim.x) { o_npos[i] = npos[e0 + i]; o_nbr[i] = nbr[e0 + i]; }
+    const int words = (int)esz * ncomb * (lsize / 4);
+    const int* src = reinterpret_cast<const int*>(reinterpret_cast<const unsigned char*>(V) + (long long)e0 * ncomb * lsize);
+    int* dst = reinterpret_cast<int*>(p_V);
+    for (int i = threadIdx.x; i < words; i += blockDim.x) dst[i] = src[i];
 }
 
 // ---- set-up kernels ---------------------------------------------------------------------
@@ -500,14 +555,14 @@ inline unsigned cdivu(long long a, long long b) { return (unsigned)((a + b - 1) 
 template <int CPT, bool FWD, bool ALL_STAGED, typename LT>
 cudaError_t window_impl(const PassArgs& a, const WindowPlan& plan, int warps, cudaStream_t st)
 {
-    const Carve c = carve(a.tab.k, plan.ncomb, plan.R, CPT, warps, (int)sizeof(LT));
+    const Carve c = carve(a.tab.k, plan.R, CPT, warps, (int)sizeof(LT), plan.max_v, plan.head_max, plan.body_max, plan.depth);
     WinLayout L;
-    L.head = (unsigned)c.head; L.head_stride = (unsigned)up16(sizeof(HeadBuf));
-    L.edge_nbr = (unsigned)c.edge_nbr; L.edge_npos = (unsigned)c.edge_npos; L.edge_V = (unsigned)c.edge_V;
-    L.edge_stride = (unsigned)c.edge_stride;
+    L.bars = (unsigned)c.bars; L.rt = (unsigned)c.rt; L.cls2 = (unsigned)c.cls2; L.cp = (unsigned)c.cp;
+    L.head = (unsigned)c.head; L.head_stride = (unsigned)c.head_stride;
+    L.body = (unsigned)c.body; L.body_stride = (unsigned)c.body_stride;
     L.ids = (unsigned)c.ids; L.ids_stride = (unsigned)c.ids_stride;
-    L.rt = (unsigned)c.rt; L.cls2 = (unsigned)c.cls2; L.cp = (unsigned)c.cp;
     L.win_lev = (unsigned)c.win_lev; L.win_id = (unsigned)c.win_id;
+    L.depth = plan.depth;
     cudaError_t e = cudaFuncSetAttribute(pass_window_kernel<CPT, FWD, ALL_STAGED, LT>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c.total);
     if (e != cudaSuccess) return e;
@@ -526,9 +581,20 @@ cudaError_t window_dispatch(const PassArgs& a, bool fwd, const WindowPlan& plan,
 
 }  // namespace
 
-size_t window_smem_bytes(int k, int ncomb, int R, int cpt, int warps, int level_bytes)
+size_t window_smem_bytes(int k, int R, int cpt, int warps, int level_bytes, int max_v, int head_max, int body_max, int depth)
 {
-    return carve(k, ncomb, R, cpt, warps, level_bytes).total;
+    return carve(k, R, cpt, warps, level_bytes, max_v, head_max, body_max, depth).total;
+}
+
+cudaError_t launch_pack_chunks(int num_chunks, const int* chunks, const int* desc, const int* vertf, const int* eptr,
+                               const unsigned long long* xvert, const int* npos, const int* nbr, const void* V, int ncomb,
+                               int lsize, unsigned char* blob, cudaStream_t st)
+{
+    if (num_chunks <= 0) return cudaSuccess;
+    pack_chunks_kernel<<<num_chunks, 128, 0, st>>>(reinterpret_cast<const int4*>(chunks), reinterpret_cast<const int4*>(desc),
+                                                   vertf, eptr, xvert, npos, nbr, V, ncomb, lsize, blob);
+    count_launches(1);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_pass_window(const PassArgs& a, bool fwd, const WindowPlan& plan, int cpt, int warps, cudaStream_t st)
