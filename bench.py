@@ -275,7 +275,7 @@ def run_gpu(args):
         "edge_relaxations_per_s": world * 2.0 * m * P / (ms * 1e-3),
         "phase_ms": {"loads_validate_viol": loads_ms, "forward": fwd_ms, "backward": bwd_ms},
         "roofline": {"bound": "hbm",
-                     "kernel": "pass_level_kernel<fwd>" if args.variant == "level_sync" else "pass_sliced_kernel<fwd>",
+                     "kernel": tfps.tfps_last_pass_kernel(g.handle) + "<forward>",
                      "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "peak_kind": f"of {peak_kind}", "bytes_per_launch": compulsory, "traffic": None,
                      "achieved_logical": logical / (fwd_ms * 1e-3) / 1e9,

@@ -186,6 +186,13 @@ int tfps_eval_batch_host(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* p
  */
 int tfps_phase_times(tfps_graph* g, float ms[3]);
 
+/*
+ * Name of the pass kernel family the most recent tfps_eval_batch call on this handle chose
+ * ("pass_window_kernel", "pass_sliced_kernel", "pass_tile_kernel", "pass_level_kernel"; "" before any call).
+ * The string is static.
+ */
+const char* tfps_last_pass_kernel(const tfps_graph* g);
+
 /* Number of kernels this library has launched in the calling process so far. */
 int64_t tfps_kernel_launches(void);
 

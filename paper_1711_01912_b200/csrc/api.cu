@@ -139,6 +139,7 @@ struct tfps_graph {
     cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
     bool ev_valid = false;
     bool ran_fwd = false, ran_bwd = false;
+    const char* last_kernel = "";
     ~tfps_graph()
     {
         for (cudaEvent_t e : ev)
@@ -920,6 +921,7 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
         long long* lev = fwd ? fwd_lev : (long long*)blevel;
         long long* cp_here = (cp && (fwd || !need_fwd)) ? (long long*)cp : nullptr;
         PassArgs a = make_args(g, fwd, P, ldp, part, lev, cp_here);
+        g->last_kernel = use_window ? "pass_window_kernel" : (sliced ? "pass_sliced_kernel" : (g->npass > 0 ? "pass_tile_kernel" : "pass_level_kernel"));
         if (use_window) {
             WindowPlan wp;
             wp.vertf = g->vertf.as<int>();
@@ -978,6 +980,8 @@ int tfps_phase_times(tfps_graph* g, float ms[3])
     if (!g->ran_bwd) ms[2] = 0.f;
     return TFPS_OK;
 }
+
+const char* tfps_last_pass_kernel(const tfps_graph* g) { return g ? g->last_kernel : ""; }
 
 int64_t tfps_kernel_launches(void) { return (int64_t)tfps::g_launches.load(std::memory_order_relaxed); }
 

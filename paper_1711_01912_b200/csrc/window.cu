@@ -118,7 +118,7 @@ __host__ __device__ inline Carve carve(int k, int R, int cpt, int warps, int lsi
     Carve c;
     const size_t slice = 32 * (size_t)cpt;
     size_t o = 0;
-    c.bars = o; o += up16(8 * (size_t)(3 * depth + 2) + 8);
+    c.bars = o; o += up16(8 * (size_t)(3 * depth + 2) + 16);   // mbarriers, abort flag, two vertex counters
     c.rt = o; o += up16(sizeof(DivConst) * (size_t)k);
     c.cls2 = o; o += up16((size_t)k * k);
     c.cp = o;   // the staging rings double as the reduction buffer of the CP maxima after the last chunk
@@ -182,6 +182,8 @@ pass_window_kernel(PassArgs a, WindowPlan wp, WinLayout L)
     DivConst* s_rt = reinterpret_cast<DivConst*>(smem + L.rt);
     long long* s_cp = reinterpret_cast<long long*>(smem + L.cp);
     volatile int* s_abort = reinterpret_cast<volatile int*>(smem + L.bars + 8 * (3 * L.depth + 2));
+    // vertices of a chunk are handed out dynamically (degrees differ): one counter per chunk parity
+    int* s_next = reinterpret_cast<int*>(smem + L.bars + 8 * (3 * L.depth + 2) + 4);
     if (*a.status != 0) return;
     const int D = L.depth, NB = 2 * D + 1, NS = D + 1;
     const unsigned head_bar0 = sbase + L.bars, stage_bar0 = head_bar0 + 8u * NB;
@@ -191,6 +193,8 @@ pass_window_kernel(PassArgs a, WindowPlan wp, WinLayout L)
         // producer lane once that lane's id-row copies have landed
         for (int j = 0; j < NS; ++j) mbar_init(stage_bar0 + 8u * j, 33);
         *s_abort = 0;
+        s_next[0] = 0;
+        s_next[1] = 0;
         mbar_init_fence();
     }
     for (int i = threadIdx.x; i < k; i += blockDim.x) s_rt[i] = a.tab.rt_div[i];
@@ -325,7 +329,18 @@ pass_window_kernel(PassArgs a, WindowPlan wp, WinLayout L)
             const int* nbr_p = reinterpret_cast<const int*>(V_b + ((esz * (unsigned)ncomb * LS + 15u) & ~15u));
             const unsigned char* idrow_p = smem + L.ids + (unsigned)ss * L.ids_stride + (unsigned)lane_col;
 
-            for (int i = warp; i < cnt; i += wpb) {
+            int* next_ctr = s_next + (ci & 1);
+            if (threadIdx.x == 0) s_next[(ci + 1) & 1] = 0;   // last used by chunk ci-1, whose warps all passed the barrier
+            const bool dynamic = cnt > wpb;   // a narrow chunk gives every warp at most one vertex: no counter needed
+            for (bool first = true;; first = false) {
+                int i = warp;
+                if (dynamic) {
+                    if (lane == 0) i = atomicAdd(next_ctr, 1);
+                    i = __shfl_sync(0xffffffffu, i, 0);
+                } else if (!first) {
+                    break;
+                }
+                if (i >= cnt) break;
                 const int vf = vertf_p[i];
                 const int v = vf & 0x7fffffff;
                 const int pos = p0 + i;

@@ -31,7 +31,7 @@ EXPORTS = [
     "tfps_strerror", "tfps_last_error", "tfps_graph_create", "tfps_graph_destroy", "tfps_graph_info",
     "tfps_devices_set", "tfps_topo_levels", "tfps_eval_workspace_bytes", "tfps_eval_batch",
     "tfps_eval_batch_host", "tfps_get_status", "tfps_transpose_u8", "tfps_phase_times", "tfps_kernel_launches",
-    "tfps_eval_cp_noalloc",
+    "tfps_eval_cp_noalloc", "tfps_last_pass_kernel",
 ]
 
 
@@ -78,6 +78,8 @@ def lib() -> ctypes.CDLL:
     L.tfps_phase_times.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
     L.tfps_kernel_launches.restype = i64
     L.tfps_kernel_launches.argtypes = []
+    L.tfps_last_pass_kernel.restype = ctypes.c_char_p
+    L.tfps_last_pass_kernel.argtypes = [vp]
     L.tfps_eval_cp_noalloc.restype = ci
     L.tfps_eval_cp_noalloc.argtypes = [vp, i64, i64, vp, vp, ci, vp]
     L.tfps_get_status.restype = ci
@@ -148,6 +150,10 @@ def tfps_phase_times(g):
     ms = (ctypes.c_float * 3)()
     _check(lib().tfps_phase_times(g, ms))
     return [float(x) for x in ms]
+
+
+def tfps_last_pass_kernel(g) -> str:
+    return lib().tfps_last_pass_kernel(g).decode()
 
 
 def tfps_kernel_launches() -> int:
