@@ -631,6 +631,7 @@ cp_reduce_kernel(PassArgs a, const int* __restrict__ list, int list_len, int per
 // shared-memory atomics), walks a chunk of vertices and merges into global
 // memory with 64-bit atomic adds (integer, order independent).  Doubles as the
 // id validator: an id >= k raises BAD_PARTITION and is counted on device 0.
+template <int C>   // candidates per thread: 1, 2 or 4
 __global__ void loads_kernel(int n, long long P, long long ldp, const uint8_t* __restrict__ part,
                              const int* __restrict__ vert, const unsigned long long* __restrict__ xvert,
                              const long long* __restrict__ mem, DevTables tab, long long* load,
@@ -638,21 +639,20 @@ __global__ void loads_kernel(int n, long long P, long long ldp, const uint8_t* _
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const int k = tab.k;
-    const int bc = blockDim.x * 4;
+    const int nthr = blockDim.x;  // accumulators are laid out [device][c][thread]: conflict-free columns
     DivConst* s_rt = reinterpret_cast<DivConst*>(smem_raw);
     long long* acc_l = reinterpret_cast<long long*>(s_rt + k);
-    long long* acc_m = acc_l + (size_t)k * bc;
+    long long* acc_m = acc_l + (size_t)k * nthr * C;
     for (int i = threadIdx.x; i < k; i += blockDim.x) s_rt[i] = tab.rt_div[i];
-    for (int i = threadIdx.x; i < k * bc; i += blockDim.x) { acc_l[i] = 0; acc_m[i] = 0; }
+    for (int i = threadIdx.x; i < k * nthr * C; i += blockDim.x) { acc_l[i] = 0; acc_m[i] = 0; }
     __syncthreads();
 
-    const long long slice0 = (long long)blockIdx.x * bc;
-    const long long j0 = slice0 + (long long)threadIdx.x * 4;
+    const long long slice0 = (long long)blockIdx.x * nthr * C;
+    const long long j0 = slice0 + (long long)threadIdx.x * C;
     const long long rem = P - j0;
-    const int nvalid = rem >= 4 ? 4 : (rem > 0 ? (int)rem : 0);
+    const int nvalid = rem >= C ? C : (rem > 0 ? (int)rem : 0);
     const long long jl = nvalid > 0 ? j0 : slice0;  // idle lanes keep the warp's shuffles company
     const int lane = threadIdx.x & 31;
-    const int nthr = blockDim.x;  // accumulators are laid out [device][c][thread]: conflict-free columns
     const int r0 = blockIdx.y * rows_per_block;
     const int r1 = r0 + rows_per_block < n ? r0 + rows_per_block : n;
     bool bad = false;
@@ -667,7 +667,10 @@ __global__ void loads_kernel(int n, long long P, long long ldp, const uint8_t* _
                 const int v = vert[pos + q];
                 Xv[q] = xvert[pos + q];
                 mv[q] = mem[v];
-                packed[q] = *reinterpret_cast<const unsigned*>(part + (long long)v * ldp + jl);
+                const uint8_t* p = part + (long long)v * ldp + jl;
+                if constexpr (C == 1) packed[q] = *p;
+                else if constexpr (C == 2) packed[q] = *reinterpret_cast<const unsigned short*>(p);
+                else packed[q] = *reinterpret_cast<const unsigned*>(p);
             }
         }
 #pragma unroll
@@ -680,7 +683,7 @@ __global__ void loads_kernel(int n, long long P, long long ldp, const uint8_t* _
                     if (k > 32 && lane + 32 < k) row_hi = ceil_quot(Xv[q], s_rt[lane + 32]);
                 }
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
+                for (int c = 0; c < C; ++c) {
                     unsigned id = (packed[q] >> (8 * c)) & 0xffu;
                     if (c >= nvalid) id = 0;
                     if (id >= (unsigned)k) { bad = true; id = 0; }
@@ -690,8 +693,8 @@ __global__ void loads_kernel(int n, long long P, long long ldp, const uint8_t* _
                         rt = id >= 32u ? hi : rt;
                     }
                     if (c < nvalid) {
-                        acc_l[(id * 4 + c) * nthr + threadIdx.x] += rt;
-                        acc_m[(id * 4 + c) * nthr + threadIdx.x] += mv[q];
+                        acc_l[(id * C + c) * nthr + threadIdx.x] += rt;
+                        acc_m[(id * C + c) * nthr + threadIdx.x] += mv[q];
                     }
                 }
             }
@@ -700,12 +703,12 @@ __global__ void loads_kernel(int n, long long P, long long ldp, const uint8_t* _
     if (bad && validate) atomicCAS(status, 0, (int)TFPS_ERR_BAD_PARTITION);
     for (int d = 0; d < k; ++d) {
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
+        for (int c = 0; c < C; ++c) {
             if (c < nvalid) {
                 if (load) atomicAdd(reinterpret_cast<unsigned long long*>(load + d * ldp + j0 + c),
-                                    (unsigned long long)acc_l[(d * 4 + c) * nthr + threadIdx.x]);
+                                    (unsigned long long)acc_l[(d * C + c) * nthr + threadIdx.x]);
                 if (memload) atomicAdd(reinterpret_cast<unsigned long long*>(memload + d * ldp + j0 + c),
-                                       (unsigned long long)acc_m[(d * 4 + c) * nthr + threadIdx.x]);
+                                       (unsigned long long)acc_m[(d * C + c) * nthr + threadIdx.x]);
             }
         }
     }
@@ -900,19 +903,22 @@ cudaError_t launch_cp_reduce(const PassArgs& a, bool from_tlevel, const int* lis
     return cudaGetLastError();
 }
 
-cudaError_t launch_loads(int n, long long P, long long ldp, const uint8_t* part, const int* vert,
-                         const unsigned long long* xvert, const long long* mem, DevTables tab, long long* load,
-                         long long* memload, int* status, bool validate, int sm_count, cudaStream_t st)
+template <int C>
+static cudaError_t loads_impl(int n, long long P, long long ldp, const uint8_t* part, const int* vert,
+                              const unsigned long long* xvert, const long long* mem, DevTables tab, long long* load,
+                              long long* memload, int* status, bool validate, int sm_count, cudaStream_t st)
 {
     const int k = tab.k;
-    // threads per block sized so that 2*k*(4*threads) int64 accumulators fit in shared memory
+    // threads per block sized so that 2*k*(C*threads) int64 accumulators fit in shared memory
     int threads = 64;
-    while (threads > 32 && sizeof(DivConst) * k + (size_t)2 * k * threads * 4 * 8 > 96 * 1024) threads >>= 1;
-    const size_t smem = sizeof(DivConst) * k + (size_t)2 * k * threads * 4 * 8;
-    cudaError_t e = allow_smem(loads_kernel, smem);
+    while (threads > 32 && sizeof(DivConst) * k + (size_t)2 * k * threads * C * 8 > 96 * 1024) threads >>= 1;
+    const size_t smem = sizeof(DivConst) * k + (size_t)2 * k * threads * C * 8;
+    cudaError_t e = allow_smem(loads_kernel<C>, smem);
     if (e != cudaSuccess) return e;
-    const unsigned gx = cdivu(P, threads * 4);
-    long long want_blocks = (long long)sm_count * 32;
+    const unsigned gx = cdivu(P, threads * C);
+    int per_sm = 64;
+    if (const char* ov = getenv("TFPS_LOADS_BLOCKS_PER_SM")) { const int q = atoi(ov); if (q >= 1 && q <= 64) per_sm = q; }
+    long long want_blocks = (long long)sm_count * per_sm;
     long long gy = (want_blocks + gx - 1) / gx;
     if (gy < 1) gy = 1;
     if (gy > n) gy = n;
@@ -920,9 +926,20 @@ cudaError_t launch_loads(int n, long long P, long long ldp, const uint8_t* part,
     int rows = (int)((n + gy - 1) / gy);
     gy = (n + rows - 1) / rows;
     count_launches(1);
-    loads_kernel<<<dim3(gx, (unsigned)gy), threads, smem, st>>>(n, P, ldp, part, vert, xvert, mem, tab, load, memload,
-                                                                status, validate ? 1 : 0, rows);
+    loads_kernel<C><<<dim3(gx, (unsigned)gy), threads, smem, st>>>(n, P, ldp, part, vert, xvert, mem, tab, load, memload,
+                                                                   status, validate ? 1 : 0, rows);
     return cudaGetLastError();
+}
+
+cudaError_t launch_loads(int n, long long P, long long ldp, const uint8_t* part, const int* vert,
+                         const unsigned long long* xvert, const long long* mem, DevTables tab, long long* load,
+                         long long* memload, int* status, bool validate, int sm_count, cudaStream_t st)
+{
+    int c = 2;  // two candidates per thread: best balance of shared-memory footprint (occupancy) and per-row work
+    if (const char* ov = getenv("TFPS_LOADS_CPT")) c = atoi(ov);   // tuning override
+    if (c == 1) return loads_impl<1>(n, P, ldp, part, vert, xvert, mem, tab, load, memload, status, validate, sm_count, st);
+    if (c == 2) return loads_impl<2>(n, P, ldp, part, vert, xvert, mem, tab, load, memload, status, validate, sm_count, st);
+    return loads_impl<4>(n, P, ldp, part, vert, xvert, mem, tab, load, memload, status, validate, sm_count, st);
 }
 
 cudaError_t launch_validate(long long n, long long P, long long ldp, const uint8_t* part, int k, int* status,
