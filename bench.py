@@ -263,6 +263,11 @@ def run_gpu(args):
     compulsory = 9.0 * n * P
     logical = 9.0 * (n + m) * P
     achieved = compulsory / (fwd_ms * 1e-3) / 1e9
+    # DRAM bytes of the forward kernel from the ncu capture summarised in profiles/pass_window_kernel_cfg3.md
+    # (P=2368: 1.3474 GB read+write = 8.682 B per vertex-candidate), scaled to this launch by n*P; only
+    # valid for the kernel and graph that capture was taken on
+    kernel_name = tfps.tfps_last_pass_kernel(g.handle)
+    traffic = 8.682 * n * P if (args.config == 3 and kernel_name == "pass_window_kernel") else None
     value = world * P / (ms * 1e-3)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
@@ -277,7 +282,7 @@ def run_gpu(args):
         "roofline": {"bound": "hbm",
                      "kernel": tfps.tfps_last_pass_kernel(g.handle) + "<forward>",
                      "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "peak_kind": f"of {peak_kind}", "bytes_per_launch": compulsory, "traffic": None,
+                     "peak_kind": f"of {peak_kind}", "bytes_per_launch": compulsory, "traffic": traffic,
                      "achieved_logical": logical / (fwd_ms * 1e-3) / 1e9,
                      "frac_logical": logical / (fwd_ms * 1e-3) / 1e9 / peak,
                      "note": "achieved counts compulsory bytes 9*n*P (1 B id read + 8 B level write per vertex-candidate); "
