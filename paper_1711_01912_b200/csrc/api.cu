@@ -951,7 +951,14 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
             plan.src_end = (int)g->h_level_ptr[1];
             CUDA_TRY(launch_pass_sliced(a, fwd, plan, cpt, warps, table, st));
         } else {
-            CUDA_TRY(launch_pass_level_sync(a, fwd, g->h_level_ptr, st));
+            // the value-array kernel is opt-in: the tile kernel measured faster on the wide power-law graph (config 5)
+            if (g->ncomb > 0 && env_int("TFPS_LEVEL_VALUES", 0) != 0) {
+                g->last_kernel = "pass_levelv_kernel";
+                CUDA_TRY(launch_pass_level_values(a, fwd, g->h_level_ptr, fwd ? g->V_f.as<long long>() : g->V_b.as<long long>(),
+                                                  fwd ? g->cls2_f.as<uint8_t>() : g->cls2_b.as<uint8_t>(), g->ncomb, st));
+            } else {
+                CUDA_TRY(launch_pass_level_sync(a, fwd, g->h_level_ptr, st));
+            }
             if (cp_here) {
                 CUDA_TRY(cudaMemsetAsync(cp_here, 0, sizeof(long long) * (size_t)P, st));
                 if (fwd) CUDA_TRY(launch_cp_reduce(a, true, g->sink_list.as<int>(), g->sink_count, st));

@@ -159,6 +159,8 @@ cudaError_t launch_default_mem(int n, const long long* out_ptr, const long long*
 
 int pick_cpt(long long P);
 cudaError_t launch_pass_level_sync(const PassArgs& a, bool fwd, const std::vector<long long>& level_ptr_host, cudaStream_t st);
+cudaError_t launch_pass_level_values(const PassArgs& a, bool fwd, const std::vector<long long>& level_ptr_host,
+                                     const long long* V, const uint8_t* cls2, int ncomb, cudaStream_t st);
 cudaError_t launch_pass_sliced(const PassArgs& a, bool fwd, const SlicedPlan& plan, int cpt, int warps, bool table,
                                cudaStream_t st);
 cudaError_t launch_pass_window(const PassArgs& a, bool fwd, const WindowPlan& plan, int cpt, int warps, cudaStream_t st);

@@ -431,6 +431,78 @@ pass_tile_kernel(PassArgs a, int pos0, int count)
     if (!waited) grid_dependency_wait();
 }
 
+// ---- level-synchronous variant on precomputed edge values ---------------------------------
+// One launch per level, a warp takes one vertex and 32*CPT candidates.  The cost of an edge comes from the
+// precomputed value array (at most COMB_MAX distinct values per edge): lanes 0..ncomb-1 fetch the edge's
+// values, every candidate picks its own with one shuffle.  No per-edge table, no block barrier.  Launches are
+// chained with programmatic dependent launch exactly as in the tile kernel.
+constexpr int LEVELV_WARPS = 8;
+
+template <int CPT, bool FWD>
+__global__ void __launch_bounds__(LEVELV_WARPS * 32)
+pass_levelv_kernel(PassArgs a, const long long* __restrict__ V, const uint8_t* __restrict__ cls2, int ncomb, int pos0,
+                   int count)
+{
+    __shared__ uint8_t s_cls2[TABLE_K_MAX * TABLE_K_MAX];
+    __shared__ DivConst s_rt[TABLE_K_MAX];
+    grid_launch_dependents();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int k = a.tab.k;
+    const bool live = *a.status == 0;
+    for (int i = threadIdx.x; i < k * k; i += blockDim.x) s_cls2[i] = cls2[i];
+    for (int i = threadIdx.x; i < k; i += blockDim.x) s_rt[i] = a.tab.rt_div[i];
+    __syncthreads();
+    const long long slice0 = (long long)blockIdx.x * 32 * CPT;
+    const LaneCtx<CPT> lc = lane_setup<CPT>(slice0, a.P, lane);
+    const long long ldp = a.ldp;
+    bool waited = false;
+    constexpr int UNR = 2;
+    for (int i = blockIdx.y * LEVELV_WARPS + warp; i < count && live; i += gridDim.y * LEVELV_WARPS) {
+        const VertexMeta vm = global_meta(a.adj, pos0 + i);
+        unsigned pv[IdWords<CPT>::N];
+        load_ids_masked<CPT>(a.part + (long long)vm.v * ldp + lc.jl, lc, pv);
+        long long best[CPT];
+#pragma unroll
+        for (int c = 0; c < CPT; ++c) best[c] = 0;
+        for (int e = vm.e0; e < vm.e1; e += UNR) {
+            long long off[UNR], vreg[UNR];
+            unsigned pu[UNR][IdWords<CPT>::N];
+#pragma unroll
+            for (int q = 0; q < UNR; ++q) {
+                if (e + q < vm.e1) {
+                    off[q] = (long long)vm.nbr[e + q] * ldp + lc.jl;
+                    vreg[q] = lane < ncomb ? V[(long long)(e + q) * ncomb + lane] : 0;
+                    load_ids_masked<CPT>(a.part + off[q], lc, pu[q]);
+                }
+            }
+            if (!waited) { grid_dependency_wait(); waited = true; }
+            long long lu[UNR][CPT];
+#pragma unroll
+            for (int q = 0; q < UNR; ++q)
+                if (e + q < vm.e1) load_levels<CPT>(a.lev + off[q], lu[q]);
+#pragma unroll
+            for (int q = 0; q < UNR; ++q) {
+                if (e + q < vm.e1) {
+#pragma unroll
+                    for (int c = 0; c < CPT; ++c) {
+                        const unsigned cls = s_cls2[id_at<CPT>(pu[q], c) * k + id_at<CPT>(pv, c)];
+                        const long long val = lu[q][c] + shfl64(vreg[q], (int)cls);
+                        best[c] = val > best[c] ? val : best[c];
+                    }
+                }
+            }
+        }
+        if (!FWD && vm.e0 == vm.e1) {  // sink: blevel = own runtime
+#pragma unroll
+            for (int c = 0; c < CPT; ++c)
+                best[c] = vm.xvert != NUM_ZERO ? ceil_quot(vm.xvert, s_rt[id_at<CPT>(pv, c)]) : 0;
+        }
+        if (!waited) { grid_dependency_wait(); waited = true; }
+        store_levels<CPT>(a.lev + (long long)vm.v * ldp + lc.jl, best, lc.nvalid);
+    }
+    if (!waited) grid_dependency_wait();
+}
+
 // ---- candidate-sliced persistent variant ---------------------------------------------
 // One block owns 32*CPT candidates and walks the whole graph chunk by chunk; a
 // chunk is a run of at most CHUNK_V positions / CHUNK_E edges inside one level
@@ -834,6 +906,45 @@ static cudaError_t tile_impl(const PassArgs& a, const std::vector<long long>& lp
     }
     count_launches(L);
     return cudaGetLastError();
+}
+
+template <int CPT, bool FWD>
+static cudaError_t levelv_impl(const PassArgs& a, const std::vector<long long>& lp, const long long* V, const uint8_t* cls2,
+                               int ncomb, cudaStream_t st)
+{
+    const unsigned gx = cdivu(a.P, 32 * CPT);
+    const int L = a.num_levels;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    for (int step = 0; step < L; ++step) {
+        const int l = FWD ? step : L - 1 - step;
+        const int pos0 = (int)lp[l];
+        const int count = (int)(lp[l + 1] - lp[l]);
+        unsigned gy = cdivu(count, LEVELV_WARPS);
+        if (gy > 65535u) gy = 65535u;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(gx, gy);
+        cfg.blockDim = dim3(LEVELV_WARPS * 32);
+        cfg.dynamicSmemBytes = 0;
+        cfg.stream = st;
+        cfg.attrs = attr;
+        cfg.numAttrs = step == 0 ? 0 : 1;  // the first level follows ordinary stream order
+        cudaError_t e = cudaLaunchKernelEx(&cfg, pass_levelv_kernel<CPT, FWD>, a, V, cls2, ncomb, pos0, count);
+        if (e != cudaSuccess) return e;
+    }
+    count_launches(L);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_pass_level_values(const PassArgs& a, bool fwd, const std::vector<long long>& lp, const long long* V,
+                                     const uint8_t* cls2, int ncomb, cudaStream_t st)
+{
+    int cpt = a.P >= 4096 ? 4 : (a.P >= 512 ? 2 : 1);
+    if (const char* ov = getenv("TFPS_TILE_CPT")) { const int q = atoi(ov); if (q == 1 || q == 2 || q == 4) cpt = q; }
+    if (cpt == 4) return fwd ? levelv_impl<4, true>(a, lp, V, cls2, ncomb, st) : levelv_impl<4, false>(a, lp, V, cls2, ncomb, st);
+    if (cpt == 2) return fwd ? levelv_impl<2, true>(a, lp, V, cls2, ncomb, st) : levelv_impl<2, false>(a, lp, V, cls2, ncomb, st);
+    return fwd ? levelv_impl<1, true>(a, lp, V, cls2, ncomb, st) : levelv_impl<1, false>(a, lp, V, cls2, ncomb, st);
 }
 
 cudaError_t launch_pass_level_sync(const PassArgs& a, bool fwd, const std::vector<long long>& lp, cudaStream_t st)

@@ -115,6 +115,17 @@ def test_config2_every_candidate(flags):
     run_and_compare(w.graph, w.devices, w.part_full(), flags)
 
 
+def test_level_kernel_on_precomputed_values(monkeypatch):
+    """The opt-in level-synchronous kernel that reads precomputed edge values (TFPS_LEVEL_VALUES=1)."""
+    monkeypatch.setenv("TFPS_LEVEL_VALUES", "1")
+    w = I.config2()
+    run_and_compare(w.graph, w.devices, w.part_full()[:, :700], 1, pad_fill=255)
+    w = I.config5(layers=12, width=64, P=100)
+    run_and_compare(w.graph, w.devices, w.part_full(), 1, pad_fill=255)
+    w = I.small_random(5, 300, 900, 3, 77)
+    run_and_compare(w.graph, w.devices, w.part_full(), 1, pad_fill=255)
+
+
 def test_config1_relabelled():
     w = I.config1()
     g2, perm = I.relabel(w.graph, 5)
