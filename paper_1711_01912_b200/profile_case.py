@@ -24,6 +24,7 @@ def main():
     ap.add_argument("--cpt", type=int, default=0)
     ap.add_argument("--warps", type=int, default=0)
     ap.add_argument("--reps", type=int, default=5)
+    ap.add_argument("--layers", type=int, default=0, help="config 5 only: fewer layers of the same width (smaller capture)")
     args = ap.parse_args()
 
     import torch
@@ -31,7 +32,7 @@ def main():
 
     os.environ["TFPS_SLICED_CPT"] = str(args.cpt)
     os.environ["TFPS_SLICED_WARPS"] = str(args.warps)
-    w = inputs.make_config(args.config)
+    w = inputs.config5(layers=args.layers) if (args.config == 5 and args.layers) else inputs.make_config(args.config)
     if args.P:
         w.P = args.P
     n, m, P = w.graph.n, w.graph.m, w.P
