@@ -404,3 +404,26 @@ def test_windowed_kernel_shapes(cpt, win_r, level32, monkeypatch):
     keep = g.dst < 16 * 300  # first 300 layers of the deep narrow graph
     g2 = I.Graph(n=16 * 300, src=g.src[keep], dst=g.dst[keep], t=g.t[keep], c=g.c[:16 * 300], mem=None, layers=300)
     run_and_compare(g2, w.devices, w.part_rows(0, 16 * 300)[:, :97], 2, pad_fill=255)
+
+
+# ------------------------------------------------------------- randomized sweep
+def test_randomized_shapes_all_variants():
+    """Forty seeded random workloads (sizes, device counts, candidate counts, dtypes, device-table structure
+    drawn at random), each evaluated by the automatic choice and by both forced kernel families."""
+    rng = np.random.default_rng(2024)
+    for trial in range(40):
+        n = int(rng.integers(1, 900))
+        m = int(rng.integers(0, 4 * n))
+        k = int(rng.choice([1, 2, 3, 4, 5, 8, 12, 16, 17, 33, 64]))
+        P = int(rng.choice([1, 7, 31, 32, 33, 64, 100, 257]))
+        tdt = np.int32 if trial % 2 else np.int64
+        w = I.small_random(5000 + trial, n, m, k, P, t_dtype=tdt, with_mem=bool(trial % 3))
+        dev = w.devices
+        if trial % 4 == 0 and k > 1:   # structured tables: two speeds, two bandwidths (value classes)
+            s = np.where(np.arange(k) % 2 == 0, 3, 11).astype(np.int32)
+            grp = np.arange(k) // 2
+            B = np.where(grp[:, None] == grp[None, :], 900, 70).astype(np.int64)
+            dev = I.Devices(k, s, dev.C, B, scale=int(rng.integers(1, 40)))
+        part = w.part_full()
+        for flags in (0, 1, 2):
+            run_and_compare(w.graph, dev, part, flags, pad_fill=255)
