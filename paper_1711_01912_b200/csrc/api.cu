@@ -872,12 +872,13 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
     const int narrow = level_bytes == 4 ? 1 : 0;
     const int head_max = std::max(g->blob_head_max[0][narrow], g->blob_head_max[1][narrow]);
     const int body_max = std::max(g->blob_body_max[0][narrow], g->blob_body_max[1][narrow]);
+    const int win_warps = std::min(32, std::max(2, warps + 1));   // consumer warps plus the producer warp
     if (use_window) {
         int r_need = 32;  // smallest power of two that keeps every edge inside the ring
         while (r_need < g->maxspan + CHUNK_V) r_need <<= 1;
         auto r_fit = [&](int c, int d) {
             const long long avail = (long long)g->smem_optin - 1024 -
-                                    (long long)window_smem_bytes(k, 0, c, warps, level_bytes, g->max_chunk_v, head_max, body_max, d);
+                                    (long long)window_smem_bytes(k, 0, c, win_warps, level_bytes, g->max_chunk_v, head_max, body_max, d);
             const long long rmax = avail / (32LL * c * (level_bytes + 1));
             int r = 0;
             for (int q = 32; q <= rmax && q <= (1 << 16); q <<= 1) r = q;
@@ -909,7 +910,7 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
             win_R = std::min(q, r_fit(cpt, win_depth));
         }
         if (win_R < CHUNK_V + 32) win_R = 0;
-        if (window_smem_bytes(k, win_R, cpt, warps, level_bytes, g->max_chunk_v, head_max, body_max, win_depth) >
+        if (window_smem_bytes(k, win_R, cpt, win_warps, level_bytes, g->max_chunk_v, head_max, body_max, win_depth) >
             (size_t)g->smem_optin)
             use_window = false;
     }
@@ -942,7 +943,7 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
             wp.R = win_R;
             wp.maxspan = g->maxspan;
             wp.all_staged = (fwd ? g->f_all_staged : g->b_all_staged) ? 1 : 0;
-            CUDA_TRY(launch_pass_window(a, fwd, wp, cpt, warps, st));
+            CUDA_TRY(launch_pass_window(a, fwd, wp, cpt, win_warps, st));
         } else if (sliced) {
             SlicedPlan plan;
             plan.vertf = g->vertf.as<int>();

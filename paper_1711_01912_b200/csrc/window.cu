@@ -118,7 +118,7 @@ __host__ __device__ inline Carve carve(int k, int R, int cpt, int warps, int lsi
     Carve c;
     const size_t slice = 32 * (size_t)cpt;
     size_t o = 0;
-    c.bars = o; o += up16(8 * (size_t)(3 * depth + 2) + 16);   // mbarriers, abort flag, two vertex counters
+    c.bars = o; o += up16(8 * (size_t)(3 * depth + 2) + 16);   // mbarriers, abort flag, two vertex counters, chunks-done counter
     c.rt = o; o += up16(sizeof(DivConst) * (size_t)k);
     c.cls2 = o; o += up16((size_t)k * k);
     c.cp = o;   // the staging rings double as the reduction buffer of the CP maxima after the last chunk
@@ -161,8 +161,9 @@ struct WinLayout {
 };
 
 // ALL_STAGED: every chunk's adjacency fits the staging buffers (no vertex with more than CHUNK_E edges).
-// Warp 0 doubles as the producer: at the top of every chunk it issues the copies for the chunk `depth`
-// ahead (heads 2*depth ahead) before it takes its share of the vertices.
+// The last warp is the producer: it runs its own loop, issuing the copies for the chunk `depth` ahead (heads
+// 2*depth ahead) as soon as the consumers report the ring slot free, and never joins the consumers' per-chunk
+// barrier (a named barrier over the consumer warps only), so its latency stays off their critical path.
 template <int CPT, bool FWD, bool ALL_STAGED, typename LT>
 __global__ void __launch_bounds__(1024)
 pass_window_kernel(PassArgs a, WindowPlan wp, WinLayout L)
@@ -171,7 +172,8 @@ pass_window_kernel(PassArgs a, WindowPlan wp, WinLayout L)
     constexpr int SLICE = 32 * CPT;
     constexpr unsigned LS = sizeof(LT);   // bytes of a level inside the block: 4 when every path length fits int32
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, wpb = blockDim.x >> 5;
-    const bool producer = warp == 0;
+    const int ncons = wpb - 1;                 // consumer warps 0..ncons-1
+    const bool producer = warp == ncons;
     const int k = a.tab.k;
     const int ncomb = wp.ncomb;
     const int R = wp.R;              // power of two (or 0)
@@ -184,6 +186,8 @@ pass_window_kernel(PassArgs a, WindowPlan wp, WinLayout L)
     volatile int* s_abort = reinterpret_cast<volatile int*>(smem + L.bars + 8 * (3 * L.depth + 2));
     // vertices of a chunk are handed out dynamically (degrees differ): one counter per chunk parity
     int* s_next = reinterpret_cast<int*>(smem + L.bars + 8 * (3 * L.depth + 2) + 4);
+    // number of chunks the consumers have finished: tells the producer which ring slots are free again
+    volatile int* s_done = reinterpret_cast<volatile int*>(smem + L.bars + 8 * (3 * L.depth + 2) + 12);
     if (*a.status != 0) return;
     const int D = L.depth, NB = 2 * D + 1, NS = D + 1;
     const unsigned head_bar0 = sbase + L.bars, stage_bar0 = head_bar0 + 8u * NB;
@@ -195,6 +199,7 @@ pass_window_kernel(PassArgs a, WindowPlan wp, WinLayout L)
         *s_abort = 0;
         s_next[0] = 0;
         s_next[1] = 0;
+        *s_done = 0;
         mbar_init_fence();
     }
     for (int i = threadIdx.x; i < k; i += blockDim.x) s_rt[i] = a.tab.rt_div[i];
@@ -283,20 +288,24 @@ pass_window_kernel(PassArgs a, WindowPlan wp, WinLayout L)
     int4 hq0, hq1, sq0, sq1;
     int hq_first = 0, sq_first = 0;
     hq0 = hq1 = sq0 = sq1 = make_int4(0, 0, 0, 0);
+    // ring positions: chunk ci (consumers), ci+D (producer: stage), ci+2D (producer: head)
+    int hs = 0, ss = 0;
+    unsigned sp = 0;
     if (producer) {
         load_desc(0, hq0, hq1);
         sq0 = hq0; sq1 = hq1;
         for (int j = 0; j < 2 * D && j < num_chunks; ++j) issue_head(bcast(hq0, j), j);       // 2D <= 16 < 32
         for (int j = 0; j < D && j < num_chunks; ++j) issue_stage(bcast(sq0, j), bcast(sq1, j), j, j, 0u);
-    }
-    // ring positions: chunk ci (consumers), ci+D (producer: stage), ci+2D (producer: head)
-    int hs = 0, ss = 0;
-    unsigned hp = 0, sp = 0;
-    int hsD = D % NB, ssD = D % NS, hs2D = (2 * D) % NB;
-    unsigned hpD = (unsigned)((D / NB) & 1);
-
-    for (int ci = 0; ci < num_chunks; ++ci) {
-        if (producer) {   // warp-uniform
+        int hsD = D % NB, ssD = D % NS, hs2D = (2 * D) % NB;
+        unsigned hpD = (unsigned)((D / NB) & 1);
+        for (int ci = 0; ci < num_chunks && !*s_abort; ++ci) {
+            // head(ci+2D) and stage(ci+D) overwrite the ring slots of chunk ci-1: wait until it is finished
+            bool freed = ci == 0;
+            for (int spin = 0; !freed && spin < WAIT_LIMIT; ++spin) {
+                freed = *s_done >= ci || *s_abort;
+                if (!freed) __nanosleep(32);
+            }
+            if (!freed) { fail_wait(); break; }
             if (ci + 2 * D < num_chunks) {
                 if (ci + 2 * D >= hq_first + 32) { hq_first += 32; load_desc(hq_first, hq0, hq1); }
                 issue_head(bcast(hq0, ci + 2 * D - hq_first), hs2D);
@@ -306,7 +315,13 @@ pass_window_kernel(PassArgs a, WindowPlan wp, WinLayout L)
                 const int src = ci + D - sq_first;
                 issue_stage(bcast(sq0, src), bcast(sq1, src), ssD, hsD, hpD);
             }
+            if (++hsD == NB) { hsD = 0; hpD ^= 1u; }
+            if (++ssD == NS) ssD = 0;
+            if (++hs2D == NB) hs2D = 0;
         }
+    }
+
+    for (int ci = 0; ci < num_chunks && !producer; ++ci) {
         // A stage is armed only after the producer has seen its head land, so seeing the stage complete
         // orders this thread after the head's arrival as well: one wait per chunk.
         if (!mbar_wait(stage_bar0 + 8u * ss, sp)) {
@@ -331,7 +346,7 @@ pass_window_kernel(PassArgs a, WindowPlan wp, WinLayout L)
 
             int* next_ctr = s_next + (ci & 1);
             if (threadIdx.x == 0) s_next[(ci + 1) & 1] = 0;   // last used by chunk ci-1, whose warps all passed the barrier
-            const bool dynamic = cnt > wpb;   // a narrow chunk gives every warp at most one vertex: no counter needed
+            const bool dynamic = cnt > ncons;   // a narrow chunk gives every warp at most one vertex: no counter needed
             for (bool first = true;; first = false) {
                 int i = warp;
                 if (dynamic) {
@@ -451,14 +466,17 @@ pass_window_kernel(PassArgs a, WindowPlan wp, WinLayout L)
                 }
             }
         }
-        __syncthreads();
+        // consumers only: results of this chunk are in the window, its ring slots are free again
+        asm volatile("bar.sync 1, %0;" ::"r"(ncons * 32) : "memory");
+        if (threadIdx.x == 0) {
+            __threadfence_block();
+            *s_done = ci + 1;
+        }
         if (*s_abort) break;
-        if (++hs == NB) { hs = 0; hp ^= 1u; }
+        if (++hs == NB) hs = 0;
         if (++ss == NS) { ss = 0; sp ^= 1u; }
-        if (++hsD == NB) { hsD = 0; hpD ^= 1u; }
-        if (++ssD == NS) ssD = 0;
-        if (++hs2D == NB) hs2D = 0;
     }
+    __syncthreads();   // producer and consumers meet again
     if (*s_abort) {
         // copies that were already requested may still be landing in this block's shared memory: give them
         // a bounded time before the block (and its shared memory) goes away
