@@ -160,16 +160,20 @@ struct WinLayout {
     int depth;
 };
 
-// ALL_STAGED: every chunk's adjacency fits the staging buffers (no vertex with more than CHUNK_E edges).
+// MODE 0: general.  MODE 1 (ALL_STAGED): every chunk's adjacency fits the staging buffers (no vertex with more
+// than CHUNK_E edges).  MODE 2: additionally every neighbour lies inside the window, so the loop carries neither
+// the distance test nor the global-memory path.
 // The last warp is the producer: it runs its own loop, issuing the copies for the chunk `depth` ahead (heads
 // 2*depth ahead) as soon as the consumers report the ring slot free, and never joins the consumers' per-chunk
 // barrier (a named barrier over the consumer warps only), so its latency stays off their critical path.
-template <int CPT, bool FWD, bool ALL_STAGED, typename LT>
+template <int CPT, bool FWD, int MODE, typename LT>
 __global__ void __launch_bounds__(1024)
 pass_window_kernel(PassArgs a, WindowPlan wp, WinLayout L)
 {
     extern __shared__ __align__(16) unsigned char smem[];
     constexpr int SLICE = 32 * CPT;
+    constexpr bool ALL_STAGED = MODE >= 1;
+    constexpr bool FULL_WINDOW = MODE == 2;
     constexpr unsigned LS = sizeof(LT);   // bytes of a level inside the block: 4 when every path length fits int32
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, wpb = blockDim.x >> 5;
     const int ncons = wpb - 1;                 // consumer warps 0..ncons-1
@@ -376,7 +380,7 @@ pass_window_kernel(PassArgs a, WindowPlan wp, WinLayout L)
                         const int span = FWD ? pos - np : np - pos;
                         LT lu[CPT];
                         unsigned pu;
-                        if (span <= hit_span) {
+                        if (FULL_WINDOW || span <= hit_span) {
                             const int slot = np & rmask;
                             load_win<CPT>(win_lev_lane + slot * SLICE, lu);
                             unsigned w[IdWords<CPT>::N];
@@ -585,7 +589,7 @@ __global__ void npos_kernel(int n, const int* __restrict__ pos_of, const int* __
 
 inline unsigned cdivu(long long a, long long b) { return (unsigned)((a + b - 1) / b); }
 
-template <int CPT, bool FWD, bool ALL_STAGED, typename LT>
+template <int CPT, bool FWD, int MODE, typename LT>
 cudaError_t window_impl(const PassArgs& a, const WindowPlan& plan, int warps, cudaStream_t st)
 {
     const Carve c = carve(a.tab.k, plan.R, CPT, warps, (int)sizeof(LT), plan.max_v, plan.head_max, plan.body_max, plan.depth);
@@ -596,10 +600,10 @@ cudaError_t window_impl(const PassArgs& a, const WindowPlan& plan, int warps, cu
     L.ids = (unsigned)c.ids; L.ids_stride = (unsigned)c.ids_stride;
     L.win_lev = (unsigned)c.win_lev; L.win_id = (unsigned)c.win_id;
     L.depth = plan.depth;
-    cudaError_t e = cudaFuncSetAttribute(pass_window_kernel<CPT, FWD, ALL_STAGED, LT>,
+    cudaError_t e = cudaFuncSetAttribute(pass_window_kernel<CPT, FWD, MODE, LT>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c.total);
     if (e != cudaSuccess) return e;
-    pass_window_kernel<CPT, FWD, ALL_STAGED, LT><<<cdivu(a.P, 32 * CPT), warps * 32, c.total, st>>>(a, plan, L);
+    pass_window_kernel<CPT, FWD, MODE, LT><<<cdivu(a.P, 32 * CPT), warps * 32, c.total, st>>>(a, plan, L);
     count_launches(1);
     return cudaGetLastError();
 }
@@ -607,9 +611,11 @@ cudaError_t window_impl(const PassArgs& a, const WindowPlan& plan, int warps, cu
 template <int CPT, typename LT>
 cudaError_t window_dispatch(const PassArgs& a, bool fwd, const WindowPlan& plan, int warps, cudaStream_t st)
 {
+    if (plan.all_staged && plan.R - CHUNK_V >= plan.maxspan)
+        return fwd ? window_impl<CPT, true, 2, LT>(a, plan, warps, st) : window_impl<CPT, false, 2, LT>(a, plan, warps, st);
     if (plan.all_staged)
-        return fwd ? window_impl<CPT, true, true, LT>(a, plan, warps, st) : window_impl<CPT, false, true, LT>(a, plan, warps, st);
-    return fwd ? window_impl<CPT, true, false, LT>(a, plan, warps, st) : window_impl<CPT, false, false, LT>(a, plan, warps, st);
+        return fwd ? window_impl<CPT, true, 1, LT>(a, plan, warps, st) : window_impl<CPT, false, 1, LT>(a, plan, warps, st);
+    return fwd ? window_impl<CPT, true, 0, LT>(a, plan, warps, st) : window_impl<CPT, false, 0, LT>(a, plan, warps, st);
 }
 
 }  // namespace
