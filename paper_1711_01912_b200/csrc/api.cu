@@ -938,6 +938,7 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
             wp.head_max = head_max;
             wp.body_max = body_max;
             wp.depth = win_depth;
+            wp.static_rounds = std::max(1, env_int("TFPS_WINDOW_STATIC_ROUNDS", 1));
             wp.cls2 = fwd ? g->cls2_f.as<uint8_t>() : g->cls2_b.as<uint8_t>();
             wp.ncomb = g->ncomb;
             wp.R = win_R;

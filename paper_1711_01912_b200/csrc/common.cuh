@@ -138,6 +138,7 @@ struct WindowPlan {
     const unsigned char* blob;
     int max_v, head_max, body_max;  // largest chunk: vertices, head bytes, body bytes
     int depth;                   // chunks staged ahead
+    int static_rounds;           // chunks of at most this many vertices per consumer warp use a fixed vertex assignment
 };
 
 // every kernel launch of the library goes through the wrappers below and is counted here

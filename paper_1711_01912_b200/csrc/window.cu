@@ -350,14 +350,12 @@ pass_window_kernel(PassArgs a, WindowPlan wp, WinLayout L)
 
             int* next_ctr = s_next + (ci & 1);
             if (threadIdx.x == 0) s_next[(ci + 1) & 1] = 0;   // last used by chunk ci-1, whose warps all passed the barrier
-            const bool dynamic = cnt > ncons;   // a narrow chunk gives every warp at most one vertex: no counter needed
-            for (bool first = true;; first = false) {
-                int i = warp;
+            const bool dynamic = cnt > ncons * wp.static_rounds;   // few vertices per warp: a fixed assignment is cheaper than the counter
+            for (int round = 0;; ++round) {
+                int i = warp + round * ncons;
                 if (dynamic) {
                     if (lane == 0) i = atomicAdd(next_ctr, 1);
                     i = __shfl_sync(0xffffffffu, i, 0);
-                } else if (!first) {
-                    break;
                 }
                 if (i >= cnt) break;
                 const int vf = vertf_p[i];
