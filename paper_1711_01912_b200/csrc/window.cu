@@ -250,7 +250,7 @@ pass_window_kernel(PassArgs a, WindowPlan wp, WinLayout L)
         return make_int4(__shfl_sync(0xffffffffu, v.x, src), __shfl_sync(0xffffffffu, v.y, src),
                          __shfl_sync(0xffffffffu, v.z, src), __shfl_sync(0xffffffffu, v.w, src));
     };
-    auto issue_head = [&](const int4& d, int slot) {   // chunk -> head ring slot
+    auto issue_head = [&](const int4& d, int slot) {   // chunk -> head ring slot (needs d.x, d.y)
         if (lane == 0) {
             const unsigned bar = head_bar0 + 8u * slot;
             mbar_expect_tx(bar, (unsigned)d.y);
@@ -307,17 +307,19 @@ pass_window_kernel(PassArgs a, WindowPlan wp, WinLayout L)
             bool freed = ci == 0;
             for (int spin = 0; !freed && spin < WAIT_LIMIT; ++spin) {
                 freed = *s_done >= ci || *s_abort;
-                if (!freed) __nanosleep(32);
             }
             if (!freed) { fail_wait(); break; }
             if (ci + 2 * D < num_chunks) {
                 if (ci + 2 * D >= hq_first + 32) { hq_first += 32; load_desc(hq_first, hq0, hq1); }
-                issue_head(bcast(hq0, ci + 2 * D - hq_first), hs2D);
+                const int src = ci + 2 * D - hq_first;
+                issue_head(make_int4(__shfl_sync(0xffffffffu, hq0.x, src), __shfl_sync(0xffffffffu, hq0.y, src), 0, 0), hs2D);
             }
             if (ci + D < num_chunks) {
                 if (ci + D >= sq_first + 32) { sq_first += 32; load_desc(sq_first, sq0, sq1); }
                 const int src = ci + D - sq_first;
-                issue_stage(bcast(sq0, src), bcast(sq1, src), ssD, hsD, hpD);
+                const int4 b0 = make_int4(0, 0, __shfl_sync(0xffffffffu, sq0.z, src), __shfl_sync(0xffffffffu, sq0.w, src));
+                const int4 b1 = make_int4(__shfl_sync(0xffffffffu, sq1.x, src), __shfl_sync(0xffffffffu, sq1.y, src), 0, 0);
+                issue_stage(b0, b1, ssD, hsD, hpD);
             }
             if (++hsD == NB) { hsD = 0; hpD ^= 1u; }
             if (++ssD == NS) ssD = 0;
