@@ -168,8 +168,10 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp,
  * host outputs, any of which may be NULL.  Copies the ids to the device, runs
  * the load kernel and BOTH passes (the level matrices live in scratch owned by
  * the handle and are copied back only when a host pointer is given), copies
- * the other results back and synchronises `stream`.  Staging and scratch
- * buffers grow on demand and stay with the handle.  Pinned host memory makes
+ * the other results back and synchronises `stream`.  Large batches go up in two
+ * column chunks on an internal copy stream so that the second half's transfer
+ * overlaps the first half's evaluation.  Staging and scratch buffers (and that
+ * stream) are created on demand and stay with the handle.  Pinned host memory makes
  * the copies asynchronous and fast; pageable memory works too.  Returns the
  * device status as tfps_get_status would.
  */

@@ -140,10 +140,16 @@ struct tfps_graph {
     bool ev_valid = false;
     bool ran_fwd = false, ran_bwd = false;
     const char* last_kernel = "";
+    // copy stream and per-chunk events of tfps_eval_batch_host (created on first use)
+    cudaStream_t copy_stream = nullptr;
+    cudaEvent_t copy_ev[9] = {};
     ~tfps_graph()
     {
         for (cudaEvent_t e : ev)
             if (e) cudaEventDestroy(e);
+        for (cudaEvent_t e : copy_ev)
+            if (e) cudaEventDestroy(e);
+        if (copy_stream) cudaStreamDestroy(copy_stream);
     }
 };
 
@@ -1070,11 +1076,39 @@ int tfps_eval_batch_host(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* p
     if (load) CUDA_TRY(g->st_load.reserve(kcells * 8));
     if (memload || viol) CUDA_TRY(g->st_mem.reserve(kcells * 8));
     if (viol) CUDA_TRY(g->st_viol.reserve((size_t)P * 8));
-    CUDA_TRY(cudaMemcpyAsync(g->st_part.p, part, cells, cudaMemcpyHostToDevice, st));
-    TFPS_TRY(tfps_eval_batch(g, P, ldp, g->st_part.as<uint8_t>(), g->st_lev.as<int64_t>(), g->st_lev2.as<int64_t>(),
-                             g->st_cp.as<int64_t>(), load ? g->st_load.as<int64_t>() : nullptr,
-                             (memload || viol) ? g->st_mem.as<int64_t>() : nullptr,
-                             viol ? g->st_viol.as<uint64_t>() : nullptr, nullptr, 0, flags, st));
+    // Candidates are independent: the id matrix goes up in column chunks on a copy stream and every chunk is
+    // evaluated as soon as it has landed, so the transfer of chunk c+1 overlaps the evaluation of chunk c.
+    // (a chunk must still fill the GPU: one wave of blocks of the sliced kernel is 64 candidates per SM)
+    int nchunks = P >= 128LL * g->sm_count * 3 / 4 ? 2 : 1;
+    long long width = (P + nchunks - 1) / nchunks;
+    width = (width + 127) / 128 * 128;   // whole candidate slices per chunk
+    nchunks = (int)((P + width - 1) / width);
+    if (nchunks > 1) {
+        if (!g->copy_stream) CUDA_TRY(cudaStreamCreateWithFlags(&g->copy_stream, cudaStreamNonBlocking));
+        for (int c = 0; c <= nchunks; ++c)
+            if (!g->copy_ev[c]) CUDA_TRY(cudaEventCreateWithFlags(&g->copy_ev[c], cudaEventDisableTiming));
+        // the staging buffers may still be in use by earlier work on the caller's stream
+        CUDA_TRY(cudaEventRecord(g->copy_ev[nchunks], st));
+        CUDA_TRY(cudaStreamWaitEvent(g->copy_stream, g->copy_ev[nchunks], 0));
+    }
+    for (int c = 0; c < nchunks; ++c) {
+        const long long j0 = (long long)c * width;
+        const long long w = std::min<long long>(width, P - j0);
+        const long long wl = std::min<long long>(width, ldp - j0);   // bytes per row to copy: whole 16-byte pieces
+        if (nchunks > 1) {
+            CUDA_TRY(cudaMemcpy2DAsync(g->st_part.as<uint8_t>() + j0, (size_t)ldp, part + j0, (size_t)ldp, (size_t)wl,
+                                       (size_t)g->n, cudaMemcpyHostToDevice, g->copy_stream));
+            CUDA_TRY(cudaEventRecord(g->copy_ev[c], g->copy_stream));
+            CUDA_TRY(cudaStreamWaitEvent(st, g->copy_ev[c], 0));
+        } else {
+            CUDA_TRY(cudaMemcpyAsync(g->st_part.p, part, cells, cudaMemcpyHostToDevice, st));
+        }
+        TFPS_TRY(tfps_eval_batch(g, w, ldp, g->st_part.as<uint8_t>() + j0, g->st_lev.as<int64_t>() + j0,
+                                 g->st_lev2.as<int64_t>() + j0, g->st_cp.as<int64_t>() + j0,
+                                 load ? g->st_load.as<int64_t>() + j0 : nullptr,
+                                 (memload || viol) ? g->st_mem.as<int64_t>() + j0 : nullptr,
+                                 viol ? g->st_viol.as<uint64_t>() + j0 : nullptr, nullptr, 0, flags, st));
+    }
     if (tlevel) CUDA_TRY(cudaMemcpyAsync(tlevel, g->st_lev.p, cells * 8, cudaMemcpyDeviceToHost, st));
     if (blevel) CUDA_TRY(cudaMemcpyAsync(blevel, g->st_lev2.p, cells * 8, cudaMemcpyDeviceToHost, st));
     if (cp) CUDA_TRY(cudaMemcpyAsync(cp, g->st_cp.p, (size_t)P * 8, cudaMemcpyDeviceToHost, st));

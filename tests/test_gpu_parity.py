@@ -241,6 +241,32 @@ def test_host_entry_point_matches():
     G.close()
 
 
+def test_host_entry_point_pipelined_in_two_column_chunks():
+    """Enough candidates for the host entry point to upload and evaluate in two column chunks."""
+    import oracle
+    w = I.config1()
+    n = w.graph.n
+    P = 15000
+    ldp = 15008
+    rng = np.random.default_rng(9)
+    buf = rng.integers(0, w.devices.k, size=(n, ldp), dtype=np.uint8)
+    G = gpu_graph(w.graph, w.devices)
+    res = G.eval_batch_host(buf, P, want=("tlevel", "blevel", "cp", "load", "memload", "viol"))
+    og = oracle_graph(w.graph)
+    d = w.devices
+    cols = [0, 1, 7423, 7424, 7551, 7552, 7553, 14999]   # both sides of the chunk boundary
+    ref = oracle.eval_batch(og, d.k, d.s, d.C, d.B, d.scale, buf, cols)
+    assert np.array_equal(res["tlevel"][:, cols], ref.tlevel)
+    assert np.array_equal(res["blevel"][:, cols], ref.blevel)
+    assert np.array_equal(res["cp"][cols], ref.cp)
+    assert np.array_equal(res["load"][:, cols], ref.load)
+    assert np.array_equal(res["memload"][:, cols], ref.memload)
+    assert np.array_equal(res["viol"][cols], ref.viol)
+    # every candidate: CP = max_v(tlevel + blevel)
+    assert np.array_equal((res["tlevel"][:, :P] + res["blevel"][:, :P]).max(axis=0), res["cp"][:P])
+    G.close()
+
+
 def test_transpose_u8():
     from paper_1711_01912_b200 import tfps
     torch = _torch()
