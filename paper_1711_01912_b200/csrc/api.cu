@@ -131,6 +131,12 @@ struct tfps_graph {
     std::vector<long long> h_in_ptr, h_in_t;
     std::vector<int> h_in_src, h_c;
     int npass = 0, use_cls = 0, ncls_w = 0;
+    // lean windowed pass: host-packed chunk records per direction (0 forward, 1 backward)
+    struct Lean {
+        bool ok = false;
+        DBuf blob, desc, vlist;
+        LeanPlan plan;
+    } lean[2];
     DBuf status;
     // scratch owned by the handle
     DBuf scr_memload;
@@ -358,6 +364,158 @@ int env_int(const char* name, int dflt)
     const char* s = getenv(name);
     if (!s || !*s) return dflt;
     return atoi(s);
+}
+
+// Packs the chunk records of the lean windowed pass for both directions (layout: LeanPlan in common.cuh).
+// Everything is computed on the host with plain integer division; `order` is the host copy of the level order.
+int build_lean(tfps_graph* g, int k, const int32_t* s, const int64_t* B, long long S, const std::vector<int>& order,
+               cudaStream_t st)
+{
+    for (auto& L : g->lean) L.ok = false;
+    const int n = (int)g->n, m = (int)g->m;
+    if (!g->fits32 || k > LEAN_K_MAX || n == 0 || env_int("TFPS_LEAN", 1) == 0) return TFPS_OK;
+    std::vector<long long> wvals;   // distinct off-diagonal bandwidths; class c+1 <-> wvals[c], class 0 = same device
+    auto cls_of = [&](long long x) {
+        for (size_t i = 0; i < wvals.size(); ++i)
+            if (wvals[i] == x) return (int)i;
+        wvals.push_back(x);
+        return (int)wvals.size() - 1;
+    };
+    for (int a = 0; a < k; ++a)
+        for (int b = 0; b < k; ++b)
+            if (a != b) cls_of(B[a * k + b]);
+    const int ncw = (int)wvals.size();
+    if (ncw > LEAN_CLS_MAX) return TFPS_OK;
+    const int KP = k <= 4 ? 4 : 8;
+    const int vstride = 16 + 4 * KP, estride = 4 * (ncw + 2);
+    const int e_cap = std::max(64, std::min(1024, 24576 / estride));   // edges per chunk
+
+    std::vector<int> pos_of((size_t)n);
+    for (int i = 0; i < n; ++i) pos_of[order[i]] = i;
+    std::vector<int> eptr[2], nbr[2];
+    std::vector<long long> tt[2];
+    for (int dir = 0; dir < 2; ++dir) {
+        eptr[dir].resize((size_t)n + 1);
+        nbr[dir].resize((size_t)m);
+        tt[dir].resize((size_t)m);
+        CUDA_TRY(cudaMemcpyAsync(eptr[dir].data(), dir == 0 ? g->f_eptr.p : g->b_eptr.p, sizeof(int) * ((size_t)n + 1),
+                                 cudaMemcpyDeviceToHost, st));
+        if (m > 0) {
+            CUDA_TRY(cudaMemcpyAsync(nbr[dir].data(), dir == 0 ? g->f_nbr.p : g->b_nbr.p, sizeof(int) * (size_t)m,
+                                     cudaMemcpyDeviceToHost, st));
+            CUDA_TRY(cudaMemcpyAsync(tt[dir].data(), dir == 0 ? g->f_t.p : g->b_t.p, sizeof(long long) * (size_t)m,
+                                     cudaMemcpyDeviceToHost, st));
+        }
+    }
+    CUDA_TRY(cudaStreamSynchronize(st));
+    auto ceil_div = [](long long a, long long S_, long long d) {
+        return (long long)(((u128)a * (u128)S_ + (u128)d - 1) / (u128)d);
+    };
+    const int src_end = (int)g->h_level_ptr[1];
+
+    for (int dir = 0; dir < 2; ++dir) {
+        tfps_graph::Lean& L = g->lean[dir];
+        const std::vector<int>& ep = eptr[dir];
+        // chunks: runs of positions inside one level; a wide level is split evenly
+        std::vector<int> ch_p0, ch_cnt;
+        bool ok = true;
+        int max_v = 1;
+        for (int li = 0; li < g->num_levels && ok; ++li) {
+            const int l = dir == 0 ? li : g->num_levels - 1 - li;
+            int p = (int)g->h_level_ptr[l];
+            const int pend = (int)g->h_level_ptr[l + 1];
+            const int width = pend - p;
+            int target = width;
+            if (width > LEAN_CHUNK_V) {
+                const int nch = (width + LEAN_CHUNK_V - 1) / LEAN_CHUNK_V;
+                target = std::min(LEAN_CHUNK_V, (((width + nch - 1) / nch) + 31) / 32 * 32);
+            }
+            while (p < pend) {
+                int q = p, edges = 0;
+                while (q < pend && q - p < target && edges + (ep[q + 1] - ep[q]) <= e_cap) { edges += ep[q + 1] - ep[q]; ++q; }
+                if (q == p) { ok = false; break; }   // a vertex with more edges than a chunk can stage
+                ch_p0.push_back(p);
+                ch_cnt.push_back(q - p);
+                max_v = std::max(max_v, q - p);
+                p = q;
+            }
+        }
+        if (!ok) continue;
+        int R = 1;
+        while (R < g->maxspan + max_v) R <<= 1;
+        const int nc = (int)ch_p0.size();
+        std::vector<int> desc((size_t)(nc + 2 * LEAN_DEPTH_MAX) * 4, 0), vlist((size_t)n);
+        std::vector<unsigned char> blob;
+        blob.reserve((size_t)n * vstride + (size_t)m * estride + (size_t)nc * 32);
+        std::vector<int> idx;
+        int rec_max = 16, vfirst = 0;
+        for (int c = 0; c < nc; ++c) {
+            const int p0 = ch_p0[c], cnt = ch_cnt[c];
+            idx.resize((size_t)cnt);
+            for (int i = 0; i < cnt; ++i) idx[i] = p0 + i;
+            // highest degree first: dealt round-robin, every round of the warps sees similar degrees
+            std::stable_sort(idx.begin(), idx.end(), [&](int a, int b) { return ep[a + 1] - ep[a] > ep[b + 1] - ep[b]; });
+            int ne = 0;
+            for (int i = 0; i < cnt; ++i) ne += ep[idx[i] + 1] - ep[idx[i]];
+            const size_t e_area = 16 + (size_t)cnt * vstride;
+            const size_t bytes = (e_area + (size_t)ne * estride + 15) & ~(size_t)15;
+            const size_t off = blob.size();
+            blob.resize(off + bytes, 0);
+            int* hdr = reinterpret_cast<int*>(blob.data() + off);
+            hdr[0] = cnt;
+            hdr[1] = (int)e_area;
+            int eb = 0;
+            for (int i = 0; i < cnt; ++i) {
+                const int p = idx[i], v = order[p];
+                int* vr = reinterpret_cast<int*>(blob.data() + off + 16 + (size_t)i * vstride);
+                const bool flag = dir == 0 ? (eptr[1][p + 1] == eptr[1][p]) : (p < src_end);
+                vr[0] = v | (flag ? (int)0x80000000u : 0);
+                vr[1] = p & (R - 1);
+                vr[2] = eb;
+                for (int d = 0; d < k; ++d) vr[4 + d] = (int)ceil_div(g->h_c[v], S, s[d]);
+                for (int q = ep[p]; q < ep[p + 1]; ++q) {
+                    int* er = reinterpret_cast<int*>(blob.data() + off + e_area + (size_t)eb);
+                    er[0] = pos_of[nbr[dir][q]] & (R - 1);
+                    er[1] = 0;
+                    for (int w = 0; w < ncw; ++w) er[2 + w] = (int)ceil_div(tt[dir][q], S, wvals[w]);
+                    eb += estride;
+                }
+                vr[3] = eb;
+                vlist[(size_t)vfirst + i] = v;
+            }
+            desc[4 * (size_t)c + 0] = (int)(off / 16);
+            desc[4 * (size_t)c + 1] = (int)bytes;
+            desc[4 * (size_t)c + 2] = cnt;
+            desc[4 * (size_t)c + 3] = vfirst;
+            vfirst += cnt;
+            rec_max = std::max(rec_max, (int)bytes);
+        }
+        if (blob.size() / 16 >= ((size_t)1 << 31)) continue;
+        TFPS_TRY(upload(L.blob, blob, st));
+        TFPS_TRY(upload(L.desc, desc, st));
+        TFPS_TRY(upload(L.vlist, vlist, st));
+        CUDA_TRY(cudaStreamSynchronize(st));
+        L.plan.blob = L.blob.as<unsigned char>();
+        L.plan.desc = L.desc.as<int4>();
+        L.plan.vlist = L.vlist.as<int>();
+        L.plan.num_chunks = nc;
+        L.plan.vstride = vstride;
+        L.plan.estride = estride;
+        L.plan.R = R;
+        L.plan.rec_max = rec_max;
+        L.plan.max_v = max_v;
+        for (int pv = 0; pv < LEAN_K_MAX; ++pv) {
+            unsigned long long row = 0;
+            for (int pu = 0; pu < LEAN_K_MAX; ++pu) {
+                unsigned long long byte = 0;
+                if (pv < k && pu < k && pu != pv) byte = 4ull * (unsigned)(cls_of(dir == 0 ? B[pu * k + pv] : B[pv * k + pu]) + 1);
+                row |= byte << (8 * pu);
+            }
+            L.plan.rows[pv] = row;
+        }
+        L.ok = true;
+    }
+    return TFPS_OK;
 }
 
 }  // namespace
@@ -674,7 +832,8 @@ int tfps_devices_set(tfps_graph* g, int k, const int32_t* s, const int64_t* C, c
                                    g->xvert.as<unsigned long long>(), g->xw_f.as<unsigned long long>(),
                                    g->xnbr_f.as<unsigned long long>(), g->xw_b.as<unsigned long long>(), st));
     g->fits32 = false;
-    if (g->ncomb > 0 && n > 0) {
+    for (auto& L : g->lean) L.ok = false;
+    if ((g->ncomb > 0 || k <= LEAN_K_MAX) && n > 0) {
         // worst-case critical path: every vertex on the slowest device, every edge over the slowest link
         std::vector<int> order((size_t)n);
         CUDA_TRY(cudaMemcpyAsync(order.data(), g->order.p, sizeof(int) * (size_t)n, cudaMemcpyDeviceToHost, st));
@@ -692,6 +851,9 @@ int tfps_devices_set(tfps_graph* g, int k, const int32_t* s, const int64_t* C, c
             worst = std::max(worst, fin[v]);
         }
         g->fits32 = worst < (1LL << 31) - 1;
+        TFPS_TRY(build_lean(g, k, s, B, scale, order, st));
+    }
+    if (g->ncomb > 0 && n > 0) {
         CUDA_TRY(g->V_f.reserve(sizeof(long long) * (size_t)m * g->ncomb + 16));
         CUDA_TRY(g->V_b.reserve(sizeof(long long) * (size_t)m * g->ncomb + 16));
         if (g->fits32) {
@@ -929,6 +1091,48 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
         long long* cp_here = (cp && (fwd || !need_fwd)) ? (long long*)cp : nullptr;
         PassArgs a = make_args(g, fwd, P, ldp, part, lev, cp_here);
         g->last_kernel = use_window ? "pass_window_kernel" : (sliced ? "pass_sliced_kernel" : (g->npass > 0 ? "pass_tile_kernel" : "pass_level_kernel"));
+        // lean windowed pass: 32-bit levels, whole window resident, host-packed records
+        if (sliced && g->lean[0].ok && g->lean[1].ok && level_bytes == 4 && ((uintptr_t)part & 15u) == 0 &&
+            env_int("TFPS_LEAN", 1) != 0) {
+            const LeanPlan& lp = g->lean[fwd ? 0 : 1].plan;
+            const int forced = env_int("TFPS_SLICED_CPT", 0);
+            const long long want_slices = std::min<long long>((3LL * g->sm_count) / 4, (P + 31) / 32);
+            int d_want = env_int("TFPS_LEAN_DEPTH", 0);
+            if (d_want < 1 || d_want > LEAN_DEPTH_MAX) d_want = 3;
+            int l_cpt = 0, l_depth = 0, l_warps = 0;
+            size_t l_smem = 0;
+            LeanArgs la;
+            for (int c = 4; c >= 1 && !l_cpt; c >>= 1) {
+                if (forced == 1 || forced == 2 || forced == 4) { if (c != forced) continue; }
+                else if ((P + 32 * c - 1) / (32 * c) < want_slices && c > 1) continue;
+                int w = warps;   // every warp consumes; each thread fetches at most two id-row pieces per chunk
+                while (w < 32 && lp.max_v * 2 * c > 2 * w * 32) w <<= 1;
+                if (lp.max_v * 2 * c > 2 * w * 32) continue;
+                for (int d = d_want; d >= 1; --d) {
+                    unsigned slot_stride = 0, stage_bytes = 0;
+                    const size_t need = lean_smem_bytes(lp, c, w, d, &slot_stride, &stage_bytes);
+                    if (need + 512 <= (size_t)g->smem_optin) {
+                        l_cpt = c; l_depth = d; l_warps = w; l_smem = need;
+                        la.slot_stride = slot_stride;
+                        la.stage_bytes = stage_bytes;
+                        break;
+                    }
+                }
+            }
+            if (l_cpt) {
+                la.part = part;
+                la.lev = lev;
+                la.cp = cp_here;
+                la.status = status;
+                la.P = P;
+                la.ldp = ldp;
+                la.plan = lp;
+                la.depth = l_depth;
+                g->last_kernel = "pass_lean_kernel";
+                CUDA_TRY(launch_pass_lean(la, fwd, l_cpt, l_warps, l_smem, st));
+                continue;
+            }
+        }
         if (use_window) {
             WindowPlan wp;
             wp.vertf = g->vertf.as<int>();

@@ -141,6 +141,49 @@ struct WindowPlan {
     int static_rounds;           // chunks of at most this many vertices per consumer warp use a fixed vertex assignment
 };
 
+// Lean windowed pass (32-bit levels, k <= LEAN_K_MAX, whole window resident).  The host packs, per direction
+// and in processing order, one record per chunk:
+//   header  int4 {vertices, byte offset of the edge area, 0, 0}
+//   vertex  [vstride bytes each]  {v | flag << 31, window slot, first edge byte, end edge byte, rt[KP]}
+//           flag: sink (forward) / source (backward): the vertex enters the CP maximum;
+//           rt[d] = ceil(c_v*S / s_d); edge bytes are relative to the edge area
+//   edge    [estride bytes each]  {window slot of the neighbour, W[0] = 0, W[1..ncls]}
+//           W[c] = ceil(t_e*S / b_c) for the c-th distinct off-diagonal bandwidth b_c
+// rows[pv] holds, in byte pu, 4 * (class of the link between a neighbour on device pu and a vertex on device
+// pv; 0 = same device), so one byte permute turns the neighbour's id into the offset of W inside the edge record.
+// The window keeps finish times (forward) or bottom levels (backward), so an edge adds the transfer term only.
+constexpr int LEAN_K_MAX = 8;
+constexpr int LEAN_CLS_MAX = 30;     // 4 * (classes + 1) must stay below 0x80 (sign-replicating byte permute)
+constexpr int LEAN_CHUNK_V = 128;
+constexpr int LEAN_DEPTH_MAX = 4;
+
+struct LeanPlan {
+    const unsigned char* blob;   // chunk records, 16-byte aligned each
+    const int4* desc;            // [num_chunks + 2*LEAN_DEPTH_MAX] {offset/16, bytes, vertices, first index into vlist}; zero padded
+    const int* vlist;            // [n] vertex ids in processing order
+    int num_chunks;
+    int vstride, estride;
+    int R;                       // window length in positions (power of two)
+    int rec_max;                 // largest record, bytes (multiple of 16)
+    int max_v;                   // most vertices in one chunk
+    unsigned long long rows[LEAN_K_MAX];
+};
+
+struct LeanArgs {
+    const uint8_t* part;
+    long long* lev;
+    long long* cp;
+    int* status;
+    long long P, ldp;
+    LeanPlan plan;
+    int depth;                   // chunks in flight (stage slots)
+    unsigned slot_stride;        // bytes of a stage slot: rec_max + max_v * slice
+    unsigned stage_bytes;        // bytes reserved for all stage slots (also the CP reduction buffer)
+};
+
+size_t lean_smem_bytes(const LeanPlan& plan, int cpt, int warps, int depth, unsigned* slot_stride, unsigned* stage_bytes);
+cudaError_t launch_pass_lean(const LeanArgs& a, bool fwd, int cpt, int warps, size_t smem, cudaStream_t st);
+
 // every kernel launch of the library goes through the wrappers below and is counted here
 void count_launches(long long n);
 
