@@ -446,9 +446,10 @@ int build_lean(tfps_graph* g, int k, const int32_t* s, const int64_t* B, long lo
         const int nc = (int)ch_p0.size();
         std::vector<int> desc((size_t)(nc + 2 * LEAN_DEPTH_MAX) * 4, 0), vlist((size_t)n);
         std::vector<unsigned char> blob;
-        blob.reserve((size_t)n * vstride + (size_t)m * estride + (size_t)nc * 32);
-        std::vector<int> idx;
+        std::vector<int> idx, sorted((size_t)n);
         int rec_max = 16, vfirst = 0;
+        // first the processing order and the descriptors (a record names the chunks that follow it) ...
+        size_t total = 0;
         for (int c = 0; c < nc; ++c) {
             const int p0 = ch_p0[c], cnt = ch_cnt[c];
             idx.resize((size_t)cnt);
@@ -456,18 +457,34 @@ int build_lean(tfps_graph* g, int k, const int32_t* s, const int64_t* B, long lo
             // highest degree first: dealt round-robin, every round of the warps sees similar degrees
             std::stable_sort(idx.begin(), idx.end(), [&](int a, int b) { return ep[a + 1] - ep[a] > ep[b + 1] - ep[b]; });
             int ne = 0;
-            for (int i = 0; i < cnt; ++i) ne += ep[idx[i] + 1] - ep[idx[i]];
-            const size_t e_area = 16 + (size_t)cnt * vstride;
+            for (int i = 0; i < cnt; ++i) { ne += ep[idx[i] + 1] - ep[idx[i]]; sorted[(size_t)vfirst + i] = idx[i]; }
+            const size_t e_area = LEAN_HDR_BYTES + (size_t)cnt * vstride;
             const size_t bytes = (e_area + (size_t)ne * estride + 15) & ~(size_t)15;
-            const size_t off = blob.size();
-            blob.resize(off + bytes, 0);
+            desc[4 * (size_t)c + 0] = (int)(total / 16);
+            desc[4 * (size_t)c + 1] = (int)bytes;
+            desc[4 * (size_t)c + 2] = cnt;
+            desc[4 * (size_t)c + 3] = vfirst;
+            vfirst += cnt;
+            total += bytes;
+            rec_max = std::max(rec_max, (int)bytes);
+        }
+        if (total / 16 >= ((size_t)1 << 31)) continue;
+        // ... then the records
+        blob.assign(total, 0);
+        for (int c = 0; c < nc; ++c) {
+            const int cnt = ch_cnt[c];
+            const size_t off = (size_t)desc[4 * (size_t)c] * 16;
+            const int first = desc[4 * (size_t)c + 3];
+            const size_t e_area = LEAN_HDR_BYTES + (size_t)cnt * vstride;
             int* hdr = reinterpret_cast<int*>(blob.data() + off);
             hdr[0] = cnt;
             hdr[1] = (int)e_area;
+            for (int d = 1; d <= LEAN_DEPTH_MAX; ++d)
+                for (int q = 0; q < 4; ++q) hdr[4 * d + q] = desc[4 * (size_t)(c + d) + q];   // zero past the end
             int eb = 0;
             for (int i = 0; i < cnt; ++i) {
-                const int p = idx[i], v = order[p];
-                int* vr = reinterpret_cast<int*>(blob.data() + off + 16 + (size_t)i * vstride);
+                const int p = sorted[(size_t)first + i], v = order[p];
+                int* vr = reinterpret_cast<int*>(blob.data() + off + LEAN_HDR_BYTES + (size_t)i * vstride);
                 const bool flag = dir == 0 ? (eptr[1][p + 1] == eptr[1][p]) : (p < src_end);
                 vr[0] = v | (flag ? (int)0x80000000u : 0);
                 vr[1] = p & (R - 1);
@@ -481,14 +498,8 @@ int build_lean(tfps_graph* g, int k, const int32_t* s, const int64_t* B, long lo
                     eb += estride;
                 }
                 vr[3] = eb;
-                vlist[(size_t)vfirst + i] = v;
+                vlist[(size_t)first + i] = v;
             }
-            desc[4 * (size_t)c + 0] = (int)(off / 16);
-            desc[4 * (size_t)c + 1] = (int)bytes;
-            desc[4 * (size_t)c + 2] = cnt;
-            desc[4 * (size_t)c + 3] = vfirst;
-            vfirst += cnt;
-            rec_max = std::max(rec_max, (int)bytes);
         }
         if (blob.size() / 16 >= ((size_t)1 << 31)) continue;
         TFPS_TRY(upload(L.blob, blob, st));
@@ -1092,27 +1103,33 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
         PassArgs a = make_args(g, fwd, P, ldp, part, lev, cp_here);
         g->last_kernel = use_window ? "pass_window_kernel" : (sliced ? "pass_sliced_kernel" : (g->npass > 0 ? "pass_tile_kernel" : "pass_level_kernel"));
         // lean windowed pass: 32-bit levels, whole window resident, host-packed records
-        if (sliced && g->lean[0].ok && g->lean[1].ok && level_bytes == 4 && ((uintptr_t)part & 15u) == 0 &&
+        if (sliced && g->lean[0].ok && g->lean[1].ok && level_bytes == 4 && ((uintptr_t)part & 15u) == 0 && ldp < (1LL << 28) &&
             env_int("TFPS_LEAN", 1) != 0) {
             const LeanPlan& lp = g->lean[fwd ? 0 : 1].plan;
+            // candidates per block (slice): the widest that keeps the window in shared memory and leaves enough
+            // blocks to occupy the machine; TFPS_SLICED_CPT = c forces 32*c
             const int forced = env_int("TFPS_SLICED_CPT", 0);
-            const long long want_slices = std::min<long long>((3LL * g->sm_count) / 4, (P + 31) / 32);
+            const long long want_slices = std::min<long long>((3LL * g->sm_count) / 4, (P + 15) / 16);
             int d_want = env_int("TFPS_LEAN_DEPTH", 0);
             if (d_want < 1 || d_want > LEAN_DEPTH_MAX) d_want = 3;
+            const int forced_warps = env_int("TFPS_SLICED_WARPS", 0);
             int l_cpt = 0, l_depth = 0, l_warps = 0;
             size_t l_smem = 0;
             LeanArgs la;
-            for (int c = 4; c >= 1 && !l_cpt; c >>= 1) {
-                if (forced == 1 || forced == 2 || forced == 4) { if (c != forced) continue; }
-                else if ((P + 32 * c - 1) / (32 * c) < want_slices && c > 1) continue;
-                int w = warps;   // every warp consumes; each thread fetches at most two id-row pieces per chunk
-                while (w < 32 && lp.max_v * 2 * c > 2 * w * 32) w <<= 1;
-                if (lp.max_v * 2 * c > 2 * w * 32) continue;
+            for (int slice = 128; slice >= 16 && !l_cpt; slice >>= 1) {
+                if (forced == 1 || forced == 2 || forced == 4) { if (slice != 32 * forced) continue; }
+                else if ((P + slice - 1) / slice < want_slices && slice > 16) continue;
+                const int vpw = 128 / slice, pr = slice / 16;
+                int w = 1;   // one round of the vertex groups covers the widest chunk when 32 warps allow it
+                while (w < 32 && w * vpw < lp.max_v) w <<= 1;
+                if (forced_warps >= 1 && forced_warps <= 32) w = forced_warps;
+                while (w < 32 && lp.max_v * pr > 2 * w * 32) w <<= 1;   // a thread fetches at most two id-row pieces per chunk
+                if (lp.max_v * pr > 2 * w * 32) continue;
                 for (int d = d_want; d >= 1; --d) {
                     unsigned slot_stride = 0, stage_bytes = 0;
-                    const size_t need = lean_smem_bytes(lp, c, w, d, &slot_stride, &stage_bytes);
+                    const size_t need = lean_smem_bytes(lp, slice, w, d, &slot_stride, &stage_bytes);
                     if (need + 512 <= (size_t)g->smem_optin) {
-                        l_cpt = c; l_depth = d; l_warps = w; l_smem = need;
+                        l_cpt = slice; l_depth = d; l_warps = w; l_smem = need;
                         la.slot_stride = slot_stride;
                         la.stage_bytes = stage_bytes;
                         break;

@@ -143,7 +143,8 @@ struct WindowPlan {
 
 // Lean windowed pass (32-bit levels, k <= LEAN_K_MAX, whole window resident).  The host packs, per direction
 // and in processing order, one record per chunk:
-//   header  int4 {vertices, byte offset of the edge area, 0, 0}
+//   header  LEAN_HDR_BYTES: int4 {vertices, byte offset of the edge area, 0, 0}, then the descriptors
+//           {offset/16, bytes, vertices, first index into vlist} of the chunks 1..LEAN_DEPTH_MAX places later (zero past the end)
 //   vertex  [vstride bytes each]  {v | flag << 31, window slot, first edge byte, end edge byte, rt[KP]}
 //           flag: sink (forward) / source (backward): the vertex enters the CP maximum;
 //           rt[d] = ceil(c_v*S / s_d); edge bytes are relative to the edge area
@@ -156,6 +157,7 @@ constexpr int LEAN_K_MAX = 8;
 constexpr int LEAN_CLS_MAX = 30;     // 4 * (classes + 1) must stay below 0x80 (sign-replicating byte permute)
 constexpr int LEAN_CHUNK_V = 128;
 constexpr int LEAN_DEPTH_MAX = 4;
+constexpr int LEAN_HDR_BYTES = 16 + 16 * LEAN_DEPTH_MAX;
 
 struct LeanPlan {
     const unsigned char* blob;   // chunk records, 16-byte aligned each
@@ -177,12 +179,12 @@ struct LeanArgs {
     long long P, ldp;
     LeanPlan plan;
     int depth;                   // chunks in flight (stage slots)
-    unsigned slot_stride;        // bytes of a stage slot: rec_max + max_v * slice
+    unsigned slot_stride;        // bytes of a stage slot: rec_max + max_v * (candidates per block)
     unsigned stage_bytes;        // bytes reserved for all stage slots (also the CP reduction buffer)
 };
 
-size_t lean_smem_bytes(const LeanPlan& plan, int cpt, int warps, int depth, unsigned* slot_stride, unsigned* stage_bytes);
-cudaError_t launch_pass_lean(const LeanArgs& a, bool fwd, int cpt, int warps, size_t smem, cudaStream_t st);
+size_t lean_smem_bytes(const LeanPlan& plan, int slice, int warps, int depth, unsigned* slot_stride, unsigned* stage_bytes);
+cudaError_t launch_pass_lean(const LeanArgs& a, bool fwd, int slice, int warps, size_t smem, cudaStream_t st);
 
 // every kernel launch of the library goes through the wrappers below and is counted here
 void count_launches(long long n);

@@ -78,7 +78,8 @@ __device__ __forceinline__ void sts128(unsigned a, unsigned x, unsigned y, unsig
 __device__ __forceinline__ void sts_u16(unsigned a, unsigned v) { asm volatile("st.shared.u16 [%0], %1;" ::"r"(a), "h"((unsigned short)v) : "memory"); }
 __device__ __forceinline__ void sts_u8(unsigned a, unsigned v) { asm volatile("st.shared.u8 [%0], %1;" ::"r"(a), "r"(v) : "memory"); }
 
-// byte permute: result byte i = byte (sel nibble i & 7) of {b, a}; nibble bit 3 replicates that byte's sign bit instead
+// byte permute: result byte i = byte (sel nibble i & 7) of {b, a}; nibble bit 3 replicates that byte's sign bit
+// instead.  (Inline PTX on purpose: the sign-replicating selector form is part of prmt, not of __byte_perm.)
 __device__ __forceinline__ unsigned prmt(unsigned a, unsigned b, unsigned sel)
 {
     unsigned d;
@@ -121,16 +122,35 @@ __device__ __forceinline__ void cp_async_arrive_on(unsigned bar)
 constexpr int WAIT_LIMIT = 1 << 20;
 __device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity)
 {
+#pragma unroll 1
     for (int i = 0; i < WAIT_LIMIT; ++i)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
 
-__device__ __forceinline__ void stg_cs_v2(long long* p, long long x, long long y)
+// streaming stores of non-negative 32-bit levels widened to int64 (the high words are zero)
+template <int OFF> __device__ __forceinline__ void stg_cs_v2(long long* p, int x, int y)
 {
-    asm volatile("st.global.cs.v2.u64 [%0], {%1, %2};" ::"l"(p), "l"(x), "l"(y) : "memory");
+    asm volatile("{\n\t.reg .b64 a, b;\n\tcvt.u64.u32 a, %1;\n\tcvt.u64.u32 b, %2;\n\tst.global.cs.v2.u64 [%0+%3], {a, b};\n\t}"
+                 ::"l"(p), "r"(x), "r"(y), "n"(OFF) : "memory");
 }
-__device__ __forceinline__ void stg_cs(long long* p, long long x) { asm volatile("st.global.cs.u64 [%0], %1;" ::"l"(p), "l"(x) : "memory"); }
+__device__ __forceinline__ void stg_cs(long long* p, int x)
+{
+    asm volatile("{\n\t.reg .b64 a;\n\tcvt.u64.u32 a, %1;\n\tst.global.cs.u64 [%0], a;\n\t}" ::"l"(p), "r"(x) : "memory");
+}
+// p + (a * b) with a 32 x 32 -> 64 bit product
+__device__ __forceinline__ const uint8_t* ptr_mad(const uint8_t* p, unsigned a, unsigned b)
+{
+    unsigned long long r;
+    asm volatile("mad.wide.u32 %0, %1, %2, %3;" : "=l"(r) : "r"(a), "r"(b), "l"((unsigned long long)p));
+    return reinterpret_cast<const uint8_t*>(r);
+}
+__device__ __forceinline__ long long* ptr_mad(long long* p, unsigned a, unsigned b)
+{
+    unsigned long long r;
+    asm("mad.wide.u32 %0, %1, %2, %3;" : "=l"(r) : "r"(a), "r"(b), "l"((unsigned long long)p));
+    return reinterpret_cast<long long*>(r);
+}
 
 template <int CPT> __device__ __forceinline__ unsigned ld_ids(unsigned a)
 {
@@ -157,25 +177,33 @@ template <int CPT> __device__ __forceinline__ void st_lev(unsigned a, const int 
     else sts128(a, (unsigned)l[0], (unsigned)l[1], (unsigned)l[2], (unsigned)l[3]);
 }
 
-template <int CPT, bool FWD>
-__global__ void __launch_bounds__(1024, 1) pass_lean_kernel(const LeanArgs a)
+// CPT candidates per lane, VPW vertices per warp: a vertex is handled by 32/VPW lanes, so a block owns
+// SLICE = 32/VPW*CPT candidates.  Several vertices per warp cut the instructions per vertex-candidate (the
+// bookkeeping of a vertex and of an edge is paid once per warp instruction, whatever the number of vertices its
+// lanes serve); the lanes of different vertices simply diverge when the degrees differ, and the host deals
+// vertices of similar degree to the same warp.  MAXT = largest block size of the instantiation (512 threads may
+// use 128 registers each, 1024 threads 64).
+template <int CPT, int VPW, bool FWD, int MAXT>
+__global__ void __launch_bounds__(MAXT, 1) pass_lean_kernel(const __grid_constant__ LeanArgs a)
 {
     extern __shared__ __align__(16) unsigned char dsm[];   // [stage slots][window]
     __shared__ __align__(16) unsigned long long s_rows[LEAN_K_MAX];
     __shared__ __align__(8) unsigned long long s_bar[LEAN_DEPTH_MAX];
+    __shared__ int s_cp[128];   // CP maxima of the block's candidates
     __shared__ int s_abort;
-    constexpr int SLICE = 32 * CPT;        // candidates of the block = bytes of an id row
+    constexpr int LPV = 32 / VPW;          // lanes per vertex
+    constexpr int SLICE = LPV * CPT;       // candidates of the block = bytes of an id row
     constexpr unsigned LEVB = SLICE * 4;   // a window row: SLICE levels, then SLICE id bytes
     constexpr unsigned ROWB = SLICE * 5;
-    constexpr int PR = 2 * CPT;            // 16-byte pieces of an id row
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nthreads = blockDim.x, nwarps = nthreads >> 5;
+    constexpr int PR = SLICE / 16;         // 16-byte pieces of an id row
+    const int tid = threadIdx.x, nthreads = blockDim.x;
     if (*a.status != 0) return;
     const int D = a.depth;
-    const int nc = a.plan.num_chunks;
     const unsigned stage0 = smem_u32(dsm), win0 = stage0 + a.stage_bytes;
     const unsigned rows_s = smem_u32(s_rows), bar0 = smem_u32(s_bar);
     volatile int* abort_p = &s_abort;
     if (tid < LEAN_K_MAX) s_rows[tid] = a.plan.rows[tid];
+    for (int t = tid; t < 128; t += nthreads) s_cp[t] = 0;
     if (tid == 0) {
         // a stage completes on the record's bulk copy (one arrival carrying the byte count) plus one arrival
         // per thread once that thread's id-row pieces have landed
@@ -185,75 +213,88 @@ __global__ void __launch_bounds__(1024, 1) pass_lean_kernel(const LeanArgs a)
     }
     __syncthreads();
 
+    const int ll = (tid & 31) % LPV;                       // lane within the vertex
+    const int group = (tid >> 5) * VPW + (tid & 31) / LPV; // vertex group of this lane
+    const int ngroups = (nthreads >> 5) * VPW;
     const long long slice0 = (long long)blockIdx.x * SLICE;
-    const long long j0 = slice0 + (long long)lane * CPT;
-    const long long rem = a.P - j0;
-    const int nvalid = rem >= CPT ? CPT : (rem > 0 ? (int)rem : 0);
-    const long long ldp = a.ldp;
-    const unsigned slice_bytes = (unsigned)((ldp - slice0) < SLICE ? (ldp - slice0) : SLICE);   // multiple of 16
-    const unsigned win_lev_lane = win0 + (unsigned)(lane * CPT * 4);
-    const unsigned id_delta = LEVB - (unsigned)(3 * lane * CPT);   // id bytes of a lane relative to its levels
-    const int vstride = a.plan.vstride, estride = a.plan.estride;
+    const unsigned win_lev_lane = win0 + (unsigned)(ll * CPT * 4);
+    const unsigned id_delta = LEVB - (unsigned)(3 * ll * CPT);   // id bytes of a lane relative to its levels
     const unsigned rec_max = (unsigned)a.plan.rec_max;
-    const int4* __restrict__ desc = a.plan.desc;
-    const int* __restrict__ vlist = a.plan.vlist;
-    const unsigned char* __restrict__ blob = a.plan.blob;
-    const uint8_t* __restrict__ part0 = a.part + slice0;
-    long long* __restrict__ out_lane = a.lev + j0;
-    const unsigned ldp8 = (unsigned)(ldp * 8);
-    int cpmax[CPT];
-#pragma unroll
-    for (int c = 0; c < CPT; ++c) cpmax[c] = 0;
+    const bool two_pieces = a.plan.max_v * PR > nthreads;   // a thread fetches one id-row piece per chunk, or two
+    const long long j0 = slice0 + (long long)(ll * CPT);
+    const bool full = j0 + CPT <= a.P;        // all CPT candidates of this lane exist
+    long long* const out_lane = a.lev + j0;
+    const unsigned ldp8 = (unsigned)(a.ldp * 8);   // the host keeps ldp below 2^28
+    unsigned k88;   // kept in a register (opaque to the compiler), so the selectors below can be immediates
+    asm volatile("mov.u32 %0, 0x88888888;" : "=r"(k88));
 
-    // copies of one chunk into a stage slot: d = its descriptor, v[s] = vertex of the id row this thread fetches
-    auto issue = [&](const int4& d, const int (&v)[2], unsigned slotb, unsigned bar) {
+    // copies of one chunk into a stage slot: d = its descriptor {offset/16, bytes, vertices, first index into
+    // vlist}, v0/v1 = vertices of the id rows this thread fetches
+    auto issue = [&](const uint4& d, unsigned v0, unsigned v1, unsigned slotb, unsigned bar) {
         if (d.y == 0) return;   // past the last chunk
+        const long long ldp = a.ldp;
+        const unsigned slice_bytes = (unsigned)((ldp - slice0) < SLICE ? (ldp - slice0) : SLICE);   // multiple of 16
+        const uint8_t* part0 = a.part + slice0;
+        const unsigned ldp32 = (unsigned)ldp;
         if (tid == 0) {
-            mbar_expect_tx(bar, (unsigned)d.y);
-            bulk_g2s(slotb, blob + 16ll * (unsigned)d.x, (unsigned)d.y, bar);
+            mbar_expect_tx(bar, d.y);
+            bulk_g2s(slotb, a.plan.blob + 16ll * d.x, d.y, bar);
         }
-#pragma unroll
-        for (int s = 0; s < 2; ++s) {
-            const int p = tid + s * nthreads;
+        {
+            const int r = tid / PR, q = tid % PR;
+            if (r < (int)d.z && (unsigned)(16 * q) < slice_bytes)
+                cp_async16(slotb + rec_max + (unsigned)(r * SLICE + 16 * q), ptr_mad(part0 + 16 * q, v0, ldp32));
+        }
+        if (two_pieces) {
+            const int p = tid + nthreads;
             const int r = p / PR, q = p % PR;
-            if (r < d.z && (unsigned)(16 * q) < slice_bytes)
-                cp_async16(slotb + rec_max + (unsigned)(r * SLICE + 16 * q), part0 + (long long)v[s] * ldp + 16 * q);
+            if (r < (int)d.z && (unsigned)(16 * q) < slice_bytes)
+                cp_async16(slotb + rec_max + (unsigned)(r * SLICE + 16 * q), ptr_mad(part0 + 16 * q, v1, ldp32));
         }
         cp_async_arrive_on(bar);
     };
-    auto fetch_v = [&](const int4& d, int (&v)[2]) {
-#pragma unroll
-        for (int s = 0; s < 2; ++s) {
-            const int r = (tid + s * nthreads) / PR;
-            v[s] = r < d.z ? __ldg(vlist + d.w + r) : 0;
+    auto fetch_v = [&](const uint4& d, unsigned& v0, unsigned& v1) {
+        const int r0 = tid / PR;
+        v0 = r0 < (int)d.z ? (unsigned)__ldg(a.plan.vlist + d.w + r0) : 0u;
+        v1 = 0;
+        if (two_pieces) {
+            const int r1 = (tid + nthreads) / PR;
+            if (r1 < (int)d.z) v1 = (unsigned)__ldg(a.plan.vlist + d.w + r1);
         }
     };
 
     for (int j = 0; j < D; ++j) {   // chunks 0..D-1 (descriptors past the end are zero)
-        const int4 d = __ldg(desc + j);
-        int v[2];
-        fetch_v(d, v);
-        issue(d, v, stage0 + (unsigned)j * a.slot_stride, bar0 + 8u * j);
+        const int4 di = __ldg(a.plan.desc + j);
+        const uint4 d = make_uint4((unsigned)di.x, (unsigned)di.y, (unsigned)di.z, (unsigned)di.w);
+        unsigned v0, v1;
+        fetch_v(d, v0, v1);
+        issue(d, v0, v1, stage0 + (unsigned)j * a.slot_stride, bar0 + 8u * j);
     }
-    int4 dC = __ldg(desc + D);   // the chunk issued after chunk 0 is done
+    const int nc = a.plan.num_chunks;
     int slot = 0;
     unsigned par = 0;
     for (int ci = 0; ci < nc; ++ci) {
-        // prefetch for the issue at the end of this iteration (chunk ci+D) and of the next one
-        const int4 dN = __ldg(desc + ci + D + 1);
-        int vA[2];
-        fetch_v(dC, vA);
         const unsigned slotb = stage0 + (unsigned)slot * a.slot_stride;
         const unsigned bar = bar0 + 8u * slot;
+        unsigned vA0 = 0, vA1 = 0;
         if (!mbar_wait(bar, par)) {
             atomicCAS(a.status, 0, (int)TFPS_ERR_TIMEOUT);
             *abort_p = 1;
         } else {
+            // the record of chunk ci names chunk ci+D: request the vertex ids of its id rows now, use them after the barrier
+            fetch_v(lds128(slotb + 16u * (unsigned)D), vA0, vA1);
             const uint4 hdr = lds128(slotb);
             const int cnt = (int)hdr.x;
-            const unsigned vbase = slotb + 16u, ebase = slotb + hdr.y;
-            const unsigned idrow = slotb + rec_max + (unsigned)(lane * CPT);
-            for (int i = warp; i < cnt; i += nwarps) {
+            const unsigned vbase = slotb + LEAN_HDR_BYTES, ebase = slotb + hdr.y;
+            const unsigned idrow = slotb + rec_max + (unsigned)(ll * CPT);
+            const int vstride = a.plan.vstride;
+            const unsigned estride = (unsigned)a.plan.estride;
+            // rounds alternate direction: group g takes entries g, 2G-1-g, 2G+g, ... of the degree-sorted list
+            for (int base = 0; base < cnt; base += 2 * ngroups) {
+#pragma unroll 1
+              for (int half = 0; half < 2; ++half) {
+                const int i = half == 0 ? base + group : base + 2 * ngroups - 1 - group;
+                if (i >= cnt) continue;
                 const unsigned vr = vbase + (unsigned)(i * vstride);
                 const uint4 rec = lds128(vr);   // {v | flag, window slot, first edge byte, end edge byte}
                 const unsigned ids = ld_ids<CPT>(idrow + (unsigned)(i * SLICE));
@@ -269,118 +310,122 @@ __global__ void __launch_bounds__(1024, 1) pass_lean_kernel(const LeanArgs a)
                     rt[c] = (int)lds32_off16(vr + (pv8 >> 1));
                     best[c] = 0;
                 }
-                for (unsigned ea = ebase + rec.z, ee = ebase + rec.w; ea < ee; ea += (unsigned)estride) {
-                    const unsigned ns = lds32(ea);
-                    const unsigned la = win_lev_lane + ns * ROWB;
-                    int lu[CPT];
-                    ld_lev<CPT>(la, lu);
-                    const unsigned pu = ld_ids<CPT>(la + id_delta);   // bytes 0x80 | device id
+                unsigned ea = ebase + rec.z;
+                const unsigned ee = ebase + rec.w;
+                if (ea < ee) {
+                    unsigned ns = lds32(ea);
+                    bool more;
+                    do {
+                        const unsigned la = win_lev_lane + ns * ROWB;
+                        const unsigned en = ea + estride;
+                        more = en < ee;
+                        if (more) ns = lds32(en);   // next edge's window slot, ahead of this edge's dependent loads
+                        int lu[CPT];
+                        ld_lev<CPT>(la, lu);
+                        const unsigned pu = ld_ids<CPT>(la + id_delta);   // bytes 0x80 | device id
 #pragma unroll
-                    for (int c = 0; c < CPT; ++c) {
-                        // selector 0x888(8|pu): byte 0 <- rows[pv][pu], bytes 1..3 <- 0 (sign of a byte below 0x80)
-                        const unsigned sel = prmt(pu, 0x88888888u, 0x4440u + (unsigned)c);
-                        const unsigned off = prmt(rlo[c], rhi[c], sel);
-                        const int w = (int)lds32_off4(ea + off);
-                        best[c] = __viaddmax_s32(lu[c], w, best[c]);
-                    }
+                        for (int c = 0; c < CPT; ++c) {
+                            // selector 0x888(8|pu): byte 0 <- rows[pv][pu], bytes 1..3 <- 0 (sign of a byte below 0x80)
+                            const unsigned sel = prmt(pu, k88, 0x4440u + (unsigned)c);
+                            const unsigned off = prmt(rlo[c], rhi[c], sel);
+                            const int w = (int)lds32_off4(ea + off);
+                            best[c] = __viaddmax_s32(lu[c], w, best[c]);
+                        }
+                        ea = en;
+                    } while (more);
                 }
                 int fin[CPT];
 #pragma unroll
                 for (int c = 0; c < CPT; ++c) fin[c] = best[c] + rt[c];
-                if ((int)rec.x < 0) {
+                if ((int)rec.x < 0) {   // sink (forward) / source (backward): enters the CP maximum; rare
 #pragma unroll
-                    for (int c = 0; c < CPT; ++c) cpmax[c] = max(cpmax[c], fin[c]);
+                    for (int c = 0; c < CPT; ++c) atomicMax(&s_cp[ll * CPT + c], fin[c]);
                 }
                 // results: global memory (start time forward, bottom level backward) and the window
-                long long* gout = out_lane + (unsigned long long)(rec.x & 0x7fffffffu) * ldp;
-                if (nvalid == CPT) {
-                    if constexpr (CPT == 1) stg_cs(gout, (long long)(FWD ? best[0] : fin[0]));
-                    else {
-#pragma unroll
-                        for (int c = 0; c < CPT; c += 2)
-                            stg_cs_v2(gout + c, (long long)(FWD ? best[c] : fin[c]), (long long)(FWD ? best[c + 1] : fin[c + 1]));
-                    }
+                long long* gout = ptr_mad(out_lane, rec.x & 0x7fffffffu, ldp8);
+                if (full) {
+                    if constexpr (CPT == 1) stg_cs(gout, FWD ? best[0] : fin[0]);
+                    if constexpr (CPT >= 2) stg_cs_v2<0>(gout, FWD ? best[0] : fin[0], FWD ? best[1] : fin[1]);
+                    if constexpr (CPT == 4) stg_cs_v2<16>(gout, FWD ? best[2] : fin[2], FWD ? best[3] : fin[3]);
                 } else {
 #pragma unroll
                     for (int c = 0; c < CPT; ++c)
-                        if (c < nvalid) stg_cs(gout + c, (long long)(FWD ? best[c] : fin[c]));
+                        if (j0 + c < a.P) stg_cs(gout + c, FWD ? best[c] : fin[c]);
                 }
                 const unsigned lo = win_lev_lane + rec.y * ROWB;
                 st_lev<CPT>(lo, fin);
                 st_ids<CPT>(lo + id_delta, (ids & 0x07070707u) | 0x80808080u);
+              }
             }
         }
+        const uint4 dA = lds128(slotb + 16u * (unsigned)D);   // descriptor of chunk ci+D, before the slot is overwritten
         __syncthreads();   // chunk ci is in the window; its stage slot is free again
         if (*abort_p) break;
-        issue(dC, vA, slotb, bar);
-        dC = dN;
+        issue(dA, vA0, vA1, slotb, bar);
         if (++slot == D) { slot = 0; par ^= 1u; }
     }
     __syncthreads();
     if (*abort_p) {
         // copies already requested may still be landing in this block's shared memory: give them a bounded
         // time before the block (and its shared memory) goes away
+#pragma unroll 1
         for (int i = 0; i < 1000; ++i) __nanosleep(1000);
         return;
     }
-    if (a.cp != nullptr) {
-        // maxima of the warps through the (now idle) stage area
-        const unsigned red = stage0 + (unsigned)((warp * 32 + lane) * CPT * 4);
-#pragma unroll
-        for (int c = 0; c < CPT; ++c) sts32(red + 4u * c, (unsigned)cpmax[c]);
-        __syncthreads();
-        if (warp == 0) {
-#pragma unroll
-            for (int c = 0; c < CPT; ++c) {
-                int m = cpmax[c];
-                for (int w = 1; w < nwarps; ++w) m = max(m, (int)lds32(stage0 + (unsigned)(((w * 32 + lane) * CPT + c) * 4)));
-                if (c < nvalid) a.cp[j0 + c] = (long long)m;
-            }
-        }
-    }
-    (void)ldp8;
+    if (a.cp != nullptr)
+        for (int t = tid; t < SLICE; t += nthreads)
+            if (slice0 + t < a.P) a.cp[slice0 + t] = (long long)s_cp[t];
 }
 
-template <int CPT>
-cudaError_t lean_impl(const LeanArgs& a, bool fwd, int warps, size_t smem, cudaStream_t st)
+template <int CPT, int VPW, int MAXT>
+cudaError_t lean_impl2(const LeanArgs& a, bool fwd, int warps, size_t smem, cudaStream_t st)
 {
-    const unsigned grid = (unsigned)((a.P + 32 * CPT - 1) / (32 * CPT));
+    constexpr int SLICE = 32 / VPW * CPT;
+    const unsigned grid = (unsigned)((a.P + SLICE - 1) / SLICE);
     cudaError_t e;
     if (fwd) {
-        e = cudaFuncSetAttribute(pass_lean_kernel<CPT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        e = cudaFuncSetAttribute(pass_lean_kernel<CPT, VPW, true, MAXT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        pass_lean_kernel<CPT, true><<<grid, warps * 32, smem, st>>>(a);
+        pass_lean_kernel<CPT, VPW, true, MAXT><<<grid, warps * 32, smem, st>>>(a);
     } else {
-        e = cudaFuncSetAttribute(pass_lean_kernel<CPT, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        e = cudaFuncSetAttribute(pass_lean_kernel<CPT, VPW, false, MAXT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        pass_lean_kernel<CPT, false><<<grid, warps * 32, smem, st>>>(a);
+        pass_lean_kernel<CPT, VPW, false, MAXT><<<grid, warps * 32, smem, st>>>(a);
     }
     count_launches(1);
     return cudaGetLastError();
+}
+
+template <int CPT, int VPW>
+cudaError_t lean_impl(const LeanArgs& a, bool fwd, int warps, size_t smem, cudaStream_t st)
+{
+    if (warps <= 16) return lean_impl2<CPT, VPW, 512>(a, fwd, warps, smem, st);
+    return lean_impl2<CPT, VPW, 1024>(a, fwd, warps, smem, st);
 }
 
 inline size_t up16(size_t x) { return (x + 15) & ~(size_t)15; }
 
 }  // namespace
 
-size_t lean_smem_bytes(const LeanPlan& plan, int cpt, int warps, int depth, unsigned* slot_stride, unsigned* stage_bytes)
+size_t lean_smem_bytes(const LeanPlan& plan, int slice, int warps, int depth, unsigned* slot_stride, unsigned* stage_bytes)
 {
-    const size_t slice = 32 * (size_t)cpt;
-    const size_t slot = (size_t)plan.rec_max + up16((size_t)plan.max_v * slice);
+    const size_t slot = (size_t)plan.rec_max + up16((size_t)plan.max_v * (size_t)slice);
     size_t stage = (size_t)depth * slot;
-    const size_t red = (size_t)warps * slice * 4;   // CP reduction buffer after the last chunk
+    const size_t red = (size_t)warps * 128 * 4;   // CP reduction buffer after the last chunk (at most 4 candidates per lane)
     if (stage < red) stage = up16(red);
     if (slot_stride) *slot_stride = (unsigned)slot;
     if (stage_bytes) *stage_bytes = (unsigned)stage;
-    return stage + (size_t)plan.R * slice * 5;
+    return stage + (size_t)plan.R * (size_t)slice * 5;
 }
 
-cudaError_t launch_pass_lean(const LeanArgs& a, bool fwd, int cpt, int warps, size_t smem, cudaStream_t st)
+// slice = candidates per block: 128, 64, 32 or 16 (4 candidates per lane, 1, 2, 4 or 8 vertices per warp)
+cudaError_t launch_pass_lean(const LeanArgs& a, bool fwd, int slice, int warps, size_t smem, cudaStream_t st)
 {
     if (a.plan.num_chunks <= 0) return cudaSuccess;
-    if (cpt == 4) return lean_impl<4>(a, fwd, warps, smem, st);
-    if (cpt == 2) return lean_impl<2>(a, fwd, warps, smem, st);
-    return lean_impl<1>(a, fwd, warps, smem, st);
+    if (slice == 128) return lean_impl<4, 1>(a, fwd, warps, smem, st);
+    if (slice == 64) return lean_impl<4, 2>(a, fwd, warps, smem, st);
+    if (slice == 32) return lean_impl<4, 4>(a, fwd, warps, smem, st);
+    return lean_impl<4, 8>(a, fwd, warps, smem, st);
 }
 
 }  // namespace tfps
