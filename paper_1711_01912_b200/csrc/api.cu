@@ -118,6 +118,8 @@ struct tfps_graph {
     int k = 0;
     long long S = 0;
     DBuf rt_div, w_div, cap, xvert, xw_f, xnbr_f, xw_b;
+    DBuf rtv;          // [n][rt_kp] runtime of every vertex on every device (loads kernel)
+    int rt_kp = 0;     // table width: power of two >= k, or 0 when k is too large for the table
     DBuf pair_f, pair_b, cls_div, sel_f, sel_b;
     // windowed pass: neighbour positions, comb tables, precomputed edge values
     DBuf pos_of, npos_f, npos_b, cls2_f, cls2_b, comb_f, comb_b, V_f, V_b, V32_f, V32_b;
@@ -842,6 +844,15 @@ int tfps_devices_set(tfps_graph* g, int k, const int32_t* s, const int64_t* C, c
                                    g->f_t.as<long long>(), g->b_nbr.as<int>(), g->b_t.as<long long>(),
                                    g->xvert.as<unsigned long long>(), g->xw_f.as<unsigned long long>(),
                                    g->xnbr_f.as<unsigned long long>(), g->xw_b.as<unsigned long long>(), st));
+    g->rt_kp = 0;
+    if (n > 0 && k <= 32) {
+        int kp = 2;   // at least two entries: rows of the table start on 16-byte boundaries
+        while (kp < k) kp <<= 1;
+        CUDA_TRY(g->rtv.reserve(sizeof(long long) * (size_t)n * kp));
+        CUDA_TRY(launch_rt_rows(n, k, kp, g->pos_of.as<int>(), g->xvert.as<unsigned long long>(), g->rt_div.as<DivConst>(),
+                                g->rtv.as<long long>(), st));
+        g->rt_kp = kp;
+    }
     g->fits32 = false;
     for (auto& L : g->lean) L.ok = false;
     if ((g->ncomb > 0 || k <= LEAN_K_MAX) && n > 0) {
@@ -1009,8 +1020,12 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
     if (load || ml) {
         if (load) CUDA_TRY(cudaMemset2DAsync(load, sizeof(long long) * (size_t)ldp, 0, sizeof(long long) * (size_t)P, (size_t)k, st));
         if (ml) CUDA_TRY(cudaMemset2DAsync(ml, sizeof(long long) * (size_t)ldp, 0, sizeof(long long) * (size_t)P, (size_t)k, st));
-        CUDA_TRY(launch_loads(n, P, ldp, part, g->order.as<int>(), g->xvert.as<unsigned long long>(), g->mem.as<long long>(),
-                              tab, (long long*)load, ml, status, validate, g->sm_count, st));
+        if (g->rt_kp > 0 && ((uintptr_t)part & 3u) == 0 && env_int("TFPS_LOADS2", 1) != 0)
+            CUDA_TRY(launch_loads2(n, P, ldp, part, g->rtv.as<long long>(), g->mem.as<long long>(), k, g->rt_kp,
+                                   (long long*)load, ml, status, validate, g->sm_count, g->smem_optin, st));
+        else
+            CUDA_TRY(launch_loads(n, P, ldp, part, g->order.as<int>(), g->xvert.as<unsigned long long>(), g->mem.as<long long>(),
+                                  tab, (long long*)load, ml, status, validate, g->sm_count, st));
         if (viol) CUDA_TRY(launch_viol(P, ldp, k, ml, tab.cap, (unsigned long long*)viol, status, st));
     } else if (validate) {
         CUDA_TRY(launch_validate(n, P, ldp, part, k, status, g->sm_count, st));

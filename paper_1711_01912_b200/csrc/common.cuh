@@ -224,6 +224,11 @@ cudaError_t launch_cp_reduce(const PassArgs& a, bool from_tlevel, const int* lis
 cudaError_t launch_loads(int n, long long P, long long ldp, const uint8_t* part, const int* vert,
                          const unsigned long long* xvert, const long long* mem, DevTables tab, long long* load,
                          long long* memload, int* status, bool validate, int sm_count, cudaStream_t st);
+cudaError_t launch_rt_rows(int n, int k, int kp, const int* pos_of, const unsigned long long* xvert, const DivConst* rt_div,
+                           long long* rtv, cudaStream_t st);
+cudaError_t launch_loads2(int n, long long P, long long ldp, const uint8_t* part, const long long* rtv, const long long* mem,
+                          int k, int kp, long long* load, long long* memload, int* status, bool validate, int sm_count,
+                          int smem_optin, cudaStream_t st);
 cudaError_t launch_validate(long long n, long long P, long long ldp, const uint8_t* part, int k, int* status,
                             int sm_count, cudaStream_t st);
 cudaError_t launch_viol(long long P, long long ldp, int k, const long long* memload, const long long* cap,
