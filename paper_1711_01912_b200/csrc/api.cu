@@ -1128,11 +1128,13 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
             int d_want = env_int("TFPS_LEAN_DEPTH", 0);
             if (d_want < 1 || d_want > LEAN_DEPTH_MAX) d_want = 3;
             const int forced_warps = env_int("TFPS_SLICED_WARPS", 0);
+            const int forced_slice = env_int("TFPS_LEAN_SLICE", 0);
             int l_cpt = 0, l_depth = 0, l_warps = 0;
             size_t l_smem = 0;
             LeanArgs la;
             for (int slice = 128; slice >= 16 && !l_cpt; slice >>= 1) {
-                if (forced == 1 || forced == 2 || forced == 4) { if (slice != 32 * forced) continue; }
+                if (forced_slice == 16 || forced_slice == 32 || forced_slice == 64 || forced_slice == 128) { if (slice != forced_slice) continue; }
+                else if (forced == 1 || forced == 2 || forced == 4) { if (slice != 32 * forced) continue; }
                 else if ((P + slice - 1) / slice < want_slices && slice > 16) continue;
                 const int vpw = 128 / slice, pr = slice / 16;
                 int w = 1;   // one round of the vertex groups covers the widest chunk when 32 warps allow it

@@ -382,6 +382,7 @@ def test_sliced_kernel_shapes(cpt, table, monkeypatch):
     monkeypatch.setenv("TFPS_SLICED_TABLE", str(table))
     monkeypatch.setenv("TFPS_SLICED_WARPS", "4")
     monkeypatch.setenv("TFPS_WINDOW", "0")
+    monkeypatch.setenv("TFPS_LEAN", "0")
     for g, dev, part in _shape_cases(cpt * 2 + table):
         run_and_compare(g, dev, part, 2, pad_fill=255)
 
@@ -419,6 +420,7 @@ def test_windowed_kernel_shapes(cpt, win_r, level32, monkeypatch):
     monkeypatch.setenv("TFPS_SLICED_CPT", str(cpt))
     monkeypatch.setenv("TFPS_SLICED_WARPS", "8")
     monkeypatch.setenv("TFPS_WINDOW", "1")
+    monkeypatch.setenv("TFPS_LEAN", "0")
     monkeypatch.setenv("TFPS_WINDOW_R", str(win_r))
     monkeypatch.setenv("TFPS_LEVEL32", str(level32))  # 32-bit levels inside the block when every path fits int32
     for g, dev, part in _shape_cases(cpt * 2 + 1):
@@ -430,6 +432,80 @@ def test_windowed_kernel_shapes(cpt, win_r, level32, monkeypatch):
     keep = g.dst < 16 * 300  # first 300 layers of the deep narrow graph
     g2 = I.Graph(n=16 * 300, src=g.src[keep], dst=g.dst[keep], t=g.t[keep], c=g.c[:16 * 300], mem=None, layers=300)
     run_and_compare(g2, w.devices, w.part_rows(0, 16 * 300)[:, :97], 2, pad_fill=255)
+
+
+def _small_costs(g):
+    """Same graph with edge sizes below 50,000, so that every path length fits 32 bits."""
+    return I.Graph(n=g.n, src=g.src, dst=g.dst, t=(g.t % 50000).astype(g.t.dtype), c=g.c, mem=g.mem, layers=g.layers)
+
+
+def _grouped_devices(k, rng):
+    """Two speeds and three bandwidths in groups of two: few distinct values, asymmetric."""
+    s = np.where(np.arange(k) % 2 == 0, 3, 11).astype(np.int32)
+    grp = np.arange(k) // 2
+    B = np.where(grp[:, None] == grp[None, :], 900, 70).astype(np.int64)
+    B[np.triu_indices(k, 1)] += 13
+    return I.Devices(k, s, np.full(k, INF, np.int64), B, scale=int(rng.integers(1, 40)))
+
+
+@pytest.mark.parametrize("depth", [1, 3])
+@pytest.mark.parametrize("slice_,warps", [(16, 1), (16, 8), (32, 4), (64, 2), (64, 32), (128, 16)])
+def test_lean_kernel_shapes(slice_, warps, depth, monkeypatch):
+    """The lean windowed pass for every block shape (candidates per block, warps, stage depth): graphs with
+    wide and narrow levels, ragged candidate counts, k up to 8 with few and with many distinct bandwidths,
+    zero costs, vertices of high degree; device tables it does not take (k > 8, more than 30 distinct
+    bandwidths) fall back to the older kernels and must agree as well."""
+    from paper_1711_01912_b200 import tfps
+    monkeypatch.setenv("TFPS_LEAN", "1")
+    monkeypatch.setenv("TFPS_LEAN_SLICE", str(slice_))
+    monkeypatch.setenv("TFPS_SLICED_WARPS", str(warps))
+    monkeypatch.setenv("TFPS_LEAN_DEPTH", str(depth))
+    rng = np.random.default_rng(slice_ * 100 + warps)
+    took = []
+    cases = []
+    for (n, m, k, P) in [(1, 0, 1, 1), (50, 120, 2, 16), (700, 2500, 8, 77), (1500, 9000, 5, 150), (400, 0, 3, 33)]:
+        w = I.small_random(9000 + n + slice_, n, m, k, P, t_dtype=np.int64 if n % 2 else np.int32, with_mem=bool(n % 3))
+        dev = w.devices if k < 4 else _grouped_devices(k, rng)
+        cases.append((_small_costs(w.graph), dev, w.part_full()))
+    w = I.small_random(9100 + slice_, 600, 2000, 6, 90)       # 30 distinct bandwidths: the most the lean pass takes
+    cases.append((_small_costs(w.graph), w.devices, w.part_full()))
+    w = I.small_random(9200 + slice_, 500, 1500, 7, 40)       # 42 distinct bandwidths: falls back
+    cases.append((_small_costs(w.graph), w.devices, w.part_full()))
+    w = I.config3()
+    g = w.graph
+    keep = g.dst < 128 * 12   # first 12 layers of the wide graph (levels of 128 vertices)
+    g3 = I.Graph(n=128 * 12, src=g.src[keep], dst=g.dst[keep], t=g.t[keep], c=g.c[:128 * 12], mem=None, layers=12)
+    cases.append((g3, w.devices, w.part_rows(0, 128 * 12)[:, :200]))
+    w = I.config4()
+    g = w.graph
+    keep = g.dst < 16 * 200
+    g4 = I.Graph(n=16 * 200, src=g.src[keep], dst=g.dst[keep], t=g.t[keep], c=g.c[:16 * 200], mem=None, layers=200)
+    cases.append((g4, w.devices, w.part_rows(0, 16 * 200)[:, :97]))
+    n = 900   # one vertex with 899 in-edges, a level of 860 vertices
+    edges = [(u, n - 1, int(rng.integers(0, 10 ** 6))) for u in range(n - 1)] + [(0, u, 5) for u in range(1, 40)]
+    gh = graph_from_edges(n, edges, rng.integers(0, 100, size=n))
+    cases.append((gh, _grouped_devices(4, rng), rng.integers(0, 4, size=(n, 45), dtype=np.uint8)))
+    for g, dev, part in cases:
+        run_and_compare(g, dev, part, 2, pad_fill=255)
+        G = gpu_graph(g, dev)
+        dpart, P, ldp = padded(part)
+        G.eval_batch(dpart, P, flags=2)
+        took.append(tfps.tfps_last_pass_kernel(G.handle) == "pass_lean_kernel")
+        G.close()
+    # which cases the lean pass takes depends on the block shape (the window of a graph with long edges does not
+    # fit beside wide slices); the deep narrow graph always fits, the table with 42 bandwidths never does
+    assert took[8] and sum(took) >= 3 and not took[6], f"kernel choice per case: {took}"
+
+
+def test_loads_kernel_table_widths():
+    """Loads, memory loads and violation flags for every width of the runtime table (k = 1 .. 32) and beyond
+    it (k = 33, 64: the shuffle-based kernel), with bounded capacities so that some flags are set."""
+    for k in (1, 2, 3, 5, 8, 9, 16, 17, 32, 33, 64):
+        w = I.small_random(7000 + k, 300, 700, k, 130, with_mem=bool(k % 2))
+        d = w.devices
+        memsum = int(np.sum(w.graph.mem)) if w.graph.mem is not None else int(np.sum(w.graph.t))
+        dev = I.Devices(k, d.s, np.full(k, max(1, memsum // max(1, k - 1)), np.int64), d.B, d.scale)
+        run_and_compare(w.graph, dev, w.part_full(), 0, pad_fill=255)
 
 
 # ------------------------------------------------------------- randomized sweep
