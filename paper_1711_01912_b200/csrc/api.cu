@@ -151,6 +151,9 @@ struct tfps_graph {
     // copy stream and per-chunk events of tfps_eval_batch_host (created on first use)
     cudaStream_t copy_stream = nullptr;
     cudaEvent_t copy_ev[9] = {};
+    // low-priority stream on which the loads kernel runs beside the lean passes (created by tfps_devices_set)
+    cudaStream_t aux_stream = nullptr;
+    cudaEvent_t aux_fork = nullptr, aux_join = nullptr;
     ~tfps_graph()
     {
         for (cudaEvent_t e : ev)
@@ -158,6 +161,9 @@ struct tfps_graph {
         for (cudaEvent_t e : copy_ev)
             if (e) cudaEventDestroy(e);
         if (copy_stream) cudaStreamDestroy(copy_stream);
+        if (aux_fork) cudaEventDestroy(aux_fork);
+        if (aux_join) cudaEventDestroy(aux_join);
+        if (aux_stream) cudaStreamDestroy(aux_stream);
     }
 };
 
@@ -934,6 +940,13 @@ int tfps_devices_set(tfps_graph* g, int k, const int32_t* s, const int64_t* C, c
             }
     }
     CUDA_TRY(cudaStreamSynchronize(st));
+    if (!g->aux_stream) {
+        int lo = 0, hi = 0;
+        CUDA_TRY(cudaDeviceGetStreamPriorityRange(&lo, &hi));   // lo = least priority
+        CUDA_TRY(cudaStreamCreateWithPriority(&g->aux_stream, cudaStreamNonBlocking, lo));
+        CUDA_TRY(cudaEventCreateWithFlags(&g->aux_fork, cudaEventDisableTiming));
+        CUDA_TRY(cudaEventCreateWithFlags(&g->aux_join, cudaEventDisableTiming));
+    }
     g->k = k;
     g->S = scale;
     g->dev_set = true;
@@ -1011,25 +1024,28 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
         CUDA_TRY(cudaEventRecord(g->ev[0], st));
     }
 
-    // loads first: the same kernel checks the ids, and a bad id stops everything after it
     long long* ml = (long long*)memload;
     if (viol && !ml) {
         CUDA_TRY(g->scr_memload.reserve(sizeof(long long) * (size_t)k * (size_t)ldp));
         ml = g->scr_memload.as<long long>();
     }
-    if (load || ml) {
-        if (load) CUDA_TRY(cudaMemset2DAsync(load, sizeof(long long) * (size_t)ldp, 0, sizeof(long long) * (size_t)P, (size_t)k, st));
-        if (ml) CUDA_TRY(cudaMemset2DAsync(ml, sizeof(long long) * (size_t)ldp, 0, sizeof(long long) * (size_t)P, (size_t)k, st));
-        if (g->rt_kp > 0 && ((uintptr_t)part & 3u) == 0 && env_int("TFPS_LOADS2", 1) != 0)
-            CUDA_TRY(launch_loads2(n, P, ldp, part, g->rtv.as<long long>(), g->mem.as<long long>(), k, g->rt_kp,
-                                   (long long*)load, ml, status, validate, g->sm_count, g->smem_optin, st));
-        else
-            CUDA_TRY(launch_loads(n, P, ldp, part, g->order.as<int>(), g->xvert.as<unsigned long long>(), g->mem.as<long long>(),
-                                  tab, (long long*)load, ml, status, validate, g->sm_count, st));
-        if (viol) CUDA_TRY(launch_viol(P, ldp, k, ml, tab.cap, (unsigned long long*)viol, status, st));
-    } else if (validate) {
-        CUDA_TRY(launch_validate(n, P, ldp, part, k, status, g->sm_count, st));
-    }
+    // loads, memory loads, violation flags and the id check, on stream `ls`
+    auto run_loads = [&](cudaStream_t ls) -> int {
+        if (load || ml) {
+            if (load) CUDA_TRY(cudaMemset2DAsync(load, sizeof(long long) * (size_t)ldp, 0, sizeof(long long) * (size_t)P, (size_t)k, ls));
+            if (ml) CUDA_TRY(cudaMemset2DAsync(ml, sizeof(long long) * (size_t)ldp, 0, sizeof(long long) * (size_t)P, (size_t)k, ls));
+            if (g->rt_kp > 0 && ((uintptr_t)part & 3u) == 0 && env_int("TFPS_LOADS2", 1) != 0)
+                CUDA_TRY(launch_loads2(n, P, ldp, part, g->rtv.as<long long>(), g->mem.as<long long>(), k, g->rt_kp,
+                                       (long long*)load, ml, status, validate, g->sm_count, g->smem_optin, ls));
+            else
+                CUDA_TRY(launch_loads(n, P, ldp, part, g->order.as<int>(), g->xvert.as<unsigned long long>(), g->mem.as<long long>(),
+                                      tab, (long long*)load, ml, status, validate, g->sm_count, ls));
+            if (viol) CUDA_TRY(launch_viol(P, ldp, k, ml, tab.cap, (unsigned long long*)viol, status, ls));
+        } else if (validate) {
+            CUDA_TRY(launch_validate(n, P, ldp, part, k, status, g->sm_count, ls));
+        }
+        return TFPS_OK;
+    };
 
     // kernel variant
     bool sliced;
@@ -1057,12 +1073,71 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
         while (warps < 32 && warps < avg_width) warps <<= 1;
     }
 
+    const int level_bytes = (g->fits32 && env_int("TFPS_LEVEL32", 1) != 0) ? 4 : 8;
+    // Lean windowed pass (32-bit levels, whole window resident, host-packed records): block shape for one direction.
+    struct LeanChoice { bool ok = false; int slice = 0, warps = 0; size_t smem = 0; LeanArgs args; };
+    auto pick_lean = [&](bool fwd) {
+        LeanChoice ch;
+        if (!(sliced && g->lean[0].ok && g->lean[1].ok && level_bytes == 4 && ((uintptr_t)part & 15u) == 0 &&
+              ldp < (1LL << 28) && env_int("TFPS_LEAN", 1) != 0))
+            return ch;
+        const LeanPlan& lp = g->lean[fwd ? 0 : 1].plan;
+        // candidates per block (slice): the widest that keeps the window in shared memory and leaves enough
+        // blocks to occupy the machine; TFPS_LEAN_SLICE (or TFPS_SLICED_CPT = c for 32*c) forces one
+        const int forced = env_int("TFPS_SLICED_CPT", 0);
+        const long long want_slices = std::min<long long>((3LL * g->sm_count) / 4, (P + 15) / 16);
+        int d_want = env_int("TFPS_LEAN_DEPTH", 0);
+        if (d_want < 1 || d_want > LEAN_DEPTH_MAX) d_want = 3;
+        const int forced_warps = env_int("TFPS_SLICED_WARPS", 0);
+        const int forced_slice = env_int("TFPS_LEAN_SLICE", 0);
+        for (int slice = 128; slice >= 16 && !ch.ok; slice >>= 1) {
+            if (forced_slice == 16 || forced_slice == 32 || forced_slice == 64 || forced_slice == 128) { if (slice != forced_slice) continue; }
+            else if (forced == 1 || forced == 2 || forced == 4) { if (slice != 32 * forced) continue; }
+            else if ((P + slice - 1) / slice < want_slices && slice > 16) continue;
+            const int vpw = 128 / slice, pr = slice / 16;
+            int w = 1;   // one round of the vertex groups covers the widest chunk when 32 warps allow it
+            while (w < 32 && w * vpw < lp.max_v) w <<= 1;
+            if (forced_warps >= 1 && forced_warps <= 32) w = forced_warps;
+            while (w < 32 && lp.max_v * pr > 2 * w * 32) w <<= 1;   // a thread fetches at most two id-row pieces per chunk
+            if (lp.max_v * pr > 2 * w * 32) continue;
+            for (int d = d_want; d >= 1; --d) {
+                unsigned slot_stride = 0, stage_bytes = 0;
+                const size_t need = lean_smem_bytes(lp, slice, w, d, &slot_stride, &stage_bytes);
+                if (need + 1024 <= (size_t)g->smem_optin) {
+                    ch.ok = true; ch.slice = slice; ch.warps = w; ch.smem = need;
+                    ch.args.slot_stride = slot_stride;
+                    ch.args.stage_bytes = stage_bytes;
+                    ch.args.depth = d;
+                    break;
+                }
+            }
+        }
+        if (ch.ok) {
+            ch.args.part = part;
+            ch.args.status = status;
+            ch.args.P = P;
+            ch.args.ldp = ldp;
+            ch.args.plan = lp;
+        }
+        return ch;
+    };
+    LeanChoice lean_f, lean_b;
+    if (need_fwd) lean_f = pick_lean(true);
+    if (need_bwd) lean_b = pick_lean(false);
+    // The lean passes cannot leave their tables on a bad id (ids are masked), so the id check need not come first:
+    // the loads kernel then runs on a low-priority stream beside them and fills the SMs the passes' last wave leaves idle.
+    const bool overlap = (load || ml) && (need_fwd || need_bwd) && (!need_fwd || lean_f.ok) && (!need_bwd || lean_b.ok) &&
+                         g->aux_stream && env_int("TFPS_OVERLAP_LOADS", 1) != 0;
+    if (!overlap) TFPS_TRY(run_loads(st));   // loads first: the same kernel checks the ids, and a bad id stops everything after it
+    else {
+        CUDA_TRY(cudaEventRecord(g->aux_fork, st));
+        CUDA_TRY(cudaStreamWaitEvent(g->aux_stream, g->aux_fork, 0));
+    }
     if (profile) CUDA_TRY(cudaEventRecord(g->ev[1], st));
     // windowed pass: needs the precomputed edge values (simple device tables)
     // (its bulk copies of id rows need a 16-byte aligned id matrix)
     bool use_window = sliced && g->ncomb > 0 && env_int("TFPS_WINDOW", 1) != 0 && ((uintptr_t)part & 15u) == 0;
     int win_R = 0, win_depth = 1;
-    const int level_bytes = (g->fits32 && env_int("TFPS_LEVEL32", 1) != 0) ? 4 : 8;
     const int narrow = level_bytes == 4 ? 1 : 0;
     const int head_max = std::max(g->blob_head_max[0][narrow], g->blob_head_max[1][narrow]);
     const int body_max = std::max(g->blob_body_max[0][narrow], g->blob_body_max[1][narrow]);
@@ -1117,53 +1192,18 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
         long long* cp_here = (cp && (fwd || !need_fwd)) ? (long long*)cp : nullptr;
         PassArgs a = make_args(g, fwd, P, ldp, part, lev, cp_here);
         g->last_kernel = use_window ? "pass_window_kernel" : (sliced ? "pass_sliced_kernel" : (g->npass > 0 ? "pass_tile_kernel" : "pass_level_kernel"));
-        // lean windowed pass: 32-bit levels, whole window resident, host-packed records
-        if (sliced && g->lean[0].ok && g->lean[1].ok && level_bytes == 4 && ((uintptr_t)part & 15u) == 0 && ldp < (1LL << 28) &&
-            env_int("TFPS_LEAN", 1) != 0) {
-            const LeanPlan& lp = g->lean[fwd ? 0 : 1].plan;
-            // candidates per block (slice): the widest that keeps the window in shared memory and leaves enough
-            // blocks to occupy the machine; TFPS_SLICED_CPT = c forces 32*c
-            const int forced = env_int("TFPS_SLICED_CPT", 0);
-            const long long want_slices = std::min<long long>((3LL * g->sm_count) / 4, (P + 15) / 16);
-            int d_want = env_int("TFPS_LEAN_DEPTH", 0);
-            if (d_want < 1 || d_want > LEAN_DEPTH_MAX) d_want = 3;
-            const int forced_warps = env_int("TFPS_SLICED_WARPS", 0);
-            const int forced_slice = env_int("TFPS_LEAN_SLICE", 0);
-            int l_cpt = 0, l_depth = 0, l_warps = 0;
-            size_t l_smem = 0;
-            LeanArgs la;
-            for (int slice = 128; slice >= 16 && !l_cpt; slice >>= 1) {
-                if (forced_slice == 16 || forced_slice == 32 || forced_slice == 64 || forced_slice == 128) { if (slice != forced_slice) continue; }
-                else if (forced == 1 || forced == 2 || forced == 4) { if (slice != 32 * forced) continue; }
-                else if ((P + slice - 1) / slice < want_slices && slice > 16) continue;
-                const int vpw = 128 / slice, pr = slice / 16;
-                int w = 1;   // one round of the vertex groups covers the widest chunk when 32 warps allow it
-                while (w < 32 && w * vpw < lp.max_v) w <<= 1;
-                if (forced_warps >= 1 && forced_warps <= 32) w = forced_warps;
-                while (w < 32 && lp.max_v * pr > 2 * w * 32) w <<= 1;   // a thread fetches at most two id-row pieces per chunk
-                if (lp.max_v * pr > 2 * w * 32) continue;
-                for (int d = d_want; d >= 1; --d) {
-                    unsigned slot_stride = 0, stage_bytes = 0;
-                    const size_t need = lean_smem_bytes(lp, slice, w, d, &slot_stride, &stage_bytes);
-                    if (need + 512 <= (size_t)g->smem_optin) {
-                        l_cpt = slice; l_depth = d; l_warps = w; l_smem = need;
-                        la.slot_stride = slot_stride;
-                        la.stage_bytes = stage_bytes;
-                        break;
-                    }
-                }
-            }
-            if (l_cpt) {
-                la.part = part;
-                la.lev = lev;
-                la.cp = cp_here;
-                la.status = status;
-                la.P = P;
-                la.ldp = ldp;
-                la.plan = lp;
-                la.depth = l_depth;
+        {
+            LeanChoice& ch = fwd ? lean_f : lean_b;
+            if (ch.ok) {
+                ch.args.lev = lev;
+                ch.args.cp = cp_here;
                 g->last_kernel = "pass_lean_kernel";
-                CUDA_TRY(launch_pass_lean(la, fwd, l_cpt, l_warps, l_smem, st));
+                CUDA_TRY(launch_pass_lean(ch.args, fwd, ch.slice, ch.warps, ch.smem, st));
+                if (overlap && fwd == need_fwd) {
+                    // the first pass is queued: now the loads, so that the pass gets the machine first
+                    TFPS_TRY(run_loads(g->aux_stream));
+                    CUDA_TRY(cudaEventRecord(g->aux_join, g->aux_stream));
+                }
                 continue;
             }
         }
@@ -1212,6 +1252,7 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
             }
         }
     }
+    if (overlap) CUDA_TRY(cudaStreamWaitEvent(st, g->aux_join, 0));
     if (profile) {
         CUDA_TRY(cudaEventRecord(g->ev[3], st));
         g->ev_valid = true;
