@@ -263,11 +263,11 @@ def run_gpu(args):
     compulsory = 9.0 * n * P
     logical = 9.0 * (n + m) * P
     achieved = compulsory / (fwd_ms * 1e-3) / 1e9
-    # DRAM bytes of the forward kernel from the ncu capture summarised in profiles/pass_window_kernel_cfg3.md
-    # (P=2368: 1.3474 GB read+write = 8.682 B per vertex-candidate), scaled to this launch by n*P; only
+    # DRAM bytes of the forward kernel from the ncu capture summarised in profiles/pass_lean_kernel_cfg3.md
+    # (P=2368: 1.3435 GB read+write = 8.657 B per vertex-candidate), scaled to this launch by n*P; only
     # valid for the kernel and graph that capture was taken on
     kernel_name = tfps.tfps_last_pass_kernel(g.handle)
-    traffic = 8.682 * n * P if (args.config == 3 and kernel_name == "pass_window_kernel") else None
+    traffic = 8.657 * n * P if (args.config == 3 and kernel_name == "pass_lean_kernel") else None
     value = world * P / (ms * 1e-3)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
@@ -278,7 +278,9 @@ def run_gpu(args):
                    "l2": f"inputs+outputs per step {(n * ldp * 17) / 1e9:.1f} GB >> 126 MB L2, no explicit flush",
                    "setup_ms_graph_levels_tables": setup_s * 1e3},
         "edge_relaxations_per_s": world * 2.0 * m * P / (ms * 1e-3),
-        "phase_ms": {"loads_validate_viol": loads_ms, "forward": fwd_ms, "backward": bwd_ms},
+        "phase_ms": {"loads_validate_viol": loads_ms, "forward": fwd_ms, "backward": bwd_ms,
+                     "note": "CUDA events on the pass stream; with the lean pass the loads kernel runs beside the passes on "
+                             "its own stream and the backward figure includes the wait for it"},
         "roofline": {"bound": "hbm",
                      "kernel": tfps.tfps_last_pass_kernel(g.handle) + "<forward>",
                      "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
@@ -286,7 +288,8 @@ def run_gpu(args):
                      "achieved_logical": logical / (fwd_ms * 1e-3) / 1e9,
                      "frac_logical": logical / (fwd_ms * 1e-3) / 1e9 / peak,
                      "note": "achieved counts compulsory bytes 9*n*P (1 B id read + 8 B level write per vertex-candidate); "
-                             "achieved_logical adds 9 B per relaxation for neighbour reads, which L2 can serve"},
+                             "achieved_logical adds 9 B per relaxation for neighbour reads, which the lean pass serves "
+                             "from its shared-memory window (they never reach DRAM)"},
         "e2e": {"value": world * P / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": n * ldp, "d2h_bytes_per_step": 8 * (2 * P + 2 * k * ldp),
                 "api": "tfps_eval_batch_host (pinned host ids in; cp, load, memload, viol out; level matrices stay on the device)"},

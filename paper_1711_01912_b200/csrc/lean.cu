@@ -1,19 +1,20 @@
 // Lean windowed candidate-sliced pass.
 //
-// Same idea as the windowed pass (one block owns 32*CPT candidates, walks the whole graph chunk by chunk and
+// Same idea as the windowed pass (one block owns a slice of 16 to 128 candidates, walks the whole graph chunk by chunk and
 // keeps the levels of the last R positions of its own candidates in a shared-memory ring, so only the
 // compulsory traffic -- one id read and one level write per vertex-candidate -- reaches global memory), cut
 // down to the instructions the recurrences need:
 //   * the host packs one record per chunk (LeanPlan): vertices in processing order (highest degree first, dealt
-//     round-robin to the warps, so a fixed assignment is balanced), per-vertex runtimes for every device, and
-//     per-edge transfer times for every distinct bandwidth;
+//     to the vertex groups in alternating direction, so a fixed assignment is balanced), per-vertex runtimes for
+//     every device, and per-edge transfer times for every distinct bandwidth;
 //   * the window keeps finish times tlevel+rt (forward) or bottom levels (backward, Eq. 12), so a relaxation
 //     only adds the transfer term: one byte permute maps the neighbour's device id to the offset of the right
 //     transfer time inside the edge record, one shared-memory load fetches it, one add-max folds it in;
 //   * all shared-memory traffic uses 32-bit shared-window addresses;
 //   * every warp consumes; the copies of the chunk `depth` ahead (one bulk copy for the record, 16-byte
-//     cp.async pieces for the id rows) are issued by all threads right after the chunk barrier, from chunk
-//     descriptors and vertex ids prefetched into registers one chunk earlier.
+//     cp.async pieces for the id rows) are issued by all threads right after the chunk barrier; the descriptor
+//     comes from the header of the current record, the vertex ids of the id rows are requested at the top of
+//     the chunk and first touched after the barrier.
 // Requirements (checked by the host): every path length fits int32, k <= 8, at most 30 distinct off-diagonal
 // bandwidths, the whole window fits in shared memory beside the stage slots.
 #include "common.cuh"
