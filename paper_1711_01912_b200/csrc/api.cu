@@ -1095,8 +1095,10 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
             else if (forced == 1 || forced == 2 || forced == 4) { if (slice != 32 * forced) continue; }
             else if ((P + slice - 1) / slice < want_slices && slice > 16) continue;
             const int vpw = 128 / slice, pr = slice / 16;
-            int w = 1;   // one round of the vertex groups covers the widest chunk when 32 warps allow it
-            while (w < 32 && w * vpw < lp.max_v) w <<= 1;
+            // warps: one round of the vertex groups covers the widest chunk, up to 16 warps (512 threads with up to
+            // 128 registers each measured faster than 1024 threads with 64: 2.95 against 3.21 ms on config 3)
+            int w = 1;
+            while (w < 16 && w * vpw < lp.max_v) w <<= 1;
             if (forced_warps >= 1 && forced_warps <= 32) w = forced_warps;
             while (w < 32 && lp.max_v * pr > 2 * w * 32) w <<= 1;   // a thread fetches at most two id-row pieces per chunk
             if (lp.max_v * pr > 2 * w * 32) continue;
