@@ -449,29 +449,51 @@ int build_lean(tfps_graph* g, int k, const int32_t* s, const int64_t* B, long lo
             }
         }
         if (!ok) continue;
-        int R = 1;
-        while (R < g->maxspan + max_v) R <<= 1;
-        const int nc = (int)ch_p0.size();
+        // records: consecutive chunks staged together (one wait and one copy issue per record, a block barrier
+        // between its chunks), as many as fit LEAN_CHUNK_V vertices, e_cap edges and LEAN_SUB_MAX chunks
+        const int nchunks = (int)ch_p0.size();
+        std::vector<int> rec_c0, rec_nc;
+        int max_rec_v = 1;
+        for (int c = 0; c < nchunks;) {
+            int q = c, vs = 0, es = 0;
+            while (q < nchunks && q - c < LEAN_SUB_MAX) {
+                const int ce = ep[ch_p0[q] + ch_cnt[q]] - ep[ch_p0[q]];
+                if (q > c && (vs + ch_cnt[q] > LEAN_CHUNK_V || es + ce > e_cap)) break;
+                vs += ch_cnt[q];
+                es += ce;
+                ++q;
+            }
+            rec_c0.push_back(c);
+            rec_nc.push_back(q - c);
+            max_rec_v = std::max(max_rec_v, vs);
+            c = q;
+        }
+        int R = 1;   // every position written while a record is processed must leave its readers' neighbours intact
+        while (R < g->maxspan + max_rec_v) R <<= 1;
+        const int nc = (int)rec_c0.size();
         std::vector<int> desc((size_t)(nc + 2 * LEAN_DEPTH_MAX) * 4, 0), vlist((size_t)n);
         std::vector<unsigned char> blob;
         std::vector<int> idx, sorted((size_t)n);
         int rec_max = 16, vfirst = 0;
-        // first the processing order and the descriptors (a record names the chunks that follow it) ...
+        // first the processing order and the descriptors (a record names the records that follow it) ...
         size_t total = 0;
-        for (int c = 0; c < nc; ++c) {
-            const int p0 = ch_p0[c], cnt = ch_cnt[c];
-            idx.resize((size_t)cnt);
-            for (int i = 0; i < cnt; ++i) idx[i] = p0 + i;
-            // highest degree first: dealt round-robin, every round of the warps sees similar degrees
-            std::stable_sort(idx.begin(), idx.end(), [&](int a, int b) { return ep[a + 1] - ep[a] > ep[b + 1] - ep[b]; });
-            int ne = 0;
-            for (int i = 0; i < cnt; ++i) { ne += ep[idx[i] + 1] - ep[idx[i]]; sorted[(size_t)vfirst + i] = idx[i]; }
+        for (int r = 0; r < nc; ++r) {
+            int cnt = 0, ne = 0;
+            for (int c = rec_c0[r]; c < rec_c0[r] + rec_nc[r]; ++c) {
+                const int p0 = ch_p0[c], cc = ch_cnt[c];
+                idx.resize((size_t)cc);
+                for (int i = 0; i < cc; ++i) idx[i] = p0 + i;
+                // highest degree first: dealt to the vertex groups in alternating direction, every round sees similar degrees
+                std::stable_sort(idx.begin(), idx.end(), [&](int a, int b) { return ep[a + 1] - ep[a] > ep[b + 1] - ep[b]; });
+                for (int i = 0; i < cc; ++i) { ne += ep[idx[i] + 1] - ep[idx[i]]; sorted[(size_t)vfirst + cnt + i] = idx[i]; }
+                cnt += cc;
+            }
             const size_t e_area = LEAN_HDR_BYTES + (size_t)cnt * vstride;
             const size_t bytes = (e_area + (size_t)ne * estride + 15) & ~(size_t)15;
-            desc[4 * (size_t)c + 0] = (int)(total / 16);
-            desc[4 * (size_t)c + 1] = (int)bytes;
-            desc[4 * (size_t)c + 2] = cnt;
-            desc[4 * (size_t)c + 3] = vfirst;
+            desc[4 * (size_t)r + 0] = (int)(total / 16);
+            desc[4 * (size_t)r + 1] = (int)bytes;
+            desc[4 * (size_t)r + 2] = cnt;
+            desc[4 * (size_t)r + 3] = vfirst;
             vfirst += cnt;
             total += bytes;
             rec_max = std::max(rec_max, (int)bytes);
@@ -479,16 +501,23 @@ int build_lean(tfps_graph* g, int k, const int32_t* s, const int64_t* B, long lo
         if (total / 16 >= ((size_t)1 << 31)) continue;
         // ... then the records
         blob.assign(total, 0);
-        for (int c = 0; c < nc; ++c) {
-            const int cnt = ch_cnt[c];
-            const size_t off = (size_t)desc[4 * (size_t)c] * 16;
-            const int first = desc[4 * (size_t)c + 3];
+        for (int r = 0; r < nc; ++r) {
+            const int cnt = desc[4 * (size_t)r + 2];
+            const size_t off = (size_t)desc[4 * (size_t)r] * 16;
+            const int first = desc[4 * (size_t)r + 3];
             const size_t e_area = LEAN_HDR_BYTES + (size_t)cnt * vstride;
             int* hdr = reinterpret_cast<int*>(blob.data() + off);
-            hdr[0] = cnt;
+            hdr[0] = rec_nc[r];
             hdr[1] = (int)e_area;
+            hdr[2] = cnt;
             for (int d = 1; d <= LEAN_DEPTH_MAX; ++d)
-                for (int q = 0; q < 4; ++q) hdr[4 * d + q] = desc[4 * (size_t)(c + d) + q];   // zero past the end
+                for (int q = 0; q < 4; ++q) hdr[4 * d + q] = desc[4 * (size_t)(r + d) + q];   // zero past the end
+            int* sub = hdr + 4 + 4 * LEAN_DEPTH_MAX;   // per chunk {first vertex of the record, vertices}
+            for (int j = 0, at = 0; j < rec_nc[r]; ++j) {
+                sub[2 * j] = at;
+                sub[2 * j + 1] = ch_cnt[rec_c0[r] + j];
+                at += ch_cnt[rec_c0[r] + j];
+            }
             int eb = 0;
             for (int i = 0; i < cnt; ++i) {
                 const int p = sorted[(size_t)first + i], v = order[p];
@@ -522,7 +551,8 @@ int build_lean(tfps_graph* g, int k, const int32_t* s, const int64_t* B, long lo
         L.plan.estride = estride;
         L.plan.R = R;
         L.plan.rec_max = rec_max;
-        L.plan.max_v = max_v;
+        L.plan.max_v = max_rec_v;
+        L.plan.max_sub = max_v;
         for (int pv = 0; pv < LEAN_K_MAX; ++pv) {
             unsigned long long row = 0;
             for (int pu = 0; pu < LEAN_K_MAX; ++pu) {
@@ -1098,7 +1128,7 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
             // warps: one round of the vertex groups covers the widest chunk, up to 16 warps (512 threads with up to
             // 128 registers each measured faster than 1024 threads with 64: 2.95 against 3.21 ms on config 3)
             int w = 1;
-            while (w < 16 && w * vpw < lp.max_v) w <<= 1;
+            while (w < 16 && w * vpw < lp.max_sub) w <<= 1;
             if (forced_warps >= 1 && forced_warps <= 32) w = forced_warps;
             while (w < 32 && lp.max_v * pr > 2 * w * 32) w <<= 1;   // a thread fetches at most two id-row pieces per chunk
             if (lp.max_v * pr > 2 * w * 32) continue;

@@ -142,9 +142,11 @@ struct WindowPlan {
 };
 
 // Lean windowed pass (32-bit levels, k <= LEAN_K_MAX, whole window resident).  The host packs, per direction
-// and in processing order, one record per chunk:
-//   header  LEAN_HDR_BYTES: int4 {vertices, byte offset of the edge area, 0, 0}, then the descriptors
-//           {offset/16, bytes, vertices, first index into vlist} of the chunks 1..LEAN_DEPTH_MAX places later (zero past the end)
+// and in processing order, records of one or more consecutive chunks (a chunk = mutually independent vertices of
+// one level; narrow levels share a record, so a deep narrow graph pays the staging once per several levels):
+//   header  LEAN_HDR_BYTES: int4 {chunks, byte offset of the edge area, vertices, 0}, then the descriptors
+//           {offset/16, bytes, vertices, first index into vlist} of the records 1..LEAN_DEPTH_MAX places later
+//           (zero past the end), then per chunk {first vertex within the record, vertices}
 //   vertex  [vstride bytes each]  {v | flag << 31, window slot, first edge byte, end edge byte, rt[KP]}
 //           flag: sink (forward) / source (backward): the vertex enters the CP maximum;
 //           rt[d] = ceil(c_v*S / s_d); edge bytes are relative to the edge area
@@ -157,17 +159,19 @@ constexpr int LEAN_K_MAX = 8;
 constexpr int LEAN_CLS_MAX = 30;     // 4 * (classes + 1) must stay below 0x80 (sign-replicating byte permute)
 constexpr int LEAN_CHUNK_V = 128;
 constexpr int LEAN_DEPTH_MAX = 4;
-constexpr int LEAN_HDR_BYTES = 16 + 16 * LEAN_DEPTH_MAX;
+constexpr int LEAN_SUB_MAX = 16;      // chunks per record
+constexpr int LEAN_HDR_BYTES = 16 + 16 * LEAN_DEPTH_MAX + 8 * LEAN_SUB_MAX;
 
 struct LeanPlan {
     const unsigned char* blob;   // chunk records, 16-byte aligned each
     const int4* desc;            // [num_chunks + 2*LEAN_DEPTH_MAX] {offset/16, bytes, vertices, first index into vlist}; zero padded
     const int* vlist;            // [n] vertex ids in processing order
-    int num_chunks;
+    int num_chunks;              // records
     int vstride, estride;
     int R;                       // window length in positions (power of two)
     int rec_max;                 // largest record, bytes (multiple of 16)
-    int max_v;                   // most vertices in one chunk
+    int max_v;                   // most vertices in one record
+    int max_sub;                 // most vertices in one chunk
     unsigned long long rows[LEAN_K_MAX];
 };
 

@@ -191,7 +191,6 @@ __global__ void __launch_bounds__(MAXT, 1) pass_lean_kernel(const __grid_constan
     __shared__ __align__(16) unsigned long long s_rows[LEAN_K_MAX];
     __shared__ __align__(8) unsigned long long s_bar[LEAN_DEPTH_MAX];
     __shared__ int s_cp[128];   // CP maxima of the block's candidates
-    __shared__ int s_abort;
     constexpr int LPV = 32 / VPW;          // lanes per vertex
     constexpr int SLICE = LPV * CPT;       // candidates of the block = bytes of an id row
     constexpr unsigned LEVB = SLICE * 4;   // a window row: SLICE levels, then SLICE id bytes
@@ -202,14 +201,12 @@ __global__ void __launch_bounds__(MAXT, 1) pass_lean_kernel(const __grid_constan
     const int D = a.depth;
     const unsigned stage0 = smem_u32(dsm), win0 = stage0 + a.stage_bytes;
     const unsigned rows_s = smem_u32(s_rows), bar0 = smem_u32(s_bar);
-    volatile int* abort_p = &s_abort;
     if (tid < LEAN_K_MAX) s_rows[tid] = a.plan.rows[tid];
     for (int t = tid; t < 128; t += nthreads) s_cp[t] = 0;
     if (tid == 0) {
         // a stage completes on the record's bulk copy (one arrival carrying the byte count) plus one arrival
         // per thread once that thread's id-row pieces have landed
         for (int j = 0; j < D; ++j) mbar_init(bar0 + 8u * j, (unsigned)nthreads + 1u);
-        s_abort = 0;
         mbar_init_fence();
     }
     __syncthreads();
@@ -272,30 +269,37 @@ __global__ void __launch_bounds__(MAXT, 1) pass_lean_kernel(const __grid_constan
         issue(d, v0, v1, stage0 + (unsigned)j * a.slot_stride, bar0 + 8u * j);
     }
     const int nc = a.plan.num_chunks;
+    // Every wait on a stage is followed by a block-wide vote, so all threads agree whether it ran out (the records
+    // hold block barriers that every thread must reach): before the loop for record 0, afterwards folded into the
+    // barrier that ends a record.
     int slot = 0;
     unsigned par = 0;
-    for (int ci = 0; ci < nc; ++ci) {
+    bool timed_out = nc > 0 && !mbar_wait(bar0, 0u);
+    bool dead = __syncthreads_or(timed_out) != 0;
+    for (int ci = 0; ci < nc && !dead; ++ci) {
         const unsigned slotb = stage0 + (unsigned)slot * a.slot_stride;
         const unsigned bar = bar0 + 8u * slot;
         unsigned vA0 = 0, vA1 = 0;
-        if (!mbar_wait(bar, par)) {
-            atomicCAS(a.status, 0, (int)TFPS_ERR_TIMEOUT);
-            *abort_p = 1;
-        } else {
+        {
             // the record of chunk ci names chunk ci+D: request the vertex ids of its id rows now, use them after the barrier
             fetch_v(lds128(slotb + 16u * (unsigned)D), vA0, vA1);
-            const uint4 hdr = lds128(slotb);
-            const int cnt = (int)hdr.x;
+            const uint4 hdr = lds128(slotb);   // {chunks, byte offset of the edge area, vertices, -}
+            const int nsub = (int)hdr.x;
             const unsigned vbase = slotb + LEAN_HDR_BYTES, ebase = slotb + hdr.y;
             const unsigned idrow = slotb + rec_max + (unsigned)(ll * CPT);
             const int vstride = a.plan.vstride;
             const unsigned estride = (unsigned)a.plan.estride;
+            for (int sub = 0; sub < nsub; ++sub) {
+            if (sub > 0) __syncthreads();   // the previous chunk of the record is in the window
+            const uint2 sc = lds64(slotb + 16u + 16u * LEAN_DEPTH_MAX + 8u * (unsigned)sub);   // {first vertex, vertices}
+            const int first = (int)sc.x, cnt = (int)sc.y;
             // rounds alternate direction: group g takes entries g, 2G-1-g, 2G+g, ... of the degree-sorted list
             for (int base = 0; base < cnt; base += 2 * ngroups) {
 #pragma unroll 1
               for (int half = 0; half < 2; ++half) {
-                const int i = half == 0 ? base + group : base + 2 * ngroups - 1 - group;
-                if (i >= cnt) continue;
+                const int il = half == 0 ? base + group : base + 2 * ngroups - 1 - group;
+                if (il >= cnt) continue;
+                const int i = first + il;
                 const unsigned vr = vbase + (unsigned)(i * vstride);
                 const uint4 rec = lds128(vr);   // {v | flag, window slot, first edge byte, end edge byte}
                 const unsigned ids = ld_ids<CPT>(idrow + (unsigned)(i * SLICE));
@@ -358,21 +362,37 @@ __global__ void __launch_bounds__(MAXT, 1) pass_lean_kernel(const __grid_constan
                 st_ids<CPT>(lo + id_delta, (ids & 0x07070707u) | 0x80808080u);
               }
             }
+            }
         }
-        const uint4 dA = lds128(slotb + 16u * (unsigned)D);   // descriptor of chunk ci+D, before the slot is overwritten
-        __syncthreads();   // chunk ci is in the window; its stage slot is free again
-        if (*abort_p) break;
-        issue(dA, vA0, vA1, slotb, bar);
-        if (++slot == D) { slot = 0; par ^= 1u; }
+        const uint4 dA = lds128(slotb + 16u * (unsigned)D);   // descriptor of record ci+D, before the slot is overwritten
+        // wait for the next record, then one barrier: record ci is in the window, its stage slot is free again,
+        // and the outcome of the wait is agreed on
+        const int nslot = slot + 1 == D ? 0 : slot + 1;
+        const unsigned npar = slot + 1 == D ? par ^ 1u : par;
+        if (D > 1) {
+            timed_out = ci + 1 < nc && !mbar_wait(bar0 + 8u * nslot, npar);
+            dead = __syncthreads_or(timed_out) != 0;
+            if (dead) break;
+            issue(dA, vA0, vA1, slotb, bar);
+        } else {   // a single stage: the next record can only be requested once this one is done with
+            __syncthreads();
+            issue(dA, vA0, vA1, slotb, bar);
+            timed_out = ci + 1 < nc && !mbar_wait(bar0 + 8u * nslot, npar);
+            dead = __syncthreads_or(timed_out) != 0;
+            if (dead) break;
+        }
+        slot = nslot;
+        par = npar;
     }
-    __syncthreads();
-    if (*abort_p) {
+    if (dead) {
+        if (timed_out) atomicCAS(a.status, 0, (int)TFPS_ERR_TIMEOUT);
         // copies already requested may still be landing in this block's shared memory: give them a bounded
         // time before the block (and its shared memory) goes away
 #pragma unroll 1
         for (int i = 0; i < 1000; ++i) __nanosleep(1000);
         return;
     }
+    __syncthreads();
     if (a.cp != nullptr)
         for (int t = tid; t < SLICE; t += nthreads)
             if (slice0 + t < a.P) a.cp[slice0 + t] = (long long)s_cp[t];
