@@ -87,9 +87,16 @@ class ClockSampler:
                 "reasons": sorted(reasons), "samples": len(sm)}
 
 
-def make_workload(cfg: int, rank: int):
+def make_workload(cfg: int, rank: int, P: int = 0):
+    """The seeded workload of a configuration.  Config 5's 8,192 candidates x 1 M vertices need 146 GB for ids and both
+    level matrices, so it is evaluated in candidate chunks: one step = one chunk of P candidates (default 4,096)."""
     from paper_1711_01912_b200 import inputs
     w = inputs.make_config(cfg)
+    w.P_full = w.P
+    if P <= 0 and cfg == 5:
+        P = 4096
+    if P > 0:
+        w.P = min(P, w.P)
     if rank:
         w.seed = w.seed + 1000 * rank  # other ranks draw other candidate partitions of the same graph
     return w
@@ -121,7 +128,7 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    w = make_workload(args.config, 0)
+    w = make_workload(args.config, 0, args.P)
     og = oracle_setup(w)
     cols, part_cols = sample_columns(w, 8)
     per = oracle_time(w, og, part_cols) / 8
@@ -163,7 +170,7 @@ def run_gpu(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
-    w = make_workload(args.config, rank)
+    w = make_workload(args.config, rank, args.P)
     n, m, k, P = w.graph.n, w.graph.m, w.devices.k, w.P
     ldp = tfps.round_up_ldp(P)
     t_setup = time.perf_counter()
@@ -264,23 +271,25 @@ def run_gpu(args):
     logical = 9.0 * (n + m) * P
     achieved = compulsory / (fwd_ms * 1e-3) / 1e9
     # DRAM bytes of the forward kernel from the ncu capture summarised in profiles/pass_lean_kernel_cfg3.md
-    # (P=2368: 1.3435 GB read+write = 8.657 B per vertex-candidate), scaled to this launch by n*P; only
+    # (P=2368: 1.3472 GB read+write = 8.681 B per vertex-candidate), scaled to this launch by n*P; only
     # valid for the kernel and graph that capture was taken on
     kernel_name = tfps.tfps_last_pass_kernel(g.handle)
-    traffic = 8.657 * n * P if (args.config == 3 and kernel_name == "pass_lean_kernel") else None
+    traffic = 8.681 * n * P if (args.config == 3 and kernel_name == "pass_lean_kernel") else None
     value = world * P / (ms * 1e-3)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
         "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int64",
         "data": "synthetic",
-        "config": {"workload": w.name, "n": n, "m": m, "levels": L, "k": k, "P": P, "ldp": ldp, "scale": w.devices.scale,
+        "config": {"workload": w.name, "n": n, "m": m, "levels": L, "k": k, "P": P, "P_of_configuration": w.P_full,
+                   "ldp": ldp, "scale": w.devices.scale,
                    "variant": args.variant, "outputs": list(want),
                    "l2": f"inputs+outputs per step {(n * ldp * 17) / 1e9:.1f} GB >> 126 MB L2, no explicit flush",
                    "setup_ms_graph_levels_tables": setup_s * 1e3},
         "edge_relaxations_per_s": world * 2.0 * m * P / (ms * 1e-3),
         "phase_ms": {"loads_validate_viol": loads_ms, "forward": fwd_ms, "backward": bwd_ms,
-                     "note": "CUDA events on the pass stream; with the lean pass the loads kernel runs beside the passes on "
-                             "its own stream and the backward figure includes the wait for it"},
+                     "note": ("CUDA events on the pass stream; the loads kernel runs beside the lean passes on its own stream "
+                              "and the backward figure includes the wait for it") if kernel_name == "pass_lean_kernel"
+                             else "CUDA events on the pass stream"},
         "roofline": {"bound": "hbm",
                      "kernel": tfps.tfps_last_pass_kernel(g.handle) + "<forward>",
                      "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
@@ -288,8 +297,9 @@ def run_gpu(args):
                      "achieved_logical": logical / (fwd_ms * 1e-3) / 1e9,
                      "frac_logical": logical / (fwd_ms * 1e-3) / 1e9 / peak,
                      "note": "achieved counts compulsory bytes 9*n*P (1 B id read + 8 B level write per vertex-candidate); "
-                             "achieved_logical adds 9 B per relaxation for neighbour reads, which the lean pass serves "
-                             "from its shared-memory window (they never reach DRAM)"},
+                             "achieved_logical adds 9 B per relaxation for neighbour reads" +
+                             (", which the lean pass serves from its shared-memory window (they never reach DRAM)"
+                              if kernel_name == "pass_lean_kernel" else ", which L2 serves when the levels in use fit")},
         "e2e": {"value": world * P / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": n * ldp, "d2h_bytes_per_step": 8 * (2 * P + 2 * k * ldp),
                 "api": "tfps_eval_batch_host (pinned host ids in; cp, load, memload, viol out; level matrices stay on the device)"},
@@ -324,7 +334,8 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--config", type=int, default=3, choices=[1, 2, 3, 4])
+    ap.add_argument("--config", type=int, default=3, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--P", type=int, default=0, help="candidates per step (default: the configuration's; config 5: a chunk of 4096)")
     ap.add_argument("--impl", default="tfps", choices=["tfps", "reference"])
     ap.add_argument("--variant", default="auto", choices=["auto", "sliced", "level_sync"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
