@@ -374,14 +374,18 @@ int env_int(const char* name, int dflt)
     return atoi(s);
 }
 
-// Packs the chunk records of the lean windowed pass for both directions (layout: LeanPlan in common.cuh).
+// Packs the chunk records of the lean windowed passes for both directions (layout: LeanPlan in common.cuh).
 // Everything is computed on the host with plain integer division; `order` is the host copy of the level order.
+// Narrow plan (pass_lean_kernel): every path fits int32 and k <= 8.  Wide plan (pass_lean64_kernel): k <= 16 and
+// every vertex runtime below 2^31.  The plan walks the vertices either in level order or, when the caller's vertex
+// numbering is itself a topological order whose edges are at least twice shorter, in that order (graphs built layer
+// by layer, as data-flow graphs usually are): a shorter longest edge is a smaller window.
 int build_lean(tfps_graph* g, int k, const int32_t* s, const int64_t* B, long long S, const std::vector<int>& order,
                cudaStream_t st)
 {
     for (auto& L : g->lean) L.ok = false;
     const int n = (int)g->n, m = (int)g->m;
-    if (!g->fits32 || k > LEAN_K_MAX || n == 0 || env_int("TFPS_LEAN", 1) == 0) return TFPS_OK;
+    if (n == 0 || env_int("TFPS_LEAN", 1) == 0) return TFPS_OK;
     std::vector<long long> wvals;   // distinct off-diagonal bandwidths; class c+1 <-> wvals[c], class 0 = same device
     auto cls_of = [&](long long x) {
         for (size_t i = 0; i < wvals.size(); ++i)
@@ -389,18 +393,26 @@ int build_lean(tfps_graph* g, int k, const int32_t* s, const int64_t* B, long lo
         wvals.push_back(x);
         return (int)wvals.size() - 1;
     };
-    for (int a = 0; a < k; ++a)
+    long long s_min = INT64_MAX;
+    for (int a = 0; a < k; ++a) {
+        s_min = std::min<long long>(s_min, s[a]);
         for (int b = 0; b < k; ++b)
             if (a != b) cls_of(B[a * k + b]);
+    }
     const int ncw = (int)wvals.size();
     if (ncw > LEAN_CLS_MAX) return TFPS_OK;
-    const int KP = k <= 4 ? 4 : 8;
-    const int vstride = 16 + 4 * KP, estride = 4 * (ncw + 2);
-    const int e_cap = std::max(64, std::min(1024, 24576 / estride));   // edges per chunk
+    const bool narrow_ok = g->fits32 && k <= LEAN_K_MAX && env_int("TFPS_LEAN_FORCE_WIDE", 0) == 0;
+    const u128 rt_max = ((u128)g->max_c * (u128)S + (u128)s_min - 1) / (u128)s_min;
+    const bool wide_ok = k <= LEAN64_K_MAX && rt_max < ((u128)1 << 31) && env_int("TFPS_LEAN64", 1) != 0;
+    if (!narrow_ok && !wide_ok) return TFPS_OK;
+    const bool wide = !narrow_ok;
+    const int KP = wide ? 16 : (k <= 4 ? 4 : 8);
+    const int vstride = 16 + 4 * KP, estride = wide ? 8 + 8 * (ncw + 1) : 4 * (ncw + 2);
+    const int e_cap = std::max(64, std::min(1024, 24576 / estride));   // edges per record
 
-    std::vector<int> pos_of((size_t)n);
+    std::vector<int> pos_of((size_t)n);   // level position of a vertex
     for (int i = 0; i < n; ++i) pos_of[order[i]] = i;
-    std::vector<int> eptr[2], nbr[2];
+    std::vector<int> eptr[2], nbr[2];     // level-ordered adjacency: [0] in-edges, [1] out-edges
     std::vector<long long> tt[2];
     for (int dir = 0; dir < 2; ++dir) {
         eptr[dir].resize((size_t)n + 1);
@@ -419,45 +431,99 @@ int build_lean(tfps_graph* g, int k, const int32_t* s, const int64_t* B, long lo
     auto ceil_div = [](long long a, long long S_, long long d) {
         return (long long)(((u128)a * (u128)S_ + (u128)d - 1) / (u128)d);
     };
-    const int src_end = (int)g->h_level_ptr[1];
+
+    // plan order: level order, or the caller's numbering when it is topological and its longest edge much shorter
+    bool id_topo = true;
+    int span_id = 0;
+    for (int v = 0; v < n && id_topo; ++v)
+        for (long long e = g->h_in_ptr[v]; e < g->h_in_ptr[v + 1]; ++e) {
+            const int u = g->h_in_src[e];
+            if (u >= v) { id_topo = false; break; }
+            span_id = std::max(span_id, v - u);
+        }
+    bool use_id = id_topo && 2LL * (span_id + LEAN_CHUNK_V) <= (long long)g->maxspan + LEAN_CHUNK_V;
+    const int forced_order = env_int("TFPS_LEAN_ORDER", 0);   // 1: level order, 2: caller's numbering (if topological)
+    if (forced_order == 1) use_id = false;
+    if (forced_order == 2) use_id = id_topo;
+    const int span = use_id ? span_id : g->maxspan;
+    // vertex at plan position q, plan position of vertex v, level position (index into eptr) of plan position q
+    auto vert_at = [&](int q) { return use_id ? q : order[q]; };
+    auto ppos = [&](int v) { return use_id ? v : pos_of[v]; };
+    auto lpos = [&](int q) { return use_id ? pos_of[q] : q; };
 
     for (int dir = 0; dir < 2; ++dir) {
         tfps_graph::Lean& L = g->lean[dir];
         const std::vector<int>& ep = eptr[dir];
-        // chunks: runs of positions inside one level; a wide level is split evenly
+        auto deg = [&](int q) { const int a = lpos(q); return ep[a + 1] - ep[a]; };
+        // chunks (first plan position, vertices) in processing order: mutually independent vertices, at most
+        // LEAN_CHUNK_V of them and e_cap edges
         std::vector<int> ch_p0, ch_cnt;
         bool ok = true;
         int max_v = 1;
-        for (int li = 0; li < g->num_levels && ok; ++li) {
-            const int l = dir == 0 ? li : g->num_levels - 1 - li;
-            int p = (int)g->h_level_ptr[l];
-            const int pend = (int)g->h_level_ptr[l + 1];
-            const int width = pend - p;
-            int target = width;
-            if (width > LEAN_CHUNK_V) {
-                const int nch = (width + LEAN_CHUNK_V - 1) / LEAN_CHUNK_V;
-                target = std::min(LEAN_CHUNK_V, (((width + nch - 1) / nch) + 31) / 32 * 32);
+        if (!use_id) {   // runs of positions inside one level; a wide level is split evenly
+            for (int li = 0; li < g->num_levels && ok; ++li) {
+                const int l = dir == 0 ? li : g->num_levels - 1 - li;
+                int p = (int)g->h_level_ptr[l];
+                const int pend = (int)g->h_level_ptr[l + 1];
+                const int width = pend - p;
+                int target = width;
+                if (width > LEAN_CHUNK_V) {
+                    const int nch = (width + LEAN_CHUNK_V - 1) / LEAN_CHUNK_V;
+                    target = std::min(LEAN_CHUNK_V, (((width + nch - 1) / nch) + 31) / 32 * 32);
+                }
+                while (p < pend) {
+                    int q = p, edges = 0;
+                    while (q < pend && q - p < target && edges + deg(q) <= e_cap) { edges += deg(q); ++q; }
+                    if (q == p) { ok = false; break; }   // a vertex with more edges than a record can stage
+                    ch_p0.push_back(p);
+                    ch_cnt.push_back(q - p);
+                    max_v = std::max(max_v, q - p);
+                    p = q;
+                }
             }
-            while (p < pend) {
-                int q = p, edges = 0;
-                while (q < pend && q - p < target && edges + (ep[q + 1] - ep[q]) <= e_cap) { edges += ep[q + 1] - ep[q]; ++q; }
-                if (q == p) { ok = false; break; }   // a vertex with more edges than a chunk can stage
-                ch_p0.push_back(p);
-                ch_cnt.push_back(q - p);
-                max_v = std::max(max_v, q - p);
-                p = q;
+        } else {   // consecutive vertices none of which has a neighbour (of this direction) inside the run
+            int lo = dir == 0 ? 0 : n - 1, cnt = 0, edges = 0;   // current run: forward [lo, lo+cnt), backward (lo-cnt, lo]
+            auto close = [&]() {
+                if (cnt == 0) return;
+                ch_p0.push_back(dir == 0 ? lo : lo - cnt + 1);
+                ch_cnt.push_back(cnt);
+                max_v = std::max(max_v, cnt);
+            };
+            for (int step = 0; step < n && ok; ++step) {
+                const int q = dir == 0 ? step : n - 1 - step;
+                const int a = lpos(q), d = ep[a + 1] - ep[a];
+                if (d > e_cap) { ok = false; break; }
+                bool indep = true;   // every neighbour lies before the run (forward) / after it (backward)
+                for (int e = ep[a]; e < ep[a + 1] && indep; ++e) {
+                    const int x = ppos(nbr[dir][e]);
+                    indep = dir == 0 ? x < lo : x > lo;
+                }
+                if (cnt > 0 && (!indep || cnt >= LEAN_CHUNK_V || edges + d > e_cap)) {
+                    close();
+                    cnt = 0;
+                    edges = 0;
+                }
+                if (cnt == 0) lo = q;
+                ++cnt;
+                edges += d;
             }
+            close();
         }
         if (!ok) continue;
         // records: consecutive chunks staged together (one wait and one copy issue per record, a block barrier
         // between its chunks), as many as fit LEAN_CHUNK_V vertices, e_cap edges and LEAN_SUB_MAX chunks
         const int nchunks = (int)ch_p0.size();
+        auto chunk_edges = [&](int c) {
+            int es = 0;
+            for (int q = ch_p0[c]; q < ch_p0[c] + ch_cnt[c]; ++q) es += deg(q);
+            return es;
+        };
         std::vector<int> rec_c0, rec_nc;
         int max_rec_v = 1;
         for (int c = 0; c < nchunks;) {
             int q = c, vs = 0, es = 0;
             while (q < nchunks && q - c < LEAN_SUB_MAX) {
-                const int ce = ep[ch_p0[q] + ch_cnt[q]] - ep[ch_p0[q]];
+                const int ce = chunk_edges(q);
                 if (q > c && (vs + ch_cnt[q] > LEAN_CHUNK_V || es + ce > e_cap)) break;
                 vs += ch_cnt[q];
                 es += ce;
@@ -468,8 +534,9 @@ int build_lean(tfps_graph* g, int k, const int32_t* s, const int64_t* B, long lo
             max_rec_v = std::max(max_rec_v, vs);
             c = q;
         }
-        int R = 1;   // every position written while a record is processed must leave its readers' neighbours intact
-        while (R < g->maxspan + max_rec_v) R <<= 1;
+        // window rows: every position written while a record is processed must leave its readers' neighbours intact
+        int R = span + max_rec_v;
+        if (!wide) { R = 1; while (R < span + max_rec_v) R <<= 1; }
         const int nc = (int)rec_c0.size();
         std::vector<int> desc((size_t)(nc + 2 * LEAN_DEPTH_MAX) * 4, 0), vlist((size_t)n);
         std::vector<unsigned char> blob;
@@ -484,8 +551,8 @@ int build_lean(tfps_graph* g, int k, const int32_t* s, const int64_t* B, long lo
                 idx.resize((size_t)cc);
                 for (int i = 0; i < cc; ++i) idx[i] = p0 + i;
                 // highest degree first: dealt to the vertex groups in alternating direction, every round sees similar degrees
-                std::stable_sort(idx.begin(), idx.end(), [&](int a, int b) { return ep[a + 1] - ep[a] > ep[b + 1] - ep[b]; });
-                for (int i = 0; i < cc; ++i) { ne += ep[idx[i] + 1] - ep[idx[i]]; sorted[(size_t)vfirst + cnt + i] = idx[i]; }
+                std::stable_sort(idx.begin(), idx.end(), [&](int x, int y) { return deg(x) > deg(y); });
+                for (int i = 0; i < cc; ++i) { ne += deg(idx[i]); sorted[(size_t)vfirst + cnt + i] = idx[i]; }
                 cnt += cc;
             }
             const size_t e_area = LEAN_HDR_BYTES + (size_t)cnt * vstride;
@@ -520,18 +587,23 @@ int build_lean(tfps_graph* g, int k, const int32_t* s, const int64_t* B, long lo
             }
             int eb = 0;
             for (int i = 0; i < cnt; ++i) {
-                const int p = sorted[(size_t)first + i], v = order[p];
+                const int p = sorted[(size_t)first + i], v = vert_at(p), a = lpos(p);
                 int* vr = reinterpret_cast<int*>(blob.data() + off + LEAN_HDR_BYTES + (size_t)i * vstride);
-                const bool flag = dir == 0 ? (eptr[1][p + 1] == eptr[1][p]) : (p < src_end);
+                // the vertex enters the CP maximum: sinks forward, sources backward
+                const bool flag = dir == 0 ? (eptr[1][a + 1] == eptr[1][a]) : (eptr[0][a + 1] == eptr[0][a]);
                 vr[0] = v | (flag ? (int)0x80000000u : 0);
-                vr[1] = p & (R - 1);
+                vr[1] = p % R;
                 vr[2] = eb;
                 for (int d = 0; d < k; ++d) vr[4 + d] = (int)ceil_div(g->h_c[v], S, s[d]);
-                for (int q = ep[p]; q < ep[p + 1]; ++q) {
-                    int* er = reinterpret_cast<int*>(blob.data() + off + e_area + (size_t)eb);
-                    er[0] = pos_of[nbr[dir][q]] & (R - 1);
-                    er[1] = 0;
-                    for (int w = 0; w < ncw; ++w) er[2 + w] = (int)ceil_div(tt[dir][q], S, wvals[w]);
+                for (int q = ep[a]; q < ep[a + 1]; ++q) {
+                    unsigned char* er = blob.data() + off + e_area + (size_t)eb;
+                    const int ns = ppos(nbr[dir][q]) % R;
+                    memcpy(er, &ns, 4);
+                    for (int w = 0; w < ncw; ++w) {
+                        const long long val = ceil_div(tt[dir][q], S, wvals[w]);
+                        if (wide) memcpy(er + 16 + 8 * w, &val, 8);                     // {slot, pad, W[0] = 0, W[1..]}
+                        else { const int v32 = (int)val; memcpy(er + 8 + 4 * w, &v32, 4); }   // {slot, W[0] = 0, W[1..]}
+                    }
                     eb += estride;
                 }
                 vr[3] = eb;
@@ -553,15 +625,24 @@ int build_lean(tfps_graph* g, int k, const int32_t* s, const int64_t* B, long lo
         L.plan.rec_max = rec_max;
         L.plan.max_v = max_rec_v;
         L.plan.max_sub = max_v;
+        L.plan.wide = wide ? 1 : 0;
+        // class of the link between a neighbour on device pu and a vertex on device pv (0 = same device), scaled to
+        // the byte offset of its transfer time inside an edge record
+        auto link = [&](int pu, int pv) {
+            if (pv >= k || pu >= k || pu == pv) return 0;
+            return cls_of(dir == 0 ? B[pu * k + pv] : B[pv * k + pu]) + 1;
+        };
         for (int pv = 0; pv < LEAN_K_MAX; ++pv) {
             unsigned long long row = 0;
-            for (int pu = 0; pu < LEAN_K_MAX; ++pu) {
-                unsigned long long byte = 0;
-                if (pv < k && pu < k && pu != pv) byte = 4ull * (unsigned)(cls_of(dir == 0 ? B[pu * k + pv] : B[pv * k + pu]) + 1);
-                row |= byte << (8 * pu);
-            }
+            for (int pu = 0; pu < LEAN_K_MAX; ++pu) row |= (unsigned long long)(4 * link(pu, pv)) << (8 * pu);
             L.plan.rows[pv] = row;
         }
+        for (int pv = 0; pv < LEAN64_K_MAX; ++pv)
+            for (int h = 0; h < 2; ++h) {
+                unsigned long long row = 0;
+                for (int b = 0; b < 8; ++b) row |= (unsigned long long)(8 * link(8 * h + b, pv)) << (8 * b);
+                L.plan.rows16[2 * pv + h] = row;
+            }
         L.ok = true;
     }
     return TFPS_OK;
@@ -891,7 +972,7 @@ int tfps_devices_set(tfps_graph* g, int k, const int32_t* s, const int64_t* C, c
     }
     g->fits32 = false;
     for (auto& L : g->lean) L.ok = false;
-    if ((g->ncomb > 0 || k <= LEAN_K_MAX) && n > 0) {
+    if ((g->ncomb > 0 || k <= LEAN64_K_MAX) && n > 0) {
         // worst-case critical path: every vertex on the slowest device, every edge over the slowest link
         std::vector<int> order((size_t)n);
         CUDA_TRY(cudaMemcpyAsync(order.data(), g->order.p, sizeof(int) * (size_t)n, cudaMemcpyDeviceToHost, st));
@@ -1108,29 +1189,36 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
     struct LeanChoice { bool ok = false; int slice = 0, warps = 0; size_t smem = 0; LeanArgs args; };
     auto pick_lean = [&](bool fwd) {
         LeanChoice ch;
-        if (!(sliced && g->lean[0].ok && g->lean[1].ok && level_bytes == 4 && ((uintptr_t)part & 15u) == 0 &&
-              ldp < (1LL << 28) && env_int("TFPS_LEAN", 1) != 0))
+        if (!(sliced && g->lean[0].ok && g->lean[1].ok && ((uintptr_t)part & 15u) == 0 && ldp < (1LL << 28) &&
+              env_int("TFPS_LEAN", 1) != 0))
             return ch;
         const LeanPlan& lp = g->lean[fwd ? 0 : 1].plan;
+        if (!lp.wide && level_bytes != 4) return ch;
+        // the wide kernel can run blocks of 8 or 16 candidates, but a block that narrow is bound by the latency of a
+        // record and measured slower than the level-synchronous kernels: only on request (TFPS_LEAN_SLICE)
+        const int forced_slice = env_int("TFPS_LEAN_SLICE", 0);
+        const int slice_min = lp.wide ? ((forced_slice == 8 || forced_slice == 16) ? forced_slice : 32) : 16;
         // candidates per block (slice): the widest that keeps the window in shared memory and leaves enough
         // blocks to occupy the machine; TFPS_LEAN_SLICE (or TFPS_SLICED_CPT = c for 32*c) forces one
         const int forced = env_int("TFPS_SLICED_CPT", 0);
-        const long long want_slices = std::min<long long>((3LL * g->sm_count) / 4, (P + 15) / 16);
+        const long long want_slices = std::min<long long>((3LL * g->sm_count) / 4, (P + slice_min - 1) / slice_min);
         int d_want = env_int("TFPS_LEAN_DEPTH", 0);
         if (d_want < 1 || d_want > LEAN_DEPTH_MAX) d_want = 3;
         const int forced_warps = env_int("TFPS_SLICED_WARPS", 0);
-        const int forced_slice = env_int("TFPS_LEAN_SLICE", 0);
-        for (int slice = 128; slice >= 16 && !ch.ok; slice >>= 1) {
-            if (forced_slice == 16 || forced_slice == 32 || forced_slice == 64 || forced_slice == 128) { if (slice != forced_slice) continue; }
+        for (int slice = 128; slice >= slice_min && !ch.ok; slice >>= 1) {
+            if (forced_slice == 8 || forced_slice == 16 || forced_slice == 32 || forced_slice == 64 || forced_slice == 128) {
+                if (slice != std::max(forced_slice, slice_min)) continue;
+            }
             else if (forced == 1 || forced == 2 || forced == 4) { if (slice != 32 * forced) continue; }
-            else if ((P + slice - 1) / slice < want_slices && slice > 16) continue;
-            const int vpw = 128 / slice, pr = slice / 16;
+            else if ((P + slice - 1) / slice < want_slices && slice > slice_min) continue;
+            const int vpw = 128 / slice, pr = std::max(1, slice / 16);
             // warps: one round of the vertex groups covers the widest chunk, up to 16 warps (512 threads with up to
             // 128 registers each measured faster than 1024 threads with 64: 2.95 against 3.21 ms on config 3)
             int w = 1;
             while (w < 16 && w * vpw < lp.max_sub) w <<= 1;
-            if (forced_warps >= 1 && forced_warps <= 32) w = forced_warps;
-            while (w < 32 && lp.max_v * pr > 2 * w * 32) w <<= 1;   // a thread fetches at most two id-row pieces per chunk
+            const int wmax = lp.wide ? 16 : 32;   // the wide kernel is built for at most 512 threads
+            if (forced_warps >= 1 && forced_warps <= wmax) w = forced_warps;
+            while (w < wmax && lp.max_v * pr > 2 * w * 32) w <<= 1;   // a thread fetches at most two id-row pieces per record
             if (lp.max_v * pr > 2 * w * 32) continue;
             for (int d = d_want; d >= 1; --d) {
                 unsigned slot_stride = 0, stage_bytes = 0;
@@ -1229,8 +1317,9 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
             if (ch.ok) {
                 ch.args.lev = lev;
                 ch.args.cp = cp_here;
-                g->last_kernel = "pass_lean_kernel";
-                CUDA_TRY(launch_pass_lean(ch.args, fwd, ch.slice, ch.warps, ch.smem, st));
+                g->last_kernel = ch.args.plan.wide ? "pass_lean64_kernel" : "pass_lean_kernel";
+                if (ch.args.plan.wide) CUDA_TRY(launch_pass_lean64(ch.args, fwd, ch.slice, ch.warps, ch.smem, st));
+                else CUDA_TRY(launch_pass_lean(ch.args, fwd, ch.slice, ch.warps, ch.smem, st));
                 if (overlap && fwd == need_fwd) {
                     // the first pass is queued: now the loads, so that the pass gets the machine first
                     TFPS_TRY(run_loads(g->aux_stream));

@@ -173,7 +173,12 @@ struct LeanPlan {
     int max_v;                   // most vertices in one record
     int max_sub;                 // most vertices in one chunk
     unsigned long long rows[LEAN_K_MAX];
+    // wide plan (pass_lean64_kernel: int64 levels, k <= LEAN64_K_MAX): vertex records carry rt[16] (int32), edge
+    // records {window slot, pad, W[0..ncls] as int64}; rows16[pv*2 + h] holds, in byte pu - 8h, 8 * class
+    int wide;
+    unsigned long long rows16[2 * 16];
 };
+constexpr int LEAN64_K_MAX = 16;
 
 struct LeanArgs {
     const uint8_t* part;
@@ -189,6 +194,7 @@ struct LeanArgs {
 
 size_t lean_smem_bytes(const LeanPlan& plan, int slice, int warps, int depth, unsigned* slot_stride, unsigned* stage_bytes);
 cudaError_t launch_pass_lean(const LeanArgs& a, bool fwd, int slice, int warps, size_t smem, cudaStream_t st);
+cudaError_t launch_pass_lean64(const LeanArgs& a, bool fwd, int slice, int warps, size_t smem, cudaStream_t st);
 
 // every kernel launch of the library goes through the wrappers below and is counted here
 void count_launches(long long n);

@@ -436,7 +436,7 @@ size_t lean_smem_bytes(const LeanPlan& plan, int slice, int warps, int depth, un
     if (stage < red) stage = up16(red);
     if (slot_stride) *slot_stride = (unsigned)slot;
     if (stage_bytes) *stage_bytes = (unsigned)stage;
-    return stage + (size_t)plan.R * (size_t)slice * 5;
+    return stage + (size_t)plan.R * (size_t)slice * (plan.wide ? 9 : 5);
 }
 
 // slice = candidates per block: 128, 64, 32 or 16 (4 candidates per lane, 1, 2, 4 or 8 vertices per warp)

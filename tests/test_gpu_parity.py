@@ -497,6 +497,73 @@ def test_lean_kernel_shapes(slice_, warps, depth, monkeypatch):
     assert took[8] and sum(took) >= 3 and not took[6], f"kernel choice per case: {took}"
 
 
+@pytest.mark.parametrize("depth", [1, 3])
+@pytest.mark.parametrize("slice_,warps", [(8, 1), (8, 8), (16, 2), (32, 4), (64, 16), (128, 8)])
+def test_lean64_kernel_shapes(slice_, warps, depth, monkeypatch):
+    """The wide lean pass (int64 levels, up to 16 devices) for every block shape: path lengths beyond 32 bits,
+    k = 9..16 with grouped tables, the cases of the narrow pass forced onto the wide kernel, zero costs, a vertex
+    of high degree, ragged candidate counts; k = 17 and tables with more than 30 bandwidths fall back."""
+    from paper_1711_01912_b200 import tfps
+    monkeypatch.setenv("TFPS_LEAN", "1")
+    monkeypatch.setenv("TFPS_LEAN_FORCE_WIDE", "1")
+    monkeypatch.setenv("TFPS_LEAN_SLICE", str(slice_))
+    monkeypatch.setenv("TFPS_SLICED_WARPS", str(warps))
+    monkeypatch.setenv("TFPS_LEAN_DEPTH", str(depth))
+    rng = np.random.default_rng(slice_ * 1000 + warps)
+    cases = []
+    for (n, m, k, P) in [(1, 0, 1, 1), (60, 150, 2, 9), (700, 2500, 16, 77), (900, 5000, 12, 130), (300, 0, 9, 33)]:
+        w = I.small_random(9500 + n + slice_, n, m, k, P, t_dtype=np.int64, with_mem=bool(n % 3))   # t up to 2^36
+        dev = w.devices if k < 4 else _grouped_devices(k, rng)
+        cases.append((w.graph, dev, w.part_full()))
+    w = I.small_random(9600 + slice_, 400, 1200, 17, 40)        # k = 17: not taken
+    cases.append((w.graph, _grouped_devices(17, rng), w.part_full()))
+    w = I.config4()
+    g = w.graph
+    keep = g.dst < 16 * 200
+    g4 = I.Graph(n=16 * 200, src=g.src[keep], dst=g.dst[keep], t=g.t[keep], c=g.c[:16 * 200], mem=None, layers=200)
+    cases.append((g4, w.devices, w.part_rows(0, 16 * 200)[:, :97]))
+    w = I.config5(layers=12, width=64, P=100)                    # k = 16, int64 path lengths, fan-in up to 64
+    cases.append((w.graph, w.devices, w.part_full()))
+    took = []
+    for g, dev, part in cases:
+        run_and_compare(g, dev, part, 2, pad_fill=255)
+        G = gpu_graph(g, dev)
+        dpart, P, ldp = padded(part)
+        G.eval_batch(dpart, P, flags=2)
+        took.append(tfps.tfps_last_pass_kernel(G.handle) == "pass_lean64_kernel")
+        G.close()
+    # the deep narrow graph always fits; k = 17 never does
+    assert took[6] and sum(took) >= 3 and not took[5], f"kernel choice per case: {took}"
+
+
+@pytest.mark.parametrize("wide", [0, 1])
+def test_lean_plan_in_callers_vertex_order(wide, monkeypatch):
+    """The lean plan walked in the caller's vertex numbering (TFPS_LEAN_ORDER=2) instead of level order: graphs
+    numbered layer by layer take it, a randomly relabelled graph is not topologically numbered and keeps the level
+    order; results are the same either way."""
+    from paper_1711_01912_b200 import tfps
+    monkeypatch.setenv("TFPS_LEAN_ORDER", "2")
+    monkeypatch.setenv("TFPS_LEAN_FORCE_WIDE", str(wide))
+    w = I.config3()
+    g = w.graph
+    keep = g.dst < 128 * 10
+    g3 = I.Graph(n=128 * 10, src=g.src[keep], dst=g.dst[keep], t=g.t[keep], c=g.c[:128 * 10], mem=None, layers=10)
+    part3 = w.part_rows(0, 128 * 10)[:, :150]
+    run_and_compare(g3, w.devices, part3, 2, pad_fill=255)
+    g3r, perm = I.relabel(g3, 5)
+    part3r = np.empty_like(part3)
+    part3r[perm] = part3
+    run_and_compare(g3r, w.devices, part3r, 2, pad_fill=255)
+    w5 = I.config5(layers=40, width=64, P=70)   # edges reach four layers back: the numbering has the shorter edges
+    dev5 = w5.devices
+    run_and_compare(w5.graph, dev5, w5.part_full(), 2, pad_fill=255)
+    w4 = I.config4()
+    g = w4.graph
+    keep = g.dst < 16 * 150
+    g4 = I.Graph(n=16 * 150, src=g.src[keep], dst=g.dst[keep], t=g.t[keep], c=g.c[:16 * 150], mem=None, layers=150)
+    run_and_compare(g4, w4.devices, w4.part_rows(0, 16 * 150)[:, :50], 2, pad_fill=255)
+
+
 def test_loads_kernel_table_widths():
     """Loads, memory loads and violation flags for every width of the runtime table (k = 1 .. 32) and beyond
     it (k = 33, 64: the shuffle-based kernel), with bounded capacities so that some flags are set."""
