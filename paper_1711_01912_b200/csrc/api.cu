@@ -110,6 +110,10 @@ struct tfps_graph {
     DBuf f_eptr, f_nbr, f_t, b_eptr, b_nbr, b_t;
     // chunk tables of the candidate-sliced pass
     DBuf vertf, f_chunks, b_chunks;
+    // work items of the tile kernel per direction: vertices with many edges cut into partial items, heaviest first
+    DBuf items[2], heavy[2];
+    std::vector<long long> h_item_ptr[2];
+    int heavy_count[2] = {0, 0};
     int f_num_chunks = 0, b_num_chunks = 0;
     bool f_all_staged = true, b_all_staged = true;
     int max_chunk_v = 1;
@@ -222,6 +226,8 @@ int upload(DBuf& buf, const std::vector<T>& v, cudaStream_t st)
     return TFPS_OK;
 }
 
+int env_int(const char* name, int dflt);
+
 int build_topo(tfps_graph* g, cudaStream_t st)
 {
     if (g->topo_built) return TFPS_OK;
@@ -316,6 +322,39 @@ int build_topo(tfps_graph* g, cudaStream_t st)
                 p = q;
             }
         }
+        {
+            // a vertex with more than 2*T edges becomes ceil(deg/T) partial items of at most T edges
+            const int T = std::max(0, env_int("TFPS_TILE_SPLIT", 8));
+            std::vector<int> items, heavy, idx;
+            std::vector<long long>& ip = g->h_item_ptr[dir];
+            ip.assign((size_t)g->num_levels + 1, 0);
+            for (int l = 0; l < g->num_levels; ++l) {
+                ip[l] = (long long)(items.size() / 4);
+                idx.clear();
+                for (int p = (int)g->h_level_ptr[l]; p < (int)g->h_level_ptr[l + 1]; ++p) idx.push_back(p);
+                std::stable_sort(idx.begin(), idx.end(), [&](int x, int y) { return eptr[x + 1] - eptr[x] > eptr[y + 1] - eptr[y]; });
+                for (int p : idx) {
+                    const int e0 = eptr[p], e1 = eptr[p + 1];
+                    if (T > 0 && e1 - e0 > 2 * T) {
+                        heavy.push_back(p);
+                        for (int e = e0; e < e1; e += T) { items.push_back(p); items.push_back(e); items.push_back(std::min(e1, e + T)); items.push_back(1); }
+                    } else {
+                        items.push_back(p); items.push_back(e0); items.push_back(e1); items.push_back(0);
+                    }
+                }
+            }
+            ip[g->num_levels] = (long long)(items.size() / 4);
+            if (!heavy.empty()) {   // positions -> vertex ids (rows of the level matrices)
+                std::vector<int> h_order((size_t)n);
+                CUDA_TRY(cudaMemcpyAsync(h_order.data(), g->order.p, sizeof(int) * (size_t)n, cudaMemcpyDeviceToHost, st));
+                CUDA_TRY(cudaStreamSynchronize(st));
+                for (int& x : heavy) x = h_order[x];
+            }
+            g->heavy_count[dir] = (int)heavy.size();
+            TFPS_TRY(upload(g->items[dir], items, st));
+            TFPS_TRY(upload(g->heavy[dir], heavy, st));
+            CUDA_TRY(cudaStreamSynchronize(st));
+        }
         (dir == 0 ? g->f_num_chunks : g->b_num_chunks) = (int)(chunks.size() / 4);
         g->h_chunks[dir] = chunks;
         TFPS_TRY(upload(dir == 0 ? g->f_chunks : g->b_chunks, chunks, st));
@@ -354,6 +393,7 @@ PassArgs make_args(const tfps_graph* g, bool fwd, long long P, long long ldp, co
     a.adj.xw = fwd ? g->xw_f.as<unsigned long long>() : g->xw_b.as<unsigned long long>();
     a.adj.xnbr = fwd ? g->xnbr_f.as<unsigned long long>() : nullptr;
     a.adj.xvert = g->xvert.as<unsigned long long>();
+    a.adj.items = g->items[fwd ? 0 : 1].as<int4>();
     a.tab = make_tables(g);
     a.level_ptr = g->level_ptr_d.as<long long>();
     a.num_levels = g->num_levels;
@@ -1364,7 +1404,13 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
                 CUDA_TRY(launch_pass_level_values(a, fwd, g->h_level_ptr, fwd ? g->V_f.as<long long>() : g->V_b.as<long long>(),
                                                   fwd ? g->cls2_f.as<uint8_t>() : g->cls2_b.as<uint8_t>(), g->ncomb, st));
             } else {
-                CUDA_TRY(launch_pass_level_sync(a, fwd, g->h_level_ptr, st));
+                {
+                    // rows of the vertices that are evaluated in partial items start at zero
+                    const int dirn = fwd ? 0 : 1;
+                    if (g->npass > 0 && g->heavy_count[dirn] > 0)
+                        CUDA_TRY(launch_zero_rows(g->heavy[dirn].as<int>(), g->heavy_count[dirn], P, ldp, lev, st));
+                    CUDA_TRY(launch_pass_level_sync(a, fwd, g->h_level_ptr, st, &g->h_item_ptr[dirn]));
+                }
             }
             if (cp_here) {
                 CUDA_TRY(cudaMemsetAsync(cp_here, 0, sizeof(long long) * (size_t)P, st));

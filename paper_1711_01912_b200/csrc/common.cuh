@@ -79,6 +79,7 @@ struct LevelAdj {
     const unsigned long long* xw;    // [m]   transfer numerator ((t*S-1)<<2 or NUM_ZERO)
     const unsigned long long* xnbr;  // [m]   neighbour's runtime numerator ((c*S-1)<<2 or NUM_ZERO)
     const unsigned long long* xvert; // [n]   own runtime numerator by position
+    const int4* items;               // work items of the tile kernel {position, first edge, end edge, partial}, by level (or NULL)
 };
 
 struct PassArgs {
@@ -214,7 +215,9 @@ cudaError_t launch_numerators(int n, int m, long long S, const int* order, const
 cudaError_t launch_default_mem(int n, const long long* out_ptr, const long long* out_t, long long* mem, cudaStream_t st);
 
 int pick_cpt(long long P);
-cudaError_t launch_pass_level_sync(const PassArgs& a, bool fwd, const std::vector<long long>& level_ptr_host, cudaStream_t st);
+cudaError_t launch_pass_level_sync(const PassArgs& a, bool fwd, const std::vector<long long>& level_ptr_host, cudaStream_t st,
+                                   const std::vector<long long>* item_ptr_host = nullptr);
+cudaError_t launch_zero_rows(const int* rows, int count, long long P, long long ldp, long long* lev, cudaStream_t st);
 cudaError_t launch_pass_level_values(const PassArgs& a, bool fwd, const std::vector<long long>& level_ptr_host,
                                      const long long* V, const uint8_t* cls2, int ncomb, cudaStream_t st);
 cudaError_t launch_pass_sliced(const PassArgs& a, bool fwd, const SlicedPlan& plan, int cpt, int warps, bool table,

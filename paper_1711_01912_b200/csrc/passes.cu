@@ -381,7 +381,20 @@ pass_tile_kernel(PassArgs a, int pos0, int count)
     bool waited = false;
 
     for (int i = blockIdx.y; i < count && live; i += gridDim.y) {
-        const VertexMeta vm = global_meta(a.adj, pos0 + i);
+        // With work items, pos0 indexes the item list: a vertex with many edges is cut into several partial items
+        // (its dependent chain of edge batches would otherwise set the duration of the whole level); partial results
+        // meet in the output row, zeroed beforehand, through 64-bit atomic maxima.
+        VertexMeta vm;
+        bool partial = false;
+        if (a.adj.items) {
+            const int4 it = a.adj.items[pos0 + i];
+            vm = global_meta(a.adj, it.x);
+            vm.e0 = it.y;
+            vm.e1 = it.z;
+            partial = it.w != 0;
+        } else {
+            vm = global_meta(a.adj, pos0 + i);
+        }
         unsigned pv[IdWords<CPT>::N];
         load_ids_masked<CPT>(a.part + (long long)vm.v * ldp + lc.jl, lc, pv);
         long long best[CPT];
@@ -425,7 +438,13 @@ pass_tile_kernel(PassArgs a, int pos0, int count)
                 if (vm.xvert != NUM_ZERO) best[c] = ceil_quot(vm.xvert, tc.s_rt[id_at<CPT>(pv, c)]);
         }
         if (!waited) { grid_dependency_wait(); waited = true; }
-        store_levels<CPT>(a.lev + (long long)vm.v * ldp + lc.jl, best, lc.nvalid);
+        if (partial) {
+#pragma unroll
+            for (int c = 0; c < CPT; ++c)
+                if (c < lc.nvalid) atomicMax(a.lev + (long long)vm.v * ldp + lc.jl + c, best[c]);
+        } else {
+            store_levels<CPT>(a.lev + (long long)vm.v * ldp + lc.jl, best, lc.nvalid);
+        }
         if (i + (int)gridDim.y < count) __syncthreads();  // tables are reused by the next vertex
     }
     if (!waited) grid_dependency_wait();
@@ -877,6 +896,13 @@ static cudaError_t level_sync_impl(const PassArgs& a, const std::vector<long lon
     return cudaGetLastError();
 }
 
+__global__ void zero_rows_kernel(const int* __restrict__ rows, long long P, long long ldp, long long* lev)
+{
+    const long long j = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (j < P) lev[(long long)rows[blockIdx.y] * ldp + j] = 0;
+}
+
+// lp: level pointers over positions, or over work items when the pass has them
 template <int CPT, bool FWD>
 static cudaError_t tile_impl(const PassArgs& a, const std::vector<long long>& lp, cudaStream_t st)
 {
@@ -947,8 +973,25 @@ cudaError_t launch_pass_level_values(const PassArgs& a, bool fwd, const std::vec
     return fwd ? levelv_impl<1, true>(a, lp, V, cls2, ncomb, st) : levelv_impl<1, false>(a, lp, V, cls2, ncomb, st);
 }
 
-cudaError_t launch_pass_level_sync(const PassArgs& a, bool fwd, const std::vector<long long>& lp, cudaStream_t st)
+cudaError_t launch_zero_rows(const int* rows, int count, long long P, long long ldp, long long* lev, cudaStream_t st)
 {
+    if (count <= 0 || P <= 0) return cudaSuccess;
+    for (int r0 = 0; r0 < count; r0 += 65535) {
+        const int c = count - r0 < 65535 ? count - r0 : 65535;
+        zero_rows_kernel<<<dim3(cdivu(P, 256), (unsigned)c), 256, 0, st>>>(rows + r0, P, ldp, lev);
+    }
+    count_launches((count + 65534) / 65535);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_pass_level_sync(const PassArgs& a0, bool fwd, const std::vector<long long>& lp0, cudaStream_t st,
+                                   const std::vector<long long>* item_ptr)
+{
+    // work items belong to the tile kernel; the other level kernels walk positions
+    PassArgs a = a0;
+    const bool use_items = a.tab.npass > 0 && a.adj.items != nullptr && item_ptr != nullptr;
+    if (!use_items) a.adj.items = nullptr;
+    const std::vector<long long>& lp = use_items ? *item_ptr : lp0;
     if (a.tab.npass > 0) {  // block-shared cost tables
         const char* ov = getenv("TFPS_TILE_CPT");  // tuning override
         if (ov && *ov == '4') return fwd ? tile_impl<4, true>(a, lp, st) : tile_impl<4, false>(a, lp, st);
