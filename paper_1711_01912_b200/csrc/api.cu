@@ -113,6 +113,7 @@ struct tfps_graph {
     // work items of the tile kernel per direction: vertices with many edges cut into partial items, heaviest first
     DBuf items[2], heavy[2];
     std::vector<long long> h_item_ptr[2];
+    std::vector<int> h_items[2];
     int heavy_count[2] = {0, 0};
     int f_num_chunks = 0, b_num_chunks = 0;
     bool f_all_staged = true, b_all_staged = true;
@@ -143,6 +144,12 @@ struct tfps_graph {
         DBuf blob, desc, vlist;
         LeanPlan plan;
     } lean[2];
+    // level-synchronous pass on vertex records (0 forward, 1 backward)
+    struct LevRec {
+        bool ok = false;
+        DBuf blob, roff, items;
+        LevRecArgs args;
+    } levrec[2];
     DBuf status;
     // scratch owned by the handle
     DBuf scr_memload;
@@ -351,6 +358,7 @@ int build_topo(tfps_graph* g, cudaStream_t st)
                 for (int& x : heavy) x = h_order[x];
             }
             g->heavy_count[dir] = (int)heavy.size();
+            g->h_items[dir] = items;
             TFPS_TRY(upload(g->items[dir], items, st));
             TFPS_TRY(upload(g->heavy[dir], heavy, st));
             CUDA_TRY(cudaStreamSynchronize(st));
@@ -682,6 +690,112 @@ int build_lean(tfps_graph* g, int k, const int32_t* s, const int64_t* B, long lo
                 unsigned long long row = 0;
                 for (int b = 0; b < 8; ++b) row |= (unsigned long long)(8 * link(8 * h + b, pv)) << (8 * b);
                 L.plan.rows16[2 * pv + h] = row;
+            }
+        L.ok = true;
+    }
+    return TFPS_OK;
+}
+
+// Packs the vertex records of the level-synchronous record pass (layout: levrec.cu) for both directions.
+int build_levrec(tfps_graph* g, int k, const int32_t* s, const int64_t* B, long long S, const std::vector<int>& order,
+                 cudaStream_t st)
+{
+    for (auto& L : g->levrec) L.ok = false;
+    const int n = (int)g->n, m = (int)g->m;
+    if (n == 0 || k > LEAN64_K_MAX || env_int("TFPS_LEVREC", 1) == 0) return TFPS_OK;
+    std::vector<long long> wvals;
+    auto cls_of = [&](long long x) {
+        for (size_t i = 0; i < wvals.size(); ++i)
+            if (wvals[i] == x) return (int)i;
+        wvals.push_back(x);
+        return (int)wvals.size() - 1;
+    };
+    long long s_min = INT64_MAX;
+    for (int a = 0; a < k; ++a) {
+        s_min = std::min<long long>(s_min, s[a]);
+        for (int b = 0; b < k; ++b)
+            if (a != b) cls_of(B[a * k + b]);
+    }
+    const int ncw = (int)wvals.size();
+    const u128 rt_max = ((u128)g->max_c * (u128)S + (u128)s_min - 1) / (u128)s_min;
+    if (ncw > LEAN_CLS_MAX || rt_max >= ((u128)1 << 31)) return TFPS_OK;
+    auto ceil_div = [](long long a, long long S_, long long d) {
+        return (long long)(((u128)a * (u128)S_ + (u128)d - 1) / (u128)d);
+    };
+    const int wbytes = 8 * (ncw + 1);
+    for (int dir = 0; dir < 2; ++dir) {
+        tfps_graph::LevRec& L = g->levrec[dir];
+        std::vector<int> ep((size_t)n + 1), nb((size_t)m);
+        std::vector<long long> tt((size_t)m);
+        CUDA_TRY(cudaMemcpyAsync(ep.data(), dir == 0 ? g->f_eptr.p : g->b_eptr.p, sizeof(int) * ((size_t)n + 1), cudaMemcpyDeviceToHost, st));
+        if (m > 0) {
+            CUDA_TRY(cudaMemcpyAsync(nb.data(), dir == 0 ? g->f_nbr.p : g->b_nbr.p, sizeof(int) * (size_t)m, cudaMemcpyDeviceToHost, st));
+            CUDA_TRY(cudaMemcpyAsync(tt.data(), dir == 0 ? g->f_t.p : g->b_t.p, sizeof(long long) * (size_t)m, cudaMemcpyDeviceToHost, st));
+        }
+        CUDA_TRY(cudaStreamSynchronize(st));
+        const int estride = 8 + wbytes + (dir == 0 ? 64 : 0);
+        // work items: the tile kernel's, with edges counted from the vertex' first edge
+        std::vector<int> items = g->h_items[dir];
+        int item_edges = 0;
+        for (size_t i = 0; i + 3 < items.size(); i += 4) {
+            const int p = items[i];
+            items[i + 1] -= ep[p];
+            items[i + 2] -= ep[p];
+            item_edges = std::max(item_edges, items[i + 2] - items[i + 1]);
+        }
+        const long long smem_need = 80 + (long long)item_edges * estride;
+        if (smem_need > 48 * 1024) continue;   // an unsplit vertex with too many edges
+        std::vector<long long> roff((size_t)n + 1);
+        size_t total = 0;   // in units of 16 bytes
+        for (int p = 0; p < n; ++p) {
+            roff[p] = (long long)total;
+            total += (16 + 64 + (size_t)(ep[p + 1] - ep[p]) * estride + 15) / 16;
+        }
+        roff[n] = (long long)total;
+        if (total * 16 >= ((size_t)1 << 34)) continue;
+        std::vector<unsigned char> blob(total * 16, 0);
+        for (int p = 0; p < n; ++p) {
+            unsigned char* r = blob.data() + (size_t)roff[p] * 16;
+            const int v = order[p], d = ep[p + 1] - ep[p];
+            int* hdr = reinterpret_cast<int*>(r);
+            hdr[0] = v;
+            hdr[1] = d;
+            for (int q = 0; q < k; ++q) hdr[4 + q] = (int)ceil_div(g->h_c[v], S, s[q]);
+            for (int e = 0; e < d; ++e) {
+                unsigned char* er = r + 80 + (size_t)e * estride;
+                const int u = nb[(size_t)ep[p] + e];
+                memcpy(er, &u, 4);
+                for (int w = 0; w < ncw; ++w) {
+                    const long long val = ceil_div(tt[(size_t)ep[p] + e], S, wvals[w]);
+                    memcpy(er + 16 + 8 * w, &val, 8);   // {neighbour, pad, W[0] = 0, W[1..]}
+                }
+                if (dir == 0)
+                    for (int q = 0; q < k; ++q) {
+                        const int rtu = (int)ceil_div(g->h_c[u], S, s[q]);
+                        memcpy(er + 8 + wbytes + 4 * q, &rtu, 4);
+                    }
+            }
+        }
+        TFPS_TRY(upload(L.blob, blob, st));
+        TFPS_TRY(upload(L.roff, roff, st));
+        TFPS_TRY(upload(L.items, items, st));
+        CUDA_TRY(cudaStreamSynchronize(st));
+        L.args.blob = L.blob.as<unsigned char>();
+        L.args.roff = L.roff.as<long long>();
+        L.args.items = L.items.as<int4>();
+        L.args.estride = estride;
+        L.args.wbytes = wbytes;
+        L.args.rec_max = (int)((smem_need + 15) & ~15LL);
+        for (int pv = 0; pv < LEAN64_K_MAX; ++pv)
+            for (int h = 0; h < 2; ++h) {
+                unsigned long long row = 0;
+                for (int b = 0; b < 8; ++b) {
+                    const int pu = 8 * h + b;
+                    int cls = 0;
+                    if (pv < k && pu < k && pu != pv) cls = cls_of(dir == 0 ? B[pu * k + pv] : B[pv * k + pu]) + 1;
+                    row |= (unsigned long long)(8 * cls) << (8 * b);
+                }
+                L.args.rows16[2 * pv + h] = row;
             }
         L.ok = true;
     }
@@ -1031,6 +1145,7 @@ int tfps_devices_set(tfps_graph* g, int k, const int32_t* s, const int64_t* C, c
         }
         g->fits32 = worst < (1LL << 31) - 1;
         TFPS_TRY(build_lean(g, k, s, B, scale, order, st));
+        TFPS_TRY(build_levrec(g, k, s, B, scale, order, st));
     }
     if (g->ncomb > 0 && n > 0) {
         CUDA_TRY(g->V_f.reserve(sizeof(long long) * (size_t)m * g->ncomb + 16));
@@ -1407,9 +1522,21 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
                 {
                     // rows of the vertices that are evaluated in partial items start at zero
                     const int dirn = fwd ? 0 : 1;
-                    if (g->npass > 0 && g->heavy_count[dirn] > 0)
+                    const bool rec = g->levrec[dirn].ok && ((uintptr_t)part & 3u) == 0 && env_int("TFPS_LEVREC", 1) != 0;
+                    if ((g->npass > 0 || rec) && g->heavy_count[dirn] > 0)
                         CUDA_TRY(launch_zero_rows(g->heavy[dirn].as<int>(), g->heavy_count[dirn], P, ldp, lev, st));
-                    CUDA_TRY(launch_pass_level_sync(a, fwd, g->h_level_ptr, st, &g->h_item_ptr[dirn]));
+                    if (rec) {   // vertex records (k <= 16): no divisions or per-edge tables in the kernel
+                        LevRecArgs la = g->levrec[dirn].args;
+                        la.part = part;
+                        la.lev = lev;
+                        la.status = status;
+                        la.P = P;
+                        la.ldp = ldp;
+                        g->last_kernel = "pass_levrec_kernel";
+                        CUDA_TRY(launch_pass_levrec(la, fwd, g->h_item_ptr[dirn], g->num_levels, st));
+                    } else {
+                        CUDA_TRY(launch_pass_level_sync(a, fwd, g->h_level_ptr, st, &g->h_item_ptr[dirn]));
+                    }
                 }
             }
             if (cp_here) {

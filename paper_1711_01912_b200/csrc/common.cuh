@@ -193,6 +193,23 @@ struct LeanArgs {
     unsigned stage_bytes;        // bytes reserved for all stage slots (also the CP reduction buffer)
 };
 
+// Level-synchronous pass on host-packed vertex records (levrec.cu).
+struct LevRecArgs {
+    const uint8_t* part;
+    long long* lev;
+    int* status;
+    long long P, ldp;
+    const unsigned char* blob;   // records, 16-byte aligned
+    const long long* roff;       // [n+1] record offsets by level position, in units of 16 bytes
+    const int4* items;           // work items {level position, first edge within the record, end edge, partial}, by level
+    int estride;                 // bytes of an edge entry
+    int wbytes;                  // bytes of the transfer times of an edge entry: 8 * (classes + 1)
+    int rec_max;                 // shared memory per block: header, runtimes and the edges of the largest item
+    unsigned long long rows16[2 * 16];   // byte [pv][pu] = 8 * class of the link
+};
+cudaError_t launch_pass_levrec(const LevRecArgs& a, bool fwd, const std::vector<long long>& item_ptr_host, int num_levels,
+                               cudaStream_t st);
+
 size_t lean_smem_bytes(const LeanPlan& plan, int slice, int warps, int depth, unsigned* slot_stride, unsigned* stage_bytes);
 cudaError_t launch_pass_lean(const LeanArgs& a, bool fwd, int slice, int warps, size_t smem, cudaStream_t st);
 cudaError_t launch_pass_lean64(const LeanArgs& a, bool fwd, int slice, int warps, size_t smem, cudaStream_t st);
