@@ -147,7 +147,7 @@ struct tfps_graph {
     // level-synchronous pass on vertex records (0 forward, 1 backward)
     struct LevRec {
         bool ok = false;
-        DBuf blob, roff, items;
+        DBuf blob, items;
         LevRecArgs args;
     } levrec[2];
     DBuf status;
@@ -735,14 +735,9 @@ int build_levrec(tfps_graph* g, int k, const int32_t* s, const int64_t* B, long 
         CUDA_TRY(cudaStreamSynchronize(st));
         const int estride = 8 + wbytes + (dir == 0 ? 64 : 0);
         // work items: the tile kernel's, with edges counted from the vertex' first edge
-        std::vector<int> items = g->h_items[dir];
+        const std::vector<int>& titems = g->h_items[dir];   // {position, first edge, end edge, partial}
         int item_edges = 0;
-        for (size_t i = 0; i + 3 < items.size(); i += 4) {
-            const int p = items[i];
-            items[i + 1] -= ep[p];
-            items[i + 2] -= ep[p];
-            item_edges = std::max(item_edges, items[i + 2] - items[i + 1]);
-        }
+        for (size_t i = 0; i + 3 < titems.size(); i += 4) item_edges = std::max(item_edges, titems[i + 2] - titems[i + 1]);
         const long long smem_need = 80 + (long long)item_edges * estride;
         if (smem_need > 48 * 1024) continue;   // an unsplit vertex with too many edges
         std::vector<long long> roff((size_t)n + 1);
@@ -752,7 +747,16 @@ int build_levrec(tfps_graph* g, int k, const int32_t* s, const int64_t* B, long 
             total += (16 + 64 + (size_t)(ep[p + 1] - ep[p]) * estride + 15) / 16;
         }
         roff[n] = (long long)total;
-        if (total * 16 >= ((size_t)1 << 34)) continue;
+        if (total >= ((size_t)1 << 31)) continue;
+        // {vertex | partial << 31, record offset / 16, first edge within the record, end edge}
+        std::vector<int> items(titems.size());
+        for (size_t i = 0; i + 3 < titems.size(); i += 4) {
+            const int p = titems[i];
+            items[i] = order[p] | (titems[i + 3] ? (int)0x80000000u : 0);
+            items[i + 1] = (int)roff[p];
+            items[i + 2] = titems[i + 1] - ep[p];
+            items[i + 3] = titems[i + 2] - ep[p];
+        }
         std::vector<unsigned char> blob(total * 16, 0);
         for (int p = 0; p < n; ++p) {
             unsigned char* r = blob.data() + (size_t)roff[p] * 16;
@@ -777,11 +781,9 @@ int build_levrec(tfps_graph* g, int k, const int32_t* s, const int64_t* B, long 
             }
         }
         TFPS_TRY(upload(L.blob, blob, st));
-        TFPS_TRY(upload(L.roff, roff, st));
         TFPS_TRY(upload(L.items, items, st));
         CUDA_TRY(cudaStreamSynchronize(st));
         L.args.blob = L.blob.as<unsigned char>();
-        L.args.roff = L.roff.as<long long>();
         L.args.items = L.items.as<int4>();
         L.args.estride = estride;
         L.args.wbytes = wbytes;

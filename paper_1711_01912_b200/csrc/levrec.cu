@@ -25,7 +25,8 @@ __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddep
 // record of a vertex (16-byte aligned, a multiple of 16 bytes):
 //   int4 {vertex, edges, 0, 0}; int rt[16]; then per edge estride bytes:
 //   {int neighbour, int pad, long long W[0..ncls] (W[0] = 0), forward only: int rtu[16]}
-// item: {level position, first edge within the record, end edge, partial}
+// item: {vertex | partial << 31, record offset / 16, first edge within the record, end edge}: everything a block
+// needs to start the record copy and the read of its own ids at once
 template <bool FWD>
 __global__ void __launch_bounds__(LEVREC_WARPS * 32)
 pass_levrec_kernel(LevRecArgs a, int item0, int count)
@@ -45,22 +46,23 @@ pass_levrec_kernel(LevRecArgs a, int item0, int count)
     bool waited = false;
 
     for (int i = blockIdx.y; i < count && live; i += gridDim.y) {
-        const int4 it = a.items[item0 + i];
-        const int deg = it.z - it.y;
-        const unsigned char* rec = a.blob + 16ll * a.roff[it.x];
+        const int4 it = __ldg(a.items + item0 + i);
+        const int deg = it.w - it.z;
+        const int v = it.x & 0x7fffffff;
+        const unsigned char* rec = a.blob + 16ll * (unsigned)it.y;
+        // own ids: requested before the record arrives
+        const unsigned ids = *reinterpret_cast<const unsigned*>(a.part + (long long)v * ldp + jl) & 0x0f0f0f0fu;
         if (i != (int)blockIdx.y) __syncthreads();   // the previous item's record is no longer read
         // header + runtimes (80 bytes), then the item's edges (estride is a multiple of 8)
         for (int q = tid; q < 5; q += LEVREC_WARPS * 32) reinterpret_cast<uint4*>(s_rec)[q] = __ldg(reinterpret_cast<const uint4*>(rec) + q);
         {
-            const unsigned long long* src = reinterpret_cast<const unsigned long long*>(rec + 80 + (size_t)it.y * estride);
+            const unsigned long long* src = reinterpret_cast<const unsigned long long*>(rec + 80 + (size_t)it.z * estride);
             unsigned long long* dst = reinterpret_cast<unsigned long long*>(s_rec + 80);
             for (int q = tid; q < deg * (estride >> 3); q += LEVREC_WARPS * 32) dst[q] = __ldg(src + q);
         }
         __syncthreads();
-        const int v = reinterpret_cast<const int*>(s_rec)[0];
         const int* rtv = reinterpret_cast<const int*>(s_rec + 16);
         const unsigned char* edges = s_rec + 80;
-        const unsigned ids = *reinterpret_cast<const unsigned*>(a.part + (long long)v * ldp + jl) & 0x0f0f0f0fu;
         const unsigned char* row[4];
         long long best[4];
 #pragma unroll
@@ -110,7 +112,7 @@ pass_levrec_kernel(LevRecArgs a, int item0, int count)
         }
         if (!waited) { grid_dependency_wait(); waited = true; }
         long long* out = a.lev + (long long)v * ldp + j0;
-        if (it.w != 0) {
+        if (it.x < 0) {   // partial item
 #pragma unroll
             for (int c = 0; c < 4; ++c)
                 if (c < nvalid) atomicMax(out + c, best[c]);
