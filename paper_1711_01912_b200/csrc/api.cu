@@ -1401,6 +1401,13 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
     LeanChoice lean_f, lean_b;
     if (need_fwd) lean_f = pick_lean(true);
     if (need_bwd) lean_b = pick_lean(false);
+    // Automatic choice: a graph whose window does not fit (no lean pass) but whose levels are wide is better served
+    // by the level-synchronous record pass than by a sliced kernel that reads its neighbours through L2.
+    if (!(flags & (TFPS_EVAL_SLICED | TFPS_EVAL_LEVEL_SYNC)) && sliced && !((!need_fwd || lean_f.ok) && (!need_bwd || lean_b.ok)) &&
+        g->levrec[0].ok && g->levrec[1].ok && env_int("TFPS_LEVREC", 1) != 0) {
+        const long long avg_width = g->num_levels > 0 ? g->n / g->num_levels : g->n;
+        if (avg_width * P >= (1LL << 18)) { sliced = false; lean_f.ok = false; lean_b.ok = false; }
+    }
     // The lean passes cannot leave their tables on a bad id (ids are masked), so the id check need not come first:
     // the loads kernel then runs on a low-priority stream beside them and fills the SMs the passes' last wave leaves idle.
     const bool overlap = (load || ml) && (need_fwd || need_bwd) && (!need_fwd || lean_f.ok) && (!need_bwd || lean_b.ok) &&

@@ -564,6 +564,31 @@ def test_lean_plan_in_callers_vertex_order(wide, monkeypatch):
     run_and_compare(g4, w4.devices, w4.part_rows(0, 16 * 150)[:, :50], 2, pad_fill=255)
 
 
+@pytest.mark.parametrize("levrec", [0, 1])
+@pytest.mark.parametrize("split", [0, 3, 8])
+def test_level_kernels_with_partial_items(split, levrec, monkeypatch):
+    """The level-synchronous kernels (record pass and tile kernel) with vertices of many edges cut into partial
+    work items of at most `split` edges (0: never): a hub with hundreds of in-edges next to vertices of degree one,
+    the power-law fan-in graph with k = 16, a graph with k = 17 (per-relaxation division kernel, no items)."""
+    from paper_1711_01912_b200 import tfps
+    monkeypatch.setenv("TFPS_TILE_SPLIT", str(split))
+    monkeypatch.setenv("TFPS_LEVREC", str(levrec))
+    rng = np.random.default_rng(77 + split)
+    n = 700
+    edges = [(u, n - 1, int(rng.integers(0, 10 ** 6))) for u in range(n - 1)] + [(0, u, 5) for u in range(1, 60)]
+    gh = graph_from_edges(n, edges, rng.integers(0, 100, size=n))
+    run_and_compare(gh, _grouped_devices(4, rng), rng.integers(0, 4, size=(n, 45), dtype=np.uint8), 1, pad_fill=255)
+    w = I.config5(layers=14, width=64, P=130)
+    out = run_and_compare(w.graph, w.devices, w.part_full(), 1, pad_fill=255)
+    G = gpu_graph(w.graph, w.devices)
+    dpart, P, ldp = padded(w.part_full())
+    G.eval_batch(dpart, P, flags=1)
+    assert tfps.tfps_last_pass_kernel(G.handle) == ("pass_levrec_kernel" if levrec else "pass_tile_kernel")
+    G.close()
+    w = I.small_random(4242 + split, 500, 3000, 17, 40)
+    run_and_compare(w.graph, w.devices, w.part_full(), 1, pad_fill=255)
+
+
 def test_loads_kernel_table_widths():
     """Loads, memory loads and violation flags for every width of the runtime table (k = 1 .. 32) and beyond
     it (k = 33, 64: the shuffle-based kernel), with bounded capacities so that some flags are set."""
