@@ -749,13 +749,15 @@ int build_levrec(tfps_graph* g, int k, const int32_t* s, const int64_t* B, long 
         roff[n] = (long long)total;
         if (total >= ((size_t)1 << 31)) continue;
         // {vertex | partial << 31, record offset / 16, first edge within the record, end edge}
-        std::vector<int> items(titems.size());
+        //   and the neighbours of the item's first four edges
+        std::vector<int> items(2 * titems.size(), 0);
         for (size_t i = 0; i + 3 < titems.size(); i += 4) {
             const int p = titems[i];
-            items[i] = order[p] | (titems[i + 3] ? (int)0x80000000u : 0);
-            items[i + 1] = (int)roff[p];
-            items[i + 2] = titems[i + 1] - ep[p];
-            items[i + 3] = titems[i + 2] - ep[p];
+            items[2 * i] = order[p] | (titems[i + 3] ? (int)0x80000000u : 0);
+            items[2 * i + 1] = (int)roff[p];
+            items[2 * i + 2] = titems[i + 1] - ep[p];
+            items[2 * i + 3] = titems[i + 2] - ep[p];
+            for (int q = 0; q < 4 && titems[i + 1] + q < titems[i + 2]; ++q) items[2 * i + 4 + q] = nb[(size_t)titems[i + 1] + q];
         }
         std::vector<unsigned char> blob(total * 16, 0);
         for (int p = 0; p < n; ++p) {

@@ -200,7 +200,8 @@ struct LevRecArgs {
     int* status;
     long long P, ldp;
     const unsigned char* blob;   // records, 16-byte aligned
-    const int4* items;           // work items {vertex | partial << 31, record offset / 16, first edge within the record, end edge}, by level
+    const int4* items;           // work items, two int4 each: {vertex | partial << 31, record offset / 16, first edge within the
+                                 // record, end edge}, {neighbours of the item's first four edges}; by level
     int estride;                 // bytes of an edge entry
     int wbytes;                  // bytes of the transfer times of an edge entry: 8 * (classes + 1)
     int rec_max;                 // shared memory per block: header, runtimes and the edges of the largest item

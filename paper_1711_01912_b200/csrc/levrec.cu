@@ -25,8 +25,9 @@ __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddep
 // record of a vertex (16-byte aligned, a multiple of 16 bytes):
 //   int4 {vertex, edges, 0, 0}; int rt[16]; then per edge estride bytes:
 //   {int neighbour, int pad, long long W[0..ncls] (W[0] = 0), forward only: int rtu[16]}
-// item: {vertex | partial << 31, record offset / 16, first edge within the record, end edge}: everything a block
-// needs to start the record copy and the read of its own ids at once
+// item (two int4): {vertex | partial << 31, record offset / 16, first edge within the record, end edge} and the
+// neighbours of its first four edges: everything a block needs to start the record copy, the read of its own ids
+// and the reads of the first neighbours' ids at once
 template <bool FWD>
 __global__ void __launch_bounds__(LEVREC_WARPS * 32)
 pass_levrec_kernel(LevRecArgs a, int item0, int count)
@@ -46,12 +47,26 @@ pass_levrec_kernel(LevRecArgs a, int item0, int count)
     bool waited = false;
 
     for (int i = blockIdx.y; i < count && live; i += gridDim.y) {
-        const int4 it = __ldg(a.items + item0 + i);
+        const int4 it = __ldg(a.items + 2 * (item0 + i));
+        const int4 nb4 = __ldg(a.items + 2 * (item0 + i) + 1);
         const int deg = it.w - it.z;
         const int v = it.x & 0x7fffffff;
         const unsigned char* rec = a.blob + 16ll * (unsigned)it.y;
         // own ids: requested before the record arrives
         const unsigned ids = *reinterpret_cast<const unsigned*>(a.part + (long long)v * ldp + jl) & 0x0f0f0f0fu;
+        // ids of the first four neighbours: their vertices come with the item, not with the record
+        long long off[LEVREC_EB];
+        unsigned pu[LEVREC_EB];
+        {
+            const int nbv[4] = {nb4.x, nb4.y, nb4.z, nb4.w};
+#pragma unroll
+            for (int q = 0; q < LEVREC_EB; ++q) {
+                if (q < deg) {
+                    off[q] = (long long)nbv[q] * ldp + jl;
+                    pu[q] = *reinterpret_cast<const unsigned*>(a.part + off[q]) & 0x0f0f0f0fu;
+                }
+            }
+        }
         if (i != (int)blockIdx.y) __syncthreads();   // the previous item's record is no longer read
         // header + runtimes (80 bytes), then the item's edges (estride is a multiple of 8)
         for (int q = tid; q < 5; q += LEVREC_WARPS * 32) reinterpret_cast<uint4*>(s_rec)[q] = __ldg(reinterpret_cast<const uint4*>(rec) + q);
@@ -72,11 +87,9 @@ pass_levrec_kernel(LevRecArgs a, int item0, int count)
         }
         for (int b0 = 0; b0 < deg; b0 += LEVREC_EB) {
             const int nb = deg - b0 < LEVREC_EB ? deg - b0 : LEVREC_EB;
-            long long off[LEVREC_EB];
-            unsigned pu[LEVREC_EB];
 #pragma unroll
             for (int q = 0; q < LEVREC_EB; ++q) {
-                if (q < nb) {
+                if (b0 > 0 && q < nb) {
                     off[q] = (long long)*reinterpret_cast<const int*>(edges + (size_t)(b0 + q) * estride) * ldp + jl;
                     pu[q] = *reinterpret_cast<const unsigned*>(a.part + off[q]) & 0x0f0f0f0fu;
                 }
