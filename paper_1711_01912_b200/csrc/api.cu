@@ -477,6 +477,7 @@ int build_lean(tfps_graph* g, int k, const int32_t* s, const int64_t* B, long lo
     }
     CUDA_TRY(cudaStreamSynchronize(st));
     auto ceil_div = [](long long a, long long S_, long long d) {
+        if (a <= (LIMIT62 / S_)) return (a * S_ + d - 1) / d;   // 64-bit arithmetic suffices (d < 2^62)
         return (long long)(((u128)a * (u128)S_ + (u128)d - 1) / (u128)d);
     };
 
@@ -585,6 +586,13 @@ int build_lean(tfps_graph* g, int k, const int32_t* s, const int64_t* B, long lo
         // window rows: every position written while a record is processed must leave its readers' neighbours intact
         int R = span + max_rec_v;
         if (!wide) { R = 1; while (R < span + max_rec_v) R <<= 1; }
+        {
+            // a plan whose window cannot fit beside one stage slot at the narrowest block the library picks by itself is not
+            // packed (narrower blocks of the wide kernel: only on request, TFPS_LEAN_SLICE)
+            const int fs = env_int("TFPS_LEAN_SLICE", 0);
+            const int slice_min = wide ? ((fs == 8 || fs == 16) ? fs : 32) : 16;
+            if ((long long)R * slice_min * (wide ? 9 : 5) + 16 * 1024 > (long long)g->smem_optin) continue;
+        }
         const int nc = (int)rec_c0.size();
         std::vector<int> desc((size_t)(nc + 2 * LEAN_DEPTH_MAX) * 4, 0), vlist((size_t)n);
         std::vector<unsigned char> blob;
@@ -720,9 +728,13 @@ int build_levrec(tfps_graph* g, int k, const int32_t* s, const int64_t* B, long 
     const u128 rt_max = ((u128)g->max_c * (u128)S + (u128)s_min - 1) / (u128)s_min;
     if (ncw > LEAN_CLS_MAX || rt_max >= ((u128)1 << 31)) return TFPS_OK;
     auto ceil_div = [](long long a, long long S_, long long d) {
+        if (a <= (LIMIT62 / S_)) return (a * S_ + d - 1) / d;   // 64-bit arithmetic suffices (d < 2^62)
         return (long long)(((u128)a * (u128)S_ + (u128)d - 1) / (u128)d);
     };
     const int wbytes = 8 * (ncw + 1);
+    std::vector<int> rtab((size_t)n * k);   // runtime of every vertex on every device
+    for (int v = 0; v < n; ++v)
+        for (int q = 0; q < k; ++q) rtab[(size_t)v * k + q] = (int)ceil_div(g->h_c[v], S, s[q]);
     for (int dir = 0; dir < 2; ++dir) {
         tfps_graph::LevRec& L = g->levrec[dir];
         std::vector<int> ep((size_t)n + 1), nb((size_t)m);
@@ -766,7 +778,7 @@ int build_levrec(tfps_graph* g, int k, const int32_t* s, const int64_t* B, long 
             int* hdr = reinterpret_cast<int*>(r);
             hdr[0] = v;
             hdr[1] = d;
-            for (int q = 0; q < k; ++q) hdr[4 + q] = (int)ceil_div(g->h_c[v], S, s[q]);
+            memcpy(hdr + 4, &rtab[(size_t)v * k], sizeof(int) * (size_t)k);
             for (int e = 0; e < d; ++e) {
                 unsigned char* er = r + 80 + (size_t)e * estride;
                 const int u = nb[(size_t)ep[p] + e];
@@ -775,11 +787,7 @@ int build_levrec(tfps_graph* g, int k, const int32_t* s, const int64_t* B, long 
                     const long long val = ceil_div(tt[(size_t)ep[p] + e], S, wvals[w]);
                     memcpy(er + 16 + 8 * w, &val, 8);   // {neighbour, pad, W[0] = 0, W[1..]}
                 }
-                if (dir == 0)
-                    for (int q = 0; q < k; ++q) {
-                        const int rtu = (int)ceil_div(g->h_c[u], S, s[q]);
-                        memcpy(er + 8 + wbytes + 4 * q, &rtu, 4);
-                    }
+                if (dir == 0) memcpy(er + 8 + wbytes, &rtab[(size_t)u * k], sizeof(int) * (size_t)k);
             }
         }
         TFPS_TRY(upload(L.blob, blob, st));

@@ -4,17 +4,18 @@
 // keeps the levels of the last R positions of its own candidates in a shared-memory ring, so only the
 // compulsory traffic -- one id read and one level write per vertex-candidate -- reaches global memory), cut
 // down to the instructions the recurrences need:
-//   * the host packs one record per chunk (LeanPlan): vertices in processing order (highest degree first, dealt
+//   * the host packs records of one or more consecutive chunks (LeanPlan; narrow levels share a record, with a
+//     block barrier between its chunks): vertices in processing order (highest degree first, dealt
 //     to the vertex groups in alternating direction, so a fixed assignment is balanced), per-vertex runtimes for
 //     every device, and per-edge transfer times for every distinct bandwidth;
 //   * the window keeps finish times tlevel+rt (forward) or bottom levels (backward, Eq. 12), so a relaxation
 //     only adds the transfer term: one byte permute maps the neighbour's device id to the offset of the right
 //     transfer time inside the edge record, one shared-memory load fetches it, one add-max folds it in;
 //   * all shared-memory traffic uses 32-bit shared-window addresses;
-//   * every warp consumes; the copies of the chunk `depth` ahead (one bulk copy for the record, 16-byte
-//     cp.async pieces for the id rows) are issued by all threads right after the chunk barrier; the descriptor
+//   * every warp consumes; the copies of the record `depth` ahead (one bulk copy for the record, 16-byte
+//     cp.async pieces for the id rows) are issued by all threads right after the record's last barrier; the descriptor
 //     comes from the header of the current record, the vertex ids of the id rows are requested at the top of
-//     the chunk and first touched after the barrier.
+//     the record and first touched after that barrier.
 // Requirements (checked by the host): every path length fits int32, k <= 8, at most 30 distinct off-diagonal
 // bandwidths, the whole window fits in shared memory beside the stage slots.
 #include "common.cuh"
