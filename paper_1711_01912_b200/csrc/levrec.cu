@@ -5,7 +5,7 @@
 // vertex, or a run of the edges of a vertex with many edges) and LEVREC_WARPS * 128 candidates: it copies the
 // vertex' record into shared memory once (its runtimes on every device; per edge the neighbour, the transfer time
 // for every distinct bandwidth and, forward, the neighbour's runtimes on every device), then every warp relaxes its
-// own 128 candidates: the neighbour's id and level come from global memory (four edges in flight), the class of the
+// own 128 candidates: the neighbour's id and level come from global memory (two edges in flight), the class of the
 // link from a 16 x 16 byte table, transfer time and neighbour runtime from the record.  No division, no per-edge
 // table, one block barrier.  Partial items meet in the output row (zeroed beforehand) through 64-bit atomic maxima.
 //   forward:  tlevel(v) = max over in-edges  of tlevel(u) + rt(u, p(u)) + w(u -> v)        (0 for sources)
@@ -17,7 +17,11 @@ namespace tfps {
 namespace {
 
 constexpr int LEVREC_WARPS = 8;
-constexpr int LEVREC_EB = 4;   // edges in flight per warp
+// Edges in flight per thread and resident blocks per SM.  Most vertices have one or two edges, so registers are
+// better spent on more resident blocks than on deeper batches: forward (the edge entry also carries the neighbour's
+// runtimes) two edges and four blocks, backward one edge and six blocks measured best (config 5: 37.5 / 30.3 ms with
+// four edges in flight and three blocks, 28.9 / 20.5 ms now).
+template <bool FWD> struct LevRecShape { static constexpr int EB = FWD ? 2 : 1, BLOCKS = FWD ? 4 : 6; };
 
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
@@ -29,9 +33,10 @@ __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddep
 // neighbours of its first four edges: everything a block needs to start the record copy, the read of its own ids
 // and the reads of the first neighbours' ids at once
 template <bool FWD>
-__global__ void __launch_bounds__(LEVREC_WARPS * 32)
+__global__ void __launch_bounds__(LEVREC_WARPS * 32, LevRecShape<FWD>::BLOCKS)
 pass_levrec_kernel(LevRecArgs a, int item0, int count)
 {
+    constexpr int LEVREC_EB = LevRecShape<FWD>::EB;
     extern __shared__ __align__(16) unsigned char s_rec[];   // header, runtimes and the item's edges
     __shared__ __align__(16) unsigned long long s_rows[2 * LEAN64_K_MAX];   // byte [pv][pu] = 8 * class of the link
     grid_launch_dependents();
@@ -54,7 +59,7 @@ pass_levrec_kernel(LevRecArgs a, int item0, int count)
         const unsigned char* rec = a.blob + 16ll * (unsigned)it.y;
         // own ids: requested before the record arrives
         const unsigned ids = *reinterpret_cast<const unsigned*>(a.part + (long long)v * ldp + jl) & 0x0f0f0f0fu;
-        // ids of the first four neighbours: their vertices come with the item, not with the record
+        // ids of the first neighbours: their vertices come with the item, not with the record
         long long off[LEVREC_EB];
         unsigned pu[LEVREC_EB];
         {
