@@ -1416,7 +1416,10 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
     if (!(flags & (TFPS_EVAL_SLICED | TFPS_EVAL_LEVEL_SYNC)) && sliced && !((!need_fwd || lean_f.ok) && (!need_bwd || lean_b.ok)) &&
         g->levrec[0].ok && g->levrec[1].ok && env_int("TFPS_LEVREC", 1) != 0) {
         const long long avg_width = g->num_levels > 0 ? g->n / g->num_levels : g->n;
-        if (avg_width * P >= (1LL << 18)) { sliced = false; lean_f.ok = false; lean_b.ok = false; }
+        // a level costs the record pass about 8 us however few candidates there are, a vertex costs a sliced kernel
+        // without a resident window about 0.07 us: levels of more than a hundred vertices favour the record pass at
+        // any P (1,590 levels of 660: 12.8 against 76.6 ms forward at P = 64), narrower ones only with enough candidates
+        if (avg_width * P >= (1LL << 18) || avg_width >= 128) { sliced = false; lean_f.ok = false; lean_b.ok = false; }
     }
     // The lean passes cannot leave their tables on a bad id (ids are masked), so the id check need not come first:
     // the loads kernel then runs on a low-priority stream beside them and fills the SMs the passes' last wave leaves idle.
