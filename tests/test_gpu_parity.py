@@ -600,6 +600,34 @@ def test_loads_kernel_table_widths():
         run_and_compare(w.graph, dev, w.part_full(), 0, pad_fill=255)
 
 
+def test_loads_kernel_value_ranges():
+    """Loads and memory loads over the value ranges an accumulator has to hold: all-small costs, all-huge costs and
+    memory sizes (sums far beyond 2^32), huge values in the first rows only, per-block sums just below / exactly at
+    2^32, with candidates that put every vertex on one device."""
+    rng = np.random.default_rng(99)
+    w = I.small_random(4242, 1500, 3000, 4, 130, with_mem=True)
+    g0 = w.graph
+    n = g0.n
+    dev = I.Devices(4, np.ones(4, np.int32), np.full(4, INF, np.int64), w.devices.B, scale=1)
+    part = w.part_full().copy()
+    part[:, 0] = 0          # every vertex on device 0
+    part[:, 1] = 3
+    cases = []
+    cases.append((rng.integers(0, 1000, size=n).astype(np.int32), rng.integers(0, 1000, size=n).astype(np.int64)))
+    cases.append((np.full(n, 2 ** 31 - 1, np.int32), rng.integers(2 ** 33, 2 ** 40, size=n).astype(np.int64)))
+    c = rng.integers(0, 1000, size=n).astype(np.int32)
+    mem = rng.integers(0, 1000, size=n).astype(np.int64)
+    c[:40] = 2 ** 31 - 1
+    mem[5:90] = 2 ** 36 + 17
+    cases.append((c, mem))
+    cases.append((np.full(n, 2 ** 24 - 1, np.int32), np.full(n, 2 ** 24 - 1, np.int64)))   # 256 rows: 2^32 - 256
+    cases.append((np.full(n, 2 ** 24, np.int32), np.full(n, 2 ** 24, np.int64)))           # 256 rows: exactly 2^32
+    cases.append((np.full(n, 5, np.int32), np.full(n, 2 ** 32 - 1, np.int64)))
+    for c, mem in cases:
+        g = I.Graph(n=n, src=g0.src, dst=g0.dst, t=g0.t, c=c, mem=mem, layers=g0.layers)
+        run_and_compare(g, dev, part, 0, pad_fill=255)
+
+
 # ------------------------------------------------------------- randomized sweep
 def test_randomized_shapes_all_variants():
     """Forty seeded random workloads (sizes, device counts, candidate counts, dtypes, device-table structure
