@@ -16,12 +16,13 @@ namespace tfps {
 
 namespace {
 
-constexpr int LEVREC_WARPS = 8;
+constexpr int LEVREC_WARPS = 4;
 // Edges in flight per thread and resident blocks per SM.  Most vertices have one or two edges, so registers are
-// better spent on more resident blocks than on deeper batches: forward (the edge entry also carries the neighbour's
-// runtimes) two edges and four blocks, backward one edge and six blocks measured best (config 5: 37.5 / 30.3 ms with
-// four edges in flight and three blocks, 28.9 / 20.5 ms now).
-template <bool FWD> struct LevRecShape { static constexpr int EB = FWD ? 2 : 1, BLOCKS = FWD ? 4 : 6; };
+// better spent on more resident warps than on deeper batches: forward (the edge entry also carries the neighbour's
+// runtimes) two edges and 32 warps, backward one edge and 48 warps measured best, in blocks of four warps (config 5,
+// forward / backward: 37.5 / 30.3 ms with four edges in flight and 24 warps in blocks of eight, 28.9 / 20.5 ms with
+// these depths in blocks of eight, 28.1 / 19.9 ms in blocks of four, 28.9 / 22.0 ms in blocks of two).
+template <bool FWD> struct LevRecShape { static constexpr int EB = FWD ? 2 : 1, BLOCKS = FWD ? 8 : 12; };
 
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
