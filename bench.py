@@ -277,9 +277,9 @@ def run_gpu(args):
     traffic = 8.681 * n * P if (args.config == 3 and kernel_name == "pass_lean_kernel") else None
     # level-synchronous record pass on config 5: DRAM bytes of all forward launches of a pass, captured with warm
     # caches on the generator's 128-layer graph at the same P (profiles/pass_levrec_kernel_cfg5.md: 6.83 GB for
-    # 268.4 M vertex-candidates = 25.46 B each) and scaled by n*P: the levels in use are the same number of rows
+    # 268.4 M vertex-candidates = 25.45 B each) and scaled by n*P: the levels in use are the same number of rows
     if args.config == 5 and kernel_name == "pass_levrec_kernel" and P == 4096:
-        traffic = 25.46 * n * P
+        traffic = 25.45 * n * P
     value = world * P / (ms * 1e-3)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
