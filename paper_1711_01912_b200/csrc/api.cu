@@ -330,8 +330,11 @@ int build_topo(tfps_graph* g, cudaStream_t st)
             }
         }
         {
-            // a vertex with more than 2*T edges becomes ceil(deg/T) partial items of at most T edges
+            // a vertex with more than `over` (default T) edges becomes ceil(deg/T) partial items of at most T edges
             const int T = std::max(0, env_int("TFPS_TILE_SPLIT", 8));
+            // largest degree left whole.  T edges: at P = 4,096 config 5's forward pass takes the same time as with 2*T
+            // (28.1 ms), at P = 1,024 it takes 11.2 instead of 15.6 ms (the level's longest chain is halved)
+            const int over = std::max(T, env_int("TFPS_TILE_SPLIT_OVER", T));
             std::vector<int> items, heavy, idx;
             std::vector<long long>& ip = g->h_item_ptr[dir];
             ip.assign((size_t)g->num_levels + 1, 0);
@@ -342,7 +345,7 @@ int build_topo(tfps_graph* g, cudaStream_t st)
                 std::stable_sort(idx.begin(), idx.end(), [&](int x, int y) { return eptr[x + 1] - eptr[x] > eptr[y + 1] - eptr[y]; });
                 for (int p : idx) {
                     const int e0 = eptr[p], e1 = eptr[p + 1];
-                    if (T > 0 && e1 - e0 > 2 * T) {
+                    if (T > 0 && e1 - e0 > over) {
                         heavy.push_back(p);
                         for (int e = e0; e < e1; e += T) { items.push_back(p); items.push_back(e); items.push_back(std::min(e1, e + T)); items.push_back(1); }
                     } else {
