@@ -276,10 +276,10 @@ def run_gpu(args):
     kernel_name = tfps.tfps_last_pass_kernel(g.handle)
     traffic = 8.681 * n * P if (args.config == 3 and kernel_name == "pass_lean_kernel") else None
     # level-synchronous record pass on config 5: DRAM bytes of all forward launches of a pass, captured with warm
-    # caches on the generator's 128-layer graph at the same P (profiles/pass_levrec_kernel_cfg5.md: 6.83 GB for
-    # 268.4 M vertex-candidates = 25.45 B each) and scaled by n*P: the levels in use are the same number of rows
+    # caches on the generator's 128-layer graph at the same P (profiles/pass_levrec_kernel_cfg5.md: 7.20 GB for
+    # 268.4 M vertex-candidates = 26.83 B each) and scaled by n*P: the levels in use are the same number of rows
     if args.config == 5 and kernel_name == "pass_levrec_kernel" and P == 4096:
-        traffic = 25.45 * n * P
+        traffic = 26.83 * n * P
     value = world * P / (ms * 1e-3)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
