@@ -80,7 +80,7 @@ const char* tfps_last_error(void);
 
 /*
  * Build a graph handle (Section 2: G, c, t; optional per-vertex memory).
- *   n, m         vertices, edges (n < 2^31, m < 2^31)
+ *   n, m         vertices, edges (n < 2^26, m < 2^31 - 64; larger sizes give TFPS_ERR_UNSUPPORTED)
  *   in_ptr[n+1], in_src[m], in_t[m]     in-edge CSR: row v lists the sources u of edges u->v and their sizes
  *   out_ptr[n+1], out_dst[m], out_t[m]  out-edge CSR; pass all three NULL to have it built by transposing.
  *                                       When given, it must hold the same multiset of (u, v, t) edges.
@@ -150,12 +150,17 @@ size_t tfps_eval_workspace_bytes(const tfps_graph* g, int64_t P, int64_t ldp, in
  *   viol         dev uint64 [P] or NULL; bit d = capacity of device d violated
  *   workspace    dev, 256-byte aligned, workspace_bytes >= tfps_eval_workspace_bytes(...); may be NULL when that is 0
  *   flags        TFPS_EVAL_* (kernel variant; validation)
+ * part and every output that is given must be 16-byte aligned (the kernels move ids
+ * and levels as 16-byte vectors; ldp is a multiple of 16, so every row then is):
+ * a misaligned pointer gives TFPS_ERR_INVALID_ARG and nothing is launched.
  * The forward pass runs when tlevel is wanted, or when cp is wanted and blevel
  * is not; the backward pass runs when blevel is wanted.  P == 0 or n == 0:
  * TFPS_OK, nothing written.  Host-detectable errors are returned at once and
  * nothing is launched.  An id >= k is found on the device: every later kernel
  * of the call then returns without touching memory, outputs are unspecified,
- * and tfps_get_status reports TFPS_ERR_BAD_PARTITION.
+ * and tfps_get_status reports TFPS_ERR_BAD_PARTITION.  The device status is
+ * sticky: until tfps_get_status has read (and cleared) it, the kernels of later
+ * calls on the handle return at once as well, although those calls return TFPS_OK.
  */
 int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp,
                     const uint8_t* part, int64_t* tlevel, int64_t* blevel,
@@ -217,8 +222,9 @@ int64_t tfps_kernel_launches(void);
  *   - n*ldp*8 must not exceed TFPS_NOALLOC_SCRATCH_BYTES, else TFPS_ERR_WORKSPACE.
  *   - tfps_devices_set must have been called (it builds everything the pass
  *     needs), else TFPS_ERR_STATE.
- *   - The first call on a device looks up the device address of the scratch
- *     array; make that first call outside of any stream capture.
+ *   - The device address of the scratch array is looked up once per device by
+ *     tfps_devices_set (a synchronous set-up call: make it outside of any stream
+ *     capture), so the evaluation call itself finds the address cached.
  *   - All calls on a device share the one array.  It keeps whatever the last call
  *     left in it; nothing in it has to start at zero, because every cell the
  *     pass reads was written earlier in the same call.  Two calls that overlap

@@ -19,7 +19,30 @@ static std::atomic<long long> g_launches{0};
 void count_launches(long long n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 }  // namespace tfps
 
+// Scratch of tfps_eval_cp_noalloc: one int64 level matrix, resident on every device that loads the library.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[TFPS_NOALLOC_SCRATCH_BYTES];
+
 namespace {
+
+std::mutex g_noalloc_mutex;
+void* g_noalloc_ptr[128] = {};  // device address of g_noalloc_scratch, by device ordinal
+
+// The array's name is only a host-side handle: the runtime is asked for its address on the current device, once
+// per device.  Called from tfps_devices_set (set-up time), so that the evaluation call itself finds the address
+// cached and touches neither the module loader nor an allocator.
+cudaError_t noalloc_scratch_address(int device, void** out)
+{
+    if (device < 0 || device >= 128) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (!g_noalloc_ptr[device]) {
+        void* p = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
+        if (e != cudaSuccess) return e;
+        g_noalloc_ptr[device] = p;
+    }
+    *out = g_noalloc_ptr[device];
+    return cudaSuccess;
+}
 
 thread_local std::string g_last_error;
 
@@ -147,9 +170,15 @@ struct tfps_graph {
     // level-synchronous pass on vertex records (0 forward, 1 backward)
     struct LevRec {
         bool ok = false;
-        DBuf blob, items;
+        bool by_id = false;    // steps follow the caller's vertex numbering
+        DBuf blob, items, step_ptr, heavy, cls;
+        std::vector<int> h_step_ptr;   // host copy: the chained variant launches step by step
+        int heavy_count = 0;   // vertices evaluated in partial items (their rows start at zero)
         LevRecArgs args;
     } levrec[2];
+    DBuf step_bar;             // barrier counters of the persistent record pass
+    bool id_topo = false;      // the caller's vertex numbering is a topological order ...
+    int span_id = 0;           // ... whose longest edge spans this many vertices
     DBuf status;
     // scratch owned by the handle
     DBuf scr_memload;
@@ -161,7 +190,7 @@ struct tfps_graph {
     const char* last_kernel = "";
     // copy stream and per-chunk events of tfps_eval_batch_host (created on first use)
     cudaStream_t copy_stream = nullptr;
-    cudaEvent_t copy_ev[9] = {};
+    cudaEvent_t copy_ev[4] = {};
     // low-priority stream on which the loads kernel runs beside the lean passes (created by tfps_devices_set)
     cudaStream_t aux_stream = nullptr;
     cudaEvent_t aux_fork = nullptr, aux_join = nullptr;
@@ -707,13 +736,16 @@ int build_lean(tfps_graph* g, int k, const int32_t* s, const int64_t* B, long lo
     return TFPS_OK;
 }
 
-// Packs the vertex records of the level-synchronous record pass (layout: levrec.cu) for both directions.
+// Packs the vertex records, work items and steps of the persistent record pass (layout: levrec.cu) for both
+// directions.  Steps are the topological levels, or -- when the caller's vertex numbering is a topological order whose
+// longest edge is at most half as long and which needs at most twice as many steps -- runs of consecutive vertices
+// none of which depends on a vertex of the same run: the rows a step reads then lie within a short range of rows.
 int build_levrec(tfps_graph* g, int k, const int32_t* s, const int64_t* B, long long S, const std::vector<int>& order,
                  cudaStream_t st)
 {
     for (auto& L : g->levrec) L.ok = false;
     const int n = (int)g->n, m = (int)g->m;
-    if (n == 0 || k > LEAN64_K_MAX || env_int("TFPS_LEVREC", 1) == 0) return TFPS_OK;
+    if (n == 0 || env_int("TFPS_LEVREC", 1) == 0) return TFPS_OK;
     std::vector<long long> wvals;
     auto cls_of = [&](long long x) {
         for (size_t i = 0; i < wvals.size(); ++i)
@@ -729,15 +761,34 @@ int build_levrec(tfps_graph* g, int k, const int32_t* s, const int64_t* B, long 
     }
     const int ncw = (int)wvals.size();
     const u128 rt_max = ((u128)g->max_c * (u128)S + (u128)s_min - 1) / (u128)s_min;
-    if (ncw > LEAN_CLS_MAX || rt_max >= ((u128)1 << 31)) return TFPS_OK;
+    if (ncw > 255 || rt_max >= ((u128)1 << 31)) return TFPS_OK;   // class indices are bytes, runtimes int32
     auto ceil_div = [](long long a, long long S_, long long d) {
         if (a <= (LIMIT62 / S_)) return (a * S_ + d - 1) / d;   // 64-bit arithmetic suffices (d < 2^62)
         return (long long)(((u128)a * (u128)S_ + (u128)d - 1) / (u128)d);
     };
-    const int wbytes = 8 * (ncw + 1);
+    const int KP = k <= 16 ? 16 : 64;
+    const int HDR = 16 + 4 * KP;
+    // speed classes: the runtime of a vertex depends on its device only through the device's speed
+    std::vector<long long> svals;
+    std::vector<int> sc_of((size_t)k);
+    for (int d = 0; d < k; ++d) {
+        size_t i = 0;
+        while (i < svals.size() && svals[i] != s[d]) ++i;
+        if (i == svals.size()) svals.push_back(s[d]);
+        sc_of[d] = (int)i;
+    }
+    const int ns = (int)svals.size();
+    // forward edge costs: one value per (link class, speed class of the neighbour's device) when those are few
+    // enough for a byte index, else transfer times per class plus the neighbour's runtimes per device (RTU form)
+    const bool rtu = (ncw + 1) * ns > 255;
     std::vector<int> rtab((size_t)n * k);   // runtime of every vertex on every device
     for (int v = 0; v < n; ++v)
         for (int q = 0; q < k; ++q) rtab[(size_t)v * k + q] = (int)ceil_div(g->h_c[v], S, s[q]);
+    std::vector<int> pos_of((size_t)n);
+    for (int i = 0; i < n; ++i) pos_of[order[i]] = i;
+    if (!g->step_bar.p) {
+        CUDA_TRY(g->step_bar.alloc(128 * STEPREC_GROUPS_MAX));
+    }
     for (int dir = 0; dir < 2; ++dir) {
         tfps_graph::LevRec& L = g->levrec[dir];
         std::vector<int> ep((size_t)n + 1), nb((size_t)m);
@@ -748,32 +799,66 @@ int build_levrec(tfps_graph* g, int k, const int32_t* s, const int64_t* B, long 
             CUDA_TRY(cudaMemcpyAsync(tt.data(), dir == 0 ? g->f_t.p : g->b_t.p, sizeof(long long) * (size_t)m, cudaMemcpyDeviceToHost, st));
         }
         CUDA_TRY(cudaStreamSynchronize(st));
-        const int estride = 8 + wbytes + (dir == 0 ? 64 : 0);
-        // work items: the tile kernel's, with edges counted from the vertex' first edge
-        const std::vector<int>& titems = g->h_items[dir];   // {position, first edge, end edge, partial}
-        int item_edges = 0;
-        for (size_t i = 0; i + 3 < titems.size(); i += 4) item_edges = std::max(item_edges, titems[i + 2] - titems[i + 1]);
-        const long long smem_need = 80 + (long long)item_edges * estride;
-        if (smem_need > 48 * 1024) continue;   // an unsplit vertex with too many edges
+        const int ncomb = (dir == 0 && !rtu) ? (ncw + 1) * ns : ncw + 1;
+        const int wbytes = 8 * ncomb;
+        const int estride = (8 + wbytes + ((dir == 0 && rtu) ? 4 * KP : 0) + 15) & ~15;
+        // a vertex with more than T edges becomes ceil(deg / T) partial items of at most T edges
+        const int T = std::max(1, std::min(std::max(1, env_int("TFPS_TILE_SPLIT", 8)), 2048 / estride));
+        // steps: lists of level positions in processing order
+        std::vector<int> sp_level, sp_id, vs_id;   // step pointers; vertices (as level positions) of the caller-order steps
+        for (int li = 0; li <= g->num_levels; ++li) sp_level.push_back((int)g->h_level_ptr[li]);
+        bool use_id = false;
+        if (g->id_topo && env_int("TFPS_STEP_ORDER", 0) != 1) {
+            vs_id.resize((size_t)n);
+            int lo = dir == 0 ? 0 : n - 1;   // first vertex of the running step
+            sp_id.push_back(0);
+            for (int stp = 0; stp < n; ++stp) {
+                const int v = dir == 0 ? stp : n - 1 - stp;
+                const int p = pos_of[v];
+                bool indep = true;   // every neighbour lies before (forward) / after (backward) the running step
+                for (int e = ep[p]; e < ep[p + 1] && indep; ++e) indep = dir == 0 ? nb[e] < lo : nb[e] > lo;
+                if (!indep) { sp_id.push_back(stp); lo = v; }
+                vs_id[(size_t)stp] = p;
+            }
+            sp_id.push_back(n);
+            const bool shorter = 2LL * g->span_id <= (long long)g->maxspan && (long long)sp_id.size() - 1 <= 2LL * g->num_levels;
+            use_id = shorter || env_int("TFPS_STEP_ORDER", 0) == 2;
+        }
+        const std::vector<int>& sp = use_id ? sp_id : sp_level;
+        const int nsteps = (int)sp.size() - 1;
         std::vector<long long> roff((size_t)n + 1);
         size_t total = 0;   // in units of 16 bytes
         for (int p = 0; p < n; ++p) {
             roff[p] = (long long)total;
-            total += (16 + 64 + (size_t)(ep[p + 1] - ep[p]) * estride + 15) / 16;
+            total += ((size_t)HDR + (size_t)(ep[p + 1] - ep[p]) * estride) / 16;
         }
         roff[n] = (long long)total;
         if (total >= ((size_t)1 << 31)) continue;
-        // {vertex | partial << 31, record offset / 16, first edge within the record, end edge}
-        //   and the neighbours of the item's first four edges
-        std::vector<int> items(2 * titems.size(), 0);
-        for (size_t i = 0; i + 3 < titems.size(); i += 4) {
-            const int p = titems[i];
-            items[2 * i] = order[p] | (titems[i + 3] ? (int)0x80000000u : 0);
-            items[2 * i + 1] = (int)roff[p];
-            items[2 * i + 2] = titems[i + 1] - ep[p];
-            items[2 * i + 3] = titems[i + 2] - ep[p];
-            for (int q = 0; q < 4 && titems[i + 1] + q < titems[i + 2]; ++q) items[2 * i + 4 + q] = nb[(size_t)titems[i + 1] + q];
+        std::vector<int> items, step_ptr((size_t)nsteps + 1, 0), heavy, idx;
+        int item_edges = 0, max_items = 1;
+        for (int sidx = 0; sidx < nsteps; ++sidx) {
+            // forward: steps in ascending order; backward: level steps in descending order (caller-order steps are built descending)
+            const int src = (dir == 1 && !use_id) ? nsteps - 1 - sidx : sidx;
+            step_ptr[sidx] = (int)(items.size() / 4);
+            idx.clear();
+            for (int q = sp[src]; q < sp[src + 1]; ++q) idx.push_back(use_id ? vs_id[(size_t)q] : q);
+            std::stable_sort(idx.begin(), idx.end(), [&](int x, int y) { return ep[x + 1] - ep[x] > ep[y + 1] - ep[y]; });
+            for (int p : idx) {
+                const int d = ep[p + 1] - ep[p];
+                if (d > T) {
+                    heavy.push_back(order[p]);
+                    for (int e = 0; e < d; e += T) {
+                        items.push_back(order[p] | (int)0x80000000u); items.push_back((int)roff[p]); items.push_back(e); items.push_back(std::min(d, e + T));
+                    }
+                    item_edges = std::max(item_edges, T);
+                } else {
+                    items.push_back(order[p]); items.push_back((int)roff[p]); items.push_back(0); items.push_back(d);
+                    item_edges = std::max(item_edges, d);
+                }
+            }
+            max_items = std::max(max_items, (int)(items.size() / 4) - step_ptr[sidx]);
         }
+        step_ptr[nsteps] = (int)(items.size() / 4);
         std::vector<unsigned char> blob(total * 16, 0);
         for (int p = 0; p < n; ++p) {
             unsigned char* r = blob.data() + (size_t)roff[p] * 16;
@@ -783,35 +868,54 @@ int build_levrec(tfps_graph* g, int k, const int32_t* s, const int64_t* B, long 
             hdr[1] = d;
             memcpy(hdr + 4, &rtab[(size_t)v * k], sizeof(int) * (size_t)k);
             for (int e = 0; e < d; ++e) {
-                unsigned char* er = r + 80 + (size_t)e * estride;
+                unsigned char* er = r + HDR + (size_t)e * estride;
                 const int u = nb[(size_t)ep[p] + e];
                 memcpy(er, &u, 4);
-                for (int w = 0; w < ncw; ++w) {
-                    const long long val = ceil_div(tt[(size_t)ep[p] + e], S, wvals[w]);
-                    memcpy(er + 16 + 8 * w, &val, 8);   // {neighbour, pad, W[0] = 0, W[1..]}
+                // {neighbour, pad, V[ncomb]}: class 0 = same device (no transfer)
+                for (int w = 0; w <= ncw; ++w) {
+                    const long long tr = w == 0 ? 0 : ceil_div(tt[(size_t)ep[p] + e], S, wvals[(size_t)w - 1]);
+                    if (dir == 0 && !rtu) {
+                        for (int q = 0; q < ns; ++q) {
+                            const long long val = tr + ceil_div(g->h_c[u], S, svals[(size_t)q]);   // + the neighbour's runtime
+                            memcpy(er + 8 + 8 * (w * ns + q), &val, 8);
+                        }
+                    } else {
+                        memcpy(er + 8 + 8 * w, &tr, 8);
+                    }
                 }
-                if (dir == 0) memcpy(er + 8 + wbytes, &rtab[(size_t)u * k], sizeof(int) * (size_t)k);
+                if (dir == 0 && rtu) memcpy(er + 8 + wbytes, &rtab[(size_t)u * k], sizeof(int) * (size_t)k);
             }
         }
+        // cost combination of a neighbour on device pu and a vertex on device pv (devices beyond k never occur: ids are
+        // checked by the loads kernel; the table is zero there)
+        std::vector<unsigned char> cls((size_t)KP * KP, 0);
+        for (int pu = 0; pu < k; ++pu)
+            for (int pv = 0; pv < k; ++pv) {
+                const int lc = pu == pv ? 0 : cls_of(dir == 0 ? B[pu * k + pv] : B[pv * k + pu]) + 1;
+                cls[(size_t)pu * KP + pv] = (unsigned char)((dir == 0 && !rtu) ? lc * ns + sc_of[pu] : lc);
+            }
         TFPS_TRY(upload(L.blob, blob, st));
         TFPS_TRY(upload(L.items, items, st));
+        TFPS_TRY(upload(L.step_ptr, step_ptr, st));
+        TFPS_TRY(upload(L.heavy, heavy, st));
+        TFPS_TRY(upload(L.cls, cls, st));
         CUDA_TRY(cudaStreamSynchronize(st));
+        L.heavy_count = (int)heavy.size();
+        L.h_step_ptr = step_ptr;
+        L.by_id = use_id;
+        L.args = LevRecArgs{};
         L.args.blob = L.blob.as<unsigned char>();
         L.args.items = L.items.as<int4>();
+        L.args.step_ptr = L.step_ptr.as<int>();
+        L.args.num_steps = nsteps;
+        L.args.max_step_items = max_items;
+        L.args.cls = L.cls.as<unsigned char>();
+        L.args.bar = g->step_bar.as<unsigned>();
+        L.args.kp = KP;
         L.args.estride = estride;
         L.args.wbytes = wbytes;
-        L.args.rec_max = (int)((smem_need + 15) & ~15LL);
-        for (int pv = 0; pv < LEAN64_K_MAX; ++pv)
-            for (int h = 0; h < 2; ++h) {
-                unsigned long long row = 0;
-                for (int b = 0; b < 8; ++b) {
-                    const int pu = 8 * h + b;
-                    int cls = 0;
-                    if (pv < k && pu < k && pu != pv) cls = cls_of(dir == 0 ? B[pu * k + pv] : B[pv * k + pu]) + 1;
-                    row |= (unsigned long long)(8 * cls) << (8 * b);
-                }
-                L.args.rows16[2 * pv + h] = row;
-            }
+        L.args.rtu = (dir == 0 && rtu) ? 1 : 0;
+        L.args.rec_max = HDR + item_edges * estride;
         L.ok = true;
     }
     return TFPS_OK;
@@ -888,6 +992,12 @@ int tfps_graph_create(tfps_graph** out, int64_t n, int64_t m,
     for (long long v = 0; v < n; ++v)
         for (long long e = h_in_ptr[v]; e < h_in_ptr[v + 1]; ++e)
             if (h_in_src[e] == v) return fail(TFPS_ERR_CYCLE, "self loop at vertex %lld", v);
+    g->id_topo = true;
+    for (long long v = 0; v < n && g->id_topo; ++v)
+        for (long long e = h_in_ptr[v]; e < h_in_ptr[v + 1]; ++e) {
+            if (h_in_src[e] >= v) { g->id_topo = false; break; }
+            g->span_id = std::max(g->span_id, (int)(v - h_in_src[e]));
+        }
 
     // out-CSR by transposing the in-CSR (rows come out sorted by target, then by in-row order)
     std::vector<long long> t_ptr((size_t)n + 1, 0), t_t((size_t)m);
@@ -1141,7 +1251,7 @@ int tfps_devices_set(tfps_graph* g, int k, const int32_t* s, const int64_t* C, c
     }
     g->fits32 = false;
     for (auto& L : g->lean) L.ok = false;
-    if ((g->ncomb > 0 || k <= LEAN64_K_MAX) && n > 0) {
+    if (n > 0) {
         // worst-case critical path: every vertex on the slowest device, every edge over the slowest link
         std::vector<int> order((size_t)n);
         CUDA_TRY(cudaMemcpyAsync(order.data(), g->order.p, sizeof(int) * (size_t)n, cudaMemcpyDeviceToHost, st));
@@ -1228,6 +1338,10 @@ int tfps_devices_set(tfps_graph* g, int k, const int32_t* s, const int64_t* C, c
         CUDA_TRY(cudaEventCreateWithFlags(&g->aux_fork, cudaEventDisableTiming));
         CUDA_TRY(cudaEventCreateWithFlags(&g->aux_join, cudaEventDisableTiming));
     }
+    if (g->device >= 0 && g->device < 128) {
+        void* scratch = nullptr;   // resolve the built-in scratch of tfps_eval_cp_noalloc now, not in the evaluation call
+        CUDA_TRY(noalloc_scratch_address(g->device, &scratch));
+    }
     g->k = k;
     g->S = scale;
     g->dev_set = true;
@@ -1275,6 +1389,14 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
     if (P == 0 || g->n == 0) return TFPS_OK;
     if (!part) return fail(TFPS_ERR_INVALID_ARG, "part is NULL");
     if (P > ((int64_t)1 << 31)) return fail(TFPS_ERR_UNSUPPORTED, "P above 2^31");
+    {
+        // the kernels read ids and read and write levels as 16-byte vectors: refuse anything else before any launch
+        const void* ptrs[] = {part, tlevel, blevel, cp, load, memload, viol};
+        const char* names[] = {"part", "tlevel", "blevel", "cp", "load", "memload", "viol"};
+        for (int i = 0; i < 7; ++i)
+            if (((uintptr_t)ptrs[i] & 15u) != 0)
+                return fail(TFPS_ERR_INVALID_ARG, "%s must be 16-byte aligned", names[i]);
+    }
 
     DeviceGuard guard(g->device);
     if (!guard.ok) return fail(TFPS_ERR_CUDA, "cannot select the handle's device");
@@ -1408,6 +1530,7 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
             ch.args.P = P;
             ch.args.ldp = ldp;
             ch.args.plan = lp;
+            ch.args.wait_limit = std::max(0, env_int("TFPS_WAIT_LIMIT", 1 << 20));
         }
         return ch;
     };
@@ -1547,19 +1670,35 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
                 {
                     // rows of the vertices that are evaluated in partial items start at zero
                     const int dirn = fwd ? 0 : 1;
-                    const bool rec = g->levrec[dirn].ok && ((uintptr_t)part & 3u) == 0 && env_int("TFPS_LEVREC", 1) != 0;
-                    if ((g->npass > 0 || rec) && g->heavy_count[dirn] > 0)
-                        CUDA_TRY(launch_zero_rows(g->heavy[dirn].as<int>(), g->heavy_count[dirn], P, ldp, lev, st));
-                    if (rec) {   // vertex records (k <= 16): no divisions or per-edge tables in the kernel
-                        LevRecArgs la = g->levrec[dirn].args;
+                    const bool rec = g->levrec[dirn].ok && env_int("TFPS_LEVREC", 1) != 0;
+                    if (rec) {   // vertex records (k <= 64): no divisions or per-edge tables in the kernel
+                        tfps_graph::LevRec& L = g->levrec[dirn];
+                        if (L.heavy_count > 0) CUDA_TRY(launch_zero_rows(L.heavy.as<int>(), L.heavy_count, P, ldp, lev, st));
+                        LevRecArgs la = L.args;
                         la.part = part;
                         la.lev = lev;
                         la.status = status;
                         la.P = P;
                         la.ldp = ldp;
-                        g->last_kernel = "pass_levrec_kernel";
-                        CUDA_TRY(launch_pass_levrec(la, fwd, g->h_item_ptr[dirn], g->num_levels, st));
+                        la.groups = std::max(1, std::min((int)STEPREC_GROUPS_MAX, env_int("TFPS_STEP_GROUPS", 2)));
+                        la.tiles_per_group = std::max(1, env_int("TFPS_STEP_TILES", 8));
+                        la.tiles_per_run = std::max(1, env_int("TFPS_STEP_RUN", 4));
+                        la.blocks_per_sm = std::max(0, env_int("TFPS_STEP_BLOCKS", 0));
+                        la.wait_limit = std::max(0, env_int("TFPS_WAIT_LIMIT", 1 << 20));
+                        la.shape = env_int("TFPS_STEP_SHAPE", 0);
+                        // One launch per step by default; the persistent form (one cooperative launch, barriers between
+                        // the steps inside the kernel) measured slower at every batch width (config 5, forward pass: 14.4
+                        // against 10.1 ms at P = 256, 18.9 against 16.0 at 1,024, 33.8 against 29.4 at 4,096) and is opt-in.
+                        if (env_int("TFPS_STEP_PERSISTENT", 0) == 1) {
+                            g->last_kernel = "pass_steprec_kernel";
+                            CUDA_TRY(launch_pass_steprec(la, fwd, g->sm_count, st));
+                        } else {
+                            g->last_kernel = "pass_stepchain_kernel";
+                            CUDA_TRY(launch_pass_stepchain(la, fwd, L.h_step_ptr, st));
+                        }
                     } else {
+                        if (g->npass > 0 && g->heavy_count[dirn] > 0)
+                            CUDA_TRY(launch_zero_rows(g->heavy[dirn].as<int>(), g->heavy_count[dirn], P, ldp, lev, st));
                         CUDA_TRY(launch_pass_level_sync(a, fwd, g->h_level_ptr, st, &g->h_item_ptr[dirn]));
                     }
                 }
@@ -1598,13 +1737,6 @@ const char* tfps_last_pass_kernel(const tfps_graph* g) { return g ? g->last_kern
 
 int64_t tfps_kernel_launches(void) { return (int64_t)tfps::g_launches.load(std::memory_order_relaxed); }
 
-// Scratch of tfps_eval_cp_noalloc: one int64 level matrix, resident on every device that loads the library.
-static __device__ __align__(256) unsigned char g_noalloc_scratch[TFPS_NOALLOC_SCRATCH_BYTES];
-
-namespace {
-std::mutex g_noalloc_mutex;
-void* g_noalloc_ptr[128] = {};  // device address of g_noalloc_scratch, by device ordinal
-}  // namespace
 
 int tfps_eval_cp_noalloc(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, int64_t* cp, int flags,
                          void* stream)
@@ -1622,16 +1754,7 @@ int tfps_eval_cp_noalloc(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* p
     DeviceGuard guard(g->device);
     if (!guard.ok) return fail(TFPS_ERR_CUDA, "cannot select the handle's device");
     void* scratch = nullptr;
-    {
-        // the array's name is only a host-side handle: ask the runtime for its address on this device, once
-        std::lock_guard<std::mutex> lock(g_noalloc_mutex);
-        if (!g_noalloc_ptr[g->device]) {
-            void* p = nullptr;
-            CUDA_TRY(cudaGetSymbolAddress(&p, g_noalloc_scratch));
-            g_noalloc_ptr[g->device] = p;
-        }
-        scratch = g_noalloc_ptr[g->device];
-    }
+    CUDA_TRY(noalloc_scratch_address(g->device, &scratch));   // cached by tfps_devices_set on this device
     return tfps_eval_batch(g, P, ldp, part, nullptr, nullptr, cp, nullptr, nullptr, nullptr, scratch,
                            TFPS_NOALLOC_SCRATCH_BYTES, flags & ~TFPS_EVAL_PROFILE, stream);
 }
@@ -1665,54 +1788,64 @@ int tfps_eval_batch_host(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* p
     DeviceGuard guard(g->device);
     if (!guard.ok) return fail(TFPS_ERR_CUDA, "cannot select the handle's device");
     cudaStream_t st = (cudaStream_t)stream;
-    const size_t cells = (size_t)g->n * (size_t)ldp;
-    const size_t kcells = (size_t)g->k * (size_t)ldp;
-    CUDA_TRY(g->st_part.reserve(cells));
-    CUDA_TRY(g->st_lev.reserve(cells * 8));
-    CUDA_TRY(g->st_lev2.reserve(cells * 8));
-    CUDA_TRY(g->st_cp.reserve((size_t)P * 8));
-    if (load) CUDA_TRY(g->st_load.reserve(kcells * 8));
-    if (memload || viol) CUDA_TRY(g->st_mem.reserve(kcells * 8));
-    if (viol) CUDA_TRY(g->st_viol.reserve((size_t)P * 8));
-    // Candidates are independent: the id matrix goes up in column chunks on a copy stream and every chunk is
-    // evaluated as soon as it has landed, so the transfer of chunk c+1 overlaps the evaluation of chunk c.
-    // (a chunk must still fill the GPU: one wave of blocks of the sliced kernel is 64 candidates per SM)
+    const int k = g->k;
+    // Candidates are independent: the id matrix goes up in column chunks on a copy stream (two staging buffers) and
+    // every chunk is evaluated as soon as it has landed, so the transfer of chunk c+1 overlaps the evaluation of
+    // chunk c; results come back per chunk.  A chunk must still fill the GPU (one wave of blocks of the sliced kernel
+    // is 64 candidates per SM) and rows shorter than 4 KiB copy far below the link rate, so chunks are as wide as the
+    // scratch allows: the two level matrices of a chunk (int64 [n][width] each) are kept below 2 x 36 GB.
     int nchunks = P >= 128LL * g->sm_count * 3 / 4 ? 2 : 1;
     long long width = (P + nchunks - 1) / nchunks;
+    const long long cap = std::max<long long>(128, ((36LL << 30) / (8LL * std::max<long long>(1, g->n))) / 128 * 128);
+    width = std::min(width, cap);
     width = (width + 127) / 128 * 128;   // whole candidate slices per chunk
+    if (width >= ldp) width = ldp;
     nchunks = (int)((P + width - 1) / width);
+    const size_t ccells = (size_t)g->n * (size_t)width;
+    const size_t kcells = (size_t)k * (size_t)width;
+    CUDA_TRY(g->st_part.reserve(ccells * (nchunks > 1 ? 2 : 1)));
+    CUDA_TRY(g->st_lev.reserve(ccells * 8));
+    CUDA_TRY(g->st_lev2.reserve(ccells * 8));
+    CUDA_TRY(g->st_cp.reserve((size_t)width * 8));
+    if (load) CUDA_TRY(g->st_load.reserve(kcells * 8));
+    if (memload || viol) CUDA_TRY(g->st_mem.reserve(kcells * 8));
+    if (viol) CUDA_TRY(g->st_viol.reserve((size_t)width * 8));
     if (nchunks > 1) {
         if (!g->copy_stream) CUDA_TRY(cudaStreamCreateWithFlags(&g->copy_stream, cudaStreamNonBlocking));
-        for (int c = 0; c <= nchunks; ++c)
+        for (int c = 0; c < 4; ++c)
             if (!g->copy_ev[c]) CUDA_TRY(cudaEventCreateWithFlags(&g->copy_ev[c], cudaEventDisableTiming));
         // the staging buffers may still be in use by earlier work on the caller's stream
-        CUDA_TRY(cudaEventRecord(g->copy_ev[nchunks], st));
-        CUDA_TRY(cudaStreamWaitEvent(g->copy_stream, g->copy_ev[nchunks], 0));
+        CUDA_TRY(cudaEventRecord(g->copy_ev[2], st));
+        CUDA_TRY(cudaStreamWaitEvent(g->copy_stream, g->copy_ev[2], 0));
     }
     for (int c = 0; c < nchunks; ++c) {
         const long long j0 = (long long)c * width;
         const long long w = std::min<long long>(width, P - j0);
         const long long wl = std::min<long long>(width, ldp - j0);   // bytes per row to copy: whole 16-byte pieces
+        uint8_t* dpart = g->st_part.as<uint8_t>() + (size_t)(c & 1) * ccells;
         if (nchunks > 1) {
-            CUDA_TRY(cudaMemcpy2DAsync(g->st_part.as<uint8_t>() + j0, (size_t)ldp, part + j0, (size_t)ldp, (size_t)wl,
-                                       (size_t)g->n, cudaMemcpyHostToDevice, g->copy_stream));
-            CUDA_TRY(cudaEventRecord(g->copy_ev[c], g->copy_stream));
-            CUDA_TRY(cudaStreamWaitEvent(st, g->copy_ev[c], 0));
+            // buffer c & 1 was last read by the evaluation of chunk c - 2
+            if (c >= 2) CUDA_TRY(cudaStreamWaitEvent(g->copy_stream, g->copy_ev[3], 0));
+            CUDA_TRY(cudaMemcpy2DAsync(dpart, (size_t)width, part + j0, (size_t)ldp, (size_t)wl, (size_t)g->n,
+                                       cudaMemcpyHostToDevice, g->copy_stream));
+            CUDA_TRY(cudaEventRecord(g->copy_ev[c & 1], g->copy_stream));
+            CUDA_TRY(cudaStreamWaitEvent(st, g->copy_ev[c & 1], 0));
         } else {
-            CUDA_TRY(cudaMemcpyAsync(g->st_part.p, part, cells, cudaMemcpyHostToDevice, st));
+            CUDA_TRY(cudaMemcpy2DAsync(dpart, (size_t)width, part, (size_t)ldp, (size_t)wl, (size_t)g->n, cudaMemcpyHostToDevice, st));
         }
-        TFPS_TRY(tfps_eval_batch(g, w, ldp, g->st_part.as<uint8_t>() + j0, g->st_lev.as<int64_t>() + j0,
-                                 g->st_lev2.as<int64_t>() + j0, g->st_cp.as<int64_t>() + j0,
-                                 load ? g->st_load.as<int64_t>() + j0 : nullptr,
-                                 (memload || viol) ? g->st_mem.as<int64_t>() + j0 : nullptr,
-                                 viol ? g->st_viol.as<uint64_t>() + j0 : nullptr, nullptr, 0, flags, st));
+        TFPS_TRY(tfps_eval_batch(g, w, width, dpart, g->st_lev.as<int64_t>(), g->st_lev2.as<int64_t>(), g->st_cp.as<int64_t>(),
+                                 load ? g->st_load.as<int64_t>() : nullptr, (memload || viol) ? g->st_mem.as<int64_t>() : nullptr,
+                                 viol ? g->st_viol.as<uint64_t>() : nullptr, nullptr, 0, flags, st));
+        if (nchunks > 1 && c + 2 < nchunks) CUDA_TRY(cudaEventRecord(g->copy_ev[3], st));   // chunk c + 1 runs between: one event suffices
+        // results of the chunk: strided copies into the caller's [.][ldp] arrays
+        const size_t wb = (size_t)w * 8;
+        if (tlevel) CUDA_TRY(cudaMemcpy2DAsync(tlevel + j0, (size_t)ldp * 8, g->st_lev.p, (size_t)width * 8, wb, (size_t)g->n, cudaMemcpyDeviceToHost, st));
+        if (blevel) CUDA_TRY(cudaMemcpy2DAsync(blevel + j0, (size_t)ldp * 8, g->st_lev2.p, (size_t)width * 8, wb, (size_t)g->n, cudaMemcpyDeviceToHost, st));
+        if (cp) CUDA_TRY(cudaMemcpyAsync(cp + j0, g->st_cp.p, wb, cudaMemcpyDeviceToHost, st));
+        if (load) CUDA_TRY(cudaMemcpy2DAsync(load + j0, (size_t)ldp * 8, g->st_load.p, (size_t)width * 8, wb, (size_t)k, cudaMemcpyDeviceToHost, st));
+        if (memload) CUDA_TRY(cudaMemcpy2DAsync(memload + j0, (size_t)ldp * 8, g->st_mem.p, (size_t)width * 8, wb, (size_t)k, cudaMemcpyDeviceToHost, st));
+        if (viol) CUDA_TRY(cudaMemcpyAsync(viol + j0, g->st_viol.p, wb, cudaMemcpyDeviceToHost, st));
     }
-    if (tlevel) CUDA_TRY(cudaMemcpyAsync(tlevel, g->st_lev.p, cells * 8, cudaMemcpyDeviceToHost, st));
-    if (blevel) CUDA_TRY(cudaMemcpyAsync(blevel, g->st_lev2.p, cells * 8, cudaMemcpyDeviceToHost, st));
-    if (cp) CUDA_TRY(cudaMemcpyAsync(cp, g->st_cp.p, (size_t)P * 8, cudaMemcpyDeviceToHost, st));
-    if (load) CUDA_TRY(cudaMemcpyAsync(load, g->st_load.p, kcells * 8, cudaMemcpyDeviceToHost, st));
-    if (memload) CUDA_TRY(cudaMemcpyAsync(memload, g->st_mem.p, kcells * 8, cudaMemcpyDeviceToHost, st));
-    if (viol) CUDA_TRY(cudaMemcpyAsync(viol, g->st_viol.p, (size_t)P * 8, cudaMemcpyDeviceToHost, st));
     return tfps_get_status(g, stream);
 }
 

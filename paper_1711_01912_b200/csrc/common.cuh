@@ -191,24 +191,38 @@ struct LeanArgs {
     int depth;                   // chunks in flight (stage slots)
     unsigned slot_stride;        // bytes of a stage slot: rec_max + max_v * (candidates per block)
     unsigned stage_bytes;        // bytes reserved for all stage slots (also the CP reduction buffer)
+    int wait_limit;              // polls before a wait for a stage gives up (TFPS_ERR_TIMEOUT)
 };
 
-// Level-synchronous pass on host-packed vertex records (levrec.cu).
+// Persistent step-synchronous pass on host-packed vertex records (levrec.cu).
 struct LevRecArgs {
     const uint8_t* part;
     long long* lev;
     int* status;
     long long P, ldp;
     const unsigned char* blob;   // records, 16-byte aligned
-    const int4* items;           // work items, two int4 each: {vertex | partial << 31, record offset / 16, first edge within the
-                                 // record, end edge}, {neighbours of the item's first four edges}; by level
-    int estride;                 // bytes of an edge entry
-    int wbytes;                  // bytes of the transfer times of an edge entry: 8 * (classes + 1)
-    int rec_max;                 // shared memory per block: header, runtimes and the edges of the largest item
-    unsigned long long rows16[2 * 16];   // byte [pv][pu] = 8 * class of the link
+    const int4* items;           // work items {vertex | partial << 31, record offset / 16, first edge within the record, end edge},
+                                 // step by step in processing order
+    const int* step_ptr;         // [num_steps + 1] first item of every step
+    int num_steps;
+    int max_step_items;          // most items in one step
+    const unsigned char* cls;    // [kp * kp] byte [pu * kp + pv] = cost combination of a neighbour on pu and a vertex on pv
+    unsigned* bar;               // one counter per phase, 128 bytes apart (zeroed by the launcher)
+    int kp;                      // device table width: 16 or 64
+    int estride;                 // bytes of an edge entry (multiple of 16)
+    int wbytes;                  // bytes of the cost values of an edge entry: 8 * combinations
+    int rtu;                     // forward records carry the neighbour's runtimes separately (too many combinations)
+    int rec_max;                 // bytes of the largest item: header, runtimes and its edges
+    int groups;                  // phases (column groups) of a walk
+    int tiles_per_group;         // tiles of a phase
+    int tiles_per_run;           // consecutive tiles of a phase a warp evaluates for one item
+    int blocks_per_sm;           // 0: as many as fit
+    int wait_limit;              // polls before a barrier wait gives up
+    int shape;                   // block shape variant (tuning)
 };
-cudaError_t launch_pass_levrec(const LevRecArgs& a, bool fwd, const std::vector<long long>& item_ptr_host, int num_levels,
-                               cudaStream_t st);
+constexpr int STEPREC_GROUPS_MAX = 4;
+cudaError_t launch_pass_steprec(const LevRecArgs& a, bool fwd, int sm_count, cudaStream_t st);
+cudaError_t launch_pass_stepchain(const LevRecArgs& a, bool fwd, const std::vector<int>& step_ptr_host, cudaStream_t st);
 
 size_t lean_smem_bytes(const LeanPlan& plan, int slice, int warps, int depth, unsigned* slot_stride, unsigned* stage_bytes);
 cudaError_t launch_pass_lean(const LeanArgs& a, bool fwd, int slice, int warps, size_t smem, cudaStream_t st);

@@ -10,118 +10,22 @@
 // Requirements (checked by the host): k <= 16, at most 30 distinct off-diagonal bandwidths, every vertex runtime
 // below 2^31, the whole window resident.
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace tfps {
 
 namespace {
 
-__device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ unsigned lds32(unsigned a)
-{
-    unsigned v;
-    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a) : "memory");
-    return v;
-}
-__device__ __forceinline__ unsigned lds32_off16(unsigned a)
-{
-    unsigned v;
-    asm volatile("ld.shared.u32 %0, [%1+16];" : "=r"(v) : "r"(a) : "memory");
-    return v;
-}
-__device__ __forceinline__ unsigned lds_u8(unsigned a)
-{
-    unsigned v;
-    asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(a) : "memory");
-    return v;
-}
-__device__ __forceinline__ uint2 lds64(unsigned a)
-{
-    uint2 v;
-    asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(a) : "memory");
-    return v;
-}
-__device__ __forceinline__ long long lds_s64_off8(unsigned a)   // int64 at a + 8
-{
-    long long v;
-    asm volatile("ld.shared.s64 %0, [%1+8];" : "=l"(v) : "r"(a) : "memory");
-    return v;
-}
-__device__ __forceinline__ uint4 lds128(unsigned a)
-{
-    uint4 v;
-    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a) : "memory");
-    return v;
-}
-__device__ __forceinline__ void lds_2x64(unsigned a, long long& x, long long& y)
-{
-    asm volatile("ld.shared.v2.s64 {%0, %1}, [%2];" : "=l"(x), "=l"(y) : "r"(a) : "memory");
-}
-__device__ __forceinline__ void sts_2x64(unsigned a, long long x, long long y)
-{
-    asm volatile("st.shared.v2.s64 [%0], {%1, %2};" ::"r"(a), "l"(x), "l"(y) : "memory");
-}
-__device__ __forceinline__ void sts32(unsigned a, unsigned v) { asm volatile("st.shared.u32 [%0], %1;" ::"r"(a), "r"(v) : "memory"); }
-
-__device__ __forceinline__ void mbar_init(unsigned bar, unsigned count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_init_fence() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
-__device__ __forceinline__ void mbar_expect_tx(unsigned bar, unsigned bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-// global -> shared bulk copy; both addresses 16-byte aligned, bytes a multiple of 16
-__device__ __forceinline__ void bulk_g2s(unsigned dst, const void* src, unsigned bytes, unsigned bar)
-{
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(unsigned bar, unsigned parity)
-{
-    unsigned ok;
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
 template <int BYTES> __device__ __forceinline__ void cp_async_piece(unsigned dst, const void* g)
 {
-    if constexpr (BYTES == 16) asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(g) : "memory");
-    else asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(dst), "l"(g) : "memory");
-}
-// one (pre-counted) arrival on the mbarrier once every cp.async this thread has issued so far has landed
-__device__ __forceinline__ void cp_async_arrive_on(unsigned bar)
-{
-    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
-}
-// Bounded wait: gives up after WAIT_LIMIT polls (each poll blocks for a hardware-defined time slice at most).
-constexpr int WAIT_LIMIT = 1 << 20;
-__device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity)
-{
-#pragma unroll 1
-    for (int i = 0; i < WAIT_LIMIT; ++i)
-        if (mbar_try_wait(bar, parity)) return true;
-    return false;
+    if constexpr (BYTES == 16) cp_async16(dst, g);
+    else cp_async8_ca(dst, g);
 }
 template <int OFF> __device__ __forceinline__ void stg_cs_v2(long long* p, long long x, long long y)
 {
     asm volatile("st.global.cs.v2.u64 [%0+%3], {%1, %2};" ::"l"(p), "l"(x), "l"(y), "n"(OFF) : "memory");
 }
 __device__ __forceinline__ void stg_cs(long long* p, long long x) { asm volatile("st.global.cs.u64 [%0], %1;" ::"l"(p), "l"(x) : "memory"); }
-// p + (a * b) with a 32 x 32 -> 64 bit product
-__device__ __forceinline__ const uint8_t* ptr_mad(const uint8_t* p, unsigned a, unsigned b)
-{
-    unsigned long long r;
-    asm volatile("mad.wide.u32 %0, %1, %2, %3;" : "=l"(r) : "r"(a), "r"(b), "l"((unsigned long long)p));
-    return reinterpret_cast<const uint8_t*>(r);
-}
-__device__ __forceinline__ long long* ptr_mad(long long* p, unsigned a, unsigned b)
-{
-    unsigned long long r;
-    asm("mad.wide.u32 %0, %1, %2, %3;" : "=l"(r) : "r"(a), "r"(b), "l"((unsigned long long)p));
-    return reinterpret_cast<long long*>(r);
-}
-
 constexpr int CPT = 4;   // candidates per lane
 
 // VPW vertices per warp: a vertex is handled by 32/VPW lanes with 4 candidates each, so a block owns
@@ -216,7 +120,7 @@ __global__ void __launch_bounds__(512, 1) pass_lean64_kernel(const __grid_consta
     // hold block barriers that every thread must reach).
     int slot = 0;
     unsigned par = 0;
-    bool timed_out = nc > 0 && !mbar_wait(bar0, 0u);
+    bool timed_out = nc > 0 && !mbar_wait(bar0, 0u, a.wait_limit);
     bool dead = __syncthreads_or(timed_out) != 0;
     for (int ci = 0; ci < nc && !dead; ++ci) {
         const unsigned slotb = stage0 + (unsigned)slot * a.slot_stride;
@@ -307,14 +211,14 @@ __global__ void __launch_bounds__(512, 1) pass_lean64_kernel(const __grid_consta
         const int nslot = slot + 1 == D ? 0 : slot + 1;
         const unsigned npar = slot + 1 == D ? par ^ 1u : par;
         if (D > 1) {
-            timed_out = ci + 1 < nc && !mbar_wait(bar0 + 8u * nslot, npar);
+            timed_out = ci + 1 < nc && !mbar_wait(bar0 + 8u * nslot, npar, a.wait_limit);
             dead = __syncthreads_or(timed_out) != 0;
             if (dead) break;
             issue(dA, vA0, vA1, slotb, bar);
         } else {   // a single stage: the next record can only be requested once this one is done with
             __syncthreads();
             issue(dA, vA0, vA1, slotb, bar);
-            timed_out = ci + 1 < nc && !mbar_wait(bar0 + 8u * nslot, npar);
+            timed_out = ci + 1 < nc && !mbar_wait(bar0 + 8u * nslot, npar, a.wait_limit);
             dead = __syncthreads_or(timed_out) != 0;
             if (dead) break;
         }

@@ -564,15 +564,17 @@ def test_lean_plan_in_callers_vertex_order(wide, monkeypatch):
     run_and_compare(g4, w4.devices, w4.part_rows(0, 16 * 150)[:, :50], 2, pad_fill=255)
 
 
-@pytest.mark.parametrize("levrec", [0, 1])
-@pytest.mark.parametrize("split", [0, 3, 8])
+@pytest.mark.parametrize("levrec", [0, 1, 2])
+@pytest.mark.parametrize("split", [1, 3, 8])
 def test_level_kernels_with_partial_items(split, levrec, monkeypatch):
-    """The level-synchronous kernels (record pass and tile kernel) with vertices of many edges cut into partial
-    work items of at most `split` edges (0: never): a hub with hundreds of in-edges next to vertices of degree one,
-    the power-law fan-in graph with k = 16, a graph with k = 17 (per-relaxation division kernel, no items)."""
+    """The step-synchronous kernels (0: tile kernel, 1: record pass with one launch per step, 2: persistent record
+    pass) with vertices of many edges cut into partial work items of at most `split` edges: a hub with hundreds of
+    in-edges next to vertices of degree one, the power-law fan-in graph with k = 16, a graph with k = 17 (record pass
+    with the 64-device tables; the tile kernel's family falls back to the per-relaxation division kernel)."""
     from paper_1711_01912_b200 import tfps
     monkeypatch.setenv("TFPS_TILE_SPLIT", str(split))
-    monkeypatch.setenv("TFPS_LEVREC", str(levrec))
+    monkeypatch.setenv("TFPS_LEVREC", "1" if levrec else "0")
+    monkeypatch.setenv("TFPS_STEP_PERSISTENT", "1" if levrec == 2 else "0")
     rng = np.random.default_rng(77 + split)
     n = 700
     edges = [(u, n - 1, int(rng.integers(0, 10 ** 6))) for u in range(n - 1)] + [(0, u, 5) for u in range(1, 60)]
@@ -583,7 +585,7 @@ def test_level_kernels_with_partial_items(split, levrec, monkeypatch):
     G = gpu_graph(w.graph, w.devices)
     dpart, P, ldp = padded(w.part_full())
     G.eval_batch(dpart, P, flags=1)
-    assert tfps.tfps_last_pass_kernel(G.handle) == ("pass_levrec_kernel" if levrec else "pass_tile_kernel")
+    assert tfps.tfps_last_pass_kernel(G.handle) == ["pass_tile_kernel", "pass_stepchain_kernel", "pass_steprec_kernel"][levrec]
     G.close()
     w = I.small_random(4242 + split, 500, 3000, 17, 40)
     run_and_compare(w.graph, w.devices, w.part_full(), 1, pad_fill=255)
@@ -649,3 +651,35 @@ def test_randomized_shapes_all_variants():
         part = w.part_full()
         for flags in (0, 1, 2):
             run_and_compare(w.graph, dev, part, flags, pad_fill=255)
+
+
+@pytest.mark.parametrize("family", ["lean", "lean64", "steprec"])
+def test_bounded_waits_run_out(family, monkeypatch):
+    """The bounded device-side waits, made to run out on the host's terms: with a limit of zero polls every wait of
+    the windowed kernels (for a staged record) and of the persistent record pass (for the other blocks' signal) gives
+    up at once; the kernels vote, let their few copies in flight land, and return.  The call reports
+    TFPS_ERR_TIMEOUT through the status word, nothing hangs or faults, and the next call on the same handle is
+    bit-exact again."""
+    from paper_1711_01912_b200 import tfps
+    if family == "steprec":
+        w = I.config5(layers=14, width=64, P=300)
+        flags = tfps.EVAL_LEVEL_SYNC
+        monkeypatch.setenv("TFPS_STEP_PERSISTENT", "1")
+    else:
+        w = I.config2()
+        w.P = 200
+        flags = tfps.EVAL_SLICED
+        if family == "lean64":
+            monkeypatch.setenv("TFPS_LEAN_FORCE_WIDE", "1")
+    G = gpu_graph(w.graph, w.devices)
+    dpart, P, ldp = padded(w.part_full()[:, :w.P])
+    monkeypatch.setenv("TFPS_WAIT_LIMIT", "0")
+    out = G.eval_batch(dpart, P, flags=flags, check=False)
+    kernel = tfps.tfps_last_pass_kernel(G.handle)
+    assert kernel == {"lean": "pass_lean_kernel", "lean64": "pass_lean64_kernel", "steprec": "pass_steprec_kernel"}[family]
+    with pytest.raises(tfps.TfpsError) as ei:
+        G.status()
+    assert ei.value.code == tfps.ERR_TIMEOUT
+    monkeypatch.delenv("TFPS_WAIT_LIMIT")
+    G.close()
+    run_and_compare(w.graph, w.devices, w.part_full()[:, :w.P], 2 if family != "steprec" else 1, pad_fill=255)

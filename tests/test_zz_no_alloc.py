@@ -6,9 +6,11 @@ that must not hit a device-wide synchronising cudaMalloc).  For them the library
 carries its own fixed scratch array.  This test drives the entry point through
 the C ABI twice in a row -- the second call finds the first call's leftovers in
 the shared array -- and requires the critical-path lengths to equal, bit for
-bit, those of the ordinary entry point with a caller workspace.  It also checks
-that a problem too large for the built-in array is refused with
-TFPS_ERR_WORKSPACE instead of being run.
+bit, those of the ordinary entry point with a caller workspace.  The device's
+free memory as the driver reports it (cudaMemGetInfo, which sees every
+allocation of the process, the library's own included) must not shrink across
+the calls.  It also checks that a problem too large for the built-in array is
+refused with TFPS_ERR_WORKSPACE instead of being run.
 
 This file is named so that pytest collects it last.
 """
@@ -38,13 +40,13 @@ def test_noalloc_matches_workspace_entry_point_twice():
         host[:, :P] = full[:, c0:c0 + P]
         part = torch.from_numpy(host).cuda()
         ref = g.eval_batch(part, P, want=("cp",), out={})["cp"]          # existing entry point, caller workspace
-        torch.cuda.synchronize()
-        before = torch.cuda.memory_allocated()
         cp = torch.full((P,), -1, dtype=torch.int64, device="cuda")
-        after_buffers = torch.cuda.memory_allocated()
+        torch.cuda.synchronize()
+        free_before, _ = torch.cuda.mem_get_info()
         tfps.tfps_eval_cp_noalloc(g.handle, P, ldp, part.data_ptr(), cp.data_ptr(), 0, stream)
         g.status()
-        assert torch.cuda.memory_allocated() == after_buffers >= before
+        free_after, _ = torch.cuda.mem_get_info()
+        assert free_after >= free_before, f"call {call}: {free_before - free_after} bytes of device memory went away"
         assert torch.equal(cp, ref[:P]), f"call {call}: cp differs from tfps_eval_batch"
     # too large for the built-in scratch: refused, nothing launched
     big_ldp = (tfps.NOALLOC_SCRATCH_BYTES // (8 * n) // 16 + 2) * 16
