@@ -56,6 +56,8 @@ def _get():
         lib.oracle_eval_partition.argtypes = (
             [ctypes.c_int64] + [P] * 8 + [ctypes.c_int32, P, P, P, ctypes.c_int64, P, P, ctypes.c_int64] + [P] * 6
         )
+        lib.oracle_eval_constraints.restype = ctypes.c_int
+        lib.oracle_eval_constraints.argtypes = [ctypes.c_int64, P, ctypes.c_int64, ctypes.c_int64, P, P, ctypes.c_int64, P, P, P, P]
         _lib = lib
     return _lib
 
@@ -164,3 +166,29 @@ def eval_batch(g: OracleGraph, k: int, s, C, B, S: int, part: np.ndarray,
         out.memload[:, i] = r.memload
         out.viol[i] = r.viol
     return out
+
+
+def eval_constraints(part: np.ndarray, pairs, devcons, cols: Optional[Sequence[int]] = None):
+    """Collocation constraints (Eq. 3: pairs of vertices that must share a device) and device constraints (Eq. 4:
+    (vertex, device) pairs that must hold) of the listed candidate columns of part[n][P].  Returns two int64 arrays:
+    the number of violated collocation pairs and of violated device constraints per candidate."""
+    lib = _get()
+    assert part.dtype == np.uint8 and part.ndim == 2
+    n = part.shape[0]
+    pairs = _arr(pairs, np.int32).reshape(-1, 2)
+    devcons = _arr(devcons, np.int32).reshape(-1, 2)
+    pa, pb = np.ascontiguousarray(pairs[:, 0]), np.ascontiguousarray(pairs[:, 1])
+    dv, dd = np.ascontiguousarray(devcons[:, 0]), np.ascontiguousarray(devcons[:, 1])
+    cols = list(range(part.shape[1])) if cols is None else list(cols)
+    coll = np.zeros(len(cols), np.int64)
+    dev = np.zeros(len(cols), np.int64)
+    for i, j in enumerate(cols):
+        col = part[:, j]
+        a, b = ctypes.c_int64(0), ctypes.c_int64(0)
+        rc = lib.oracle_eval_constraints(n, ctypes.c_void_p(col.ctypes.data), col.strides[0] if n > 1 else 1,
+                                         pairs.shape[0], _p(pa), _p(pb), devcons.shape[0], _p(dv), _p(dd),
+                                         ctypes.byref(a), ctypes.byref(b))
+        if rc:
+            raise OracleError(rc)
+        coll[i], dev[i] = a.value, b.value
+    return coll, dev

@@ -247,3 +247,31 @@ done:
     free(rt); free(tl); free(bl);
     return rc;
 }
+
+/*
+ * Placement constraints of one candidate partition p (uint8, byte stride pstride).
+ *   collocation constraints (Section 2, Eq. 3): for every listed pair (a, b), p(a) = p(b) must hold;
+ *   device constraints (Section 2, Eq. 4): for every listed pair (v, d), p(v) = d must hold.
+ * Every listed pair is one requirement; *coll_viol and *dev_viol count the requirements that do not hold
+ * (a vertex listed with two different devices therefore always violates at least one of them).
+ * Pins: tests/test_oracle_constraints.py (a worked example, closed forms on the partition v mod k, invariants).
+ */
+int oracle_eval_constraints(int64_t n, const uint8_t *p, int64_t pstride,
+                            int64_t npairs, const int32_t *pair_a, const int32_t *pair_b,
+                            int64_t ndev, const int32_t *dc_v, const int32_t *dc_d,
+                            int64_t *coll_viol, int64_t *dev_viol)
+{
+    int64_t cv = 0, dv = 0;
+    if (n < 0 || npairs < 0 || ndev < 0 || !coll_viol || !dev_viol) return ORACLE_BAD_ARG;
+    for (int64_t i = 0; i < npairs; ++i) {
+        if (pair_a[i] < 0 || pair_a[i] >= n || pair_b[i] < 0 || pair_b[i] >= n) return ORACLE_BAD_ARG;
+        if (p[(int64_t)pair_a[i] * pstride] != p[(int64_t)pair_b[i] * pstride]) ++cv;
+    }
+    for (int64_t i = 0; i < ndev; ++i) {
+        if (dc_v[i] < 0 || dc_v[i] >= n || dc_d[i] < 0 || dc_d[i] > 255) return ORACLE_BAD_ARG;
+        if ((int32_t)p[(int64_t)dc_v[i] * pstride] != dc_d[i]) ++dv;
+    }
+    *coll_viol = cv;
+    *dev_viol = dv;
+    return ORACLE_OK;
+}
