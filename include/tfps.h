@@ -79,6 +79,26 @@ const char* tfps_strerror(int status);
 const char* tfps_last_error(void);
 
 /*
+ * Tuning and test overrides.  The library chooses kernel family and block shape
+ * by itself; the environment variables below override single choices and exist
+ * for measurements and tests.  They are read at every call (TFPS_TILE_SPLIT,
+ * TFPS_STEP_ORDER, TFPS_LEAN*, TFPS_LEVREC when tfps_devices_set packs its
+ * records), change speed only, never results:
+ *   TFPS_LEAN=0 / TFPS_LEAN64=0 / TFPS_LEVREC=0   switch a kernel family off
+ *   TFPS_LEAN_FORCE_WIDE=1, TFPS_LEAN_ORDER=1|2    64-bit plan; plan in level order | in the caller's numbering
+ *   TFPS_LEAN_SLICE, TFPS_LEAN_CPT, TFPS_LEAN_DEPTH, TFPS_SLICED_CPT, TFPS_SLICED_WARPS, TFPS_SLICED_TABLE, TFPS_LEVEL32
+ *                                                  candidates per block / per lane, stage depth, warps, cost tables
+ *   TFPS_OVERLAP_LOADS=0, TFPS_OVERLAP_PASSES=0    loads kernel / backward pass on the caller's stream only
+ *   TFPS_LOADS2=0, TFPS_LOADS_CPT, TFPS_LOADS_BLOCKS_PER_SM   shape of the load kernel
+ *   TFPS_TILE_SPLIT                                edges per work item of the record passes (default 8)
+ *   TFPS_STEP_ORDER=1|2                            steps = topological levels | runs of the caller's numbering
+ *   TFPS_STEP_PERSISTENT=1, TFPS_STEP_GROUPS, TFPS_STEP_TILES, TFPS_STEP_RUN, TFPS_STEP_SHAPE, TFPS_STEP_BLOCKS
+ *                                                  persistent record pass and its shape
+ *   TFPS_WAIT_LIMIT                                polls before a device-side wait gives up (default 2^20;
+ *                                                  0 makes every wait run out at once: TFPS_ERR_TIMEOUT)
+ */
+
+/*
  * Build a graph handle (Section 2: G, c, t; optional per-vertex memory).
  *   n, m         vertices, edges (n < 2^26, m < 2^31 - 64; larger sizes give TFPS_ERR_UNSUPPORTED)
  *   in_ptr[n+1], in_src[m], in_t[m]     in-edge CSR: row v lists the sources u of edges u->v and their sizes
@@ -194,14 +214,30 @@ int tfps_eval_batch_host(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* p
 int tfps_phase_times(tfps_graph* g, float ms[3]);
 
 /*
- * Name of the pass kernel family the most recent tfps_eval_batch call on this handle chose
- * ("pass_window_kernel", "pass_sliced_kernel", "pass_tile_kernel", "pass_level_kernel"; "" before any call).
+ * Name of the pass kernel family the most recent tfps_eval_batch call on this handle chose ("" before any call):
+ *   "pass_lean_kernel"       candidate-sliced, shared-memory window, 32-bit levels inside (k <= 8, paths < 2^31)
+ *   "pass_lean64_kernel"     the same with 64-bit levels (k <= 16)
+ *   "pass_sliced_kernel"     candidate-sliced without a window (neighbours through L2)
+ *   "pass_stepchain_kernel"  step-synchronous on vertex records, one chained launch per step (k <= 64)
+ *   "pass_steprec_kernel"    the same as one persistent cooperative launch with bounded barriers (opt-in)
+ *   "pass_level_kernel"      step-synchronous with a division per relaxation (any device table)
  * The string is static.
  */
 const char* tfps_last_pass_kernel(const tfps_graph* g);
 
 /* Number of kernels this library has launched in the calling process so far. */
 int64_t tfps_kernel_launches(void);
+
+/*
+ * Diagnostic (no counterpart in the paper): the rate, in GB/s, at which the SMs of
+ * the current device gather pseudo-random 1 KiB row segments of a buffer of
+ * `working_set_bytes` (16 bytes per lane and load, every warp reads `rows_per_warp`
+ * rows).  It is the access pattern of the step-synchronous passes -- a neighbour's
+ * levels and ids for one tile of candidates -- without their arithmetic, and so
+ * the ceiling those passes can reach.  Allocates and frees its own buffer,
+ * synchronises the device.  *gbytes_per_s is a host output.
+ */
+int tfps_probe_gather_bandwidth(size_t working_set_bytes, int rows_per_warp, double* gbytes_per_s);
 
 /*
  * Critical-path lengths without any allocation.  (The paper has no counterpart

@@ -9,8 +9,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libtfps.so")
-SOURCES = ["api.cu", "topo.cu", "passes.cu", "window.cu", "lean.cu", "lean64.cu", "levrec.cu", "loads.cu"]
-HEADERS = [os.path.join(CSRC, "common.cuh"), os.path.join(ROOT, "include", "tfps.h")]
+SOURCES = ["api.cu", "topo.cu", "passes.cu", "lean.cu", "lean64.cu", "levrec.cu", "loads.cu", "probe.cu"]
+HEADERS = [os.path.join(CSRC, "common.cuh"), os.path.join(CSRC, "ptx.cuh"), os.path.join(ROOT, "include", "tfps.h")]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a",

@@ -133,11 +133,6 @@ struct tfps_graph {
     DBuf f_eptr, f_nbr, f_t, b_eptr, b_nbr, b_t;
     // chunk tables of the candidate-sliced pass
     DBuf vertf, f_chunks, b_chunks;
-    // work items of the tile kernel per direction: vertices with many edges cut into partial items, heaviest first
-    DBuf items[2], heavy[2];
-    std::vector<long long> h_item_ptr[2];
-    std::vector<int> h_items[2];
-    int heavy_count[2] = {0, 0};
     int f_num_chunks = 0, b_num_chunks = 0;
     bool f_all_staged = true, b_all_staged = true;
     int max_chunk_v = 1;
@@ -149,14 +144,10 @@ struct tfps_graph {
     DBuf rtv;          // [n][rt_kp] runtime of every vertex on every device (loads kernel)
     int rt_kp = 0;     // table width: power of two >= k, or 0 when k is too large for the table
     DBuf pair_f, pair_b, cls_div, sel_f, sel_b;
-    // windowed pass: neighbour positions, comb tables, precomputed edge values
-    DBuf pos_of, npos_f, npos_b, cls2_f, cls2_b, comb_f, comb_b, V_f, V_b, V32_f, V32_b;
-    int ncomb = 0, maxspan = 0, smem_optin = 0;
+    // level position of every vertex; longest edge in level positions
+    DBuf pos_of;
+    int maxspan = 0, smem_optin = 0;
     bool fits32 = false;  // every path length under any partition fits int32
-    // packed chunk records of the windowed pass, [direction][0: int64 values, 1: int32 values]
-    DBuf blob[2][2], blob_desc[2][2];
-    int blob_head_max[2][2] = {}, blob_body_max[2][2] = {};
-    std::vector<int> h_chunks[2];
     // host copies of the in-edge CSR for the worst-case path bound
     std::vector<long long> h_in_ptr, h_in_t;
     std::vector<int> h_in_src, h_c;
@@ -194,6 +185,9 @@ struct tfps_graph {
     // low-priority stream on which the loads kernel runs beside the lean passes (created by tfps_devices_set)
     cudaStream_t aux_stream = nullptr;
     cudaEvent_t aux_fork = nullptr, aux_join = nullptr;
+    // second pass stream: the backward lean pass runs beside the forward one (both only read the ids)
+    cudaStream_t pass2_stream = nullptr;
+    cudaEvent_t pass2_join = nullptr;
     ~tfps_graph()
     {
         for (cudaEvent_t e : ev)
@@ -204,6 +198,8 @@ struct tfps_graph {
         if (aux_fork) cudaEventDestroy(aux_fork);
         if (aux_join) cudaEventDestroy(aux_join);
         if (aux_stream) cudaStreamDestroy(aux_stream);
+        if (pass2_join) cudaEventDestroy(pass2_join);
+        if (pass2_stream) cudaStreamDestroy(pass2_stream);
     }
 };
 
@@ -317,10 +313,7 @@ int build_topo(tfps_graph* g, cudaStream_t st)
         CUDA_TRY(span.alloc(sizeof(int)));
         CUDA_TRY(cudaMemsetAsync(span.p, 0, sizeof(int), st));
         CUDA_TRY(g->pos_of.alloc(sizeof(int) * (size_t)n));
-        CUDA_TRY(g->npos_f.alloc(sizeof(int) * (size_t)m));
-        CUDA_TRY(g->npos_b.alloc(sizeof(int) * (size_t)m));
-        CUDA_TRY(launch_positions(n, m, g->order.as<int>(), g->pos_of.as<int>(), g->f_nbr.as<int>(), g->b_nbr.as<int>(),
-                                  g->f_eptr.as<int>(), g->npos_f.as<int>(), g->npos_b.as<int>(), span.as<int>(), st));
+        CUDA_TRY(launch_positions(n, g->order.as<int>(), g->pos_of.as<int>(), g->f_nbr.as<int>(), g->f_eptr.as<int>(), span.as<int>(), st));
         CUDA_TRY(cudaMemcpyAsync(&g->maxspan, span.p, sizeof(int), cudaMemcpyDeviceToHost, st));
         CUDA_TRY(cudaStreamSynchronize(st));
     }
@@ -358,45 +351,7 @@ int build_topo(tfps_graph* g, cudaStream_t st)
                 p = q;
             }
         }
-        {
-            // a vertex with more than `over` (default T) edges becomes ceil(deg/T) partial items of at most T edges
-            const int T = std::max(0, env_int("TFPS_TILE_SPLIT", 8));
-            // largest degree left whole.  T edges: at P = 4,096 config 5's forward pass takes the same time as with 2*T
-            // (28.1 ms), at P = 1,024 it takes 11.2 instead of 15.6 ms (the level's longest chain is halved)
-            const int over = std::max(T, env_int("TFPS_TILE_SPLIT_OVER", T));
-            std::vector<int> items, heavy, idx;
-            std::vector<long long>& ip = g->h_item_ptr[dir];
-            ip.assign((size_t)g->num_levels + 1, 0);
-            for (int l = 0; l < g->num_levels; ++l) {
-                ip[l] = (long long)(items.size() / 4);
-                idx.clear();
-                for (int p = (int)g->h_level_ptr[l]; p < (int)g->h_level_ptr[l + 1]; ++p) idx.push_back(p);
-                std::stable_sort(idx.begin(), idx.end(), [&](int x, int y) { return eptr[x + 1] - eptr[x] > eptr[y + 1] - eptr[y]; });
-                for (int p : idx) {
-                    const int e0 = eptr[p], e1 = eptr[p + 1];
-                    if (T > 0 && e1 - e0 > over) {
-                        heavy.push_back(p);
-                        for (int e = e0; e < e1; e += T) { items.push_back(p); items.push_back(e); items.push_back(std::min(e1, e + T)); items.push_back(1); }
-                    } else {
-                        items.push_back(p); items.push_back(e0); items.push_back(e1); items.push_back(0);
-                    }
-                }
-            }
-            ip[g->num_levels] = (long long)(items.size() / 4);
-            if (!heavy.empty()) {   // positions -> vertex ids (rows of the level matrices)
-                std::vector<int> h_order((size_t)n);
-                CUDA_TRY(cudaMemcpyAsync(h_order.data(), g->order.p, sizeof(int) * (size_t)n, cudaMemcpyDeviceToHost, st));
-                CUDA_TRY(cudaStreamSynchronize(st));
-                for (int& x : heavy) x = h_order[x];
-            }
-            g->heavy_count[dir] = (int)heavy.size();
-            g->h_items[dir] = items;
-            TFPS_TRY(upload(g->items[dir], items, st));
-            TFPS_TRY(upload(g->heavy[dir], heavy, st));
-            CUDA_TRY(cudaStreamSynchronize(st));
-        }
         (dir == 0 ? g->f_num_chunks : g->b_num_chunks) = (int)(chunks.size() / 4);
-        g->h_chunks[dir] = chunks;
         TFPS_TRY(upload(dir == 0 ? g->f_chunks : g->b_chunks, chunks, st));
         CUDA_TRY(cudaStreamSynchronize(st));
     }
@@ -433,7 +388,6 @@ PassArgs make_args(const tfps_graph* g, bool fwd, long long P, long long ldp, co
     a.adj.xw = fwd ? g->xw_f.as<unsigned long long>() : g->xw_b.as<unsigned long long>();
     a.adj.xnbr = fwd ? g->xnbr_f.as<unsigned long long>() : nullptr;
     a.adj.xvert = g->xvert.as<unsigned long long>();
-    a.adj.items = g->items[fwd ? 0 : 1].as<int4>();
     a.tab = make_tables(g);
     a.level_ptr = g->level_ptr_d.as<long long>();
     a.num_levels = g->num_levels;
@@ -1187,45 +1141,6 @@ int tfps_devices_set(tfps_graph* g, int k, const int32_t* s, const int64_t* C, c
         TFPS_TRY(upload(g->sel_f, sf, st));
         TFPS_TRY(upload(g->sel_b, sb, st));
 
-        // comb ids for the windowed pass: (transfer class or "same device", speed class), or the pair itself
-        const int ncs = (int)svals.size();
-        int ncomb = 0;
-        const bool by_class = use_cls && (ncw + 1) * ncs <= COMB_MAX;
-        if (by_class) ncomb = (ncw + 1) * ncs;
-        else if (k * k <= COMB_MAX) ncomb = k * k;
-        g->ncomb = ncomb;
-        if (ncomb > 0) {
-            std::vector<uint8_t> c2f((size_t)k * k), c2b((size_t)k * k);
-            std::vector<CombDiv> cf((size_t)COMB_MAX), cb((size_t)COMB_MAX);
-            const DivConst none = DivConst{0ull, 0u, 1u};
-            for (auto& x : cf) { x.w = none; x.s = make_div(1); }
-            for (auto& x : cb) { x.w = none; x.s = make_div(1); }
-            for (int nb = 0; nb < k; ++nb)
-                for (int vv = 0; vv < k; ++vv) {
-                    const int i = nb * k + vv;
-                    const bool same = nb == vv;
-                    const long long bf = same ? 0 : B[nb * k + vv], bb = same ? 0 : B[vv * k + nb];
-                    int idf, idb;
-                    if (by_class) {
-                        idf = (same ? ncw : cls_of(wvals, bf)) * ncs + cls_of(svals, s[nb]);
-                        idb = (same ? ncw : cls_of(wvals, bb)) * ncs + cls_of(svals, s[vv]);
-                    } else {
-                        idf = idb = i;
-                    }
-                    c2f[i] = (uint8_t)idf;
-                    c2b[i] = (uint8_t)idb;
-                    cf[idf].w = same ? none : make_div((unsigned long long)bf);
-                    cf[idf].s = make_div((unsigned long long)s[nb]);
-                    cb[idb].w = same ? none : make_div((unsigned long long)bb);
-                    cb[idb].s = make_div((unsigned long long)s[vv]);
-                }
-            TFPS_TRY(upload(g->cls2_f, c2f, st));
-            TFPS_TRY(upload(g->cls2_b, c2b, st));
-            TFPS_TRY(upload(g->comb_f, cf, st));
-            TFPS_TRY(upload(g->comb_b, cb, st));
-        }
-    } else {
-        g->ncomb = 0;
     }
     TFPS_TRY(upload(g->rt_div, rt, st));
     TFPS_TRY(upload(g->w_div, w, st));
@@ -1272,64 +1187,6 @@ int tfps_devices_set(tfps_graph* g, int k, const int32_t* s, const int64_t* C, c
         TFPS_TRY(build_lean(g, k, s, B, scale, order, st));
         TFPS_TRY(build_levrec(g, k, s, B, scale, order, st));
     }
-    if (g->ncomb > 0 && n > 0) {
-        CUDA_TRY(g->V_f.reserve(sizeof(long long) * (size_t)m * g->ncomb + 16));
-        CUDA_TRY(g->V_b.reserve(sizeof(long long) * (size_t)m * g->ncomb + 16));
-        if (g->fits32) {
-            CUDA_TRY(g->V32_f.reserve(sizeof(int) * (size_t)m * g->ncomb + 16));
-            CUDA_TRY(g->V32_b.reserve(sizeof(int) * (size_t)m * g->ncomb + 16));
-        }
-        CUDA_TRY(launch_edge_values(n, g->f_eptr.as<int>(), g->xw_f.as<unsigned long long>(),
-                                    g->xnbr_f.as<unsigned long long>(), g->xvert.as<unsigned long long>(),
-                                    g->comb_f.as<CombDiv>(), g->ncomb, g->V_f.as<long long>(),
-                                    g->fits32 ? g->V32_f.as<int>() : nullptr, st));
-        CUDA_TRY(launch_edge_values(n, g->b_eptr.as<int>(), g->xw_b.as<unsigned long long>(), nullptr,
-                                    g->xvert.as<unsigned long long>(), g->comb_b.as<CombDiv>(), g->ncomb,
-                                    g->V_b.as<long long>(), g->fits32 ? g->V32_b.as<int>() : nullptr, st));
-    }
-    if (g->ncomb > 0 && n > 0) {
-        auto up16 = [](size_t x) { return (x + 15) & ~(size_t)15; };
-        for (int dir = 0; dir < 2; ++dir)
-            for (int narrow = 0; narrow < (g->fits32 ? 2 : 1); ++narrow) {
-                const size_t ls = narrow ? 4 : 8;
-                const std::vector<int>& ch = g->h_chunks[dir];
-                const int nc = (int)(ch.size() / 4);
-                std::vector<int> desc((size_t)nc * 8, 0);
-                size_t off = 0;
-                int head_max = 16, body_max = 16;
-                for (int c = 0; c < nc; ++c) {
-                    const size_t cnt = (size_t)ch[4 * c + 1];
-                    const size_t es = ch[4 * c + 3] <= CHUNK_E ? (size_t)ch[4 * c + 3] : 0;
-                    const size_t head = 16 + up16(4 * cnt);
-                    const size_t nbr_bytes = up16(4 * es);
-                    const size_t body = up16(4 * (cnt + 1)) + up16(8 * cnt) + up16(4 * es) + up16(ls * es * (size_t)g->ncomb) + nbr_bytes;
-                    desc[8 * c + 0] = (int)(off / 16);
-                    desc[8 * c + 1] = (int)head;
-                    off += head;
-                    desc[8 * c + 2] = (int)(off / 16);
-                    desc[8 * c + 3] = (int)body;
-                    off += body;
-                    desc[8 * c + 4] = (int)(body - nbr_bytes);
-                    desc[8 * c + 5] = (int)cnt;
-                    head_max = std::max(head_max, (int)head);
-                    body_max = std::max(body_max, (int)body);
-                }
-                if (off / 16 >= (size_t)1 << 31) return fail(TFPS_ERR_UNSUPPORTED, "chunk records exceed 32 GiB");
-                g->blob_head_max[dir][narrow] = head_max;
-                g->blob_body_max[dir][narrow] = body_max;
-                CUDA_TRY(g->blob[dir][narrow].reserve(off + 16));
-                TFPS_TRY(upload(g->blob_desc[dir][narrow], desc, st));
-                const void* V = narrow ? (dir == 0 ? g->V32_f.p : g->V32_b.p) : (dir == 0 ? g->V_f.p : g->V_b.p);
-                CUDA_TRY(launch_pack_chunks(nc, dir == 0 ? g->f_chunks.as<int>() : g->b_chunks.as<int>(),
-                                            g->blob_desc[dir][narrow].as<int>(), g->vertf.as<int>(),
-                                            dir == 0 ? g->f_eptr.as<int>() : g->b_eptr.as<int>(),
-                                            g->xvert.as<unsigned long long>(),
-                                            dir == 0 ? g->npos_f.as<int>() : g->npos_b.as<int>(),
-                                            dir == 0 ? g->f_nbr.as<int>() : g->b_nbr.as<int>(), V, g->ncomb, (int)ls,
-                                            g->blob[dir][narrow].as<unsigned char>(), st));
-                CUDA_TRY(cudaStreamSynchronize(st));  // desc (host vector) was uploaded asynchronously
-            }
-    }
     CUDA_TRY(cudaStreamSynchronize(st));
     if (!g->aux_stream) {
         int lo = 0, hi = 0;
@@ -1337,6 +1194,8 @@ int tfps_devices_set(tfps_graph* g, int k, const int32_t* s, const int64_t* C, c
         CUDA_TRY(cudaStreamCreateWithPriority(&g->aux_stream, cudaStreamNonBlocking, lo));
         CUDA_TRY(cudaEventCreateWithFlags(&g->aux_fork, cudaEventDisableTiming));
         CUDA_TRY(cudaEventCreateWithFlags(&g->aux_join, cudaEventDisableTiming));
+        CUDA_TRY(cudaStreamCreateWithFlags(&g->pass2_stream, cudaStreamNonBlocking));
+        CUDA_TRY(cudaEventCreateWithFlags(&g->pass2_join, cudaEventDisableTiming));
     }
     if (g->device >= 0 && g->device < 128) {
         void* scratch = nullptr;   // resolve the built-in scratch of tfps_eval_cp_noalloc now, not in the evaluation call
@@ -1478,7 +1337,7 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
 
     const int level_bytes = (g->fits32 && env_int("TFPS_LEVEL32", 1) != 0) ? 4 : 8;
     // Lean windowed pass (32-bit levels, whole window resident, host-packed records): block shape for one direction.
-    struct LeanChoice { bool ok = false; int slice = 0, warps = 0; size_t smem = 0; LeanArgs args; };
+    struct LeanChoice { bool ok = false; int slice = 0, cpt = 4, warps = 0; size_t smem = 0; LeanArgs args; };
     auto pick_lean = [&](bool fwd) {
         LeanChoice ch;
         if (!(sliced && g->lean[0].ok && g->lean[1].ok && ((uintptr_t)part & 15u) == 0 && ldp < (1LL << 28) &&
@@ -1503,7 +1362,15 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
             }
             else if (forced == 1 || forced == 2 || forced == 4) { if (slice != 32 * forced) continue; }
             else if ((P + slice - 1) / slice < want_slices && slice > slice_min) continue;
-            const int vpw = 128 / slice, pr = std::max(1, slice / 16);
+            // candidates per lane of the narrow kernel: 4; 2 where the levels are narrow and the slices small, so that a
+            // level's dependent chain is shorter (config 4: 8.75 against 9.69 ms per step); TFPS_LEAN_CPT forces 1, 2 or 4
+            int cpt = 4;
+            if (!lp.wide) {
+                if (lp.max_sub <= 32 && slice <= 32) cpt = 2;
+                const int want_cpt = env_int("TFPS_LEAN_CPT", 0);
+                if ((want_cpt == 1 && slice <= 32) || (want_cpt == 2 && slice <= 64) || want_cpt == 4) cpt = want_cpt;
+            }
+            const int vpw = 32 * cpt / slice, pr = std::max(1, slice / 16);
             // warps: one round of the vertex groups covers the widest chunk, up to 16 warps (512 threads with up to
             // 128 registers each measured faster than 1024 threads with 64: 2.95 against 3.21 ms on config 3)
             int w = 1;
@@ -1516,7 +1383,7 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
                 unsigned slot_stride = 0, stage_bytes = 0;
                 const size_t need = lean_smem_bytes(lp, slice, w, d, &slot_stride, &stage_bytes);
                 if (need + 1024 <= (size_t)g->smem_optin) {
-                    ch.ok = true; ch.slice = slice; ch.warps = w; ch.smem = need;
+                    ch.ok = true; ch.slice = slice; ch.cpt = cpt; ch.warps = w; ch.smem = need;
                     ch.args.slot_stride = slot_stride;
                     ch.args.stage_bytes = stage_bytes;
                     ch.args.depth = d;
@@ -1551,62 +1418,16 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
     // the loads kernel then runs on a low-priority stream beside them and fills the SMs the passes' last wave leaves idle.
     const bool overlap = (load || ml) && (need_fwd || need_bwd) && (!need_fwd || lean_f.ok) && (!need_bwd || lean_b.ok) &&
                          g->aux_stream && env_int("TFPS_OVERLAP_LOADS", 1) != 0;
+    // Both lean passes only read the ids and write their own level matrix: the backward pass then runs on a second
+    // stream beside the forward pass, so that the blocks of both fill the machine together (config 3: 2 x 256 blocks
+    // are 3.5 waves of 148 instead of 2 x 2).  Not with phase timing, which brackets the passes on one stream.
+    const bool overlap_passes = overlap && need_fwd && need_bwd && !profile && g->pass2_stream && env_int("TFPS_OVERLAP_PASSES", 1) != 0;
     if (!overlap) TFPS_TRY(run_loads(st));   // loads first: the same kernel checks the ids, and a bad id stops everything after it
     else {
         CUDA_TRY(cudaEventRecord(g->aux_fork, st));
         CUDA_TRY(cudaStreamWaitEvent(g->aux_stream, g->aux_fork, 0));
     }
     if (profile) CUDA_TRY(cudaEventRecord(g->ev[1], st));
-    // windowed pass: needs the precomputed edge values (simple device tables)
-    // (its bulk copies of id rows need a 16-byte aligned id matrix)
-    bool use_window = sliced && g->ncomb > 0 && env_int("TFPS_WINDOW", 1) != 0 && ((uintptr_t)part & 15u) == 0;
-    int win_R = 0, win_depth = 1;
-    const int narrow = level_bytes == 4 ? 1 : 0;
-    const int head_max = std::max(g->blob_head_max[0][narrow], g->blob_head_max[1][narrow]);
-    const int body_max = std::max(g->blob_body_max[0][narrow], g->blob_body_max[1][narrow]);
-    const int win_warps = std::min(32, std::max(2, warps + 1));   // consumer warps plus the producer warp
-    if (use_window) {
-        int r_need = 32;  // smallest power of two that keeps every edge inside the ring
-        while (r_need < g->maxspan + CHUNK_V) r_need <<= 1;
-        auto r_fit = [&](int c, int d) {
-            const long long avail = (long long)g->smem_optin - 1024 -
-                                    (long long)window_smem_bytes(k, 0, c, win_warps, level_bytes, g->max_chunk_v, head_max, body_max, d);
-            const long long rmax = avail / (32LL * c * (level_bytes + 1));
-            int r = 0;
-            for (int q = 32; q <= rmax && q <= (1 << 16); q <<= 1) r = q;
-            return r;
-        };
-        // staging depth: about 256 vertices of adjacency and ids in flight ahead of the chunk being processed
-        int d_want = env_int("TFPS_WINDOW_DEPTH", 0);
-        if (d_want < 1 || d_want > 8) d_want = std::max(2, std::min(8, (256 + g->max_chunk_v - 1) / g->max_chunk_v));
-        const int forced = env_int("TFPS_SLICED_CPT", 0);
-        int chosen = 0;
-        if (forced == 1 || forced == 2 || forced == 4) chosen = forced;
-        const long long want_slices = std::min<long long>((3LL * g->sm_count) / 4, (P + 31) / 32);
-        win_depth = 0;
-        for (int c = chosen ? chosen : 4; c >= 1 && !win_depth; c >>= 1) {   // widest lane that holds the whole window
-            if (!chosen && (P + 32 * c - 1) / (32 * c) < want_slices && c > 1) continue;
-            for (int d = d_want; d >= 1 && !win_depth; --d)
-                if (r_fit(c, d) >= r_need) { cpt = c; win_depth = d; }
-            if (chosen) break;
-        }
-        if (!win_depth) {   // partial window at the width the slice count allows
-            cpt = chosen ? chosen : (cpt > 4 ? 4 : cpt);
-            win_depth = std::min(d_want, 2);
-        }
-        win_R = std::min(r_fit(cpt, win_depth), r_need);
-        const int forced_r = env_int("TFPS_WINDOW_R", -1);
-        if (forced_r >= 0) {
-            int q = 0;
-            for (int t = 32; t <= forced_r; t <<= 1) q = t;
-            win_R = std::min(q, r_fit(cpt, win_depth));
-        }
-        if (win_R < CHUNK_V + 32) win_R = 0;
-        if (window_smem_bytes(k, win_R, cpt, win_warps, level_bytes, g->max_chunk_v, head_max, body_max, win_depth) >
-            (size_t)g->smem_optin)
-            use_window = false;
-    }
-
     for (int pass = 0; pass < 2; ++pass) {
         const bool fwd = pass == 0;
         if (profile && !fwd) CUDA_TRY(cudaEventRecord(g->ev[2], st));
@@ -1614,16 +1435,22 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
         long long* lev = fwd ? fwd_lev : (long long*)blevel;
         long long* cp_here = (cp && (fwd || !need_fwd)) ? (long long*)cp : nullptr;
         PassArgs a = make_args(g, fwd, P, ldp, part, lev, cp_here);
-        g->last_kernel = use_window ? "pass_window_kernel" : (sliced ? "pass_sliced_kernel" : (g->npass > 0 ? "pass_tile_kernel" : "pass_level_kernel"));
+        g->last_kernel = sliced ? "pass_sliced_kernel" : "pass_level_kernel";
         {
             LeanChoice& ch = fwd ? lean_f : lean_b;
             if (ch.ok) {
                 ch.args.lev = lev;
                 ch.args.cp = cp_here;
                 g->last_kernel = ch.args.plan.wide ? "pass_lean64_kernel" : "pass_lean_kernel";
-                if (ch.args.plan.wide) CUDA_TRY(launch_pass_lean64(ch.args, fwd, ch.slice, ch.warps, ch.smem, st));
-                else CUDA_TRY(launch_pass_lean(ch.args, fwd, ch.slice, ch.warps, ch.smem, st));
-                if (overlap && fwd == need_fwd) {
+                cudaStream_t ps = st;
+                if (overlap_passes && !fwd) {
+                    ps = g->pass2_stream;
+                    CUDA_TRY(cudaStreamWaitEvent(ps, g->aux_fork, 0));
+                }
+                if (ch.args.plan.wide) CUDA_TRY(launch_pass_lean64(ch.args, fwd, ch.slice, ch.warps, ch.smem, ps));
+                else CUDA_TRY(launch_pass_lean(ch.args, fwd, ch.slice, ch.cpt, ch.warps, ch.smem, ps));
+                if (overlap_passes && !fwd) CUDA_TRY(cudaEventRecord(g->pass2_join, ps));
+                if (overlap && (overlap_passes ? !fwd : fwd == need_fwd)) {
                     // the first pass is queued: now the loads, so that the pass gets the machine first
                     TFPS_TRY(run_loads(g->aux_stream));
                     CUDA_TRY(cudaEventRecord(g->aux_join, g->aux_stream));
@@ -1631,29 +1458,7 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
                 continue;
             }
         }
-        if (use_window) {
-            WindowPlan wp;
-            wp.vertf = g->vertf.as<int>();
-            wp.chunks = fwd ? g->f_chunks.as<int>() : g->b_chunks.as<int>();
-            wp.num_chunks = fwd ? g->f_num_chunks : g->b_num_chunks;
-            wp.src_end = (int)g->h_level_ptr[1];
-            wp.npos = fwd ? g->npos_f.as<int>() : g->npos_b.as<int>();
-            wp.V = level_bytes == 4 ? (fwd ? g->V32_f.p : g->V32_b.p) : (fwd ? g->V_f.p : g->V_b.p);
-            wp.level_bytes = level_bytes;
-            wp.desc = g->blob_desc[fwd ? 0 : 1][narrow].as<int>();
-            wp.blob = g->blob[fwd ? 0 : 1][narrow].as<unsigned char>();
-            wp.max_v = g->max_chunk_v;
-            wp.head_max = head_max;
-            wp.body_max = body_max;
-            wp.depth = win_depth;
-            wp.static_rounds = std::max(1, env_int("TFPS_WINDOW_STATIC_ROUNDS", 1));
-            wp.cls2 = fwd ? g->cls2_f.as<uint8_t>() : g->cls2_b.as<uint8_t>();
-            wp.ncomb = g->ncomb;
-            wp.R = win_R;
-            wp.maxspan = g->maxspan;
-            wp.all_staged = (fwd ? g->f_all_staged : g->b_all_staged) ? 1 : 0;
-            CUDA_TRY(launch_pass_window(a, fwd, wp, cpt, win_warps, st));
-        } else if (sliced) {
+        if (sliced) {
             SlicedPlan plan;
             plan.vertf = g->vertf.as<int>();
             plan.chunks = fwd ? g->f_chunks.as<int>() : g->b_chunks.as<int>();
@@ -1661,14 +1466,8 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
             plan.src_end = (int)g->h_level_ptr[1];
             CUDA_TRY(launch_pass_sliced(a, fwd, plan, cpt, warps, table, st));
         } else {
-            // the value-array kernel is opt-in: the tile kernel measured faster on the wide power-law graph (config 5)
-            if (g->ncomb > 0 && env_int("TFPS_LEVEL_VALUES", 0) != 0) {
-                g->last_kernel = "pass_levelv_kernel";
-                CUDA_TRY(launch_pass_level_values(a, fwd, g->h_level_ptr, fwd ? g->V_f.as<long long>() : g->V_b.as<long long>(),
-                                                  fwd ? g->cls2_f.as<uint8_t>() : g->cls2_b.as<uint8_t>(), g->ncomb, st));
-            } else {
+            {
                 {
-                    // rows of the vertices that are evaluated in partial items start at zero
                     const int dirn = fwd ? 0 : 1;
                     const bool rec = g->levrec[dirn].ok && env_int("TFPS_LEVREC", 1) != 0;
                     if (rec) {   // vertex records (k <= 64): no divisions or per-edge tables in the kernel
@@ -1696,10 +1495,8 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
                             g->last_kernel = "pass_stepchain_kernel";
                             CUDA_TRY(launch_pass_stepchain(la, fwd, L.h_step_ptr, st));
                         }
-                    } else {
-                        if (g->npass > 0 && g->heavy_count[dirn] > 0)
-                            CUDA_TRY(launch_zero_rows(g->heavy[dirn].as<int>(), g->heavy_count[dirn], P, ldp, lev, st));
-                        CUDA_TRY(launch_pass_level_sync(a, fwd, g->h_level_ptr, st, &g->h_item_ptr[dirn]));
+                    } else {   // runtimes beyond int32 or more than 255 distinct bandwidths: division per relaxation
+                        CUDA_TRY(launch_pass_level_sync(a, fwd, g->h_level_ptr, st));
                     }
                 }
             }
@@ -1711,6 +1508,7 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
         }
     }
     if (overlap) CUDA_TRY(cudaStreamWaitEvent(st, g->aux_join, 0));
+    if (overlap_passes) CUDA_TRY(cudaStreamWaitEvent(st, g->pass2_join, 0));
     if (profile) {
         CUDA_TRY(cudaEventRecord(g->ev[3], st));
         g->ev_valid = true;

@@ -79,7 +79,6 @@ struct LevelAdj {
     const unsigned long long* xw;    // [m]   transfer numerator ((t*S-1)<<2 or NUM_ZERO)
     const unsigned long long* xnbr;  // [m]   neighbour's runtime numerator ((c*S-1)<<2 or NUM_ZERO)
     const unsigned long long* xvert; // [n]   own runtime numerator by position
-    const int4* items;               // work items of the tile kernel {position, first edge, end edge, partial}, by level (or NULL)
 };
 
 struct PassArgs {
@@ -106,40 +105,6 @@ struct SlicedPlan {
     const int* chunks;   // [num_chunks][4] = {first position, vertices, first edge, edges}
     int num_chunks;
     int src_end;         // positions below this are sources (level 0)
-};
-
-// Precomputed edge values for the windowed pass.  When the device tables are
-// simple enough the cost of an edge takes at most COMB_MAX distinct values over
-// all (neighbour device, vertex device) pairs: comb id = cls2[nb*k+vv], and
-// V[e*ncomb + c] holds the cost of edge e for comb c (same meaning as the table
-// T of the sliced pass), filled once per tfps_devices_set.
-constexpr int COMB_MAX = 16;
-
-struct CombDiv {
-    DivConst w;   // transfer divisor; w.pad != 0: no transfer term (same device)
-    DivConst s;   // speed divisor
-};
-
-struct WindowPlan {
-    const int* vertf;            // [n] vertex id by position, bit 31 set for sinks
-    const int* chunks;           // [num_chunks][4]
-    int num_chunks;
-    int src_end;
-    const int* npos;             // [m] position of the neighbour (level-ordered adjacency of this direction)
-    const void* V;               // [m][ncomb] edge values: int64, or int32 when level_bytes == 4
-    int level_bytes;             // 8, or 4 when every path length is known to fit int32
-    const uint8_t* cls2;         // [k*k] comb id of (nb, vv)
-    int ncomb;
-    int R;                       // window length in positions: a power of two, or 0 for no window
-    int maxspan;                 // largest |pos(v) - pos(u)| over all edges
-    int all_staged;              // no vertex has more than CHUNK_E edges
-    // packed chunk records staged by bulk copies: desc[2*c] = {head offset/16, head bytes, body offset/16, body bytes},
-    // desc[2*c+1] = {body bytes without the trailing neighbour-id array, vertices, 0, 0}
-    const int* desc;
-    const unsigned char* blob;
-    int max_v, head_max, body_max;  // largest chunk: vertices, head bytes, body bytes
-    int depth;                   // chunks staged ahead
-    int static_rounds;           // chunks of at most this many vertices per consumer warp use a fixed vertex assignment
 };
 
 // Lean windowed pass (32-bit levels, k <= LEAN_K_MAX, whole window resident).  The host packs, per direction
@@ -225,7 +190,7 @@ cudaError_t launch_pass_steprec(const LevRecArgs& a, bool fwd, int sm_count, cud
 cudaError_t launch_pass_stepchain(const LevRecArgs& a, bool fwd, const std::vector<int>& step_ptr_host, cudaStream_t st);
 
 size_t lean_smem_bytes(const LeanPlan& plan, int slice, int warps, int depth, unsigned* slot_stride, unsigned* stage_bytes);
-cudaError_t launch_pass_lean(const LeanArgs& a, bool fwd, int slice, int warps, size_t smem, cudaStream_t st);
+cudaError_t launch_pass_lean(const LeanArgs& a, bool fwd, int slice, int cpt, int warps, size_t smem, cudaStream_t st);
 cudaError_t launch_pass_lean64(const LeanArgs& a, bool fwd, int slice, int warps, size_t smem, cudaStream_t st);
 
 // every kernel launch of the library goes through the wrappers below and is counted here
@@ -246,23 +211,12 @@ cudaError_t launch_numerators(int n, int m, long long S, const int* order, const
 cudaError_t launch_default_mem(int n, const long long* out_ptr, const long long* out_t, long long* mem, cudaStream_t st);
 
 int pick_cpt(long long P);
-cudaError_t launch_pass_level_sync(const PassArgs& a, bool fwd, const std::vector<long long>& level_ptr_host, cudaStream_t st,
-                                   const std::vector<long long>* item_ptr_host = nullptr);
+cudaError_t launch_pass_level_sync(const PassArgs& a, bool fwd, const std::vector<long long>& level_ptr_host, cudaStream_t st);
 cudaError_t launch_zero_rows(const int* rows, int count, long long P, long long ldp, long long* lev, cudaStream_t st);
-cudaError_t launch_pass_level_values(const PassArgs& a, bool fwd, const std::vector<long long>& level_ptr_host,
-                                     const long long* V, const uint8_t* cls2, int ncomb, cudaStream_t st);
 cudaError_t launch_pass_sliced(const PassArgs& a, bool fwd, const SlicedPlan& plan, int cpt, int warps, bool table,
                                cudaStream_t st);
-cudaError_t launch_pass_window(const PassArgs& a, bool fwd, const WindowPlan& plan, int cpt, int warps, cudaStream_t st);
-size_t window_smem_bytes(int k, int R, int cpt, int warps, int level_bytes, int max_v, int head_max, int body_max, int depth);
-cudaError_t launch_pack_chunks(int num_chunks, const int* chunks, const int* desc, const int* vertf, const int* eptr,
-                               const unsigned long long* xvert, const int* npos, const int* nbr, const void* V, int ncomb,
-                               int lsize, unsigned char* blob, cudaStream_t st);
-cudaError_t launch_edge_values(int n, const int* eptr, const unsigned long long* xw, const unsigned long long* xnbr,
-                               const unsigned long long* xvert, const CombDiv* comb, int ncomb, long long* V, int* V32,
-                               cudaStream_t st);
-cudaError_t launch_positions(int n, int m, const int* order, int* pos_of, const int* nbr_f, const int* nbr_b,
-                             const int* eptr_f, int* npos_f, int* npos_b, int* maxspan, cudaStream_t st);
+cudaError_t launch_positions(int n, const int* order, int* pos_of, const int* nbr_f, const int* eptr_f, int* maxspan,
+                             cudaStream_t st);
 cudaError_t launch_vertf(int n, const int* order, const uint8_t* sink_flag, int* vertf, cudaStream_t st);
 cudaError_t launch_cp_reduce(const PassArgs& a, bool from_tlevel, const int* list, int list_len, cudaStream_t st);
 cudaError_t launch_loads(int n, long long P, long long ldp, const uint8_t* part, const int* vert,

@@ -321,14 +321,27 @@ size_t lean_smem_bytes(const LeanPlan& plan, int slice, int warps, int depth, un
     return stage + (size_t)plan.R * (size_t)slice * (plan.wide ? 9 : 5);
 }
 
-// slice = candidates per block: 128, 64, 32 or 16 (4 candidates per lane, 1, 2, 4 or 8 vertices per warp)
-cudaError_t launch_pass_lean(const LeanArgs& a, bool fwd, int slice, int warps, size_t smem, cudaStream_t st)
+// slice = candidates per block (16 ... 128), cpt = candidates per lane (4, 2 or 1): a vertex is served by slice / cpt
+// lanes.  Four candidates per lane amortise a vertex' and an edge's bookkeeping best; fewer shorten the dependent
+// chain of a level when the graph is deep and narrow and the batch too small to fill the machine anyway.
+cudaError_t launch_pass_lean(const LeanArgs& a, bool fwd, int slice, int cpt, int warps, size_t smem, cudaStream_t st)
 {
     if (a.plan.num_chunks <= 0) return cudaSuccess;
-    if (slice == 128) return lean_impl<4, 1>(a, fwd, warps, smem, st);
-    if (slice == 64) return lean_impl<4, 2>(a, fwd, warps, smem, st);
-    if (slice == 32) return lean_impl<4, 4>(a, fwd, warps, smem, st);
-    return lean_impl<4, 8>(a, fwd, warps, smem, st);
+    const int lpv = slice / cpt;   // lanes per vertex
+    if (cpt == 4) {
+        if (lpv == 32) return lean_impl<4, 1>(a, fwd, warps, smem, st);
+        if (lpv == 16) return lean_impl<4, 2>(a, fwd, warps, smem, st);
+        if (lpv == 8) return lean_impl<4, 4>(a, fwd, warps, smem, st);
+        if (lpv == 4) return lean_impl<4, 8>(a, fwd, warps, smem, st);
+    } else if (cpt == 2) {
+        if (lpv == 32) return lean_impl<2, 1>(a, fwd, warps, smem, st);
+        if (lpv == 16) return lean_impl<2, 2>(a, fwd, warps, smem, st);
+        if (lpv == 8) return lean_impl<2, 4>(a, fwd, warps, smem, st);
+    } else if (cpt == 1) {
+        if (lpv == 32) return lean_impl<1, 1>(a, fwd, warps, smem, st);
+        if (lpv == 16) return lean_impl<1, 2>(a, fwd, warps, smem, st);
+    }
+    return cudaErrorInvalidValue;
 }
 
 }  // namespace tfps

@@ -338,190 +338,6 @@ pass_level_kernel(PassArgs a, int pos0, int count)
         relax_vertex<CPT, FWD>(a, s_w, s_rt, global_meta(a.adj, pos0 + i), lc, false, unused);
 }
 
-// ---- level-synchronous tile variant (k <= TABLE_K_MAX) ---------------------------
-// One launch per level.  A block of TILE_WARPS warps takes ONE vertex and
-// TILE_WARPS*32*CPT candidates: the per-edge cost tables are built once per block
-// (warp w builds the table of edge w of the batch) and shared through shared
-// memory, so their cost is spread over the whole candidate tile.
-//
-// Launches are chained with programmatic dependent launch: a block first reads
-// what does not depend on the previous level (adjacency, partition ids) and
-// builds its tables, and only then waits for the previous level's grid before
-// it touches neighbour levels.  Every block executes the wait, so the completion
-// of a level's grid implies the completion of all earlier levels.
-constexpr int TILE_WARPS = 4;
-constexpr int TILE_EB = 4;  // edges per batch = tables resident per block
-
-__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-
-template <int CPT, bool FWD>
-__global__ void __launch_bounds__(TILE_WARPS * 32)
-pass_tile_kernel(PassArgs a, int pos0, int count)
-{
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    long long* s_T = reinterpret_cast<long long*>(smem_raw);  // [TILE_EB][npass*32]
-    grid_launch_dependents();
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int k = a.tab.k;
-    const int tsz = a.tab.npass * 32;
-    const bool live = *a.status == 0;
-    TableCtx tc;
-    tc.s_pair = FWD ? a.tab.pair_f : a.tab.pair_b;
-    tc.s_rt = a.tab.rt_div;
-    tc.s_sel = FWD ? a.tab.sel_f : a.tab.sel_b;
-    tc.T = s_T + (size_t)warp * tsz;   // table slot this warp fills
-    tc.my_cls = a.tab.cls_div[lane];
-    tc.npass = a.tab.npass;
-    tc.use_cls = a.tab.use_cls;
-    tc.ncls_w = a.tab.ncls_w;
-    const long long slice0 = ((long long)blockIdx.x * TILE_WARPS + warp) * 32 * CPT;
-    const LaneCtx<CPT> lc = lane_setup<CPT>(slice0, a.P, lane);
-    const long long ldp = a.ldp;
-    bool waited = false;
-
-    for (int i = blockIdx.y; i < count && live; i += gridDim.y) {
-        // With work items, pos0 indexes the item list: a vertex with many edges is cut into several partial items
-        // (its dependent chain of edge batches would otherwise set the duration of the whole level); partial results
-        // meet in the output row, zeroed beforehand, through 64-bit atomic maxima.
-        VertexMeta vm;
-        bool partial = false;
-        if (a.adj.items) {
-            const int4 it = a.adj.items[pos0 + i];
-            vm = global_meta(a.adj, it.x);
-            vm.e0 = it.y;
-            vm.e1 = it.z;
-            partial = it.w != 0;
-        } else {
-            vm = global_meta(a.adj, pos0 + i);
-        }
-        unsigned pv[IdWords<CPT>::N];
-        load_ids_masked<CPT>(a.part + (long long)vm.v * ldp + lc.jl, lc, pv);
-        long long best[CPT];
-#pragma unroll
-        for (int c = 0; c < CPT; ++c) best[c] = 0;
-
-        for (int b0 = vm.e0; b0 < vm.e1; b0 += TILE_EB) {
-            const int nb = vm.e1 - b0 < TILE_EB ? vm.e1 - b0 : TILE_EB;
-            long long off[TILE_EB];
-            unsigned pu[TILE_EB][IdWords<CPT>::N];
-#pragma unroll
-            for (int q = 0; q < TILE_EB; ++q) {
-                if (q < nb) {
-                    off[q] = (long long)vm.nbr[b0 + q] * ldp + lc.jl;
-                    load_ids_masked<CPT>(a.part + off[q], lc, pu[q]);
-                }
-            }
-            if (b0 != vm.e0) __syncthreads();  // lookups of the previous batch are done
-            if (warp < nb) build_edge_table<FWD>(tc, vm.xw[b0 + warp], FWD ? vm.xnbr[b0 + warp] : vm.xvert, lane);
-            if (!waited) { grid_dependency_wait(); waited = true; }
-            long long lu[TILE_EB][CPT];
-#pragma unroll
-            for (int q = 0; q < TILE_EB; ++q)
-                if (q < nb) load_levels<CPT>(a.lev + off[q], lu[q]);
-            __syncthreads();  // tables of this batch are visible
-#pragma unroll
-            for (int q = 0; q < TILE_EB; ++q) {
-                if (q < nb) {
-                    const long long* T = s_T + (size_t)q * tsz;
-#pragma unroll
-                    for (int c = 0; c < CPT; ++c) {
-                        const long long val = lu[q][c] + T[id_at<CPT>(pu[q], c) * k + id_at<CPT>(pv, c)];
-                        best[c] = val > best[c] ? val : best[c];
-                    }
-                }
-            }
-        }
-        if (!FWD && vm.e0 == vm.e1) {  // sink: blevel = own runtime
-#pragma unroll
-            for (int c = 0; c < CPT; ++c)
-                if (vm.xvert != NUM_ZERO) best[c] = ceil_quot(vm.xvert, tc.s_rt[id_at<CPT>(pv, c)]);
-        }
-        if (!waited) { grid_dependency_wait(); waited = true; }
-        if (partial) {
-#pragma unroll
-            for (int c = 0; c < CPT; ++c)
-                if (c < lc.nvalid) atomicMax(a.lev + (long long)vm.v * ldp + lc.jl + c, best[c]);
-        } else {
-            store_levels<CPT>(a.lev + (long long)vm.v * ldp + lc.jl, best, lc.nvalid);
-        }
-        if (i + (int)gridDim.y < count) __syncthreads();  // tables are reused by the next vertex
-    }
-    if (!waited) grid_dependency_wait();
-}
-
-// ---- level-synchronous variant on precomputed edge values ---------------------------------
-// One launch per level, a warp takes one vertex and 32*CPT candidates.  The cost of an edge comes from the
-// precomputed value array (at most COMB_MAX distinct values per edge): lanes 0..ncomb-1 fetch the edge's
-// values, every candidate picks its own with one shuffle.  No per-edge table, no block barrier.  Launches are
-// chained with programmatic dependent launch exactly as in the tile kernel.
-constexpr int LEVELV_WARPS = 8;
-
-template <int CPT, bool FWD>
-__global__ void __launch_bounds__(LEVELV_WARPS * 32)
-pass_levelv_kernel(PassArgs a, const long long* __restrict__ V, const uint8_t* __restrict__ cls2, int ncomb, int pos0,
-                   int count)
-{
-    __shared__ uint8_t s_cls2[TABLE_K_MAX * TABLE_K_MAX];
-    __shared__ DivConst s_rt[TABLE_K_MAX];
-    grid_launch_dependents();
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int k = a.tab.k;
-    const bool live = *a.status == 0;
-    for (int i = threadIdx.x; i < k * k; i += blockDim.x) s_cls2[i] = cls2[i];
-    for (int i = threadIdx.x; i < k; i += blockDim.x) s_rt[i] = a.tab.rt_div[i];
-    __syncthreads();
-    const long long slice0 = (long long)blockIdx.x * 32 * CPT;
-    const LaneCtx<CPT> lc = lane_setup<CPT>(slice0, a.P, lane);
-    const long long ldp = a.ldp;
-    bool waited = false;
-    constexpr int UNR = 2;
-    for (int i = blockIdx.y * LEVELV_WARPS + warp; i < count && live; i += gridDim.y * LEVELV_WARPS) {
-        const VertexMeta vm = global_meta(a.adj, pos0 + i);
-        unsigned pv[IdWords<CPT>::N];
-        load_ids_masked<CPT>(a.part + (long long)vm.v * ldp + lc.jl, lc, pv);
-        long long best[CPT];
-#pragma unroll
-        for (int c = 0; c < CPT; ++c) best[c] = 0;
-        for (int e = vm.e0; e < vm.e1; e += UNR) {
-            long long off[UNR], vreg[UNR];
-            unsigned pu[UNR][IdWords<CPT>::N];
-#pragma unroll
-            for (int q = 0; q < UNR; ++q) {
-                if (e + q < vm.e1) {
-                    off[q] = (long long)vm.nbr[e + q] * ldp + lc.jl;
-                    vreg[q] = lane < ncomb ? V[(long long)(e + q) * ncomb + lane] : 0;
-                    load_ids_masked<CPT>(a.part + off[q], lc, pu[q]);
-                }
-            }
-            if (!waited) { grid_dependency_wait(); waited = true; }
-            long long lu[UNR][CPT];
-#pragma unroll
-            for (int q = 0; q < UNR; ++q)
-                if (e + q < vm.e1) load_levels<CPT>(a.lev + off[q], lu[q]);
-#pragma unroll
-            for (int q = 0; q < UNR; ++q) {
-                if (e + q < vm.e1) {
-#pragma unroll
-                    for (int c = 0; c < CPT; ++c) {
-                        const unsigned cls = s_cls2[id_at<CPT>(pu[q], c) * k + id_at<CPT>(pv, c)];
-                        const long long val = lu[q][c] + shfl64(vreg[q], (int)cls);
-                        best[c] = val > best[c] ? val : best[c];
-                    }
-                }
-            }
-        }
-        if (!FWD && vm.e0 == vm.e1) {  // sink: blevel = own runtime
-#pragma unroll
-            for (int c = 0; c < CPT; ++c)
-                best[c] = vm.xvert != NUM_ZERO ? ceil_quot(vm.xvert, s_rt[id_at<CPT>(pv, c)]) : 0;
-        }
-        if (!waited) { grid_dependency_wait(); waited = true; }
-        store_levels<CPT>(a.lev + (long long)vm.v * ldp + lc.jl, best, lc.nvalid);
-    }
-    if (!waited) grid_dependency_wait();
-}
-
 // ---- candidate-sliced persistent variant ---------------------------------------------
 // One block owns 32*CPT candidates and walks the whole graph chunk by chunk; a
 // chunk is a run of at most CHUNK_V positions / CHUNK_E edges inside one level
@@ -903,76 +719,6 @@ __global__ void zero_rows_kernel(const int* __restrict__ rows, long long P, long
 }
 
 // lp: level pointers over positions, or over work items when the pass has them
-template <int CPT, bool FWD>
-static cudaError_t tile_impl(const PassArgs& a, const std::vector<long long>& lp, cudaStream_t st)
-{
-    const size_t smem = sizeof(long long) * (size_t)TILE_EB * a.tab.npass * 32;
-    cudaError_t e = allow_smem(pass_tile_kernel<CPT, FWD>, smem);
-    if (e != cudaSuccess) return e;
-    const unsigned gx = cdivu(a.P, TILE_WARPS * 32 * CPT);
-    const int L = a.num_levels;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    for (int step = 0; step < L; ++step) {
-        const int l = FWD ? step : L - 1 - step;
-        const int pos0 = (int)lp[l];
-        const int count = (int)(lp[l + 1] - lp[l]);
-        unsigned gy = (unsigned)count;
-        if (gy > 65535u) gy = 65535u;
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(gx, gy);
-        cfg.blockDim = dim3(TILE_WARPS * 32);
-        cfg.dynamicSmemBytes = smem;
-        cfg.stream = st;
-        cfg.attrs = attr;
-        cfg.numAttrs = step == 0 ? 0 : 1;  // the first level follows ordinary stream order
-        e = cudaLaunchKernelEx(&cfg, pass_tile_kernel<CPT, FWD>, a, pos0, count);
-        if (e != cudaSuccess) return e;
-    }
-    count_launches(L);
-    return cudaGetLastError();
-}
-
-template <int CPT, bool FWD>
-static cudaError_t levelv_impl(const PassArgs& a, const std::vector<long long>& lp, const long long* V, const uint8_t* cls2,
-                               int ncomb, cudaStream_t st)
-{
-    const unsigned gx = cdivu(a.P, 32 * CPT);
-    const int L = a.num_levels;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    for (int step = 0; step < L; ++step) {
-        const int l = FWD ? step : L - 1 - step;
-        const int pos0 = (int)lp[l];
-        const int count = (int)(lp[l + 1] - lp[l]);
-        unsigned gy = cdivu(count, LEVELV_WARPS);
-        if (gy > 65535u) gy = 65535u;
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(gx, gy);
-        cfg.blockDim = dim3(LEVELV_WARPS * 32);
-        cfg.dynamicSmemBytes = 0;
-        cfg.stream = st;
-        cfg.attrs = attr;
-        cfg.numAttrs = step == 0 ? 0 : 1;  // the first level follows ordinary stream order
-        cudaError_t e = cudaLaunchKernelEx(&cfg, pass_levelv_kernel<CPT, FWD>, a, V, cls2, ncomb, pos0, count);
-        if (e != cudaSuccess) return e;
-    }
-    count_launches(L);
-    return cudaGetLastError();
-}
-
-cudaError_t launch_pass_level_values(const PassArgs& a, bool fwd, const std::vector<long long>& lp, const long long* V,
-                                     const uint8_t* cls2, int ncomb, cudaStream_t st)
-{
-    int cpt = a.P >= 4096 ? 4 : (a.P >= 512 ? 2 : 1);
-    if (const char* ov = getenv("TFPS_TILE_CPT")) { const int q = atoi(ov); if (q == 1 || q == 2 || q == 4) cpt = q; }
-    if (cpt == 4) return fwd ? levelv_impl<4, true>(a, lp, V, cls2, ncomb, st) : levelv_impl<4, false>(a, lp, V, cls2, ncomb, st);
-    if (cpt == 2) return fwd ? levelv_impl<2, true>(a, lp, V, cls2, ncomb, st) : levelv_impl<2, false>(a, lp, V, cls2, ncomb, st);
-    return fwd ? levelv_impl<1, true>(a, lp, V, cls2, ncomb, st) : levelv_impl<1, false>(a, lp, V, cls2, ncomb, st);
-}
-
 cudaError_t launch_zero_rows(const int* rows, int count, long long P, long long ldp, long long* lev, cudaStream_t st)
 {
     if (count <= 0 || P <= 0) return cudaSuccess;
@@ -984,26 +730,8 @@ cudaError_t launch_zero_rows(const int* rows, int count, long long P, long long 
     return cudaGetLastError();
 }
 
-cudaError_t launch_pass_level_sync(const PassArgs& a0, bool fwd, const std::vector<long long>& lp0, cudaStream_t st,
-                                   const std::vector<long long>* item_ptr)
+cudaError_t launch_pass_level_sync(const PassArgs& a, bool fwd, const std::vector<long long>& lp, cudaStream_t st)
 {
-    // work items belong to the tile kernel; the other level kernels walk positions
-    PassArgs a = a0;
-    const bool use_items = a.tab.npass > 0 && a.adj.items != nullptr && item_ptr != nullptr;
-    if (!use_items) a.adj.items = nullptr;
-    const std::vector<long long>& lp = use_items ? *item_ptr : lp0;
-    if (a.tab.npass > 0) {  // block-shared cost tables
-        const char* ov = getenv("TFPS_TILE_CPT");  // tuning override
-        if (ov && *ov == '4') return fwd ? tile_impl<4, true>(a, lp, st) : tile_impl<4, false>(a, lp, st);
-        if (ov && *ov == '2') return fwd ? tile_impl<2, true>(a, lp, st) : tile_impl<2, false>(a, lp, st);
-        if (ov && *ov == '1') return fwd ? tile_impl<1, true>(a, lp, st) : tile_impl<1, false>(a, lp, st);
-        const long long tiles4 = (a.P + TILE_WARPS * 32 * 4 - 1) / (TILE_WARPS * 32 * 4);
-        const long long width = a.num_levels > 0 ? a.n / a.num_levels : a.n;
-        if (tiles4 * width >= 2048 || a.P >= 4096)
-            return fwd ? tile_impl<4, true>(a, lp, st) : tile_impl<4, false>(a, lp, st);
-        if (a.P >= 256) return fwd ? tile_impl<2, true>(a, lp, st) : tile_impl<2, false>(a, lp, st);
-        return fwd ? tile_impl<1, true>(a, lp, st) : tile_impl<1, false>(a, lp, st);
-    }
     const int cpt = pick_cpt(a.P);
     if (cpt == 2) return fwd ? level_sync_impl<2, true>(a, lp, st) : level_sync_impl<2, false>(a, lp, st);
     return fwd ? level_sync_impl<1, true>(a, lp, st) : level_sync_impl<1, false>(a, lp, st);

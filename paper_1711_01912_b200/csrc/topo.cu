@@ -326,4 +326,39 @@ cudaError_t launch_default_mem(int n, const long long* out_ptr, const long long*
     return cudaGetLastError();
 }
 
+namespace {
+
+__global__ void pos_of_kernel(int n, const int* __restrict__ order, int* pos_of)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) pos_of[order[i]] = i;
+}
+
+// the longest in-edge in level positions: one thread per position walks its in-edges
+__global__ void maxspan_kernel(int n, const int* __restrict__ pos_of, const int* __restrict__ eptr_f,
+                               const int* __restrict__ nbr_f, int* maxspan)
+{
+    const int p = blockIdx.x * blockDim.x + threadIdx.x;
+    if (p >= n) return;
+    int mx = 0;
+    for (int q = eptr_f[p]; q < eptr_f[p + 1]; ++q) {
+        const int s = p - pos_of[nbr_f[q]];
+        mx = s > mx ? s : mx;
+    }
+    if (mx > 0) atomicMax(maxspan, mx);
+}
+
+}  // namespace
+
+// pos_of[v] = level position of vertex v; *maxspan (zeroed by the caller) = largest pos(v) - pos(u) over all edges u -> v
+cudaError_t launch_positions(int n, const int* order, int* pos_of, const int* nbr_f, const int* eptr_f, int* maxspan,
+                             cudaStream_t st)
+{
+    if (n <= 0) return cudaSuccess;
+    pos_of_kernel<<<cdiv(n, 256), 256, 0, st>>>(n, order, pos_of);
+    maxspan_kernel<<<cdiv(n, 256), 256, 0, st>>>(n, pos_of, eptr_f, nbr_f, maxspan);
+    count_launches(2);
+    return cudaGetLastError();
+}
+
 }  // namespace tfps

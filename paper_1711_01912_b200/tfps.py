@@ -31,7 +31,7 @@ EXPORTS = [
     "tfps_strerror", "tfps_last_error", "tfps_graph_create", "tfps_graph_destroy", "tfps_graph_info",
     "tfps_devices_set", "tfps_topo_levels", "tfps_eval_workspace_bytes", "tfps_eval_batch",
     "tfps_eval_batch_host", "tfps_get_status", "tfps_transpose_u8", "tfps_phase_times", "tfps_kernel_launches",
-    "tfps_eval_cp_noalloc", "tfps_last_pass_kernel",
+    "tfps_eval_cp_noalloc", "tfps_last_pass_kernel", "tfps_probe_gather_bandwidth",
 ]
 
 
@@ -78,6 +78,8 @@ def lib() -> ctypes.CDLL:
     L.tfps_phase_times.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
     L.tfps_kernel_launches.restype = i64
     L.tfps_kernel_launches.argtypes = []
+    L.tfps_probe_gather_bandwidth.restype = ci
+    L.tfps_probe_gather_bandwidth.argtypes = [sz, ci, ctypes.POINTER(ctypes.c_double)]
     L.tfps_last_pass_kernel.restype = ctypes.c_char_p
     L.tfps_last_pass_kernel.argtypes = [vp]
     L.tfps_eval_cp_noalloc.restype = ci
@@ -160,6 +162,13 @@ def tfps_kernel_launches() -> int:
     return int(lib().tfps_kernel_launches())
 
 
+def tfps_probe_gather_bandwidth(working_set_bytes: int, rows_per_warp: int = 4096) -> float:
+    """GB/s at which the current device gathers pseudo-random 1 KiB row segments of a buffer of that size."""
+    out = ctypes.c_double(0.0)
+    _check(lib().tfps_probe_gather_bandwidth(int(working_set_bytes), int(rows_per_warp), ctypes.byref(out)))
+    return float(out.value)
+
+
 NOALLOC_SCRATCH_BYTES = 32 << 20
 
 
@@ -199,9 +208,10 @@ def round_up_ldp(P: int) -> int:
 
 
 class Graph:
-    """Owns a tfps_graph handle built from host numpy CSR arrays."""
+    """Owns a tfps_graph handle built from host numpy CSR arrays (or, with ``device_arrays``, from copies of them
+    placed in device memory first: the library then fetches them itself, ptr_space = TFPS_DEVICE)."""
 
-    def __init__(self, n, in_ptr, in_src, in_t, c, out_ptr=None, out_dst=None, out_t=None, mem=None):
+    def __init__(self, n, in_ptr, in_src, in_t, c, out_ptr=None, out_dst=None, out_t=None, mem=None, device_arrays=False):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("tfps needs a CUDA device; there is no CPU fallback")
@@ -218,10 +228,19 @@ class Graph:
             mem_a = _np(mem, np.int32 if mem_dt == I32 else np.int64)
         self.n = int(n)
         self.m = int(self._keep[1].shape[0])
+        space = HOST
+        if device_arrays:
+            def dev(a):
+                return None if a is None else torch.from_numpy(a).cuda() if a.size else torch.zeros(1, dtype=torch.from_numpy(a).dtype, device="cuda")
+            self._keep = [dev(a) for a in self._keep]
+            outs = [dev(a) for a in outs]
+            mem_a = dev(mem_a)
+            torch.cuda.synchronize()
+            space = DEVICE
         self.handle = tfps_graph_create(self.n, self.m, _addr(self._keep[0]), _addr(self._keep[1]),
                                         _addr(self._keep[2]), _addr(outs[0]), _addr(outs[1]), _addr(outs[2]),
                                         I32 if t_np == np.int32 else I64, _addr(self._keep[3]), _addr(mem_a), mem_dt,
-                                        HOST, _stream())
+                                        space, _stream())
         self._keep = None
         self.k = 0
 

@@ -115,15 +115,34 @@ def test_config2_every_candidate(flags):
     run_and_compare(w.graph, w.devices, w.part_full(), flags)
 
 
-def test_level_kernel_on_precomputed_values(monkeypatch):
-    """The opt-in level-synchronous kernel that reads precomputed edge values (TFPS_LEVEL_VALUES=1)."""
-    monkeypatch.setenv("TFPS_LEVEL_VALUES", "1")
-    w = I.config2()
-    run_and_compare(w.graph, w.devices, w.part_full()[:, :700], 1, pad_fill=255)
-    w = I.config5(layers=12, width=64, P=100)
-    run_and_compare(w.graph, w.devices, w.part_full(), 1, pad_fill=255)
-    w = I.small_random(5, 300, 900, 3, 77)
-    run_and_compare(w.graph, w.devices, w.part_full(), 1, pad_fill=255)
+@pytest.mark.parametrize("device_arrays", [False, True])
+@pytest.mark.parametrize("give_out_edges", [False, True])
+def test_graph_create_spaces_and_transposed_out_edges(device_arrays, give_out_edges):
+    """tfps_graph_create from host arrays and from device arrays (ptr_space = TFPS_DEVICE), with the out-edge CSR
+    given and with all three out-edge arrays NULL (built by transposing the in-edges): same results as the oracle,
+    with and without per-vertex memory, int32 and int64 edge sizes."""
+    from paper_1711_01912_b200 import tfps
+    import oracle
+    torch = _torch()
+    for w in (I.config1(), I.small_random(321, 400, 1500, 5, 70, t_dtype=np.int32, with_mem=False),
+              I.small_random(322, 300, 900, 3, 40, with_mem=True)):
+        g, d = w.graph, w.devices
+        c = I.to_csr(g)
+        outs = (c.out_ptr, c.out_dst, c.out_t) if give_out_edges else (None, None, None)
+        G = tfps.Graph(g.n, c.in_ptr, c.in_src, c.in_t, g.c, outs[0], outs[1], outs[2], g.mem, device_arrays=device_arrays)
+        G.devices_set(d.k, d.s, d.C, d.B, d.scale)
+        part = w.part_full()
+        dpart, P, ldp = padded(part)
+        ref = oracle.eval_batch(oracle_graph(g), d.k, d.s, d.C, d.B, d.scale, part)
+        for flags in VARIANTS:
+            out = G.eval_batch(dpart, P, flags=flags, out={})
+            assert np.array_equal(out["tlevel"].cpu().numpy()[:, :P], ref.tlevel)
+            assert np.array_equal(out["blevel"].cpu().numpy()[:, :P], ref.blevel)
+            assert np.array_equal(out["cp"].cpu().numpy()[:P], ref.cp)
+            assert np.array_equal(out["load"].cpu().numpy()[:, :P], ref.load)
+            assert np.array_equal(out["memload"].cpu().numpy()[:, :P], ref.memload)
+            assert np.array_equal(out["viol"].cpu().numpy().view(np.uint64)[:P], ref.viol)
+        G.close()
 
 
 def test_config1_relabelled():
@@ -353,6 +372,14 @@ def test_error_codes():
     with pytest.raises(tfps.TfpsError) as ei:
         tfps.tfps_eval_batch(G.handle, 16, 16, part.data_ptr(), None, None, cp.data_ptr(), None, None, None, None, 0, 0, 0)
     assert ei.value.code == tfps.ERR_WORKSPACE
+    # pointers the 16-byte vector accesses of the kernels cannot take are refused before anything is launched
+    lev = torch.zeros((5 * 16 + 2,), dtype=torch.int64, device="cuda")
+    for bad in (dict(part=part.data_ptr() + 1), dict(tlevel=lev.data_ptr() + 8), dict(blevel=lev.data_ptr() + 8), dict(cp=cp.data_ptr() + 8)):
+        a = dict(part=part.data_ptr(), tlevel=lev.data_ptr(), blevel=None, cp=cp.data_ptr())
+        a.update(bad)
+        with pytest.raises(tfps.TfpsError) as ei:
+            tfps.tfps_eval_batch(G.handle, 16, 16, a["part"], a["tlevel"], a["blevel"], a["cp"], None, None, None, None, 0, 0, 0)
+        assert ei.value.code == tfps.ERR_INVALID_ARG, bad
     # P == 0: nothing happens
     tfps.tfps_eval_batch(G.handle, 0, 16, part.data_ptr(), None, None, None, None, None, None, None, 0, 0, 0)
     # id >= k is reported through the status word and the context stays usable
@@ -381,7 +408,6 @@ def test_sliced_kernel_shapes(cpt, table, monkeypatch):
     monkeypatch.setenv("TFPS_SLICED_CPT", str(cpt))
     monkeypatch.setenv("TFPS_SLICED_TABLE", str(table))
     monkeypatch.setenv("TFPS_SLICED_WARPS", "4")
-    monkeypatch.setenv("TFPS_WINDOW", "0")
     monkeypatch.setenv("TFPS_LEAN", "0")
     for g, dev, part in _shape_cases(cpt * 2 + table):
         run_and_compare(g, dev, part, 2, pad_fill=255)
@@ -409,31 +435,6 @@ def _shape_cases(seed):
     return cases
 
 
-@pytest.mark.parametrize("level32", [0, 1])
-@pytest.mark.parametrize("win_r", [-1, 160, 0])
-@pytest.mark.parametrize("cpt", [1, 2, 4])
-def test_windowed_kernel_shapes(cpt, win_r, level32, monkeypatch):
-    """The windowed pass with the whole window resident (-1: automatic), with a
-    window too short for many edges (hits and misses mixed) and with no window at
-    all, for every lane width; the cases with many distinct costs or k > 16 fall
-    back to the sliced kernel and must still agree."""
-    monkeypatch.setenv("TFPS_SLICED_CPT", str(cpt))
-    monkeypatch.setenv("TFPS_SLICED_WARPS", "8")
-    monkeypatch.setenv("TFPS_WINDOW", "1")
-    monkeypatch.setenv("TFPS_LEAN", "0")
-    monkeypatch.setenv("TFPS_WINDOW_R", str(win_r))
-    monkeypatch.setenv("TFPS_LEVEL32", str(level32))  # 32-bit levels inside the block when every path fits int32
-    for g, dev, part in _shape_cases(cpt * 2 + 1):
-        run_and_compare(g, dev, part, 2, pad_fill=255)
-    w = I.config2()
-    run_and_compare(w.graph, w.devices, w.part_full()[:, :333], 2, pad_fill=255)
-    w = I.config4()
-    g = w.graph
-    keep = g.dst < 16 * 300  # first 300 layers of the deep narrow graph
-    g2 = I.Graph(n=16 * 300, src=g.src[keep], dst=g.dst[keep], t=g.t[keep], c=g.c[:16 * 300], mem=None, layers=300)
-    run_and_compare(g2, w.devices, w.part_rows(0, 16 * 300)[:, :97], 2, pad_fill=255)
-
-
 def _small_costs(g):
     """Same graph with edge sizes below 50,000, so that every path length fits 32 bits."""
     return I.Graph(n=g.n, src=g.src, dst=g.dst, t=(g.t % 50000).astype(g.t.dtype), c=g.c, mem=g.mem, layers=g.layers)
@@ -446,6 +447,35 @@ def _grouped_devices(k, rng):
     B = np.where(grp[:, None] == grp[None, :], 900, 70).astype(np.int64)
     B[np.triu_indices(k, 1)] += 13
     return I.Devices(k, s, np.full(k, INF, np.int64), B, scale=int(rng.integers(1, 40)))
+
+
+@pytest.mark.parametrize("slice_,cpt", [(16, 1), (16, 2), (16, 4), (32, 1), (32, 2), (64, 2)])
+def test_lean_kernel_candidates_per_lane(slice_, cpt, monkeypatch):
+    """The lean windowed pass with 1, 2 or 4 candidates per lane (a vertex is served by slice / cpt lanes): the deep
+    narrow graph, the wide graph, a random graph with k = 8 and ragged candidate counts."""
+    from paper_1711_01912_b200 import tfps
+    monkeypatch.setenv("TFPS_LEAN_SLICE", str(slice_))
+    monkeypatch.setenv("TFPS_LEAN_CPT", str(cpt))
+    rng = np.random.default_rng(slice_ * 10 + cpt)
+    w = I.config4()
+    g = w.graph
+    keep = g.dst < 16 * 120
+    g4 = I.Graph(n=16 * 120, src=g.src[keep], dst=g.dst[keep], t=g.t[keep], c=g.c[:16 * 120], mem=None, layers=120)
+    cases = [(g4, w.devices, w.part_rows(0, 16 * 120)[:, :83])]
+    w = I.config3()
+    g = w.graph
+    keep = g.dst < 128 * 8
+    g3 = I.Graph(n=128 * 8, src=g.src[keep], dst=g.dst[keep], t=g.t[keep], c=g.c[:128 * 8], mem=None, layers=8)
+    cases.append((g3, w.devices, w.part_rows(0, 128 * 8)[:, :130]))
+    w = I.small_random(9300 + slice_ + cpt, 700, 2500, 8, 77)
+    cases.append((_small_costs(w.graph), _grouped_devices(8, rng), w.part_full()))
+    for g, dev, part in cases:
+        run_and_compare(g, dev, part, 2, pad_fill=255)
+    G = gpu_graph(cases[0][0], cases[0][1])
+    dpart, P, ldp = padded(cases[0][2])
+    G.eval_batch(dpart, P, flags=2)
+    assert tfps.tfps_last_pass_kernel(G.handle) == "pass_lean_kernel"
+    G.close()
 
 
 @pytest.mark.parametrize("depth", [1, 3])
@@ -567,10 +597,10 @@ def test_lean_plan_in_callers_vertex_order(wide, monkeypatch):
 @pytest.mark.parametrize("levrec", [0, 1, 2])
 @pytest.mark.parametrize("split", [1, 3, 8])
 def test_level_kernels_with_partial_items(split, levrec, monkeypatch):
-    """The step-synchronous kernels (0: tile kernel, 1: record pass with one launch per step, 2: persistent record
-    pass) with vertices of many edges cut into partial work items of at most `split` edges: a hub with hundreds of
-    in-edges next to vertices of degree one, the power-law fan-in graph with k = 16, a graph with k = 17 (record pass
-    with the 64-device tables; the tile kernel's family falls back to the per-relaxation division kernel)."""
+    """The step-synchronous kernels (0: per-relaxation division kernel, 1: record pass with one launch per step,
+    2: persistent record pass) with vertices of many edges cut into partial work items of at most `split` edges: a
+    hub with hundreds of in-edges next to vertices of degree one, the power-law fan-in graph with k = 16, a graph
+    with k = 17 (record pass with the 64-device tables)."""
     from paper_1711_01912_b200 import tfps
     monkeypatch.setenv("TFPS_TILE_SPLIT", str(split))
     monkeypatch.setenv("TFPS_LEVREC", "1" if levrec else "0")
@@ -585,7 +615,7 @@ def test_level_kernels_with_partial_items(split, levrec, monkeypatch):
     G = gpu_graph(w.graph, w.devices)
     dpart, P, ldp = padded(w.part_full())
     G.eval_batch(dpart, P, flags=1)
-    assert tfps.tfps_last_pass_kernel(G.handle) == ["pass_tile_kernel", "pass_stepchain_kernel", "pass_steprec_kernel"][levrec]
+    assert tfps.tfps_last_pass_kernel(G.handle) == ["pass_level_kernel", "pass_stepchain_kernel", "pass_steprec_kernel"][levrec]
     G.close()
     w = I.small_random(4242 + split, 500, 3000, 17, 40)
     run_and_compare(w.graph, w.devices, w.part_full(), 1, pad_fill=255)
