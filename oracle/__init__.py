@@ -58,6 +58,8 @@ def _get():
         )
         lib.oracle_eval_constraints.restype = ctypes.c_int
         lib.oracle_eval_constraints.argtypes = [ctypes.c_int64, P, ctypes.c_int64, ctypes.c_int64, P, P, ctypes.c_int64, P, P, P, P]
+        lib.oracle_critical_mask.restype = ctypes.c_int
+        lib.oracle_critical_mask.argtypes = [ctypes.c_int64, P, ctypes.c_int64, P, ctypes.c_int64, ctypes.c_int64, P, ctypes.c_int64]
         _lib = lib
     return _lib
 
@@ -192,3 +194,19 @@ def eval_constraints(part: np.ndarray, pairs, devcons, cols: Optional[Sequence[i
             raise OracleError(rc)
         coll[i], dev[i] = a.value, b.value
     return coll, dev
+
+
+def critical_mask(tlevel: np.ndarray, blevel: np.ndarray, cp: np.ndarray) -> np.ndarray:
+    """mask[v][j] = 1 where vertex v lies on a longest path of candidate j (tlevel + blevel == cp), from the
+    [n][q] level matrices and the [q] critical-path lengths of an OracleBatch."""
+    lib = _get()
+    tl = _arr(tlevel, np.int64)
+    bl = _arr(blevel, np.int64)
+    n, q = tl.shape
+    mask = np.zeros((n, q), np.uint8)
+    for j in range(q):
+        rc = lib.oracle_critical_mask(n, ctypes.c_void_p(tl[:, j].ctypes.data), q, ctypes.c_void_p(bl[:, j].ctypes.data), q,
+                                      int(cp[j]), ctypes.c_void_p(mask[:, j].ctypes.data), q)
+        if rc:
+            raise OracleError(rc)
+    return mask

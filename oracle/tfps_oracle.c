@@ -275,3 +275,22 @@ int oracle_eval_constraints(int64_t n, const uint8_t *p, int64_t pstride,
     *dev_viol = dv;
     return ORACLE_OK;
 }
+
+/*
+ * Critical vertices of one evaluated candidate (Section 3.2: the critical path is the longest path from a source to
+ * a sink): vertex v lies on a longest path exactly when the longest path into it plus the longest path out of it
+ * spans the whole critical-path length, tlevel(v) + blevel(v) = CP (tlevel excludes v's own runtime, blevel includes
+ * it, so a vertex is counted once).  mask[v] = 1 for those vertices, else 0; strides in elements.
+ * Pins: tests/test_oracle_constraints.py (the critical sets of the worked DAGs, a chain, properties).
+ */
+int oracle_critical_mask(int64_t n, const int64_t *tlevel, int64_t tstride, const int64_t *blevel, int64_t bstride,
+                         int64_t cp, uint8_t *mask, int64_t mstride)
+{
+    if (n < 0 || !tlevel || !blevel || !mask) return ORACLE_BAD_ARG;
+    for (int64_t v = 0; v < n; ++v) {
+        i128 total = (i128)tlevel[v * tstride] + (i128)blevel[v * bstride];
+        if (!fits(total)) return ORACLE_OVERFLOW;
+        mask[v * mstride] = (int64_t)total == cp ? 1 : 0;
+    }
+    return ORACLE_OK;
+}

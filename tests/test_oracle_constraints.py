@@ -1,11 +1,14 @@
 """Pins of the oracle's placement-constraint check (collocation constraints, Eq. 3; device constraints, Eq. 4):
 a worked example, closed forms on the partition p(v) = v mod k, and invariants that a dropped term, a swapped
-operand or an off-by-one in the indexing would break."""
+operand or an off-by-one in the indexing would break; and of its critical-vertex mask (Section 3.2): the critical
+sets of the worked DAGs, derived by hand from their edge lists, a chain, and path properties."""
 from __future__ import annotations
 
 import numpy as np
 
 import oracle
+from helpers import graph_from_edges, load_golden, oracle_graph
+from paper_1711_01912_b200 import inputs as I
 
 
 def _col(p):
@@ -74,3 +77,53 @@ def test_invariants_on_random_inputs():
     # selected columns
     c4, d4 = oracle.eval_constraints(part, pairs, devs, cols=[4, 0, 24])
     assert c4.tolist() == coll[[4, 0, 24]].tolist() and d4.tolist() == dev[[4, 0, 24]].tolist()
+
+
+# ---------------------------------------------------------------------------------------- critical vertices
+def test_critical_sets_of_the_worked_dags():
+    """Longest paths found by hand from the edge lists and the costs of the worked examples:
+    diamond 0->1, 0->2, 1->3, 2->3 with p = [0,1,0,1]: 0->2->3 (16 + 0 + 24 + 2 + 2 = 44), so {0, 2, 3};
+    everything on the fast device: 0->1->3 (4 + 8 + 2 = 14), so {0, 1, 3};
+    two-sink DAG: the direct edge 0->5 (30 + 75 + 12 = 117), so {0, 5}."""
+    gd = load_golden("w1_diamond.json")
+    og = oracle_graph(graph_from_edges(gd["n"], gd["edges"], gd["c"]))
+    want = {0: {0, 2, 3}, 1: {0, 1, 3}, 2: {0, 2, 3}}
+    for i, cs in enumerate(gd["cases"]):
+        part = np.asarray(cs["p"], np.uint8).reshape(-1, 1)
+        r = oracle.eval_batch(og, gd["k"], gd["s"], np.full(gd["k"], np.iinfo(np.int64).max), np.asarray(cs["B"]), gd["S"], part)
+        mask = oracle.critical_mask(r.tlevel, r.blevel, r.cp)
+        assert set(np.nonzero(mask[:, 0])[0].tolist()) == want[i], (i, mask[:, 0])
+    gd = load_golden("w2_two_sinks.json")
+    og = oracle_graph(graph_from_edges(gd["n"], gd["edges"], gd["c"]))
+    cs = gd["cases"][0]
+    part = np.asarray(cs["p"], np.uint8).reshape(-1, 1)
+    r = oracle.eval_batch(og, gd["k"], gd["s"], np.full(gd["k"], np.iinfo(np.int64).max), np.asarray(cs["B"]), gd["S"], part)
+    mask = oracle.critical_mask(r.tlevel, r.blevel, r.cp)
+    assert set(np.nonzero(mask[:, 0])[0].tolist()) == {0, 5}
+
+
+def test_critical_mask_properties():
+    # a chain: every vertex is critical under every partition
+    n = 30
+    g = graph_from_edges(n, [(i, i + 1, 1000 + i) for i in range(n - 1)], np.arange(1, n + 1))
+    rng = np.random.default_rng(3)
+    part = rng.integers(0, 3, size=(n, 9), dtype=np.uint8)
+    s, B = [1, 2, 5], np.array([[0, 7, 9], [3, 0, 11], [5, 2, 0]])
+    r = oracle.eval_batch(oracle_graph(g), 3, s, np.full(3, np.iinfo(np.int64).max), B, 6, part)
+    assert oracle.critical_mask(r.tlevel, r.blevel, r.cp).all()
+    # random layered graph: the critical vertices contain a source and a sink, every critical vertex that is not a sink
+    # has a critical successor, and no vertex exceeds the critical-path length
+    w = I.small_random(55, 120, 400, 4, 12)
+    og = oracle_graph(w.graph)
+    d = w.devices
+    part = w.part_full()
+    r = oracle.eval_batch(og, d.k, d.s, d.C, d.B, d.scale, part)
+    mask = oracle.critical_mask(r.tlevel, r.blevel, r.cp)
+    assert (r.tlevel + r.blevel <= r.cp[None, :]).all()
+    c = I.to_csr(w.graph)
+    for j in range(part.shape[1]):
+        crit = np.nonzero(mask[:, j])[0]
+        assert any(c.in_ptr[v] == c.in_ptr[v + 1] for v in crit) and any(c.out_ptr[v] == c.out_ptr[v + 1] for v in crit)
+        for v in crit:
+            succ = c.out_dst[c.out_ptr[v]:c.out_ptr[v + 1]]
+            assert len(succ) == 0 or mask[succ, j].any()
