@@ -273,6 +273,39 @@ int tfps_probe_gather_bandwidth(size_t working_set_bytes, int rows_per_warp, dou
 int tfps_eval_cp_noalloc(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, int64_t* cp,
                          int flags, void* stream);
 
+/*
+ * Placement constraints (Section 2).  tfps_constraints_set stores the lists with
+ * the handle (host arrays, copied; an earlier set is replaced; synchronous):
+ *   pair_a[npairs], pair_b[npairs]      collocation constraints (Eq. 3): vertices pair_a[i] and
+ *                                       pair_b[i] must be placed on the same device
+ *   dc_vertex[ndev], dc_device[ndev]    device constraints (Eq. 4): vertex dc_vertex[i] must be
+ *                                       placed on device dc_device[i] (0 .. TFPS_K_MAX - 1)
+ * Every listed pair is one requirement; a vertex index outside 0..n-1 gives
+ * TFPS_ERR_INVALID_ARG.  tfps_eval_constraints counts, for each of the P candidates
+ * of `part` (dev uint8 [n][ldp], 16-byte aligned), the requirements that do not hold:
+ *   coll_viol    dev int32 [P] or NULL: violated collocation pairs
+ *   dev_viol     dev int32 [P] or NULL: violated device constraints
+ * Asynchronous on `stream`; needs neither the device tables nor the topological
+ * levels.  With empty lists the outputs are zero.
+ */
+int tfps_constraints_set(tfps_graph* g, int64_t npairs, const int32_t* pair_a, const int32_t* pair_b,
+                         int64_t ndev, const int32_t* dc_vertex, const int32_t* dc_device);
+int tfps_eval_constraints(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part,
+                          int32_t* coll_viol, int32_t* dev_viol, void* stream);
+
+/*
+ * Critical vertices of evaluated candidates (Section 3.2: the critical path is the
+ * longest path from a source to a sink).  mask[v*ldp+j] = 1 where vertex v lies on
+ * a longest path of candidate j, i.e. tlevel + blevel == cp, else 0.
+ *   tlevel, blevel   dev int64 [n][ldp] as written by tfps_eval_batch
+ *   cp               dev int64 [P]
+ *   mask             dev uint8 [n][ldp]; padding columns are not written
+ * All four 16-byte aligned, ldp a multiple of 16; TFPS_ERR_INVALID_ARG otherwise
+ * (nothing is launched).  Asynchronous on `stream`; needs no graph handle.
+ */
+int tfps_critical_mask(int64_t n, int64_t P, int64_t ldp, const int64_t* tlevel, const int64_t* blevel,
+                       const int64_t* cp, uint8_t* mask, void* stream);
+
 /* Synchronise `stream`, return the sticky device-side status of the handle and clear it. */
 int tfps_get_status(tfps_graph* g, void* stream);
 

@@ -171,6 +171,9 @@ struct tfps_graph {
     bool id_topo = false;      // the caller's vertex numbering is a topological order ...
     int span_id = 0;           // ... whose longest edge spans this many vertices
     DBuf status;
+    // placement constraints (tfps_constraints_set)
+    DBuf cons_a, cons_b, cons_v, cons_d;
+    int cons_pairs = 0, cons_dev = 0;
     // scratch owned by the handle
     DBuf scr_memload;
     DBuf st_part, st_lev, st_lev2, st_cp, st_load, st_mem, st_viol;
@@ -793,26 +796,28 @@ int build_levrec(tfps_graph* g, int k, const int32_t* s, const int64_t* B, long 
         for (int sidx = 0; sidx < nsteps; ++sidx) {
             // forward: steps in ascending order; backward: level steps in descending order (caller-order steps are built descending)
             const int src = (dir == 1 && !use_id) ? nsteps - 1 - sidx : sidx;
-            step_ptr[sidx] = (int)(items.size() / 4);
+            step_ptr[sidx] = (int)(items.size() / 8);
             idx.clear();
             for (int q = sp[src]; q < sp[src + 1]; ++q) idx.push_back(use_id ? vs_id[(size_t)q] : q);
             std::stable_sort(idx.begin(), idx.end(), [&](int x, int y) { return ep[x + 1] - ep[x] > ep[y + 1] - ep[y]; });
+            auto push_item = [&](int p, bool partial, int e0, int e1) {   // descriptor, then the neighbours of its first four edges
+                items.push_back(order[p] | (partial ? (int)0x80000000u : 0)); items.push_back((int)roff[p]); items.push_back(e0); items.push_back(e1);
+                for (int q = 0; q < 4; ++q) items.push_back(e0 + q < e1 ? nb[(size_t)ep[p] + e0 + q] : 0);
+            };
             for (int p : idx) {
                 const int d = ep[p + 1] - ep[p];
                 if (d > T) {
                     heavy.push_back(order[p]);
-                    for (int e = 0; e < d; e += T) {
-                        items.push_back(order[p] | (int)0x80000000u); items.push_back((int)roff[p]); items.push_back(e); items.push_back(std::min(d, e + T));
-                    }
+                    for (int e = 0; e < d; e += T) push_item(p, true, e, std::min(d, e + T));
                     item_edges = std::max(item_edges, T);
                 } else {
-                    items.push_back(order[p]); items.push_back((int)roff[p]); items.push_back(0); items.push_back(d);
+                    push_item(p, false, 0, d);
                     item_edges = std::max(item_edges, d);
                 }
             }
-            max_items = std::max(max_items, (int)(items.size() / 4) - step_ptr[sidx]);
+            max_items = std::max(max_items, (int)(items.size() / 8) - step_ptr[sidx]);
         }
-        step_ptr[nsteps] = (int)(items.size() / 4);
+        step_ptr[nsteps] = (int)(items.size() / 8);
         std::vector<unsigned char> blob(total * 16, 0);
         for (int p = 0; p < n; ++p) {
             unsigned char* r = blob.data() + (size_t)roff[p] * 16;
@@ -1555,6 +1560,65 @@ int tfps_eval_cp_noalloc(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* p
     CUDA_TRY(noalloc_scratch_address(g->device, &scratch));   // cached by tfps_devices_set on this device
     return tfps_eval_batch(g, P, ldp, part, nullptr, nullptr, cp, nullptr, nullptr, nullptr, scratch,
                            TFPS_NOALLOC_SCRATCH_BYTES, flags & ~TFPS_EVAL_PROFILE, stream);
+}
+
+int tfps_constraints_set(tfps_graph* g, int64_t npairs, const int32_t* pair_a, const int32_t* pair_b,
+                         int64_t ndev, const int32_t* dc_vertex, const int32_t* dc_device)
+{
+    if (!g) return fail(TFPS_ERR_INVALID_ARG, "graph is NULL");
+    if (npairs < 0 || ndev < 0 || npairs > INT32_MAX || ndev > INT32_MAX) return fail(TFPS_ERR_INVALID_ARG, "bad list length");
+    if ((npairs > 0 && (!pair_a || !pair_b)) || (ndev > 0 && (!dc_vertex || !dc_device)))
+        return fail(TFPS_ERR_INVALID_ARG, "a non-empty list needs both of its arrays");
+    for (int64_t i = 0; i < npairs; ++i)
+        if (pair_a[i] < 0 || pair_a[i] >= g->n || pair_b[i] < 0 || pair_b[i] >= g->n)
+            return fail(TFPS_ERR_INVALID_ARG, "collocation pair %lld names a vertex outside 0..n-1", (long long)i);
+    for (int64_t i = 0; i < ndev; ++i)
+        if (dc_vertex[i] < 0 || dc_vertex[i] >= g->n || dc_device[i] < 0 || dc_device[i] >= (int)TFPS_K_MAX)
+            return fail(TFPS_ERR_INVALID_ARG, "device constraint %lld names a vertex outside 0..n-1 or a device outside 0..%d",
+                        (long long)i, (int)TFPS_K_MAX - 1);
+    DeviceGuard guard(g->device);
+    if (!guard.ok) return fail(TFPS_ERR_CUDA, "cannot select the handle's device");
+    cudaStream_t st = 0;
+    g->cons_pairs = g->cons_dev = 0;
+    TFPS_TRY(upload(g->cons_a, std::vector<int>(pair_a, pair_a + npairs), st));
+    TFPS_TRY(upload(g->cons_b, std::vector<int>(pair_b, pair_b + npairs), st));
+    TFPS_TRY(upload(g->cons_v, std::vector<int>(dc_vertex, dc_vertex + ndev), st));
+    TFPS_TRY(upload(g->cons_d, std::vector<int>(dc_device, dc_device + ndev), st));
+    CUDA_TRY(cudaStreamSynchronize(st));
+    g->cons_pairs = (int)npairs;
+    g->cons_dev = (int)ndev;
+    return TFPS_OK;
+}
+
+int tfps_eval_constraints(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, int32_t* coll_viol, int32_t* dev_viol,
+                          void* stream)
+{
+    if (!g) return fail(TFPS_ERR_INVALID_ARG, "graph is NULL");
+    if (P < 0 || ldp < P || (ldp % 16) != 0) return fail(TFPS_ERR_INVALID_ARG, "need 0 <= P <= ldp and ldp %% 16 == 0");
+    if (P == 0 || g->n == 0 || (!coll_viol && !dev_viol)) return TFPS_OK;
+    if (!part) return fail(TFPS_ERR_INVALID_ARG, "part is NULL");
+    if (P > ((int64_t)1 << 31)) return fail(TFPS_ERR_UNSUPPORTED, "P above 2^31");
+    if (((uintptr_t)part & 15u) != 0 || ((uintptr_t)coll_viol & 3u) != 0 || ((uintptr_t)dev_viol & 3u) != 0)
+        return fail(TFPS_ERR_INVALID_ARG, "part must be 16-byte aligned, the outputs 4-byte aligned");
+    DeviceGuard guard(g->device);
+    if (!guard.ok) return fail(TFPS_ERR_CUDA, "cannot select the handle's device");
+    CUDA_TRY(launch_constraints(P, ldp, part, g->cons_pairs, g->cons_a.as<int>(), g->cons_b.as<int>(), g->cons_dev,
+                                g->cons_v.as<int>(), g->cons_d.as<int>(), coll_viol, dev_viol, g->status.as<int>(),
+                                (cudaStream_t)stream));
+    return TFPS_OK;
+}
+
+int tfps_critical_mask(int64_t n, int64_t P, int64_t ldp, const int64_t* tlevel, const int64_t* blevel, const int64_t* cp,
+                       uint8_t* mask, void* stream)
+{
+    if (n < 0 || P < 0 || ldp < P || (ldp % 16) != 0) return fail(TFPS_ERR_INVALID_ARG, "need n >= 0, 0 <= P <= ldp and ldp %% 16 == 0");
+    if (n == 0 || P == 0) return TFPS_OK;
+    if (!tlevel || !blevel || !cp || !mask) return fail(TFPS_ERR_INVALID_ARG, "tlevel, blevel, cp and mask are required");
+    if ((((uintptr_t)tlevel | (uintptr_t)blevel | (uintptr_t)mask | (uintptr_t)cp) & 15u) != 0)
+        return fail(TFPS_ERR_INVALID_ARG, "tlevel, blevel, cp and mask must be 16-byte aligned");
+    CUDA_TRY(launch_critical_mask(n, P, ldp, (const long long*)tlevel, (const long long*)blevel, (const long long*)cp, mask,
+                                  (cudaStream_t)stream));
+    return TFPS_OK;
 }
 
 int tfps_get_status(tfps_graph* g, void* stream)

@@ -231,6 +231,11 @@ cudaError_t launch_validate(long long n, long long P, long long ldp, const uint8
                             int sm_count, cudaStream_t st);
 cudaError_t launch_viol(long long P, long long ldp, int k, const long long* memload, const long long* cap,
                         unsigned long long* viol, const int* status, cudaStream_t st);
+cudaError_t launch_constraints(long long P, long long ldp, const uint8_t* part, int npairs, const int* pair_a, const int* pair_b,
+                               int ndev, const int* dc_v, const int* dc_d, int* coll_viol, int* dev_viol, const int* status,
+                               cudaStream_t st);
+cudaError_t launch_critical_mask(long long n, long long P, long long ldp, const long long* tlevel, const long long* blevel,
+                                 const long long* cp, uint8_t* mask, cudaStream_t st);
 cudaError_t launch_transpose_u8(const uint8_t* src, uint8_t* dst, long long P, long long n, long long ldp, cudaStream_t st);
 
 }  // namespace tfps

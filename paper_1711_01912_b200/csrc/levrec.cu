@@ -35,7 +35,8 @@ namespace {
 //            neighbour's runtime on such a device; RTU form (too many combinations): comb = class, V = transfer
 //            time, and rtu[d] = the neighbour's runtime on device d is added separately.
 // cls[pu * KP + pv] = comb of a neighbour on device pu and a vertex on device pv.
-// item (int4): {vertex | partial << 31, record offset / 16, first edge within the record, end edge}
+// item (two int4): {vertex | partial << 31, record offset / 16, first edge within the record, end edge} and the
+// neighbours of the item's first four edges (the chained kernel starts their loads before the record has arrived)
 //
 // A lane holds 2 * CG candidates of its warp's tile (tile width TW = 64 * CG): columns {2 * lane, 2 * lane + 1} of
 // each of the CG 64-column groups, so that every 16-byte level access of a warp is one contiguous 512-byte access.
@@ -212,7 +213,7 @@ pass_steprec_kernel(const __grid_constant__ LevRecArgs a)
         int4 dA = make_int4(0, 0, 0, -1);
         auto front_fetch = [&]() {
             if (f_step < num_steps) {
-                dA = __ldg(a.items + item_of(f_i0, f_j));
+                dA = __ldg(a.items + 2 * item_of(f_i0, f_j));
                 ++f_j;
                 f_settle();
             } else {
@@ -456,7 +457,7 @@ cudaError_t steprec_shape(const LevRecArgs& a, int sm_count, cudaStream_t st)
 
 // ---- the same pass as one launch per step --------------------------------------------------------------------------
 // For wide batches, where a step has enough blocks to fill the machine: a block takes ONE work item and CHAIN_WARPS *
-// 128 candidates (4 contiguous candidates per lane), stages the item's record in shared memory and relaxes its edges
+// 128 candidates (4 candidates per lane), stages the item's record in shared memory and relaxes its edges
 // with plain (L1-allocating) loads, so that rows many items of a step share -- the rows of hub vertices -- are served
 // by L1.  The launches of a pass are chained with programmatic dependent launch: a block reads what does not depend
 // on the previous step (item, record, own ids) before it waits for it.
@@ -474,6 +475,8 @@ pass_stepchain_kernel(const __grid_constant__ LevRecArgs a, int item0, int count
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const bool live = *a.status == 0;
     for (int i = tid; i < KP * KP / 4; i += CHAIN_WARPS * 32) reinterpret_cast<unsigned*>(s_cls)[i] = __ldg(reinterpret_cast<const unsigned*>(a.cls) + i);
+    // a lane's four candidates are contiguous (one 32-bit id load, two 16-byte level loads whose second half is served
+    // by L1; splitting a lane's candidates so that every load is contiguous across the warp measured the same)
     const long long j0 = ((long long)blockIdx.x * CHAIN_WARPS + warp) * 128 + lane * 4;
     const long long rem = a.P - j0;
     const int nvalid = rem >= 4 ? 4 : (rem > 0 ? (int)rem : 0);
@@ -483,12 +486,25 @@ pass_stepchain_kernel(const __grid_constant__ LevRecArgs a, int item0, int count
     bool waited = false;
 
     for (int i = blockIdx.y; i < count && live; i += gridDim.y) {
-        const int4 it = __ldg(a.items + item0 + i);
+        const int4 it = __ldg(a.items + 2 * (item0 + i));
+        const int4 nb4 = __ldg(a.items + 2 * (item0 + i) + 1);   // neighbours of the item's first four edges
         const int deg = it.w - it.z;
         const int v = it.x & 0x7fffffff;
         const unsigned char* rec = a.blob + 16ll * (unsigned)it.y;
-        // own ids: requested before the record arrives
+        // own ids and the ids of the first neighbours: requested before the record arrives
         const unsigned ids = __ldg(reinterpret_cast<const unsigned*>(a.part + (long long)v * ldp + jl)) & IDMASK;
+        long long off[EB];
+        unsigned pu[EB];
+        {
+            const int nbv[4] = {nb4.x, nb4.y, nb4.z, nb4.w};
+#pragma unroll
+            for (int q = 0; q < EB; ++q) {
+                if (q < deg) {
+                    off[q] = (long long)nbv[q] * ldp + jl;
+                    pu[q] = __ldg(reinterpret_cast<const unsigned*>(a.part + off[q])) & IDMASK;
+                }
+            }
+        }
         if (i != (int)blockIdx.y) __syncthreads();   // the previous item's record is no longer read
         for (int q = tid; q < HDR / 16; q += CHAIN_WARPS * 32) reinterpret_cast<uint4*>(s_rec)[q] = __ldg(reinterpret_cast<const uint4*>(rec) + q);
         {
@@ -502,11 +518,9 @@ pass_stepchain_kernel(const __grid_constant__ LevRecArgs a, int item0, int count
         long long best[4] = {0, 0, 0, 0};
         for (int b0 = 0; b0 < deg; b0 += EB) {
             const int nb = deg - b0 < EB ? deg - b0 : EB;
-            long long off[EB];
-            unsigned pu[EB];
 #pragma unroll
             for (int q = 0; q < EB; ++q) {
-                if (q < nb) {
+                if (b0 > 0 && q < nb) {
                     off[q] = (long long)*reinterpret_cast<const int*>(edges + (size_t)(b0 + q) * estride) * ldp + jl;
                     pu[q] = __ldg(reinterpret_cast<const unsigned*>(a.part + off[q])) & IDMASK;
                 }
@@ -559,11 +573,9 @@ pass_stepchain_kernel(const __grid_constant__ LevRecArgs a, int item0, int count
     if (!waited) asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
-template <bool FWD, bool RTU, int KP>
+template <bool FWD, bool RTU, int KP, int EB, int MINB>
 cudaError_t stepchain_launch(const LevRecArgs& a, const std::vector<int>& sp, cudaStream_t st)
 {
-    // forward (and the RTU form) two edges in flight and 32 resident warps per SM, backward one edge and 48 warps
-    constexpr int EB = FWD ? 2 : 1, MINB = FWD ? 8 : 12;
     auto kernel = pass_stepchain_kernel<FWD, RTU, KP, EB, MINB>;
     const size_t smem = (size_t)a.rec_max;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -604,9 +616,12 @@ cudaError_t launch_pass_steprec(const LevRecArgs& a, bool fwd, int sm_count, cud
 cudaError_t launch_pass_stepchain(const LevRecArgs& a, bool fwd, const std::vector<int>& step_ptr_host, cudaStream_t st)
 {
     if (a.num_steps <= 0) return cudaSuccess;
-    if (!fwd) return a.kp == 16 ? stepchain_launch<false, false, 16>(a, step_ptr_host, st) : stepchain_launch<false, false, 64>(a, step_ptr_host, st);
-    if (a.rtu) return a.kp == 16 ? stepchain_launch<true, true, 16>(a, step_ptr_host, st) : stepchain_launch<true, true, 64>(a, step_ptr_host, st);
-    return a.kp == 16 ? stepchain_launch<true, false, 16>(a, step_ptr_host, st) : stepchain_launch<true, false, 64>(a, step_ptr_host, st);
+    // edges in flight per thread and resident blocks per SM: forward two edges and 32 warps, backward one edge and 48
+    // (config 5, P = 4,096: 27.3 / 21.3 ms; forward with 40 warps 31.6, with four edges and 24 warps 36.9; backward
+    // with 40 warps 21.0, with two edges and 32 warps 24.2)
+    if (!fwd) return a.kp == 16 ? stepchain_launch<false, false, 16, 1, 12>(a, step_ptr_host, st) : stepchain_launch<false, false, 64, 1, 10>(a, step_ptr_host, st);
+    if (a.rtu) return a.kp == 16 ? stepchain_launch<true, true, 16, 2, 8>(a, step_ptr_host, st) : stepchain_launch<true, true, 64, 2, 8>(a, step_ptr_host, st);
+    return a.kp == 16 ? stepchain_launch<true, false, 16, 2, 8>(a, step_ptr_host, st) : stepchain_launch<true, false, 64, 2, 8>(a, step_ptr_host, st);
 }
 
 }  // namespace tfps

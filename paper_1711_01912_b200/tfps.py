@@ -31,7 +31,7 @@ EXPORTS = [
     "tfps_strerror", "tfps_last_error", "tfps_graph_create", "tfps_graph_destroy", "tfps_graph_info",
     "tfps_devices_set", "tfps_topo_levels", "tfps_eval_workspace_bytes", "tfps_eval_batch",
     "tfps_eval_batch_host", "tfps_get_status", "tfps_transpose_u8", "tfps_phase_times", "tfps_kernel_launches",
-    "tfps_eval_cp_noalloc", "tfps_last_pass_kernel", "tfps_probe_gather_bandwidth",
+    "tfps_eval_cp_noalloc", "tfps_last_pass_kernel", "tfps_probe_gather_bandwidth", "tfps_constraints_set", "tfps_eval_constraints", "tfps_critical_mask",
 ]
 
 
@@ -78,6 +78,12 @@ def lib() -> ctypes.CDLL:
     L.tfps_phase_times.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
     L.tfps_kernel_launches.restype = i64
     L.tfps_kernel_launches.argtypes = []
+    L.tfps_constraints_set.restype = ci
+    L.tfps_constraints_set.argtypes = [vp, i64, vp, vp, i64, vp, vp]
+    L.tfps_eval_constraints.restype = ci
+    L.tfps_eval_constraints.argtypes = [vp, i64, i64, vp, vp, vp, vp]
+    L.tfps_critical_mask.restype = ci
+    L.tfps_critical_mask.argtypes = [i64, i64, i64, vp, vp, vp, vp, vp]
     L.tfps_probe_gather_bandwidth.restype = ci
     L.tfps_probe_gather_bandwidth.argtypes = [sz, ci, ctypes.POINTER(ctypes.c_double)]
     L.tfps_last_pass_kernel.restype = ctypes.c_char_p
@@ -160,6 +166,18 @@ def tfps_last_pass_kernel(g) -> str:
 
 def tfps_kernel_launches() -> int:
     return int(lib().tfps_kernel_launches())
+
+
+def tfps_constraints_set(g, npairs, pair_a, pair_b, ndev, dc_vertex, dc_device) -> None:
+    _check(lib().tfps_constraints_set(g, npairs, pair_a, pair_b, ndev, dc_vertex, dc_device))
+
+
+def tfps_eval_constraints(g, P, ldp, part, coll_viol, dev_viol, stream) -> None:
+    _check(lib().tfps_eval_constraints(g, P, ldp, part, coll_viol, dev_viol, stream))
+
+
+def tfps_critical_mask(n, P, ldp, tlevel, blevel, cp, mask, stream) -> None:
+    _check(lib().tfps_critical_mask(n, P, ldp, tlevel, blevel, cp, mask, stream))
 
 
 def tfps_probe_gather_bandwidth(working_set_bytes: int, rows_per_warp: int = 4096) -> float:
@@ -322,8 +340,36 @@ class Graph:
                 res[name] = a
         return res
 
+    def constraints_set(self, pairs, devcons):
+        """pairs: [npairs][2] vertices that must share a device (Eq. 3); devcons: [ndev][2] (vertex, device) (Eq. 4)."""
+        pairs = _np(pairs, np.int32).reshape(-1, 2)
+        devcons = _np(devcons, np.int32).reshape(-1, 2)
+        pa, pb = np.ascontiguousarray(pairs[:, 0]), np.ascontiguousarray(pairs[:, 1])
+        dv, dd = np.ascontiguousarray(devcons[:, 0]), np.ascontiguousarray(devcons[:, 1])
+        tfps_constraints_set(self.handle, pairs.shape[0], _addr(pa), _addr(pb), devcons.shape[0], _addr(dv), _addr(dd))
+
+    def eval_constraints(self, part, P=None):
+        """Violated collocation pairs and device constraints per candidate: two int32 CUDA tensors [P]."""
+        import torch
+        n, ldp = part.shape
+        P = ldp if P is None else int(P)
+        coll = torch.empty(max(P, 1), dtype=torch.int32, device=part.device)
+        dev = torch.empty(max(P, 1), dtype=torch.int32, device=part.device)
+        tfps_eval_constraints(self.handle, P, ldp, _addr(part), _addr(coll), _addr(dev), _stream())
+        return coll[:P], dev[:P]
+
     def status(self):
         tfps_get_status(self.handle, _stream())
+
+
+def critical_mask(out: Dict, P: int):
+    """uint8 CUDA tensor [n][ldp]: 1 where a vertex lies on a longest path of the candidate (from eval_batch outputs)."""
+    import torch
+    tl, bl, cp = out["tlevel"], out["blevel"], out["cp"]
+    n, ldp = tl.shape
+    mask = torch.zeros((n, ldp), dtype=torch.uint8, device=tl.device)
+    tfps_critical_mask(n, int(P), ldp, _addr(tl), _addr(bl), _addr(cp), _addr(mask), _stream())
+    return mask
 
 
 def transpose_u8(src, ldp: Optional[int] = None):
