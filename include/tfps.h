@@ -94,6 +94,8 @@ const char* tfps_last_error(void);
  *   TFPS_STEP_ORDER=1|2                            steps = topological levels | runs of the caller's numbering
  *   TFPS_STEP_PERSISTENT=1, TFPS_STEP_GROUPS, TFPS_STEP_TILES, TFPS_STEP_RUN, TFPS_STEP_SHAPE, TFPS_STEP_BLOCKS
  *                                                  persistent record pass and its shape
+ *   TFPS_STEP_FLOW=1                               dataflow record pass (ready bits per vertex and tile of 128
+ *                                                  candidates instead of grid-wide steps; k <= 16, P <= 4096)
  *   TFPS_WAIT_LIMIT                                polls before a device-side wait gives up (default 2^20;
  *                                                  0 makes every wait run out at once: TFPS_ERR_TIMEOUT)
  */
@@ -220,6 +222,8 @@ int tfps_phase_times(tfps_graph* g, float ms[3]);
  *   "pass_sliced_kernel"     candidate-sliced without a window (neighbours through L2)
  *   "pass_stepchain_kernel"  step-synchronous on vertex records, one chained launch per step (k <= 64)
  *   "pass_steprec_kernel"    the same as one persistent cooperative launch with bounded barriers (opt-in)
+ *   "pass_flow_kernel"       the same records as one persistent launch without steps: an item waits (bounded) for the
+ *                            ready bits of exactly the rows it reads (opt-in)
  *   "pass_level_kernel"      step-synchronous with a division per relaxation (any device table)
  * The string is static.
  */

@@ -162,7 +162,7 @@ struct tfps_graph {
     struct LevRec {
         bool ok = false;
         bool by_id = false;    // steps follow the caller's vertex numbering
-        DBuf blob, items, step_ptr, heavy, cls;
+        DBuf blob, items, step_ptr, heavy, cls, flags, part_cnt, item_aux;
         std::vector<int> h_step_ptr;   // host copy: the chained variant launches step by step
         int heavy_count = 0;   // vertices evaluated in partial items (their rows start at zero)
         LevRecArgs args;
@@ -791,7 +791,7 @@ int build_levrec(tfps_graph* g, int k, const int32_t* s, const int64_t* B, long 
         }
         roff[n] = (long long)total;
         if (total >= ((size_t)1 << 31)) continue;
-        std::vector<int> items, step_ptr((size_t)nsteps + 1, 0), heavy, idx;
+        std::vector<int> items, step_ptr((size_t)nsteps + 1, 0), heavy, idx, aux;
         int item_edges = 0, max_items = 1;
         for (int sidx = 0; sidx < nsteps; ++sidx) {
             // forward: steps in ascending order; backward: level steps in descending order (caller-order steps are built descending)
@@ -803,6 +803,8 @@ int build_levrec(tfps_graph* g, int k, const int32_t* s, const int64_t* B, long 
             auto push_item = [&](int p, bool partial, int e0, int e1) {   // descriptor, then the neighbours of its first four edges
                 items.push_back(order[p] | (partial ? (int)0x80000000u : 0)); items.push_back((int)roff[p]); items.push_back(e0); items.push_back(e1);
                 for (int q = 0; q < 4; ++q) items.push_back(e0 + q < e1 ? nb[(size_t)ep[p] + e0 + q] : 0);
+                aux.push_back(partial ? (int)heavy.size() - 1 : 0);   // which of the cut vertices, and into how many items
+                aux.push_back(partial ? (ep[p + 1] - ep[p] + T - 1) / T : 1);
             };
             for (int p : idx) {
                 const int d = ep[p + 1] - ep[p];
@@ -858,6 +860,9 @@ int build_levrec(tfps_graph* g, int k, const int32_t* s, const int64_t* B, long 
         TFPS_TRY(upload(L.step_ptr, step_ptr, st));
         TFPS_TRY(upload(L.heavy, heavy, st));
         TFPS_TRY(upload(L.cls, cls, st));
+        TFPS_TRY(upload(L.item_aux, aux, st));
+        CUDA_TRY(L.flags.alloc(sizeof(unsigned) * (size_t)std::max(1, n)));
+        CUDA_TRY(L.part_cnt.alloc(sizeof(int) * 32 * std::max<size_t>(1, heavy.size())));
         CUDA_TRY(cudaStreamSynchronize(st));
         L.heavy_count = (int)heavy.size();
         L.h_step_ptr = step_ptr;
@@ -875,6 +880,12 @@ int build_levrec(tfps_graph* g, int k, const int32_t* s, const int64_t* B, long 
         L.args.wbytes = wbytes;
         L.args.rtu = (dir == 0 && rtu) ? 1 : 0;
         L.args.rec_max = HDR + item_edges * estride;
+        L.args.flags = L.flags.as<unsigned>();
+        L.args.part_cnt = L.part_cnt.as<int>();
+        L.args.item_aux = L.item_aux.as<int2>();
+        L.args.num_items = (int)(items.size() / 8);
+        L.args.num_vertices = n;
+        L.args.num_heavy = (int)heavy.size();
         L.ok = true;
     }
     return TFPS_OK;
@@ -1493,7 +1504,10 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
                         // One launch per step by default; the persistent form (one cooperative launch, barriers between
                         // the steps inside the kernel) measured slower at every batch width (config 5, forward pass: 14.4
                         // against 10.1 ms at P = 256, 18.9 against 16.0 at 1,024, 33.8 against 29.4 at 4,096) and is opt-in.
-                        if (env_int("TFPS_STEP_PERSISTENT", 0) == 1) {
+                        if (env_int("TFPS_STEP_FLOW", 0) == 1 && flow_applies(la)) {
+                            g->last_kernel = "pass_flow_kernel";
+                            CUDA_TRY(launch_pass_flow(la, fwd, g->sm_count, st));
+                        } else if (env_int("TFPS_STEP_PERSISTENT", 0) == 1) {
                             g->last_kernel = "pass_steprec_kernel";
                             CUDA_TRY(launch_pass_steprec(la, fwd, g->sm_count, st));
                         } else {

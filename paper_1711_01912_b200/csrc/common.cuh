@@ -184,10 +184,17 @@ struct LevRecArgs {
     int blocks_per_sm;           // 0: as many as fit
     int wait_limit;              // polls before a barrier wait gives up
     int shape;                   // block shape variant (tuning)
+    // dataflow form (flow.cu)
+    unsigned* flags;             // [num_vertices] ready bits of every vertex, one per candidate tile (zeroed by the launcher)
+    int* part_cnt;               // [num_heavy][32] finished partial items per vertex cut into several and tile (zeroed by the launcher)
+    const int2* item_aux;        // [num_items] partial items: {index of the vertex among the cut ones, number of its items}
+    int num_items, num_vertices, num_heavy;
 };
 constexpr int STEPREC_GROUPS_MAX = 4;
 cudaError_t launch_pass_steprec(const LevRecArgs& a, bool fwd, int sm_count, cudaStream_t st);
 cudaError_t launch_pass_stepchain(const LevRecArgs& a, bool fwd, const std::vector<int>& step_ptr_host, cudaStream_t st);
+bool flow_applies(const LevRecArgs& a);   // the dataflow form covers k <= 16, items of at most eight edges of at most 64 bytes, P <= 4096
+cudaError_t launch_pass_flow(const LevRecArgs& a, bool fwd, int sm_count, cudaStream_t st);
 
 size_t lean_smem_bytes(const LeanPlan& plan, int slice, int warps, int depth, unsigned* slot_stride, unsigned* stage_bytes);
 cudaError_t launch_pass_lean(const LeanArgs& a, bool fwd, int slice, int cpt, int warps, size_t smem, cudaStream_t st);

@@ -621,6 +621,35 @@ def test_level_kernels_with_partial_items(split, levrec, monkeypatch):
     run_and_compare(w.graph, w.devices, w.part_full(), 1, pad_fill=255)
 
 
+@pytest.mark.parametrize("split", [1, 3, 8])
+def test_dataflow_record_pass(split, monkeypatch):
+    """The dataflow form of the record pass (ready bits per vertex and candidate tile instead of grid-wide steps): a
+    ragged pair of tiles, exactly one tile, nine tiles with a ragged last one, sixteen tiles, a hub of hundreds
+    of in-edges cut into partial items next to vertices without edges, a chain (every item waits for the one before);
+    batches beyond 32 tiles take the chained launches."""
+    from paper_1711_01912_b200 import tfps
+    monkeypatch.setenv("TFPS_TILE_SPLIT", str(split))
+    monkeypatch.setenv("TFPS_STEP_FLOW", "1")
+    rng = np.random.default_rng(177 + split)
+    for P in (300, 256, 2100, 4096):
+        w = I.config5(layers=14, width=64, P=P)
+        run_and_compare(w.graph, w.devices, w.part_full(), 1, pad_fill=255)
+    G = gpu_graph(w.graph, w.devices)
+    dpart, P, ldp = padded(w.part_full())
+    G.eval_batch(dpart, P, flags=1)
+    assert tfps.tfps_last_pass_kernel(G.handle) == "pass_flow_kernel"
+    G.close()
+    n = 700
+    edges = [(u, n - 1, int(rng.integers(0, 10 ** 6))) for u in range(n - 1)] + [(0, u, 5) for u in range(1, 60)]
+    gh = graph_from_edges(n, edges, rng.integers(0, 100, size=n))
+    run_and_compare(gh, _grouped_devices(4, rng), rng.integers(0, 4, size=(n, 270), dtype=np.uint8), 1, pad_fill=255)
+    n = 3000
+    chain = graph_from_edges(n, [(u, u + 1, int(rng.integers(0, 10 ** 5))) for u in range(n - 1)], rng.integers(0, 100, size=n))
+    run_and_compare(chain, _grouped_devices(4, rng), rng.integers(0, 4, size=(n, 200), dtype=np.uint8), 1, pad_fill=255)
+    w = I.config5(layers=9, width=32, P=8300)
+    run_and_compare(w.graph, w.devices, w.part_full(), 1, pad_fill=255)
+
+
 def test_loads_kernel_table_widths():
     """Loads, memory loads and violation flags for every width of the runtime table (k = 1 .. 32) and beyond
     it (k = 33, 64: the shuffle-based kernel), with bounded capacities so that some flags are set."""
@@ -683,7 +712,7 @@ def test_randomized_shapes_all_variants():
             run_and_compare(w.graph, dev, part, flags, pad_fill=255)
 
 
-@pytest.mark.parametrize("family", ["lean", "lean64", "steprec"])
+@pytest.mark.parametrize("family", ["lean", "lean64", "steprec", "flow"])
 def test_bounded_waits_run_out(family, monkeypatch):
     """The bounded device-side waits, made to run out on the host's terms: with a limit of zero polls every wait of
     the windowed kernels (for a staged record) and of the persistent record pass (for the other blocks' signal) gives
@@ -691,10 +720,10 @@ def test_bounded_waits_run_out(family, monkeypatch):
     TFPS_ERR_TIMEOUT through the status word, nothing hangs or faults, and the next call on the same handle is
     bit-exact again."""
     from paper_1711_01912_b200 import tfps
-    if family == "steprec":
+    if family in ("steprec", "flow"):
         w = I.config5(layers=14, width=64, P=300)
         flags = tfps.EVAL_LEVEL_SYNC
-        monkeypatch.setenv("TFPS_STEP_PERSISTENT", "1")
+        monkeypatch.setenv("TFPS_STEP_PERSISTENT" if family == "steprec" else "TFPS_STEP_FLOW", "1")
     else:
         w = I.config2()
         w.P = 200
@@ -706,10 +735,11 @@ def test_bounded_waits_run_out(family, monkeypatch):
     monkeypatch.setenv("TFPS_WAIT_LIMIT", "0")
     out = G.eval_batch(dpart, P, flags=flags, check=False)
     kernel = tfps.tfps_last_pass_kernel(G.handle)
-    assert kernel == {"lean": "pass_lean_kernel", "lean64": "pass_lean64_kernel", "steprec": "pass_steprec_kernel"}[family]
+    assert kernel == {"lean": "pass_lean_kernel", "lean64": "pass_lean64_kernel", "steprec": "pass_steprec_kernel",
+                      "flow": "pass_flow_kernel"}[family]
     with pytest.raises(tfps.TfpsError) as ei:
         G.status()
     assert ei.value.code == tfps.ERR_TIMEOUT
     monkeypatch.delenv("TFPS_WAIT_LIMIT")
     G.close()
-    run_and_compare(w.graph, w.devices, w.part_full()[:, :w.P], 2 if family != "steprec" else 1, pad_fill=255)
+    run_and_compare(w.graph, w.devices, w.part_full()[:, :w.P], 2 if family in ("lean", "lean64") else 1, pad_fill=255)
