@@ -294,3 +294,196 @@ int oracle_critical_mask(int64_t n, const int64_t *tlevel, int64_t tstride, cons
     }
     return ORACLE_OK;
 }
+
+/*
+ * Vertex ranks (Section 3.2, Eq. 5 and Eq. 6), independent of any partition:
+ *      upRank(v)   = c_v + max over successors x of upRank(x)      (the maximum over no successor is 0: a sink has c_v)
+ *      downRank(v) = c_v + max over predecessors u of downRank(u)  (a source has c_v)
+ *      totalRank(v) = upRank(v) + downRank(v)                      (Section 3.2.1: "the sum of the upward rank and the
+ *                                                                   downward rank"; c_v is in both terms, as printed)
+ * topo: any topological order.  Any of up, down, total may be NULL.
+ * Pins: tests/test_oracle_ranks.py (hand values on the worked DAGs, chain closed form, all source-to-sink paths
+ * enumerated on small graphs, the single-device unit-speed evaluation of the same graph).
+ */
+int oracle_ranks(int64_t n, const int64_t *in_ptr, const int32_t *in_src, const int64_t *out_ptr, const int32_t *out_dst,
+                 const int32_t *c, const int32_t *topo, int64_t *up, int64_t *down, int64_t *total)
+{
+    if (n < 0) return ORACLE_BAD_ARG;
+    int64_t *u = (int64_t *)malloc(sizeof(int64_t) * (size_t)(n + 1));
+    int64_t *d = (int64_t *)malloc(sizeof(int64_t) * (size_t)(n + 1));
+    if (!u || !d) { free(u); free(d); return ORACLE_BAD_ARG; }
+    int rc = ORACLE_OK;
+    for (int64_t i = 0; i < n && rc == ORACLE_OK; ++i) {          /* Eq. 6, sources first */
+        int32_t v = topo[i];
+        i128 best = 0;
+        for (int64_t e = in_ptr[v]; e < in_ptr[v + 1]; ++e)
+            if ((i128)d[in_src[e]] > best) best = d[in_src[e]];
+        best += c[v];
+        if (!fits(best)) rc = ORACLE_OVERFLOW; else d[v] = (int64_t)best;
+    }
+    for (int64_t i = n - 1; i >= 0 && rc == ORACLE_OK; --i) {     /* Eq. 5, sinks first */
+        int32_t v = topo[i];
+        i128 best = 0;
+        for (int64_t e = out_ptr[v]; e < out_ptr[v + 1]; ++e)
+            if ((i128)u[out_dst[e]] > best) best = u[out_dst[e]];
+        best += c[v];
+        if (!fits(best)) rc = ORACLE_OVERFLOW; else u[v] = (int64_t)best;
+    }
+    for (int64_t v = 0; v < n && rc == ORACLE_OK; ++v) {
+        i128 t = (i128)u[v] + (i128)d[v];
+        if (!fits(t)) { rc = ORACLE_OVERFLOW; break; }
+        if (up) up[v] = u[v];
+        if (down) down[v] = d[v];
+        if (total) total[v] = (int64_t)t;
+    }
+    free(u); free(d);
+    return rc;
+}
+
+/* devices from the fastest to the slowest (equal speeds: lower index first) */
+static void devices_by_speed(int32_t k, const int32_t *s, int32_t *ord)
+{
+    for (int32_t i = 0; i < k; ++i) ord[i] = i;
+    for (int32_t i = 1; i < k; ++i) {          /* insertion sort, stable */
+        int32_t x = ord[i], j = i;
+        while (j > 0 && s[ord[j - 1]] < s[x]) { ord[j] = ord[j - 1]; --j; }
+        ord[j] = x;
+    }
+}
+
+static const int64_t *rank_keys;   /* keys of the sort below (the oracle is single-threaded) */
+static int rank_order(const void *pa, const void *pb)
+{
+    int64_t a = *(const int64_t *)pa, b = *(const int64_t *)pb;
+    if (rank_keys[a] != rank_keys[b]) return rank_keys[a] > rank_keys[b] ? -1 : 1;
+    return a < b ? -1 : (a > b ? 1 : 0);
+}
+
+/*
+ * Batch Split (Section 3.2.1): the vertices are taken in descending order of total rank (equal ranks: ascending
+ * vertex id) and each is assigned, independently of the others, to the fastest feasible device.  Feasible = the
+ * device's static memory use stays below its capacity with the vertex on it (Eq. 2: usage < C).  A vertex no device
+ * can take goes to the fastest device and is counted in *unplaced (the paper does not say; the instance is then
+ * infeasible).  part[v] receives the device.
+ * Pins: tests/test_oracle_ranks.py (worked example, closed forms, capacity invariants).
+ */
+int oracle_batch_split(int64_t n, const int64_t *total, const int64_t *mem, int32_t k, const int32_t *s,
+                       const int64_t *C, uint8_t *part, int64_t *unplaced)
+{
+    if (n < 0 || k < 1 || k > 64 || !unplaced) return ORACLE_BAD_ARG;
+    int32_t ord[64];
+    i128 used[64];
+    devices_by_speed(k, s, ord);
+    for (int32_t d = 0; d < k; ++d) used[d] = 0;
+    int64_t *idx = (int64_t *)malloc(sizeof(int64_t) * (size_t)(n + 1));
+    if (!idx) return ORACLE_BAD_ARG;
+    for (int64_t v = 0; v < n; ++v) idx[v] = v;
+    rank_keys = total;
+    qsort(idx, (size_t)n, sizeof(int64_t), rank_order);   /* descending total rank, ascending id */
+    int64_t bad = 0;
+    for (int64_t i = 0; i < n; ++i) {
+        int64_t v = idx[i];
+        int32_t chosen = -1;
+        for (int32_t q = 0; q < k && chosen < 0; ++q) {
+            int32_t d = ord[q];
+            if (used[d] + (i128)mem[v] < (i128)C[d]) chosen = d;
+        }
+        if (chosen < 0) { chosen = ord[0]; ++bad; }
+        used[chosen] += mem[v];
+        part[v] = (uint8_t)chosen;
+    }
+    *unplaced = bad;
+    free(idx);
+    return ORACLE_OK;
+}
+
+/*
+ * The critical path of the Critical Path strategy (Section 3.2.2, steps (1)-(4)): the sink with the largest downward
+ * rank (equal ranks: the smallest id), then backwards along predecessors of largest downward rank (equal: smallest id)
+ * until a source is reached.  path receives the vertices from the source to the sink, *len their number.
+ * The summed cost of the path is the chosen sink's downward rank, whatever the tie rule.
+ */
+int oracle_critical_path(int64_t n, const int64_t *in_ptr, const int32_t *in_src, const int64_t *out_ptr,
+                         const int64_t *down, int32_t *path, int64_t *len)
+{
+    if (n < 0 || !len) return ORACLE_BAD_ARG;
+    *len = 0;
+    if (n == 0) return ORACLE_OK;
+    int64_t best = -1;
+    for (int64_t v = 0; v < n; ++v)
+        if (out_ptr[v + 1] == out_ptr[v] && (best < 0 || down[v] > down[best])) best = v;
+    if (best < 0) return ORACLE_CYCLE;
+    int64_t cnt = 0;
+    for (int64_t v = best;;) {
+        path[cnt++] = (int32_t)v;
+        if (in_ptr[v + 1] == in_ptr[v]) break;
+        int64_t u = -1;
+        for (int64_t e = in_ptr[v]; e < in_ptr[v + 1]; ++e) {
+            int64_t x = in_src[e];
+            if (u < 0 || down[x] > down[u] || (down[x] == down[u] && x < u)) u = x;
+        }
+        v = u;
+        if (cnt > n) return ORACLE_CYCLE;
+    }
+    for (int64_t i = 0; i < cnt / 2; ++i) { int32_t t = path[i]; path[i] = path[cnt - 1 - i]; path[cnt - 1 - i] = t; }
+    *len = cnt;
+    return ORACLE_OK;
+}
+
+/*
+ * Critical Path partitioning (Section 3.2.2, Eq. 7).  The critical path goes to the fastest device that can hold all
+ * of it (static memory below capacity, Eq. 2); if none can, it is divided among the fastest devices: the path is
+ * walked from its source and every vertex goes to the fastest device that still has room for it.  Every other
+ * vertex v, in ascending id, goes to the feasible device d that minimises (sum of the execution times of the vertices
+ * already on d) + (execution time of v on d), execution time = ceil(c * S / s_d) ticks (equal sums: lower device
+ * index).  A vertex no device can take is placed by the same rule over all devices and counted in *unplaced.
+ */
+int oracle_cp_partition(int64_t n, const int32_t *path, int64_t len, const int32_t *c, const int64_t *mem,
+                        int32_t k, const int32_t *s, const int64_t *C, int64_t S, uint8_t *part, int64_t *unplaced)
+{
+    if (n < 0 || len < 0 || len > n || k < 1 || k > 64 || S < 1 || !unplaced) return ORACLE_BAD_ARG;
+    int32_t ord[64];
+    i128 used[64], load[64];
+    devices_by_speed(k, s, ord);
+    for (int32_t d = 0; d < k; ++d) { used[d] = 0; load[d] = 0; }
+    uint8_t *on_path = (uint8_t *)calloc((size_t)(n + 1), 1);
+    if (!on_path) return ORACLE_BAD_ARG;
+    int64_t bad = 0;
+    i128 path_mem = 0;
+    for (int64_t i = 0; i < len; ++i) { on_path[path[i]] = 1; path_mem += mem[path[i]]; }
+    int32_t whole = -1;
+    for (int32_t q = 0; q < k && whole < 0; ++q)
+        if (path_mem < (i128)C[ord[q]]) whole = ord[q];
+    for (int64_t i = 0; i < len; ++i) {
+        int64_t v = path[i];
+        int32_t chosen = whole;
+        for (int32_t q = 0; q < k && chosen < 0; ++q)
+            if (used[ord[q]] + (i128)mem[v] < (i128)C[ord[q]]) chosen = ord[q];
+        if (chosen < 0) { chosen = ord[0]; ++bad; }
+        int64_t rt;
+        if (ceil_scaled(c[v], S, s[chosen], &rt)) { free(on_path); return ORACLE_OVERFLOW; }
+        used[chosen] += mem[v];
+        load[chosen] += rt;
+        part[v] = (uint8_t)chosen;
+    }
+    for (int64_t v = 0; v < n; ++v) {
+        if (on_path[v]) continue;
+        int32_t chosen = -1, any = -1;
+        i128 best = 0, best_any = 0;
+        for (int32_t d = 0; d < k; ++d) {
+            int64_t rt;
+            if (ceil_scaled(c[v], S, s[d], &rt)) { free(on_path); return ORACLE_OVERFLOW; }
+            i128 sum = load[d] + rt;                                 /* Eq. 7 */
+            if (any < 0 || sum < best_any) { any = d; best_any = sum; }
+            if (used[d] + (i128)mem[v] < (i128)C[d] && (chosen < 0 || sum < best)) { chosen = d; best = sum; }
+        }
+        if (chosen < 0) { chosen = any; best = best_any; ++bad; }
+        if (!fits(best)) { free(on_path); return ORACLE_OVERFLOW; }
+        used[chosen] += mem[v];
+        load[chosen] = best;
+        part[v] = (uint8_t)chosen;
+    }
+    *unplaced = bad;
+    free(on_path);
+    return ORACLE_OK;
+}
