@@ -60,6 +60,14 @@ def _get():
         lib.oracle_eval_constraints.argtypes = [ctypes.c_int64, P, ctypes.c_int64, ctypes.c_int64, P, P, ctypes.c_int64, P, P, P, P]
         lib.oracle_critical_mask.restype = ctypes.c_int
         lib.oracle_critical_mask.argtypes = [ctypes.c_int64, P, ctypes.c_int64, P, ctypes.c_int64, ctypes.c_int64, P, ctypes.c_int64]
+        lib.oracle_ranks.restype = ctypes.c_int
+        lib.oracle_ranks.argtypes = [ctypes.c_int64] + [P] * 9
+        lib.oracle_batch_split.restype = ctypes.c_int
+        lib.oracle_batch_split.argtypes = [ctypes.c_int64, P, P, ctypes.c_int32, P, P, P, P]
+        lib.oracle_critical_path.restype = ctypes.c_int
+        lib.oracle_critical_path.argtypes = [ctypes.c_int64, P, P, P, P, P, P]
+        lib.oracle_cp_partition.restype = ctypes.c_int
+        lib.oracle_cp_partition.argtypes = [ctypes.c_int64, P, ctypes.c_int64, P, P, ctypes.c_int32, P, P, ctypes.c_int64, P, P]
         _lib = lib
     return _lib
 
@@ -210,3 +218,59 @@ def critical_mask(tlevel: np.ndarray, blevel: np.ndarray, cp: np.ndarray) -> np.
         if rc:
             raise OracleError(rc)
     return mask
+
+
+def ranks(g: OracleGraph):
+    """(upRank, downRank, totalRank) of every vertex, int64 [n] each (Eq. 5, Eq. 6, Section 3.2.1)."""
+    lib = _get()
+    up = np.zeros(g.n, np.int64)
+    down = np.zeros(g.n, np.int64)
+    total = np.zeros(g.n, np.int64)
+    rc = lib.oracle_ranks(g.n, _p(g.in_ptr), _p(g.in_src), _p(g.out_ptr), _p(g.out_dst), _p(g.c), _p(g.topo),
+                          _p(up), _p(down), _p(total))
+    if rc:
+        raise OracleError(rc)
+    return up, down, total
+
+
+def batch_split(total, mem, k: int, s, C):
+    """Batch Split partition (Section 3.2.1): (part uint8 [n], number of vertices no device could take)."""
+    lib = _get()
+    total = _arr(total, np.int64)
+    mem = _arr(mem, np.int64)
+    s = _arr(s, np.int32)
+    C = _arr(C, np.int64)
+    n = total.shape[0]
+    part = np.zeros(n, np.uint8)
+    bad = ctypes.c_int64(0)
+    rc = lib.oracle_batch_split(n, _p(total), _p(mem), k, _p(s), _p(C), _p(part), ctypes.byref(bad))
+    if rc:
+        raise OracleError(rc)
+    return part, int(bad.value)
+
+
+def critical_path(g: OracleGraph, down) -> np.ndarray:
+    """Vertices of the critical path of the Critical Path strategy, source to sink (Section 3.2.2, steps 1-4)."""
+    lib = _get()
+    down = _arr(down, np.int64)
+    path = np.zeros(max(1, g.n), np.int32)
+    ln = ctypes.c_int64(0)
+    rc = lib.oracle_critical_path(g.n, _p(g.in_ptr), _p(g.in_src), _p(g.out_ptr), _p(down), _p(path), ctypes.byref(ln))
+    if rc:
+        raise OracleError(rc)
+    return path[: int(ln.value)].copy()
+
+
+def cp_partition(g: OracleGraph, path, k: int, s, C, S: int):
+    """Critical Path partition (Section 3.2.2, Eq. 7): (part uint8 [n], number of vertices no device could take)."""
+    lib = _get()
+    path = _arr(path, np.int32)
+    s = _arr(s, np.int32)
+    C = _arr(C, np.int64)
+    part = np.zeros(g.n, np.uint8)
+    bad = ctypes.c_int64(0)
+    rc = lib.oracle_cp_partition(g.n, _p(path), path.shape[0], _p(g.c), _p(g.mem), k, _p(s), _p(C), S, _p(part),
+                                 ctypes.byref(bad))
+    if rc:
+        raise OracleError(rc)
+    return part, int(bad.value)
