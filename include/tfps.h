@@ -310,6 +310,56 @@ int tfps_eval_constraints(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* 
 int tfps_critical_mask(int64_t n, int64_t P, int64_t ldp, const int64_t* tlevel, const int64_t* blevel,
                        const int64_t* cp, uint8_t* mask, void* stream);
 
+/*
+ * Vertex ranks (Section 3.2, Eq. 5 and Eq. 6), independent of any partition and of the
+ * device tables:
+ *   upRank(v)    = c_v + max over successors x of upRank(x)      (a sink: c_v)
+ *   downRank(v)  = c_v + max over predecessors u of downRank(u)  (a source: c_v)
+ *   totalRank(v) = upRank(v) + downRank(v)                       (Section 3.2.1; c_v is in both)
+ *   up, down, total   dev int64 [n] each, any of them NULL when not wanted
+ * One launch per topological level and direction.  Asynchronous on `stream`.
+ * TFPS_ERR_OVERFLOW if twice the sum of all costs could reach 2^62.
+ */
+int tfps_ranks(tfps_graph* g, int64_t* up, int64_t* down, int64_t* total, void* stream);
+
+/*
+ * The critical path of the Critical Path strategy (Section 3.2.2, steps 1-4): the sink of
+ * largest downward rank (equal ranks: the smallest id), then backwards along predecessors
+ * of largest downward rank (equal: the smallest id) to a source.
+ *   down   dev int64 [n] from tfps_ranks
+ *   path   dev int32 [n]; receives the path's vertices from the source to the sink
+ *   len    host; number of vertices written
+ * Synchronises `stream` (the length comes back to the host).
+ */
+int tfps_critical_path(tfps_graph* g, const int64_t* down, int32_t* path, int64_t* len, void* stream);
+
+/*
+ * Batch Split (Section 3.2.1): vertices in descending order of total rank (equal ranks:
+ * ascending id), each assigned to the fastest device (equal speeds: lower index) whose
+ * static memory use stays BELOW its capacity with the vertex on it (Eq. 2).  A vertex no
+ * device can take goes to the fastest device and is counted.  Uses the device tables of
+ * tfps_devices_set (speeds, capacities) and the graph's per-vertex memory.
+ *   total      dev int64 [n] from tfps_ranks
+ *   part       dev uint8 [n]; receives the device of every vertex
+ *   unplaced   host; number of vertices no device could take
+ * Synchronises `stream`.  TFPS_ERR_STATE before tfps_devices_set.
+ */
+int tfps_batch_split(tfps_graph* g, const int64_t* total, uint8_t* part, int64_t* unplaced, void* stream);
+
+/*
+ * Critical Path partitioning (Section 3.2.2, Eq. 7).  The path goes to the fastest device
+ * that can hold all of it (memory below capacity); if none can, it is walked from its
+ * source and every vertex goes to the fastest device that still has room.  Every other
+ * vertex, in ascending id, goes to the feasible device d that minimises (execution times
+ * already on d) + ceil(c_v * scale / s_d) (equal sums: lower index); without a feasible
+ * device the same rule runs over all devices and the vertex is counted.
+ *   path, len  dev int32 [len] from tfps_critical_path (len = 0: no path)
+ *   part       dev uint8 [n]
+ *   unplaced   host
+ * Synchronises `stream`.  TFPS_ERR_STATE before tfps_devices_set.
+ */
+int tfps_cp_partition(tfps_graph* g, const int32_t* path, int64_t len, uint8_t* part, int64_t* unplaced, void* stream);
+
 /* Synchronise `stream`, return the sticky device-side status of the handle and clear it. */
 int tfps_get_status(tfps_graph* g, void* stream);
 

@@ -173,6 +173,8 @@ struct tfps_graph {
     DBuf status;
     // placement constraints (tfps_constraints_set)
     DBuf cons_a, cons_b, cons_v, cons_d;
+    // rank-driven partitioners: device speeds, devices from the fastest to the slowest, scratch
+    DBuf speed_d, ord_d, part_idx, part_flag, part_scr, rank_up, rank_down;
     int cons_pairs = 0, cons_dev = 0;
     // scratch owned by the handle
     DBuf scr_memload;
@@ -1219,6 +1221,14 @@ int tfps_devices_set(tfps_graph* g, int k, const int32_t* s, const int64_t* C, c
     }
     g->k = k;
     g->S = scale;
+    {
+        std::vector<int> speed(s, s + k), ord((size_t)k);
+        for (int d = 0; d < k; ++d) ord[d] = d;
+        std::stable_sort(ord.begin(), ord.end(), [&](int a, int b) { return s[a] > s[b]; });   // equal speeds: lower index first
+        TFPS_TRY(upload(g->speed_d, speed, st));
+        TFPS_TRY(upload(g->ord_d, ord, st));
+        CUDA_TRY(cudaStreamSynchronize(st));
+    }
     g->dev_set = true;
     return TFPS_OK;
 }
@@ -1632,6 +1642,92 @@ int tfps_critical_mask(int64_t n, int64_t P, int64_t ldp, const int64_t* tlevel,
         return fail(TFPS_ERR_INVALID_ARG, "tlevel, blevel, cp and mask must be 16-byte aligned");
     CUDA_TRY(launch_critical_mask(n, P, ldp, (const long long*)tlevel, (const long long*)blevel, (const long long*)cp, mask,
                                   (cudaStream_t)stream));
+    return TFPS_OK;
+}
+
+int tfps_ranks(tfps_graph* g, int64_t* up, int64_t* down, int64_t* total, void* stream)
+{
+    if (!g) return fail(TFPS_ERR_INVALID_ARG, "graph is NULL");
+    DeviceGuard guard(g->device);
+    if (!guard.ok) return fail(TFPS_ERR_CUDA, "cannot select the handle's device");
+    cudaStream_t st = (cudaStream_t)stream;
+    TFPS_TRY(build_topo(g, st));
+    if (g->n == 0) return TFPS_OK;
+    // a rank is at most the sum of all costs, which tfps_graph_create has bounded; the total rank at most twice that
+    if (g->sum_c >= (u128)(LIMIT62 / 2)) return fail(TFPS_ERR_OVERFLOW, "a total rank could reach 2^62");
+    const size_t bytes = sizeof(long long) * (size_t)g->n;
+    if (!up) { CUDA_TRY(g->rank_up.reserve(bytes)); up = g->rank_up.as<int64_t>(); }
+    if (!down) { CUDA_TRY(g->rank_down.reserve(bytes)); down = g->rank_down.as<int64_t>(); }
+    CUDA_TRY(launch_ranks((int)g->n, g->h_level_ptr, g->order.as<int>(), g->in_ptr.as<long long>(), g->in_src.as<int>(),
+                          g->out_ptr.as<long long>(), g->out_dst.as<int>(), g->c.as<int>(), (long long*)up, (long long*)down,
+                          (long long*)total, st));
+    return TFPS_OK;
+}
+
+int tfps_critical_path(tfps_graph* g, const int64_t* down, int32_t* path, int64_t* len, void* stream)
+{
+    if (!g || !len) return fail(TFPS_ERR_INVALID_ARG, "graph and len are required");
+    *len = 0;
+    if (g->n == 0) return TFPS_OK;
+    if (!down || !path) return fail(TFPS_ERR_INVALID_ARG, "down and path are required");
+    DeviceGuard guard(g->device);
+    if (!guard.ok) return fail(TFPS_ERR_CUDA, "cannot select the handle's device");
+    cudaStream_t st = (cudaStream_t)stream;
+    CUDA_TRY(g->part_scr.reserve(sizeof(long long) * 4));
+    CUDA_TRY(launch_critical_path((int)g->n, g->in_ptr.as<long long>(), g->in_src.as<int>(), g->out_ptr.as<long long>(),
+                                  (const long long*)down, path, g->part_scr.as<long long>(), st));
+    long long h = 0;
+    CUDA_TRY(cudaMemcpyAsync(&h, g->part_scr.as<long long>() + 2, sizeof(long long), cudaMemcpyDeviceToHost, st));
+    CUDA_TRY(cudaStreamSynchronize(st));
+    *len = h;
+    return TFPS_OK;
+}
+
+int tfps_batch_split(tfps_graph* g, const int64_t* total, uint8_t* part, int64_t* unplaced, void* stream)
+{
+    if (!g || !unplaced) return fail(TFPS_ERR_INVALID_ARG, "graph and unplaced are required");
+    *unplaced = 0;
+    if (!g->dev_set) return fail(TFPS_ERR_STATE, "tfps_devices_set has not been called");
+    if (g->n == 0) return TFPS_OK;
+    if (!total || !part) return fail(TFPS_ERR_INVALID_ARG, "total and part are required");
+    DeviceGuard guard(g->device);
+    if (!guard.ok) return fail(TFPS_ERR_CUDA, "cannot select the handle's device");
+    cudaStream_t st = (cudaStream_t)stream;
+    int npad = 1;
+    while (npad < g->n) npad <<= 1;
+    CUDA_TRY(g->part_idx.reserve(sizeof(int) * (size_t)npad));
+    CUDA_TRY(g->part_scr.reserve(sizeof(long long) * 4));
+    long long* d_unplaced = g->part_scr.as<long long>() + 3;
+    CUDA_TRY(launch_batch_split((int)g->n, npad, g->k, (const long long*)total, g->mem.as<long long>(), g->ord_d.as<int>(),
+                                g->cap.as<long long>(), g->part_idx.as<int>(), part, d_unplaced, st));
+    long long h = 0;
+    CUDA_TRY(cudaMemcpyAsync(&h, d_unplaced, sizeof(long long), cudaMemcpyDeviceToHost, st));
+    CUDA_TRY(cudaStreamSynchronize(st));
+    *unplaced = h;
+    return TFPS_OK;
+}
+
+int tfps_cp_partition(tfps_graph* g, const int32_t* path, int64_t len, uint8_t* part, int64_t* unplaced, void* stream)
+{
+    if (!g || !unplaced) return fail(TFPS_ERR_INVALID_ARG, "graph and unplaced are required");
+    *unplaced = 0;
+    if (!g->dev_set) return fail(TFPS_ERR_STATE, "tfps_devices_set has not been called");
+    if (len < 0 || len > g->n) return fail(TFPS_ERR_INVALID_ARG, "need 0 <= len <= n");
+    if (g->n == 0) return TFPS_OK;
+    if (!part || (len > 0 && !path)) return fail(TFPS_ERR_INVALID_ARG, "part (and path when len > 0) are required");
+    DeviceGuard guard(g->device);
+    if (!guard.ok) return fail(TFPS_ERR_CUDA, "cannot select the handle's device");
+    cudaStream_t st = (cudaStream_t)stream;
+    CUDA_TRY(g->part_flag.reserve((size_t)g->n));
+    CUDA_TRY(g->part_scr.reserve(sizeof(long long) * 4));
+    long long* d_unplaced = g->part_scr.as<long long>() + 3;
+    CUDA_TRY(launch_cp_partition((int)g->n, g->k, g->S, path, len, g->c.as<int>(), g->mem.as<long long>(),
+                                 g->speed_d.as<int>(), g->ord_d.as<int>(), g->cap.as<long long>(),
+                                 g->part_flag.as<uint8_t>(), part, d_unplaced, st));
+    long long h = 0;
+    CUDA_TRY(cudaMemcpyAsync(&h, d_unplaced, sizeof(long long), cudaMemcpyDeviceToHost, st));
+    CUDA_TRY(cudaStreamSynchronize(st));
+    *unplaced = h;
     return TFPS_OK;
 }
 

@@ -243,6 +243,17 @@ cudaError_t launch_constraints(long long P, long long ldp, const uint8_t* part, 
                                cudaStream_t st);
 cudaError_t launch_critical_mask(long long n, long long P, long long ldp, const long long* tlevel, const long long* blevel,
                                  const long long* cp, uint8_t* mask, cudaStream_t st);
+// rank-driven partitioners (partition.cu)
+cudaError_t launch_ranks(int n, const std::vector<long long>& level_ptr, const int* order, const long long* in_ptr,
+                         const int* in_src, const long long* out_ptr, const int* out_dst, const int* c, long long* up,
+                         long long* down, long long* total, cudaStream_t st);
+cudaError_t launch_critical_path(int n, const long long* in_ptr, const int* in_src, const long long* out_ptr,
+                                 const long long* down, int* path, long long* scratch, cudaStream_t st);
+cudaError_t launch_batch_split(int n, int npad, int k, const long long* total, const long long* mem, const int* ord,
+                               const long long* cap, int* idx, uint8_t* part, long long* unplaced, cudaStream_t st);
+cudaError_t launch_cp_partition(int n, int k, long long S, const int* path, long long len, const int* c, const long long* mem,
+                                const int* speed, const int* ord, const long long* cap, uint8_t* on_path, uint8_t* part,
+                                long long* unplaced, cudaStream_t st);
 cudaError_t launch_transpose_u8(const uint8_t* src, uint8_t* dst, long long P, long long n, long long ldp, cudaStream_t st);
 
 }  // namespace tfps

@@ -32,6 +32,7 @@ EXPORTS = [
     "tfps_devices_set", "tfps_topo_levels", "tfps_eval_workspace_bytes", "tfps_eval_batch",
     "tfps_eval_batch_host", "tfps_get_status", "tfps_transpose_u8", "tfps_phase_times", "tfps_kernel_launches",
     "tfps_eval_cp_noalloc", "tfps_last_pass_kernel", "tfps_probe_gather_bandwidth", "tfps_constraints_set", "tfps_eval_constraints", "tfps_critical_mask",
+    "tfps_ranks", "tfps_critical_path", "tfps_batch_split", "tfps_cp_partition",
 ]
 
 
@@ -84,6 +85,14 @@ def lib() -> ctypes.CDLL:
     L.tfps_eval_constraints.argtypes = [vp, i64, i64, vp, vp, vp, vp]
     L.tfps_critical_mask.restype = ci
     L.tfps_critical_mask.argtypes = [i64, i64, i64, vp, vp, vp, vp, vp]
+    L.tfps_ranks.restype = ci
+    L.tfps_ranks.argtypes = [vp, vp, vp, vp, vp]
+    L.tfps_critical_path.restype = ci
+    L.tfps_critical_path.argtypes = [vp, vp, vp, ctypes.POINTER(ctypes.c_int64), vp]
+    L.tfps_batch_split.restype = ci
+    L.tfps_batch_split.argtypes = [vp, vp, vp, ctypes.POINTER(ctypes.c_int64), vp]
+    L.tfps_cp_partition.restype = ci
+    L.tfps_cp_partition.argtypes = [vp, vp, i64, vp, ctypes.POINTER(ctypes.c_int64), vp]
     L.tfps_probe_gather_bandwidth.restype = ci
     L.tfps_probe_gather_bandwidth.argtypes = [sz, ci, ctypes.POINTER(ctypes.c_double)]
     L.tfps_last_pass_kernel.restype = ctypes.c_char_p
@@ -178,6 +187,28 @@ def tfps_eval_constraints(g, P, ldp, part, coll_viol, dev_viol, stream) -> None:
 
 def tfps_critical_mask(n, P, ldp, tlevel, blevel, cp, mask, stream) -> None:
     _check(lib().tfps_critical_mask(n, P, ldp, tlevel, blevel, cp, mask, stream))
+
+
+def tfps_ranks(handle, up, down, total, stream) -> None:
+    _check(lib().tfps_ranks(handle, up, down, total, stream))
+
+
+def tfps_critical_path(handle, down, path, stream) -> int:
+    ln = ctypes.c_int64(0)
+    _check(lib().tfps_critical_path(handle, down, path, ctypes.byref(ln), stream))
+    return int(ln.value)
+
+
+def tfps_batch_split(handle, total, part, stream) -> int:
+    bad = ctypes.c_int64(0)
+    _check(lib().tfps_batch_split(handle, total, part, ctypes.byref(bad), stream))
+    return int(bad.value)
+
+
+def tfps_cp_partition(handle, path, length, part, stream) -> int:
+    bad = ctypes.c_int64(0)
+    _check(lib().tfps_cp_partition(handle, path, length, part, ctypes.byref(bad), stream))
+    return int(bad.value)
 
 
 def tfps_probe_gather_bandwidth(working_set_bytes: int, rows_per_warp: int = 4096) -> float:
@@ -357,6 +388,34 @@ class Graph:
         dev = torch.empty(max(P, 1), dtype=torch.int32, device=part.device)
         tfps_eval_constraints(self.handle, P, ldp, _addr(part), _addr(coll), _addr(dev), _stream())
         return coll[:P], dev[:P]
+
+    def ranks(self):
+        """(upRank, downRank, totalRank): three int64 CUDA tensors [n] (Eq. 5, Eq. 6, Section 3.2.1)."""
+        import torch
+        up, down, total = (torch.zeros(max(self.n, 1), dtype=torch.int64, device="cuda") for _ in range(3))
+        tfps_ranks(self.handle, _addr(up), _addr(down), _addr(total), _stream())
+        return up[:self.n], down[:self.n], total[:self.n]
+
+    def critical_path(self, down):
+        """int32 CUDA tensor: the vertices of the critical path from its source to its sink (Section 3.2.2)."""
+        import torch
+        path = torch.zeros(max(self.n, 1), dtype=torch.int32, device="cuda")
+        ln = tfps_critical_path(self.handle, _addr(down), _addr(path), _stream())
+        return path[:ln]
+
+    def batch_split(self, total):
+        """(uint8 CUDA tensor [n] of devices, number of vertices no device could take): Batch Split (Section 3.2.1)."""
+        import torch
+        part = torch.zeros(max(self.n, 1), dtype=torch.uint8, device="cuda")
+        bad = tfps_batch_split(self.handle, _addr(total), _addr(part), _stream())
+        return part[:self.n], bad
+
+    def cp_partition(self, path):
+        """(uint8 CUDA tensor [n] of devices, unplaced count): Critical Path partitioning (Section 3.2.2, Eq. 7)."""
+        import torch
+        part = torch.zeros(max(self.n, 1), dtype=torch.uint8, device="cuda")
+        bad = tfps_cp_partition(self.handle, _addr(path) if path.numel() else None, int(path.numel()), _addr(part), _stream())
+        return part[:self.n], bad
 
     def status(self):
         tfps_get_status(self.handle, _stream())
