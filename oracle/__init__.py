@@ -68,6 +68,9 @@ def _get():
         lib.oracle_critical_path.argtypes = [ctypes.c_int64, P, P, P, P, P, P]
         lib.oracle_cp_partition.restype = ctypes.c_int
         lib.oracle_cp_partition.argtypes = [ctypes.c_int64, P, ctypes.c_int64, P, P, ctypes.c_int32, P, P, ctypes.c_int64, P, P]
+        lib.oracle_simulate.restype = ctypes.c_int
+        lib.oracle_simulate.argtypes = ([ctypes.c_int64] + [P] * 5 + [ctypes.c_int32, P, P, ctypes.c_int64, P, ctypes.c_int64,
+                                        ctypes.c_int32, P, ctypes.c_int64, P, P])
         _lib = lib
     return _lib
 
@@ -274,3 +277,20 @@ def cp_partition(g: OracleGraph, path, k: int, s, C, S: int):
     if rc:
         raise OracleError(rc)
     return part, int(bad.value)
+
+
+def simulate(g: OracleGraph, k: int, s, B, S: int, p, policy: int, prio=None):
+    """List-scheduling simulation of one candidate (Section 4): (start times int64 [n], makespan).
+    policy 0 = FIFO, 1 = PCT with prio = the candidate's path computation times (blevel, Eq. 12)."""
+    lib = _get()
+    s = _arr(s, np.int32)
+    B = _arr(B, np.int64)
+    p = _arr(p, np.uint8)
+    pr = None if prio is None else _arr(prio, np.int64)
+    start = np.zeros(g.n, np.int64)
+    mk = ctypes.c_int64(0)
+    rc = lib.oracle_simulate(g.n, _p(g.in_ptr), _p(g.out_ptr), _p(g.out_dst), _p(g.out_t), _p(g.c), k, _p(s), _p(B), S,
+                             _p(p), 1, policy, _p(pr), 1, _p(start), ctypes.byref(mk))
+    if rc:
+        raise OracleError(rc)
+    return start, int(mk.value)

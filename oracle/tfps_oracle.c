@@ -487,3 +487,110 @@ int oracle_cp_partition(int64_t n, const int32_t *path, int64_t len, const int32
     free(on_path);
     return ORACLE_OK;
 }
+
+/*
+ * List-scheduling simulation of one candidate partition (Section 4, criteria (1)-(6); the event-based simulation of
+ * Section 5).  Every device executes the vertices assigned to it, one at a time and without interruption (criteria
+ * 1-3, 5); a vertex is executable once every predecessor has finished and its tensor has arrived,
+ *      ready(v) = max over in-edges (u->v) of finish(u) + w(u->v),   0 for a source           (criterion 4)
+ * with the execution and transfer times of the evaluation (rt, w; transfers do not queue: the paper models none);
+ * an idle device that has an executable vertex starts one at once, otherwise it stays idle (criterion 6).
+ * Which one: policy 0 = FIFO (the vertex that became executable first; equal times: the smaller id),
+ *            policy 1 = PCT (Section 4.1: the largest path computation time, Eq. 12, passed in as prio[]; equal: the
+ *                       smaller id).
+ * Events are taken in time order; at one time T first every execution that ends at T is completed (and its
+ * successors' ready times updated), then every idle device starts its best executable vertex; a vertex of zero
+ * execution time ends at T as well, so the two steps repeat at T until nothing changes.
+ * start[v] receives the start time of v (the schedule f of Section 2), *makespan the time the last vertex ends.
+ * The per-device lists are plain arrays scanned linearly.
+ */
+int oracle_simulate(int64_t n,
+                    const int64_t *in_ptr, const int64_t *out_ptr, const int32_t *out_dst, const int64_t *out_t,
+                    const int32_t *c, int32_t k, const int32_t *s, const int64_t *B, int64_t S,
+                    const uint8_t *p, int64_t p_stride, int32_t policy, const int64_t *prio, int64_t prio_stride,
+                    int64_t *start, int64_t *makespan)
+{
+    if (n < 0 || k < 1 || k > 64 || S < 1 || policy < 0 || policy > 1 || !makespan) return ORACLE_BAD_ARG;
+    if (policy == 1 && !prio) return ORACLE_BAD_ARG;
+    *makespan = 0;
+    if (n == 0) return ORACLE_OK;
+    int rc = ORACLE_OK;
+    int64_t *rt = (int64_t *)malloc(sizeof(int64_t) * (size_t)n);
+    int64_t *ready = (int64_t *)calloc((size_t)n, sizeof(int64_t));
+    int64_t *left = (int64_t *)malloc(sizeof(int64_t) * (size_t)n);       /* predecessors not finished yet */
+    int64_t *list = (int64_t *)malloc(sizeof(int64_t) * (size_t)n);       /* per device: vertices whose ready time is known */
+    int64_t first[65], count[64], running[64], busy_until[64];
+    if (!rt || !ready || !left || !list) { rc = ORACLE_BAD_ARG; goto done; }
+    for (int32_t d = 0; d <= k; ++d) first[d] = 0;
+    for (int64_t v = 0; v < n; ++v) {
+        int32_t d = p[v * p_stride];
+        if (d >= k) { rc = ORACLE_BAD_PARTITION; goto done; }
+        if (ceil_scaled(c[v], S, s[d], &rt[v])) { rc = ORACLE_OVERFLOW; goto done; }
+        first[d + 1] += 1;
+        left[v] = in_ptr[v + 1] - in_ptr[v];
+    }
+    for (int32_t d = 0; d < k; ++d) { first[d + 1] += first[d]; count[d] = 0; running[d] = -1; busy_until[d] = 0; }
+    for (int64_t v = 0; v < n; ++v)
+        if (left[v] == 0) { int32_t d = p[v * p_stride]; list[first[d] + count[d]++] = v; }
+    int64_t T = 0, done_cnt = 0, last = 0;
+    while (done_cnt < n) {
+        /* every idle device starts its best executable vertex */
+        for (int32_t d = 0; d < k; ++d) {
+            if (running[d] >= 0) continue;
+            int64_t best = -1, at = -1;
+            for (int64_t i = 0; i < count[d]; ++i) {
+                int64_t v = list[first[d] + i];
+                if (ready[v] > T) continue;
+                int better;
+                if (best < 0) better = 1;
+                else if (policy == 0) better = ready[v] < ready[best] || (ready[v] == ready[best] && v < best);
+                else better = prio[v * prio_stride] > prio[best * prio_stride] ||
+                              (prio[v * prio_stride] == prio[best * prio_stride] && v < best);
+                if (better) { best = v; at = i; }
+            }
+            if (best < 0) continue;
+            list[first[d] + at] = list[first[d] + --count[d]];
+            i128 fin = (i128)T + (i128)rt[best];
+            if (!fits(fin)) { rc = ORACLE_OVERFLOW; goto done; }
+            running[d] = best;
+            busy_until[d] = (int64_t)fin;
+            if (start) start[best] = T;
+        }
+        /* the next time anything happens: an execution ends, or an idle device's earliest vertex becomes executable */
+        int64_t next = -1;
+        for (int32_t d = 0; d < k; ++d) {
+            if (running[d] >= 0) {
+                if (next < 0 || busy_until[d] < next) next = busy_until[d];
+            } else {
+                for (int64_t i = 0; i < count[d]; ++i) {
+                    int64_t r = ready[list[first[d] + i]];
+                    if (next < 0 || r < next) next = r;
+                }
+            }
+        }
+        if (next < 0) { rc = ORACLE_CYCLE; goto done; }   /* nothing runs and nothing is pending: not a DAG */
+        T = next;
+        /* executions that end at T */
+        for (int32_t d = 0; d < k; ++d) {
+            if (running[d] < 0 || busy_until[d] != T) continue;
+            int64_t u = running[d];
+            running[d] = -1;
+            ++done_cnt;
+            if (T > last) last = T;
+            for (int64_t e = out_ptr[u]; e < out_ptr[u + 1]; ++e) {
+                int64_t x = out_dst[e];
+                int32_t dx = p[x * p_stride];
+                int64_t w = 0;
+                if (dx != d && ceil_scaled(out_t[e], S, B[(int64_t)d * k + dx], &w)) { rc = ORACLE_OVERFLOW; goto done; }
+                i128 arr = (i128)T + (i128)w;
+                if (!fits(arr)) { rc = ORACLE_OVERFLOW; goto done; }
+                if ((int64_t)arr > ready[x]) ready[x] = (int64_t)arr;
+                if (--left[x] == 0) list[first[dx] + count[dx]++] = x;
+            }
+        }
+    }
+    *makespan = last;
+done:
+    free(rt); free(ready); free(left); free(list);
+    return rc;
+}
