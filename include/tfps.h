@@ -360,6 +360,30 @@ int tfps_batch_split(tfps_graph* g, const int64_t* total, uint8_t* part, int64_t
  */
 int tfps_cp_partition(tfps_graph* g, const int32_t* path, int64_t len, uint8_t* part, int64_t* unplaced, void* stream);
 
+/*
+ * Batched list-scheduling simulation (Section 4, criteria (1)-(6); the event-based
+ * simulation of Section 5), every candidate on its own.  A device executes its vertices
+ * one at a time without interruption; a vertex is executable once every predecessor has
+ * finished and its tensor has arrived (finish + transfer time of the evaluation; transfers
+ * do not queue); an idle device with an executable vertex starts one at once:
+ *   TFPS_SCHED_FIFO  the vertex that became executable first
+ *   TFPS_SCHED_PCT   the vertex with the largest path computation time (Section 4.1,
+ *                    Eq. 12): prio = the blevel matrix tfps_eval_batch wrote for `part`
+ * equal keys: the smaller vertex id.  At one time T first the executions that end at T are
+ * completed, then the idle devices start; both repeat at T while executions of zero length end.
+ *   part       dev uint8 [n][ldp]
+ *   prio       dev int64 [n][ldp] (PCT) or NULL (FIFO)
+ *   start      dev int64 [n][ldp] or NULL; start time of every vertex (the schedule f of
+ *              Section 2); padding columns are not written
+ *   makespan   dev int64 [P]; time the last vertex ends (-1 for a candidate with an id >= k,
+ *              which also raises TFPS_ERR_BAD_PARTITION in the status word)
+ * One warp per candidate; scratch of 16 bytes per vertex and candidate in flight is owned
+ * by the handle (allocated on first use).  Asynchronous on `stream`.
+ */
+enum { TFPS_SCHED_FIFO = 0, TFPS_SCHED_PCT = 1 };
+int tfps_simulate(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, int policy, const int64_t* prio,
+                  int64_t* start, int64_t* makespan, void* stream);
+
 /* Synchronise `stream`, return the sticky device-side status of the handle and clear it. */
 int tfps_get_status(tfps_graph* g, void* stream);
 

@@ -174,7 +174,8 @@ struct tfps_graph {
     // placement constraints (tfps_constraints_set)
     DBuf cons_a, cons_b, cons_v, cons_d;
     // rank-driven partitioners: device speeds, devices from the fastest to the slowest, scratch
-    DBuf speed_d, ord_d, part_idx, part_flag, part_scr, rank_up, rank_down;
+    DBuf speed_d, ord_d, bw_d, part_idx, part_flag, part_scr, rank_up, rank_down;
+    DBuf sim_ready, sim_left, sim_list;   // scratch of the scheduling simulation
     int cons_pairs = 0, cons_dev = 0;
     // scratch owned by the handle
     DBuf scr_memload;
@@ -1227,6 +1228,9 @@ int tfps_devices_set(tfps_graph* g, int k, const int32_t* s, const int64_t* C, c
         std::stable_sort(ord.begin(), ord.end(), [&](int a, int b) { return s[a] > s[b]; });   // equal speeds: lower index first
         TFPS_TRY(upload(g->speed_d, speed, st));
         TFPS_TRY(upload(g->ord_d, ord, st));
+        std::vector<long long> bw(B, B + (size_t)k * k);
+        for (int d = 0; d < k; ++d) bw[(size_t)d * k + d] = 1;   // the diagonal is never used as a divisor
+        TFPS_TRY(upload(g->bw_d, bw, st));
         CUDA_TRY(cudaStreamSynchronize(st));
     }
     g->dev_set = true;
@@ -1728,6 +1732,39 @@ int tfps_cp_partition(tfps_graph* g, const int32_t* path, int64_t len, uint8_t* 
     CUDA_TRY(cudaMemcpyAsync(&h, d_unplaced, sizeof(long long), cudaMemcpyDeviceToHost, st));
     CUDA_TRY(cudaStreamSynchronize(st));
     *unplaced = h;
+    return TFPS_OK;
+}
+
+int tfps_simulate(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, int policy, const int64_t* prio,
+                  int64_t* start, int64_t* makespan, void* stream)
+{
+    if (!g) return fail(TFPS_ERR_INVALID_ARG, "graph is NULL");
+    if (P < 0 || ldp < P) return fail(TFPS_ERR_INVALID_ARG, "need 0 <= P <= ldp");
+    if (policy != TFPS_SCHED_FIFO && policy != TFPS_SCHED_PCT) return fail(TFPS_ERR_INVALID_ARG, "unknown scheduling policy %d", policy);
+    if (!g->dev_set) return fail(TFPS_ERR_STATE, "tfps_devices_set has not been called");
+    if (P == 0) return TFPS_OK;
+    if (!part || !makespan) return fail(TFPS_ERR_INVALID_ARG, "part and makespan are required");
+    if (policy == TFPS_SCHED_PCT && !prio) return fail(TFPS_ERR_INVALID_ARG, "the PCT policy needs the path computation times (blevel)");
+    DeviceGuard guard(g->device);
+    if (!guard.ok) return fail(TFPS_ERR_CUDA, "cannot select the handle's device");
+    cudaStream_t st = (cudaStream_t)stream;
+    if (g->n == 0) {
+        CUDA_TRY(cudaMemsetAsync(makespan, 0, sizeof(int64_t) * (size_t)P, st));
+        return TFPS_OK;
+    }
+    // one warp per candidate in flight; its scratch is 16 bytes per vertex, kept below 8 GB in all
+    const int wpb = simulate_warps_per_block();
+    long long warps = std::min<long long>((P + wpb - 1) / wpb * wpb, (long long)g->sm_count * 16);
+    warps = std::min(warps, std::max<long long>(wpb, ((8LL << 30) / (16LL * g->n)) / wpb * wpb));
+    const int blocks = (int)(warps / wpb);
+    CUDA_TRY(g->sim_ready.reserve(sizeof(long long) * (size_t)warps * (size_t)g->n));
+    CUDA_TRY(g->sim_left.reserve(sizeof(int) * (size_t)warps * (size_t)g->n));
+    CUDA_TRY(g->sim_list.reserve(sizeof(int) * (size_t)warps * (size_t)g->n));
+    CUDA_TRY(launch_simulate((int)g->n, g->k, P, ldp, g->S, part, g->in_ptr.as<long long>(), g->out_ptr.as<long long>(),
+                             g->out_dst.as<int>(), g->out_t.as<long long>(), g->c.as<int>(), g->speed_d.as<int>(),
+                             g->bw_d.as<long long>(), policy, (const long long*)prio, (long long*)start, (long long*)makespan,
+                             blocks, g->sim_ready.as<long long>(), g->sim_left.as<int>(), g->sim_list.as<int>(),
+                             g->status.as<int>(), st));
     return TFPS_OK;
 }
 

@@ -254,6 +254,13 @@ cudaError_t launch_batch_split(int n, int npad, int k, const long long* total, c
 cudaError_t launch_cp_partition(int n, int k, long long S, const int* path, long long len, const int* c, const long long* mem,
                                 const int* speed, const int* ord, const long long* cap, uint8_t* on_path, uint8_t* part,
                                 long long* unplaced, cudaStream_t st);
+// batched list-scheduling simulation (simulate.cu)
+cudaError_t launch_simulate(int n, int k, long long P, long long ldp, long long S, const uint8_t* part,
+                            const long long* in_ptr, const long long* out_ptr, const int* out_dst, const long long* out_t,
+                            const int* c, const int* speed, const long long* B, int policy, const long long* prio,
+                            long long* start, long long* makespan, int blocks, long long* ready, int* left, int* list,
+                            int* status, cudaStream_t st);
+int simulate_warps_per_block();
 cudaError_t launch_transpose_u8(const uint8_t* src, uint8_t* dst, long long P, long long n, long long ldp, cudaStream_t st);
 
 }  // namespace tfps

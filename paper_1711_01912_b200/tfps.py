@@ -32,7 +32,7 @@ EXPORTS = [
     "tfps_devices_set", "tfps_topo_levels", "tfps_eval_workspace_bytes", "tfps_eval_batch",
     "tfps_eval_batch_host", "tfps_get_status", "tfps_transpose_u8", "tfps_phase_times", "tfps_kernel_launches",
     "tfps_eval_cp_noalloc", "tfps_last_pass_kernel", "tfps_probe_gather_bandwidth", "tfps_constraints_set", "tfps_eval_constraints", "tfps_critical_mask",
-    "tfps_ranks", "tfps_critical_path", "tfps_batch_split", "tfps_cp_partition",
+    "tfps_ranks", "tfps_critical_path", "tfps_batch_split", "tfps_cp_partition", "tfps_simulate",
 ]
 
 
@@ -93,6 +93,8 @@ def lib() -> ctypes.CDLL:
     L.tfps_batch_split.argtypes = [vp, vp, vp, ctypes.POINTER(ctypes.c_int64), vp]
     L.tfps_cp_partition.restype = ci
     L.tfps_cp_partition.argtypes = [vp, vp, i64, vp, ctypes.POINTER(ctypes.c_int64), vp]
+    L.tfps_simulate.restype = ci
+    L.tfps_simulate.argtypes = [vp, i64, i64, vp, ci, vp, vp, vp, vp]
     L.tfps_probe_gather_bandwidth.restype = ci
     L.tfps_probe_gather_bandwidth.argtypes = [sz, ci, ctypes.POINTER(ctypes.c_double)]
     L.tfps_last_pass_kernel.restype = ctypes.c_char_p
@@ -209,6 +211,13 @@ def tfps_cp_partition(handle, path, length, part, stream) -> int:
     bad = ctypes.c_int64(0)
     _check(lib().tfps_cp_partition(handle, path, length, part, ctypes.byref(bad), stream))
     return int(bad.value)
+
+
+SCHED_FIFO, SCHED_PCT = 0, 1
+
+
+def tfps_simulate(handle, P, ldp, part, policy, prio, start, makespan, stream) -> None:
+    _check(lib().tfps_simulate(handle, P, ldp, part, policy, prio, start, makespan, stream))
 
 
 def tfps_probe_gather_bandwidth(working_set_bytes: int, rows_per_warp: int = 4096) -> float:
@@ -416,6 +425,15 @@ class Graph:
         part = torch.zeros(max(self.n, 1), dtype=torch.uint8, device="cuda")
         bad = tfps_cp_partition(self.handle, _addr(path) if path.numel() else None, int(path.numel()), _addr(part), _stream())
         return part[:self.n], bad
+
+    def simulate(self, part, P, policy=SCHED_FIFO, prio=None, want_start=True):
+        """List-scheduling simulation of every candidate (Section 4): (start int64 [n][ldp] or None, makespan int64 [P])."""
+        import torch
+        n, ldp = part.shape
+        start = torch.zeros((n, ldp), dtype=torch.int64, device=part.device) if want_start else None
+        mk = torch.zeros(max(int(P), 1), dtype=torch.int64, device=part.device)
+        tfps_simulate(self.handle, int(P), ldp, _addr(part), policy, _addr(prio), _addr(start), _addr(mk), _stream())
+        return start, mk[:int(P)]
 
     def status(self):
         tfps_get_status(self.handle, _stream())
