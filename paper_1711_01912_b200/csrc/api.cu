@@ -1754,7 +1754,7 @@ int tfps_simulate(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, in
     }
     // one warp per candidate in flight; its scratch is 16 bytes per vertex, kept below 8 GB in all
     const int wpb = simulate_warps_per_block();
-    long long warps = std::min<long long>((P + wpb - 1) / wpb * wpb, (long long)g->sm_count * 16);
+    long long warps = std::min<long long>((P + wpb - 1) / wpb * wpb, (long long)g->sm_count * 32);
     warps = std::min(warps, std::max<long long>(wpb, ((8LL << 30) / (16LL * g->n)) / wpb * wpb));
     const int blocks = (int)(warps / wpb);
     CUDA_TRY(g->sim_ready.reserve(sizeof(long long) * (size_t)warps * (size_t)g->n));

@@ -111,63 +111,85 @@ simulate_kernel(const SimArgs a)
         int done = 0;
         bool stuck = false;
         while (done < n) {
-            // every idle device that has pending vertices looks for its best executable one
+            // every idle device that has pending vertices looks for its best executable one (lane d answers for the
+            // devices d and d + 32; only the devices that have something to decide are visited)
             long long next = BIG;
-            for (int d = 0; d < k; ++d) {
-                if (D.run[d] >= 0) { next = D.busy[d] < next ? D.busy[d] : next; continue; }
-                const int cnt = D.count[d], f = D.first[d];
-                if (cnt == 0) continue;
-                long long key = BIG, soon = BIG;
-                int id = 0x7fffffff, at = -1;
-                for (int i = lane; i < cnt; i += 32) {
-                    const int v = __ldcg(list + f + i);
-                    const long long r = __ldcg(ready + v);   // updated by atomics: read where they are performed
-                    if (r > T) { soon = r < soon ? r : soon; continue; }
-                    const long long kv = a.policy == 0 ? r : -a.prio[(size_t)v * a.ldp + j];
-                    if (kv < key || (kv == key && v < id)) { key = kv; id = v; at = i; }
-                }
-                warp_min3(key, id, at);
-                if (at < 0) {   // nothing executable yet: the device idles until its earliest vertex is
-#pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) {
-                        const long long os = __shfl_xor_sync(0xffffffffu, soon, o);
-                        soon = os < soon ? os : soon;
+            const unsigned want0 = __ballot_sync(0xffffffffu, lane < k && D.run[lane] < 0 && D.count[lane] > 0);
+            const unsigned want1 = __ballot_sync(0xffffffffu, lane + 32 < k && D.run[lane + 32] < 0 && D.count[lane + 32] > 0);
+            for (int half = 0; half < 2; ++half) {
+                unsigned want = half ? want1 : want0;
+                while (want) {
+                    const int d = 32 * half + __ffs(want) - 1;
+                    want &= want - 1;
+                    const int cnt = D.count[d], f = D.first[d];
+                    long long key = BIG, soon = BIG;
+                    int id = 0x7fffffff, at = -1;
+                    for (int i = lane; i < cnt; i += 32) {
+                        const int v = __ldcg(list + f + i);
+                        const long long r = __ldcg(ready + v);   // updated by atomics: read where they are performed
+                        if (r > T) { soon = r < soon ? r : soon; continue; }
+                        const long long kv = a.policy == 0 ? r : -a.prio[(size_t)v * a.ldp + j];
+                        if (kv < key || (kv == key && v < id)) { key = kv; id = v; at = i; }
                     }
-                    next = soon < next ? soon : next;
-                    continue;
+                    warp_min3(key, id, at);
+                    if (at < 0) {   // nothing executable yet: the device idles until its earliest vertex is
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) {
+                            const long long os = __shfl_xor_sync(0xffffffffu, soon, o);
+                            soon = os < soon ? os : soon;
+                        }
+                        next = soon < next ? soon : next;
+                        continue;
+                    }
+                    const int v = id;
+                    const long long fin = T + ceil_div_pos((long long)a.c[v] * a.S, a.speed[d]);
+                    if (lane == 0) {
+                        list[f + at] = __ldcg(list + f + cnt - 1);
+                        D.count[d] = cnt - 1;
+                        D.run[d] = v;
+                        D.busy[d] = fin;
+                        if (a.start) a.start[(size_t)v * a.ldp + j] = T;
+                    }
                 }
-                const int v = id;
-                const long long fin = T + ceil_div_pos((long long)a.c[v] * a.S, a.speed[d]);
-                if (lane == 0) {
-                    list[f + at] = __ldcg(list + f + cnt - 1);
-                    D.count[d] = cnt - 1;
-                    D.run[d] = v;
-                    D.busy[d] = fin;
-                    if (a.start) a.start[(size_t)v * a.ldp + j] = T;
+            }
+            __syncwarp();
+            {   // the earliest end of a running execution
+                long long mine = lane < k && D.run[lane] >= 0 ? D.busy[lane] : BIG;
+                const long long other = lane + 32 < k && D.run[lane + 32] >= 0 ? D.busy[lane + 32] : BIG;
+                mine = other < mine ? other : mine;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    const long long om = __shfl_xor_sync(0xffffffffu, mine, o);
+                    mine = om < mine ? om : mine;
                 }
-                __syncwarp();
-                next = fin < next ? fin : next;
+                next = mine < next ? mine : next;
             }
             if (next == BIG) { stuck = true; break; }   // nothing runs and nothing is pending (cannot happen on a DAG)
             T = next;
             // executions that end at T
-            for (int d = 0; d < k; ++d) {
-                if (D.run[d] < 0 || D.busy[d] != T) continue;
-                const int u = D.run[d];
-                __syncwarp();
-                if (lane == 0) D.run[d] = -1;
-                ++done;
-                last = T;
-                const long long e0 = a.out_ptr[u], e1 = a.out_ptr[u + 1];
-                for (long long e = e0 + lane; e < e1; e += 32) {
-                    const int x = a.out_dst[e];
-                    const int dx = pj[(size_t)x * a.ldp];
-                    const long long w = dx == d ? 0 : ceil_div_pos(a.out_t[e] * a.S, a.B[(size_t)d * k + dx]);
-                    atomicMax(&ready[x], T + w);
-                    __threadfence_block();
-                    if (atomicSub(&left[x], 1) == 1) list[D.first[dx] + atomicAdd(&D.count[dx], 1)] = x;
+            const unsigned end0 = __ballot_sync(0xffffffffu, lane < k && D.run[lane] >= 0 && D.busy[lane] == T);
+            const unsigned end1 = __ballot_sync(0xffffffffu, lane + 32 < k && D.run[lane + 32] >= 0 && D.busy[lane + 32] == T);
+            for (int half = 0; half < 2; ++half) {
+                unsigned ends = half ? end1 : end0;
+                while (ends) {
+                    const int d = 32 * half + __ffs(ends) - 1;
+                    ends &= ends - 1;
+                    const int u = D.run[d];
+                    __syncwarp();
+                    if (lane == 0) D.run[d] = -1;
+                    ++done;
+                    last = T;
+                    const long long e0 = a.out_ptr[u], e1 = a.out_ptr[u + 1];
+                    for (long long e = e0 + lane; e < e1; e += 32) {
+                        const int x = a.out_dst[e];
+                        const int dx = pj[(size_t)x * a.ldp];
+                        const long long w = dx == d ? 0 : ceil_div_pos(a.out_t[e] * a.S, a.B[(size_t)d * k + dx]);
+                        atomicMax(&ready[x], T + w);
+                        __threadfence_block();
+                        if (atomicSub(&left[x], 1) == 1) list[D.first[dx] + atomicAdd(&D.count[dx], 1)] = x;
+                    }
+                    __syncwarp();
                 }
-                __syncwarp();
             }
         }
         if (lane == 0) {
