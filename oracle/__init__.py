@@ -70,7 +70,7 @@ def _get():
         lib.oracle_cp_partition.argtypes = [ctypes.c_int64, P, ctypes.c_int64, P, P, ctypes.c_int32, P, P, ctypes.c_int64, P, P]
         lib.oracle_simulate.restype = ctypes.c_int
         lib.oracle_simulate.argtypes = ([ctypes.c_int64] + [P] * 5 + [ctypes.c_int32, P, P, ctypes.c_int64, P, ctypes.c_int64,
-                                        ctypes.c_int32, P, ctypes.c_int64, P, P])
+                                        ctypes.c_int32, P, ctypes.c_int64, P, P, P])
         _lib = lib
     return _lib
 
@@ -279,9 +279,10 @@ def cp_partition(g: OracleGraph, path, k: int, s, C, S: int):
     return part, int(bad.value)
 
 
-def simulate(g: OracleGraph, k: int, s, B, S: int, p, policy: int, prio=None):
+def simulate(g: OracleGraph, k: int, s, B, S: int, p, policy: int, prio=None, msr_weights=(1, 1, 1, 5)):
     """List-scheduling simulation of one candidate (Section 4): (start times int64 [n], makespan).
-    policy 0 = FIFO, 1 = PCT with prio = the candidate's path computation times (blevel, Eq. 12)."""
+    policy 0 = FIFO, 1 = PCT with prio = the candidate's path computation times (blevel, Eq. 12), 2 = MSR (Eq. 13)
+    with the weights (alpha, beta, gamma, delta)."""
     lib = _get()
     s = _arr(s, np.int32)
     B = _arr(B, np.int64)
@@ -289,8 +290,9 @@ def simulate(g: OracleGraph, k: int, s, B, S: int, p, policy: int, prio=None):
     pr = None if prio is None else _arr(prio, np.int64)
     start = np.zeros(g.n, np.int64)
     mk = ctypes.c_int64(0)
+    w = _arr(msr_weights, np.int64)
     rc = lib.oracle_simulate(g.n, _p(g.in_ptr), _p(g.out_ptr), _p(g.out_dst), _p(g.out_t), _p(g.c), k, _p(s), _p(B), S,
-                             _p(p), 1, policy, _p(pr), 1, _p(start), ctypes.byref(mk))
+                             _p(p), 1, policy, _p(pr), 1, _p(w), _p(start), ctypes.byref(mk))
     if rc:
         raise OracleError(rc)
     return start, int(mk.value)

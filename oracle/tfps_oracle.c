@@ -497,7 +497,12 @@ int oracle_cp_partition(int64_t n, const int32_t *path, int64_t len, const int32
  * an idle device that has an executable vertex starts one at once, otherwise it stays idle (criterion 6).
  * Which one: policy 0 = FIFO (the vertex that became executable first; equal times: the smaller id),
  *            policy 1 = PCT (Section 4.1: the largest path computation time, Eq. 12, passed in as prio[]; equal: the
- *                       smaller id).
+ *                       smaller id),
+ *            policy 2 = MSR (Section 4.2, Eq. 13: the largest successor rank; equal: the smaller id).  The score of v is
+ *                       the sum over its out-edges (v->x) of  alpha + beta [p(x) != p(v)] + gamma [x has one in-edge]
+ *                       + delta [the device of x is idle and x has one in-edge], msr_w = {alpha, beta, gamma, delta};
+ *                       "idle" is what held when the start step began: no execution on that device (the devices that
+ *                       decide in this step are idle themselves).
  * Events are taken in time order; at one time T first every execution that ends at T is completed (and its
  * successors' ready times updated), then every idle device starts its best executable vertex; a vertex of zero
  * execution time ends at T as well, so the two steps repeat at T until nothing changes.
@@ -508,10 +513,11 @@ int oracle_simulate(int64_t n,
                     const int64_t *in_ptr, const int64_t *out_ptr, const int32_t *out_dst, const int64_t *out_t,
                     const int32_t *c, int32_t k, const int32_t *s, const int64_t *B, int64_t S,
                     const uint8_t *p, int64_t p_stride, int32_t policy, const int64_t *prio, int64_t prio_stride,
-                    int64_t *start, int64_t *makespan)
+                    const int64_t *msr_w, int64_t *start, int64_t *makespan)
 {
-    if (n < 0 || k < 1 || k > 64 || S < 1 || policy < 0 || policy > 1 || !makespan) return ORACLE_BAD_ARG;
+    if (n < 0 || k < 1 || k > 64 || S < 1 || policy < 0 || policy > 2 || !makespan) return ORACLE_BAD_ARG;
     if (policy == 1 && !prio) return ORACLE_BAD_ARG;
+    if (policy == 2 && !msr_w) return ORACLE_BAD_ARG;
     *makespan = 0;
     if (n == 0) return ORACLE_OK;
     int rc = ORACLE_OK;
@@ -520,7 +526,9 @@ int oracle_simulate(int64_t n,
     int64_t *left = (int64_t *)malloc(sizeof(int64_t) * (size_t)n);       /* predecessors not finished yet */
     int64_t *list = (int64_t *)malloc(sizeof(int64_t) * (size_t)n);       /* per device: vertices whose ready time is known */
     int64_t first[65], count[64], running[64], busy_until[64];
-    if (!rt || !ready || !left || !list) { rc = ORACLE_BAD_ARG; goto done; }
+    int idle_then[64];
+    int64_t *score = (int64_t *)calloc((size_t)n, sizeof(int64_t));       /* MSR score at the running start step */
+    if (!rt || !ready || !left || !list || !score) { rc = ORACLE_BAD_ARG; goto done; }
     for (int32_t d = 0; d <= k; ++d) first[d] = 0;
     for (int64_t v = 0; v < n; ++v) {
         int32_t d = p[v * p_stride];
@@ -535,15 +543,31 @@ int oracle_simulate(int64_t n,
     int64_t T = 0, done_cnt = 0, last = 0;
     while (done_cnt < n) {
         /* every idle device starts its best executable vertex */
+        for (int32_t d = 0; d < k; ++d) idle_then[d] = running[d] < 0;
         for (int32_t d = 0; d < k; ++d) {
             if (running[d] >= 0) continue;
             int64_t best = -1, at = -1;
             for (int64_t i = 0; i < count[d]; ++i) {
                 int64_t v = list[first[d] + i];
                 if (ready[v] > T) continue;
+                if (policy == 2) {                                   /* Eq. 13 */
+                    i128 sc = 0;
+                    for (int64_t e = out_ptr[v]; e < out_ptr[v + 1]; ++e) {
+                        int64_t x = out_dst[e];
+                        int32_t dx = p[x * p_stride];
+                        int single = in_ptr[x + 1] - in_ptr[x] == 1;
+                        sc += msr_w[0];
+                        if (dx != d) sc += msr_w[1];
+                        if (single) sc += msr_w[2];
+                        if (single && idle_then[dx]) sc += msr_w[3];
+                    }
+                    if (!fits(sc)) { rc = ORACLE_OVERFLOW; goto done; }
+                    score[v] = (int64_t)sc;
+                }
                 int better;
                 if (best < 0) better = 1;
                 else if (policy == 0) better = ready[v] < ready[best] || (ready[v] == ready[best] && v < best);
+                else if (policy == 2) better = score[v] > score[best] || (score[v] == score[best] && v < best);
                 else better = prio[v * prio_stride] > prio[best * prio_stride] ||
                               (prio[v * prio_stride] == prio[best * prio_stride] && v < best);
                 if (better) { best = v; at = i; }
@@ -591,6 +615,6 @@ int oracle_simulate(int64_t n,
     }
     *makespan = last;
 done:
-    free(rt); free(ready); free(left); free(list);
+    free(rt); free(ready); free(left); free(list); free(score);
     return rc;
 }

@@ -27,7 +27,15 @@ def test_hand_worked_schedule():
     assert start.tolist() == g["pct_policy"]["start"] and mk == g["pct_policy"]["makespan"]
 
 
-def _tick_simulation(n, edges, c, k, s, B, S, p, policy, prio):
+def test_hand_worked_msr_schedule():
+    g = load_golden("sim_msr_worked.json")
+    og = oracle_graph(graph_from_edges(g["n"], g["edges"], g["c"]))
+    for case in g["cases"]:
+        start, mk = oracle.simulate(og, g["k"], g["s"], g["B"], g["S"], g["p"], 2, None, case["weights"])
+        assert start.tolist() == case["start"] and mk == case["makespan"], case
+
+
+def _tick_simulation(n, edges, c, k, s, B, S, p, policy, prio, weights=(1, 1, 1, 5)):
     """The same rules, one tick at a time (python ints): at every tick first the executions that end are completed,
     then idle devices pick; repeated within the tick while zero-length executions keep ending."""
     rt = [cdiv(c[v] * S, s[p[v]]) for v in range(n)]
@@ -36,6 +44,10 @@ def _tick_simulation(n, edges, c, k, s, B, S, p, policy, prio):
     for (u, v, t) in edges:
         succ[u].append((v, 0 if p[u] == p[v] else cdiv(t * S, B[p[u]][p[v]])))
         left[v] += 1
+    indeg = list(left)
+    out = [[] for _ in range(n)]
+    for (u, v, t) in edges:
+        out[u].append(v)
     ready = [0] * n
     known = [left[v] == 0 for v in range(n)]
     started = [False] * n
@@ -60,11 +72,18 @@ def _tick_simulation(n, edges, c, k, s, B, S, p, policy, prio):
                         left[x] -= 1
                         if left[x] == 0:
                             known[x] = True
+            idle = [running[d] is None for d in range(k)]          # as the devices stand before anybody starts
+
+            def msr(v):
+                a, b, g_, dl = weights
+                return sum(a + b * (p[x] != p[v]) + g_ * (indeg[x] == 1) + dl * (idle[p[x]] and indeg[x] == 1) for x in out[v])
+
             for d in range(k):
                 if running[d] is None:
                     cand = [v for v in range(n) if p[v] == d and known[v] and not started[v] and ready[v] <= T]
                     if cand:
-                        key = (lambda v: (ready[v], v)) if policy == 0 else (lambda v: (-prio[v], v))
+                        key = ((lambda v: (ready[v], v)) if policy == 0 else (lambda v: (-prio[v], v)) if policy == 1
+                               else (lambda v: (-msr(v), v)))
                         v = min(cand, key=key)
                         started[v] = True
                         start[v] = T
@@ -99,9 +118,11 @@ def test_against_tick_by_tick_simulation():
         S = int(rng.integers(1, 4))
         og = oracle_graph(graph_from_edges(n, edges, c))
         r = _evaluate(og, k, s, B, S, p)
-        for policy in (0, 1):
-            start, mk = oracle.simulate(og, k, s, B, S, p, policy, r.blevel)
-            ts, tm = _tick_simulation(n, edges, c.tolist(), k, s.tolist(), B.tolist(), S, p.tolist(), policy, r.blevel.tolist())
+        weights = [int(x) for x in rng.integers(0, 6, size=4)]
+        for policy in (0, 1, 2):
+            start, mk = oracle.simulate(og, k, s, B, S, p, policy, r.blevel, weights)
+            ts, tm = _tick_simulation(n, edges, c.tolist(), k, s.tolist(), B.tolist(), S, p.tolist(), policy, r.blevel.tolist(),
+                                      weights)
             assert start.tolist() == ts and mk == tm, (trial, policy)
 
 
@@ -151,7 +172,7 @@ def test_criteria_hold_on_the_schedule():
         og = oracle_graph(graph_from_edges(n, edges, c))
         r = _evaluate(og, k, s, B, S, p)
         rt = np.array([cdiv(int(c[v]) * S, int(s[p[v]])) for v in range(n)])
-        for policy in (0, 1):
+        for policy in (0, 1, 2):
             start, mk = oracle.simulate(og, k, s, B, S, p, policy, r.blevel)
             fin = start + rt
             assert mk == fin.max()
