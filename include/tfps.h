@@ -369,6 +369,11 @@ int tfps_cp_partition(tfps_graph* g, const int32_t* path, int64_t len, uint8_t* 
  *   TFPS_SCHED_FIFO  the vertex that became executable first
  *   TFPS_SCHED_PCT   the vertex with the largest path computation time (Section 4.1,
  *                    Eq. 12): prio = the blevel matrix tfps_eval_batch wrote for `part`
+ *   TFPS_SCHED_MSR   the vertex with the largest successor rank (Section 4.2, Eq. 13): the
+ *                    sum over its out-edges (v->x) of alpha + beta [x on another device]
+ *                    + gamma [x has one in-edge] + delta [x has one in-edge and its device
+ *                    executes nothing as the deciding step begins]; weights from
+ *                    tfps_msr_weights_set (default 1, 1, 1, 5: Section 5.1)
  * equal keys: the smaller vertex id.  At one time T first the executions that end at T are
  * completed, then the idle devices start; both repeat at T while executions of zero length end.
  *   part       dev uint8 [n][ldp]
@@ -380,7 +385,9 @@ int tfps_cp_partition(tfps_graph* g, const int32_t* path, int64_t len, uint8_t* 
  * One warp per candidate; scratch of 16 bytes per vertex and candidate in flight is owned
  * by the handle (allocated on first use).  Asynchronous on `stream`.
  */
-enum { TFPS_SCHED_FIFO = 0, TFPS_SCHED_PCT = 1 };
+enum { TFPS_SCHED_FIFO = 0, TFPS_SCHED_PCT = 1, TFPS_SCHED_MSR = 2 };
+/* MSR weights alpha, beta, gamma, delta of Eq. 13, each in 0 .. 2^20 (host call, takes effect at the next tfps_simulate) */
+int tfps_msr_weights_set(tfps_graph* g, int64_t alpha, int64_t beta, int64_t gamma, int64_t delta);
 int tfps_simulate(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, int policy, const int64_t* prio,
                   int64_t* start, int64_t* makespan, void* stream);
 

@@ -176,6 +176,7 @@ struct tfps_graph {
     // rank-driven partitioners: device speeds, devices from the fastest to the slowest, scratch
     DBuf speed_d, ord_d, bw_d, part_idx, part_flag, part_scr, rank_up, rank_down;
     DBuf sim_ready, sim_left, sim_list;   // scratch of the scheduling simulation
+    long long msr_w[4] = {1, 1, 1, 5};     // MSR weights alpha, beta, gamma, delta (Section 5.1)
     int cons_pairs = 0, cons_dev = 0;
     // scratch owned by the handle
     DBuf scr_memload;
@@ -1735,12 +1736,22 @@ int tfps_cp_partition(tfps_graph* g, const int32_t* path, int64_t len, uint8_t* 
     return TFPS_OK;
 }
 
+int tfps_msr_weights_set(tfps_graph* g, int64_t alpha, int64_t beta, int64_t gamma, int64_t delta)
+{
+    if (!g) return fail(TFPS_ERR_INVALID_ARG, "graph is NULL");
+    const int64_t w[4] = {alpha, beta, gamma, delta};
+    for (int i = 0; i < 4; ++i)
+        if (w[i] < 0 || w[i] > (1LL << 20)) return fail(TFPS_ERR_INVALID_ARG, "MSR weights must lie in 0 .. 2^20");
+    for (int i = 0; i < 4; ++i) g->msr_w[i] = w[i];
+    return TFPS_OK;
+}
+
 int tfps_simulate(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, int policy, const int64_t* prio,
                   int64_t* start, int64_t* makespan, void* stream)
 {
     if (!g) return fail(TFPS_ERR_INVALID_ARG, "graph is NULL");
     if (P < 0 || ldp < P) return fail(TFPS_ERR_INVALID_ARG, "need 0 <= P <= ldp");
-    if (policy != TFPS_SCHED_FIFO && policy != TFPS_SCHED_PCT) return fail(TFPS_ERR_INVALID_ARG, "unknown scheduling policy %d", policy);
+    if (policy != TFPS_SCHED_FIFO && policy != TFPS_SCHED_PCT && policy != TFPS_SCHED_MSR) return fail(TFPS_ERR_INVALID_ARG, "unknown scheduling policy %d", policy);
     if (!g->dev_set) return fail(TFPS_ERR_STATE, "tfps_devices_set has not been called");
     if (P == 0) return TFPS_OK;
     if (!part || !makespan) return fail(TFPS_ERR_INVALID_ARG, "part and makespan are required");
@@ -1762,8 +1773,8 @@ int tfps_simulate(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, in
     CUDA_TRY(g->sim_list.reserve(sizeof(int) * (size_t)warps * (size_t)g->n));
     CUDA_TRY(launch_simulate((int)g->n, g->k, P, ldp, g->S, part, g->in_ptr.as<long long>(), g->out_ptr.as<long long>(),
                              g->out_dst.as<int>(), g->out_t.as<long long>(), g->c.as<int>(), g->speed_d.as<int>(),
-                             g->bw_d.as<long long>(), policy, (const long long*)prio, (long long*)start, (long long*)makespan,
-                             blocks, g->sim_ready.as<long long>(), g->sim_left.as<int>(), g->sim_list.as<int>(),
+                             g->bw_d.as<long long>(), policy, (const long long*)prio, g->msr_w, (long long*)start,
+                             (long long*)makespan, blocks, g->sim_ready.as<long long>(), g->sim_left.as<int>(), g->sim_list.as<int>(),
                              g->status.as<int>(), st));
     return TFPS_OK;
 }

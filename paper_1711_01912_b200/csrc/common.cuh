@@ -258,8 +258,8 @@ cudaError_t launch_cp_partition(int n, int k, long long S, const int* path, long
 cudaError_t launch_simulate(int n, int k, long long P, long long ldp, long long S, const uint8_t* part,
                             const long long* in_ptr, const long long* out_ptr, const int* out_dst, const long long* out_t,
                             const int* c, const int* speed, const long long* B, int policy, const long long* prio,
-                            long long* start, long long* makespan, int blocks, long long* ready, int* left, int* list,
-                            int* status, cudaStream_t st);
+                            const long long* msr_w, long long* start, long long* makespan, int blocks, long long* ready,
+                            int* left, int* list, int* status, cudaStream_t st);
 int simulate_warps_per_block();
 cudaError_t launch_transpose_u8(const uint8_t* src, uint8_t* dst, long long P, long long n, long long ldp, cudaStream_t st);
 

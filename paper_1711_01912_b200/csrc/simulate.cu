@@ -4,8 +4,9 @@
 // A device executes its vertices one at a time without interruption; a vertex is executable once every predecessor
 // has finished and its tensor has arrived (ready = max over in-edges of finish + transfer time, transfers do not
 // queue); an idle device with an executable vertex starts one at once: FIFO takes the one that became executable first,
-// PCT the one with the largest path computation time (Eq. 12, the blevel matrix of tfps_eval_batch); equal keys go to
-// the smaller vertex id.  Events are taken in time order: at a time T every execution that ends at T is completed,
+// PCT the one with the largest path computation time (Eq. 12, the blevel matrix of tfps_eval_batch), MSR the one with
+// the largest successor rank (Eq. 13, computed from the out-edges when the device decides); equal keys go to the
+// smaller vertex id.  Events are taken in time order: at a time T every execution that ends at T is completed,
 // then every idle device starts its best executable vertex, and the two steps repeat at T while executions of zero
 // length keep ending.
 //
@@ -53,7 +54,8 @@ struct SimArgs {
     const int* c;
     const int* speed;             // [k]
     const long long* B;           // [k][k] row = source device
-    int policy;                   // 0 FIFO, 1 PCT
+    int policy;                   // 0 FIFO, 1 PCT, 2 MSR
+    long long w_alpha, w_beta, w_gamma, w_delta;   // MSR weights (Eq. 13)
     const long long* prio;        // [n][ldp] (PCT)
     long long* start;             // [n][ldp] or null
     long long* makespan;          // [P]
@@ -114,6 +116,10 @@ simulate_kernel(const SimArgs a)
             // every idle device that has pending vertices looks for its best executable one (lane d answers for the
             // devices d and d + 32; only the devices that have something to decide are visited)
             long long next = BIG;
+            // MSR looks at which devices execute nothing as this step begins (Eq. 13: idle successors' devices)
+            const unsigned long long idle_then =
+                (unsigned long long)__ballot_sync(0xffffffffu, lane < k && D.run[lane] < 0) |
+                (unsigned long long)__ballot_sync(0xffffffffu, lane + 32 < k && D.run[lane + 32] < 0) << 32;
             const unsigned want0 = __ballot_sync(0xffffffffu, lane < k && D.run[lane] < 0 && D.count[lane] > 0);
             const unsigned want1 = __ballot_sync(0xffffffffu, lane + 32 < k && D.run[lane + 32] < 0 && D.count[lane + 32] > 0);
             for (int half = 0; half < 2; ++half) {
@@ -128,7 +134,22 @@ simulate_kernel(const SimArgs a)
                         const int v = __ldcg(list + f + i);
                         const long long r = __ldcg(ready + v);   // updated by atomics: read where they are performed
                         if (r > T) { soon = r < soon ? r : soon; continue; }
-                        const long long kv = a.policy == 0 ? r : -a.prio[(size_t)v * a.ldp + j];
+                        long long kv;
+                        if (a.policy == 0) {
+                            kv = r;
+                        } else if (a.policy == 1) {
+                            kv = -a.prio[(size_t)v * a.ldp + j];
+                        } else {   // Eq. 13, summed over the out-edges
+                            long long sc = 0;
+                            for (long long e = a.out_ptr[v]; e < a.out_ptr[v + 1]; ++e) {
+                                const int x = a.out_dst[e];
+                                const int dx = pj[(size_t)x * a.ldp];
+                                const bool single = a.in_ptr[x + 1] - a.in_ptr[x] == 1;
+                                sc += a.w_alpha + (dx != d ? a.w_beta : 0) + (single ? a.w_gamma : 0) +
+                                      (single && ((idle_then >> dx) & 1ull) ? a.w_delta : 0);
+                            }
+                            kv = -sc;
+                        }
                         if (kv < key || (kv == key && v < id)) { key = kv; id = v; at = i; }
                     }
                     warp_min3(key, id, at);
@@ -206,10 +227,11 @@ simulate_kernel(const SimArgs a)
 cudaError_t launch_simulate(int n, int k, long long P, long long ldp, long long S, const uint8_t* part,
                             const long long* in_ptr, const long long* out_ptr, const int* out_dst, const long long* out_t,
                             const int* c, const int* speed, const long long* B, int policy, const long long* prio,
-                            long long* start, long long* makespan, int blocks, long long* ready, int* left, int* list,
-                            int* status, cudaStream_t st)
+                            const long long* msr_w, long long* start, long long* makespan, int blocks, long long* ready,
+                            int* left, int* list, int* status, cudaStream_t st)
 {
     SimArgs a;
+    a.w_alpha = msr_w[0]; a.w_beta = msr_w[1]; a.w_gamma = msr_w[2]; a.w_delta = msr_w[3];
     a.n = n; a.k = k; a.P = P; a.ldp = ldp; a.S = S; a.part = part;
     a.in_ptr = in_ptr; a.out_ptr = out_ptr; a.out_dst = out_dst; a.out_t = out_t; a.c = c; a.speed = speed; a.B = B;
     a.policy = policy; a.prio = prio; a.start = start; a.makespan = makespan;

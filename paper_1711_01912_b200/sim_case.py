@@ -51,7 +51,7 @@ def main():
     print(f"{w.name} n={n} m={w.graph.m} k={w.devices.k} P={P}: ranks {ms_rank:.3f} ms, critical path + CP partition "
           f"{ms_cp:.3f} ms ({cp_bad} unplaced), Batch Split {ms_bs:.3f} ms ({bs_bad} unplaced)", flush=True)
     out = G.eval_batch(part, P)
-    for name, policy in (("FIFO", tfps.SCHED_FIFO), ("PCT", tfps.SCHED_PCT)):
+    for name, policy in (("FIFO", tfps.SCHED_FIFO), ("PCT", tfps.SCHED_PCT), ("MSR", tfps.SCHED_MSR)):
         prio = out["blevel"] if policy == tfps.SCHED_PCT else None
         ms, (_, mk) = timed(lambda: G.simulate(part, P, policy, prio, want_start=False))
         G.status()
@@ -63,7 +63,7 @@ def main():
     two[:, 0] = cp_part
     two[:, 1] = bs_part
     o2 = G.eval_batch(two, 2)
-    for name, policy in (("FIFO", tfps.SCHED_FIFO), ("PCT", tfps.SCHED_PCT)):
+    for name, policy in (("FIFO", tfps.SCHED_FIFO), ("PCT", tfps.SCHED_PCT), ("MSR", tfps.SCHED_MSR)):
         _, mk = G.simulate(two, 2, policy, o2["blevel"] if policy == tfps.SCHED_PCT else None, want_start=False)
         G.status()
         print(f"  {name}: makespan of the Critical Path partition {int(mk[0]):,} (CP {int(o2['cp'][0]):,}), of the Batch Split "

@@ -32,7 +32,7 @@ EXPORTS = [
     "tfps_devices_set", "tfps_topo_levels", "tfps_eval_workspace_bytes", "tfps_eval_batch",
     "tfps_eval_batch_host", "tfps_get_status", "tfps_transpose_u8", "tfps_phase_times", "tfps_kernel_launches",
     "tfps_eval_cp_noalloc", "tfps_last_pass_kernel", "tfps_probe_gather_bandwidth", "tfps_constraints_set", "tfps_eval_constraints", "tfps_critical_mask",
-    "tfps_ranks", "tfps_critical_path", "tfps_batch_split", "tfps_cp_partition", "tfps_simulate",
+    "tfps_ranks", "tfps_critical_path", "tfps_batch_split", "tfps_cp_partition", "tfps_simulate", "tfps_msr_weights_set",
 ]
 
 
@@ -93,6 +93,8 @@ def lib() -> ctypes.CDLL:
     L.tfps_batch_split.argtypes = [vp, vp, vp, ctypes.POINTER(ctypes.c_int64), vp]
     L.tfps_cp_partition.restype = ci
     L.tfps_cp_partition.argtypes = [vp, vp, i64, vp, ctypes.POINTER(ctypes.c_int64), vp]
+    L.tfps_msr_weights_set.restype = ci
+    L.tfps_msr_weights_set.argtypes = [vp, i64, i64, i64, i64]
     L.tfps_simulate.restype = ci
     L.tfps_simulate.argtypes = [vp, i64, i64, vp, ci, vp, vp, vp, vp]
     L.tfps_probe_gather_bandwidth.restype = ci
@@ -213,7 +215,11 @@ def tfps_cp_partition(handle, path, length, part, stream) -> int:
     return int(bad.value)
 
 
-SCHED_FIFO, SCHED_PCT = 0, 1
+SCHED_FIFO, SCHED_PCT, SCHED_MSR = 0, 1, 2
+
+
+def tfps_msr_weights_set(handle, alpha, beta, gamma, delta) -> None:
+    _check(lib().tfps_msr_weights_set(handle, alpha, beta, gamma, delta))
 
 
 def tfps_simulate(handle, P, ldp, part, policy, prio, start, makespan, stream) -> None:

@@ -1,4 +1,4 @@
-"""GPU parity of the batched list-scheduling simulation (Section 4, criteria 1-6; FIFO and PCT) against the oracle,
+"""GPU parity of the batched list-scheduling simulation (Section 4, criteria 1-6; FIFO, PCT and MSR) against the oracle,
 through the C ABI: start time of every vertex and the makespan of every compared candidate, bit-exact."""
 from __future__ import annotations
 
@@ -14,8 +14,8 @@ pytestmark = pytest.mark.gpu
 INF = np.iinfo(np.int64).max
 
 
-def _compare(g, dev, part, cols=None, pad_fill=0):
-    """Simulate all candidates on the GPU under both policies; compare the listed columns (default all)."""
+def _compare(g, dev, part, cols=None, pad_fill=0, msr_weights=None):
+    """Simulate all candidates on the GPU under the three policies; compare the listed columns (default all)."""
     import oracle
     import torch
     from paper_1711_01912_b200 import tfps
@@ -25,7 +25,9 @@ def _compare(g, dev, part, cols=None, pad_fill=0):
     out = G.eval_batch(dpart, P)
     cols = list(range(P)) if cols is None else list(cols)
     res = {}
-    for policy in (tfps.SCHED_FIFO, tfps.SCHED_PCT):
+    weights = (1, 1, 1, 5) if msr_weights is None else msr_weights
+    tfps.tfps_msr_weights_set(G.handle, *weights)
+    for policy in (tfps.SCHED_FIFO, tfps.SCHED_PCT, tfps.SCHED_MSR):
         start, mk = G.simulate(dpart, P, policy, out["blevel"] if policy == tfps.SCHED_PCT else None)
         G.status()
         hs, hm = start.cpu().numpy(), mk.cpu().numpy()
@@ -33,7 +35,7 @@ def _compare(g, dev, part, cols=None, pad_fill=0):
             assert not hs[:, P:].any()   # padding columns are not written
         for j in cols:
             r = oracle.eval_partition(og, dev.k, dev.s, dev.C, dev.B, dev.scale, part[:, j])
-            ostart, omk = oracle.simulate(og, dev.k, dev.s, dev.B, dev.scale, part[:, j], policy, r.blevel)
+            ostart, omk = oracle.simulate(og, dev.k, dev.s, dev.B, dev.scale, part[:, j], policy, r.blevel, weights)
             assert hm[j] == omk, (policy, j)
             assert np.array_equal(hs[:, j], ostart), (policy, j)
         res[policy] = hm
@@ -53,6 +55,17 @@ def test_hand_worked_schedule():
     res = _compare(G, dev, part)
     from paper_1711_01912_b200 import tfps
     assert (res[tfps.SCHED_FIFO] == g["fifo"]["makespan"]).all() and (res[tfps.SCHED_PCT] == g["pct_policy"]["makespan"]).all()
+
+
+def test_hand_worked_msr_schedule():
+    from paper_1711_01912_b200 import tfps
+    g = load_golden("sim_msr_worked.json")
+    G = graph_from_edges(g["n"], g["edges"], g["c"])
+    dev = I.Devices(g["k"], np.asarray(g["s"], np.int32), np.full(g["k"], INF, np.int64), np.asarray(g["B"], np.int64), g["S"])
+    part = np.repeat(np.asarray(g["p"], np.uint8)[:, None], 3, axis=1)
+    for case in g["cases"]:
+        res = _compare(G, dev, part, msr_weights=tuple(case["weights"]))
+        assert (res[tfps.SCHED_MSR] == case["makespan"]).all()
 
 
 def test_small_configs_every_candidate():
@@ -77,7 +90,7 @@ def test_zero_cost_vertices_and_parallel_edges():
     c = rng.integers(0, 4, size=n)                                # many vertices of zero execution time
     g = graph_from_edges(n, edges, c)
     dev = I.Devices(k, np.array([1, 2, 5], np.int32), np.full(k, INF, np.int64), rng.integers(1, 9, size=(k, k)).astype(np.int64), 2)
-    _compare(g, dev, rng.integers(0, k, size=(n, P), dtype=np.uint8))
+    _compare(g, dev, rng.integers(0, k, size=(n, P), dtype=np.uint8), msr_weights=(3, 0, 2, 7))
 
 
 def test_config2_sampled_candidates_and_more_candidates_than_warps():
