@@ -244,6 +244,17 @@ int64_t tfps_kernel_launches(void);
 int tfps_probe_gather_bandwidth(size_t working_set_bytes, int rows_per_warp, double* gbytes_per_s);
 
 /*
+ * Diagnostic (no counterpart in the paper): the same with the passes' writes.  A buffer of
+ * `total_bytes` is written once, row by row (1 KiB rows in ascending order, dealt to the
+ * warps round robin); before a warp writes a row it reads `reads` rows picked pseudo-randomly
+ * among the `window_bytes` before it, and what it writes depends on what it read.  Reports
+ * (reads + 1) KiB per row over the time of the third launch, in GB/s: what the memory system
+ * sustains for a wavefront that reads its recent output out of L2 while the older output is
+ * written back to DRAM.  Allocates and frees its own buffer, synchronises the device.
+ */
+int tfps_probe_wavefront_bandwidth(size_t total_bytes, size_t window_bytes, int reads, double* gbytes_per_s);
+
+/*
  * Critical-path lengths without any allocation.  (The paper has no counterpart
  * of this call; it exists for callers of this library that are not allowed to
  * allocate device memory when they evaluate: code running inside a framework's

@@ -38,9 +38,66 @@ __global__ void __launch_bounds__(128) gather_probe_kernel(const uint4* __restri
     if (acc == 0x12345u) *sink = acc;   // keeps the loads alive
 }
 
+// The same with the pass' writes: row r of the buffer is WRITTEN once (1 KiB, by the warp r mod warps, rows in
+// ascending order per warp) after `reads` rows picked pseudo-randomly among the `window` rows before it have been read;
+// what is written depends on what was read, as in the pass.  The buffer is far larger than L2, the window is not.
+__global__ void __launch_bounds__(128)
+wavefront_probe_kernel(uint4* buf, unsigned rows, unsigned window, int reads)
+{
+    const unsigned warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    const unsigned warps = (gridDim.x * blockDim.x) >> 5;
+    for (unsigned r = warp; r < rows; r += warps) {
+        uint4 acc0 = make_uint4(r, 0u, 0u, 0u), acc1 = acc0;
+        for (int q = 0; q < reads; ++q) {
+            const unsigned back = 1u + mix32(r * 31u + (unsigned)q * 104729u) % window;
+            if (back > r) continue;
+            const uint4* p = buf + (size_t)(r - back) * 64 + lane;
+            const uint4 a = __ldcg(p), b = __ldcg(p + 32);
+            acc0.x += a.x; acc0.y ^= a.y; acc0.z += a.z; acc0.w ^= a.w;
+            acc1.x += b.x; acc1.y ^= b.y; acc1.z += b.z; acc1.w ^= b.w;
+        }
+        uint4* o = buf + (size_t)r * 64 + lane;
+        o[0] = acc0;
+        o[32] = acc1;
+    }
+}
+
 }  // namespace
 
 }  // namespace tfps
+
+extern "C" int tfps_probe_wavefront_bandwidth(size_t total_bytes, size_t window_bytes, int reads, double* gbytes_per_s)
+{
+    using namespace tfps;
+    if (!gbytes_per_s || total_bytes < 1024 || window_bytes < 1024 || reads < 0 || reads > 64) return TFPS_ERR_INVALID_ARG;
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+        return TFPS_ERR_CUDA;
+    void* buf = nullptr;
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    int rc = TFPS_ERR_CUDA;
+    const unsigned rows = (unsigned)std::min<size_t>(total_bytes / 1024, 0x7fffffffu);
+    const unsigned window = (unsigned)std::max<size_t>(1, std::min<size_t>(window_bytes / 1024, rows));
+    const int grid = sms * 8, threads = 128;
+    float ms = 0.f;
+    if (cudaMalloc(&buf, (size_t)rows * 1024) != cudaSuccess) goto done;
+    if (cudaMemset(buf, 1, (size_t)rows * 1024) != cudaSuccess) goto done;
+    if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) goto done;
+    for (int rep = 0; rep < 3; ++rep) {   // the last repetition is the one reported
+        if (cudaEventRecord(e0) != cudaSuccess) goto done;
+        wavefront_probe_kernel<<<grid, threads>>>(static_cast<uint4*>(buf), rows, window, reads);
+        if (cudaEventRecord(e1) != cudaSuccess || cudaEventSynchronize(e1) != cudaSuccess) goto done;
+    }
+    count_launches(3);
+    if (cudaEventElapsedTime(&ms, e0, e1) != cudaSuccess || ms <= 0.f) goto done;
+    *gbytes_per_s = (double)rows * 1024.0 * (reads + 1) / (ms * 1e-3) / 1e9;
+    rc = TFPS_OK;
+done:
+    if (e0) cudaEventDestroy(e0);
+    if (e1) cudaEventDestroy(e1);
+    if (buf) cudaFree(buf);
+    return rc;
+}
 
 extern "C" int tfps_probe_gather_bandwidth(size_t working_set_bytes, int rows_per_warp, double* gbytes_per_s)
 {

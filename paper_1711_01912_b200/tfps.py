@@ -32,7 +32,7 @@ EXPORTS = [
     "tfps_devices_set", "tfps_topo_levels", "tfps_eval_workspace_bytes", "tfps_eval_batch",
     "tfps_eval_batch_host", "tfps_get_status", "tfps_transpose_u8", "tfps_phase_times", "tfps_kernel_launches",
     "tfps_eval_cp_noalloc", "tfps_last_pass_kernel", "tfps_probe_gather_bandwidth", "tfps_constraints_set", "tfps_eval_constraints", "tfps_critical_mask",
-    "tfps_ranks", "tfps_critical_path", "tfps_batch_split", "tfps_cp_partition", "tfps_simulate", "tfps_msr_weights_set",
+    "tfps_ranks", "tfps_critical_path", "tfps_batch_split", "tfps_cp_partition", "tfps_simulate", "tfps_msr_weights_set", "tfps_probe_wavefront_bandwidth",
 ]
 
 
@@ -97,6 +97,8 @@ def lib() -> ctypes.CDLL:
     L.tfps_msr_weights_set.argtypes = [vp, i64, i64, i64, i64]
     L.tfps_simulate.restype = ci
     L.tfps_simulate.argtypes = [vp, i64, i64, vp, ci, vp, vp, vp, vp]
+    L.tfps_probe_wavefront_bandwidth.restype = ci
+    L.tfps_probe_wavefront_bandwidth.argtypes = [sz, sz, ci, ctypes.POINTER(ctypes.c_double)]
     L.tfps_probe_gather_bandwidth.restype = ci
     L.tfps_probe_gather_bandwidth.argtypes = [sz, ci, ctypes.POINTER(ctypes.c_double)]
     L.tfps_last_pass_kernel.restype = ctypes.c_char_p
@@ -224,6 +226,12 @@ def tfps_msr_weights_set(handle, alpha, beta, gamma, delta) -> None:
 
 def tfps_simulate(handle, P, ldp, part, policy, prio, start, makespan, stream) -> None:
     _check(lib().tfps_simulate(handle, P, ldp, part, policy, prio, start, makespan, stream))
+
+
+def tfps_probe_wavefront_bandwidth(total_bytes: int, window_bytes: int, reads: int) -> float:
+    out = ctypes.c_double(0.0)
+    _check(lib().tfps_probe_wavefront_bandwidth(total_bytes, window_bytes, reads, ctypes.byref(out)))
+    return out.value
 
 
 def tfps_probe_gather_bandwidth(working_set_bytes: int, rows_per_warp: int = 4096) -> float:
