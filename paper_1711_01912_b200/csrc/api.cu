@@ -1754,15 +1754,16 @@ int tfps_simulate(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, in
     if (policy != TFPS_SCHED_FIFO && policy != TFPS_SCHED_PCT && policy != TFPS_SCHED_MSR) return fail(TFPS_ERR_INVALID_ARG, "unknown scheduling policy %d", policy);
     if (!g->dev_set) return fail(TFPS_ERR_STATE, "tfps_devices_set has not been called");
     if (P == 0) return TFPS_OK;
-    if (!part || !makespan) return fail(TFPS_ERR_INVALID_ARG, "part and makespan are required");
-    if (policy == TFPS_SCHED_PCT && !prio) return fail(TFPS_ERR_INVALID_ARG, "the PCT policy needs the path computation times (blevel)");
+    if (!makespan) return fail(TFPS_ERR_INVALID_ARG, "makespan is required");
+    if (policy == TFPS_SCHED_PCT && !prio && g->n > 0) return fail(TFPS_ERR_INVALID_ARG, "the PCT policy needs the path computation times (blevel)");
     DeviceGuard guard(g->device);
     if (!guard.ok) return fail(TFPS_ERR_CUDA, "cannot select the handle's device");
     cudaStream_t st = (cudaStream_t)stream;
-    if (g->n == 0) {
+    if (g->n == 0) {   // nothing to execute: every schedule ends at 0
         CUDA_TRY(cudaMemsetAsync(makespan, 0, sizeof(int64_t) * (size_t)P, st));
         return TFPS_OK;
     }
+    if (!part) return fail(TFPS_ERR_INVALID_ARG, "part is required");
     // one warp per candidate in flight; its scratch is 16 bytes per vertex, kept below 8 GB in all
     const int wpb = simulate_warps_per_block();
     long long warps = std::min<long long>((P + wpb - 1) / wpb * wpb, (long long)g->sm_count * 32);

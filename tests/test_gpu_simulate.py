@@ -112,3 +112,44 @@ def test_ids_out_of_range_are_reported():
     assert ei.value.code == tfps.ERR_BAD_PARTITION
     assert int(mk[3]) == -1 and int(mk[2]) > 0
     G.close()
+
+
+def test_degenerate_calls():
+    """Empty graph, zero candidates, calls before tfps_devices_set, an unknown policy, bad weights."""
+    import torch
+    from paper_1711_01912_b200 import tfps
+    empty = graph_from_edges(0, [], [])
+    dev = I.Devices(2, np.array([1, 2], np.int32), np.full(2, INF, np.int64), np.array([[1, 5], [5, 1]], np.int64), 4)
+    G = gpu_graph(empty, dev)
+    up, down, total = G.ranks()
+    assert up.numel() == 0 and G.critical_path(down).numel() == 0
+    part, bad = G.batch_split(total)
+    assert part.numel() == 0 and bad == 0
+    part, bad = G.cp_partition(torch.zeros(0, dtype=torch.int32, device="cuda"))
+    assert part.numel() == 0 and bad == 0
+    ids = torch.zeros((0, 16), dtype=torch.uint8, device="cuda")
+    _, mk = G.simulate(ids, 5, want_start=False)
+    assert mk.tolist() == [0] * 5
+    G.close()
+    w = I.config1()
+    G = gpu_graph(w.graph)                                # devices not set
+    dpart, P, ldp = padded(w.part_full())
+    up, down, total = G.ranks()                           # ranks need no device tables
+    assert int(up.max()) == int(down.max()) > 0
+    for call in (lambda: G.batch_split(total), lambda: G.cp_partition(G.critical_path(down)), lambda: G.simulate(dpart, P)):
+        with pytest.raises(tfps.TfpsError) as ei:
+            call()
+        assert ei.value.code == tfps.ERR_STATE
+    G.devices_set(w.devices.k, w.devices.s, w.devices.C, w.devices.B, w.devices.scale)
+    _, mk = G.simulate(dpart, 0)
+    assert mk.numel() == 0
+    with pytest.raises(tfps.TfpsError) as ei:
+        G.simulate(dpart, P, policy=7)
+    assert ei.value.code == tfps.ERR_INVALID_ARG
+    with pytest.raises(tfps.TfpsError) as ei:
+        G.simulate(dpart, P, policy=tfps.SCHED_PCT)       # PCT without the path computation times
+    assert ei.value.code == tfps.ERR_INVALID_ARG
+    with pytest.raises(tfps.TfpsError) as ei:
+        tfps.tfps_msr_weights_set(G.handle, 1, -1, 1, 5)
+    assert ei.value.code == tfps.ERR_INVALID_ARG
+    G.close()
