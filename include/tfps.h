@@ -250,9 +250,11 @@ int tfps_probe_gather_bandwidth(size_t working_set_bytes, int rows_per_warp, dou
  * among the `window_bytes` before it, and what it writes depends on what it read.  Reports
  * (reads + 1) KiB per row over the time of the third launch, in GB/s: what the memory system
  * sustains for a wavefront that reads its recent output out of L2 while the older output is
- * written back to DRAM.  Allocates and frees its own buffer, synchronises the device.
+ * written back to DRAM.  layout 0: every 16-byte load of a warp covers 512 contiguous
+ * bytes, read past L1; layout 1: a lane reads 32 contiguous bytes as two loads through L1
+ * (the chained record pass' layout).  Allocates and frees its own buffer, synchronises the device.
  */
-int tfps_probe_wavefront_bandwidth(size_t total_bytes, size_t window_bytes, int reads, double* gbytes_per_s);
+int tfps_probe_wavefront_bandwidth(size_t total_bytes, size_t window_bytes, int reads, int layout, double* gbytes_per_s);
 
 /*
  * Critical-path lengths without any allocation.  (The paper has no counterpart

@@ -41,24 +41,31 @@ __global__ void __launch_bounds__(128) gather_probe_kernel(const uint4* __restri
 // The same with the pass' writes: row r of the buffer is WRITTEN once (1 KiB, by the warp r mod warps, rows in
 // ascending order per warp) after `reads` rows picked pseudo-randomly among the `window` rows before it have been read;
 // what is written depends on what was read, as in the pass.  The buffer is far larger than L2, the window is not.
+// LAYOUT 0: a lane's two 16-byte pieces of a row are 512 bytes apart (every load instruction covers 512 contiguous
+// bytes), read past L1; LAYOUT 1: a lane reads 32 contiguous bytes as two loads through L1 (the chained record pass'
+// layout: every load instruction touches 32 sectors and uses half of each).
+template <int LAYOUT>
 __global__ void __launch_bounds__(128)
 wavefront_probe_kernel(uint4* buf, unsigned rows, unsigned window, int reads)
 {
     const unsigned warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     const unsigned warps = (gridDim.x * blockDim.x) >> 5;
+    const unsigned at = LAYOUT == 0 ? lane : 2 * lane, next = LAYOUT == 0 ? 32 : 1;
     for (unsigned r = warp; r < rows; r += warps) {
         uint4 acc0 = make_uint4(r, 0u, 0u, 0u), acc1 = acc0;
         for (int q = 0; q < reads; ++q) {
             const unsigned back = 1u + mix32(r * 31u + (unsigned)q * 104729u) % window;
             if (back > r) continue;
-            const uint4* p = buf + (size_t)(r - back) * 64 + lane;
-            const uint4 a = __ldcg(p), b = __ldcg(p + 32);
+            const uint4* p = buf + (size_t)(r - back) * 64 + at;
+            uint4 a, b;
+            if (LAYOUT == 0) { a = __ldcg(p); b = __ldcg(p + next); }
+            else { a = p[0]; b = p[next]; }
             acc0.x += a.x; acc0.y ^= a.y; acc0.z += a.z; acc0.w ^= a.w;
             acc1.x += b.x; acc1.y ^= b.y; acc1.z += b.z; acc1.w ^= b.w;
         }
-        uint4* o = buf + (size_t)r * 64 + lane;
+        uint4* o = buf + (size_t)r * 64 + at;
         o[0] = acc0;
-        o[32] = acc1;
+        o[next] = acc1;
     }
 }
 
@@ -66,10 +73,11 @@ wavefront_probe_kernel(uint4* buf, unsigned rows, unsigned window, int reads)
 
 }  // namespace tfps
 
-extern "C" int tfps_probe_wavefront_bandwidth(size_t total_bytes, size_t window_bytes, int reads, double* gbytes_per_s)
+extern "C" int tfps_probe_wavefront_bandwidth(size_t total_bytes, size_t window_bytes, int reads, int layout, double* gbytes_per_s)
 {
     using namespace tfps;
-    if (!gbytes_per_s || total_bytes < 1024 || window_bytes < 1024 || reads < 0 || reads > 64) return TFPS_ERR_INVALID_ARG;
+    if (!gbytes_per_s || total_bytes < 1024 || window_bytes < 1024 || reads < 0 || reads > 64 || layout < 0 || layout > 1)
+        return TFPS_ERR_INVALID_ARG;
     int dev = 0, sms = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
         return TFPS_ERR_CUDA;
@@ -85,7 +93,8 @@ extern "C" int tfps_probe_wavefront_bandwidth(size_t total_bytes, size_t window_
     if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) goto done;
     for (int rep = 0; rep < 3; ++rep) {   // the last repetition is the one reported
         if (cudaEventRecord(e0) != cudaSuccess) goto done;
-        wavefront_probe_kernel<<<grid, threads>>>(static_cast<uint4*>(buf), rows, window, reads);
+        if (layout == 0) wavefront_probe_kernel<0><<<grid, threads>>>(static_cast<uint4*>(buf), rows, window, reads);
+        else wavefront_probe_kernel<1><<<grid, threads>>>(static_cast<uint4*>(buf), rows, window, reads);
         if (cudaEventRecord(e1) != cudaSuccess || cudaEventSynchronize(e1) != cudaSuccess) goto done;
     }
     count_launches(3);

@@ -23,11 +23,12 @@ def main():
         gbs = tfps.tfps_probe_gather_bandwidth(mb << 20, args.rows_per_warp)
         print(f"working set {mb:5d} MiB: {gbs:8.0f} GB/s gathered", flush=True)
     # the wavefront of a pass: 4 GiB written once, every row after reading rows among the last `window` MiB
-    for window in args.window_mb:
-        for reads in (0, 1, 2, 3):
-            gbs = tfps.tfps_probe_wavefront_bandwidth(4 << 30, window << 20, reads)
-            print(f"wavefront, window {window:4d} MiB, {reads} rows read per row written: {gbs:8.0f} GB/s "
-                  f"(read + written)", flush=True)
+    for layout in (0, 1):
+        for window in args.window_mb:
+            for reads in (0, 1, 2, 3):
+                gbs = tfps.tfps_probe_wavefront_bandwidth(4 << 30, window << 20, reads, layout)
+                print(f"wavefront, layout {layout}, window {window:4d} MiB, {reads} rows read per row written: {gbs:8.0f} GB/s "
+                      f"(read + written)", flush=True)
 
 
 if __name__ == "__main__":

@@ -98,7 +98,7 @@ def lib() -> ctypes.CDLL:
     L.tfps_simulate.restype = ci
     L.tfps_simulate.argtypes = [vp, i64, i64, vp, ci, vp, vp, vp, vp]
     L.tfps_probe_wavefront_bandwidth.restype = ci
-    L.tfps_probe_wavefront_bandwidth.argtypes = [sz, sz, ci, ctypes.POINTER(ctypes.c_double)]
+    L.tfps_probe_wavefront_bandwidth.argtypes = [sz, sz, ci, ci, ctypes.POINTER(ctypes.c_double)]
     L.tfps_probe_gather_bandwidth.restype = ci
     L.tfps_probe_gather_bandwidth.argtypes = [sz, ci, ctypes.POINTER(ctypes.c_double)]
     L.tfps_last_pass_kernel.restype = ctypes.c_char_p
@@ -228,9 +228,9 @@ def tfps_simulate(handle, P, ldp, part, policy, prio, start, makespan, stream) -
     _check(lib().tfps_simulate(handle, P, ldp, part, policy, prio, start, makespan, stream))
 
 
-def tfps_probe_wavefront_bandwidth(total_bytes: int, window_bytes: int, reads: int) -> float:
+def tfps_probe_wavefront_bandwidth(total_bytes: int, window_bytes: int, reads: int, layout: int = 0) -> float:
     out = ctypes.c_double(0.0)
-    _check(lib().tfps_probe_wavefront_bandwidth(total_bytes, window_bytes, reads, ctypes.byref(out)))
+    _check(lib().tfps_probe_wavefront_bandwidth(total_bytes, window_bytes, reads, layout, ctypes.byref(out)))
     return out.value
 
 
