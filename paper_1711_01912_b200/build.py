@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libtfps.so")
-SOURCES = ["api.cu", "topo.cu", "passes.cu", "lean.cu", "lean64.cu", "levrec.cu", "flow.cu", "loads.cu", "constraints.cu", "partition.cu", "simulate.cu", "probe.cu"]
+SOURCES = ["api.cu", "topo.cu", "passes.cu", "lean.cu", "lean64.cu", "levrec.cu", "ring.cu", "flow.cu", "loads.cu", "constraints.cu", "partition.cu", "simulate.cu", "probe.cu"]
 HEADERS = [os.path.join(CSRC, "common.cuh"), os.path.join(CSRC, "ptx.cuh"), os.path.join(ROOT, "include", "tfps.h")]
 
 NVCC_FLAGS = [

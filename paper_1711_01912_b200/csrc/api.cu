@@ -1,6 +1,7 @@
 // Host runtime and C ABI of libtfps: graph handle, CSR validation, device
 // tables (exact-division constants), topological structure, launch logic.
 #include <algorithm>
+#include <array>
 #include <atomic>
 #include <cstdarg>
 #include <cstdio>
@@ -168,6 +169,13 @@ struct tfps_graph {
         LevRecArgs args;
     } levrec[2];
     DBuf step_bar;             // barrier counters of the persistent record pass
+    // ring pass: host-packed records per direction (0 forward, 1 backward)
+    struct Ring {
+        bool ok = false;
+        DBuf blob, desc, vlist, cls, sc;
+        RingArgs args;
+        size_t smem = 0;
+    } ring[2];
     bool id_topo = false;      // the caller's vertex numbering is a topological order ...
     int span_id = 0;           // ... whose longest edge spans this many vertices
     DBuf status;
@@ -895,6 +903,300 @@ int build_levrec(tfps_graph* g, int k, const int32_t* s, const int64_t* B, long 
     return TFPS_OK;
 }
 
+// Packs the records of the ring pass (layout: common.cuh, kernel: ring.cu) for both directions.  Processing order and
+// steps: the caller's vertex numbering cut into runs of mutually independent vertices when it is a topological order
+// and its ring is shorter, else the topological levels.  The ring length R is the longest stretch, over the steps,
+// from the oldest vertex a step reads to the last vertex it writes.
+int build_ring(tfps_graph* g, int k, const int32_t* s, const int64_t* B, long long S, const std::vector<int>& order,
+               cudaStream_t st)
+{
+    for (auto& L : g->ring) L.ok = false;
+    const int n = (int)g->n, m = (int)g->m;
+    if (n == 0 || env_int("TFPS_RING", 1) == 0) return TFPS_OK;
+    std::vector<long long> wvals, svals;
+    auto cls_of = [&](long long x) {
+        for (size_t i = 0; i < wvals.size(); ++i)
+            if (wvals[i] == x) return (int)i;
+        wvals.push_back(x);
+        return (int)wvals.size() - 1;
+    };
+    long long s_min = INT64_MAX;
+    std::vector<int> sc_of((size_t)k);
+    for (int a = 0; a < k; ++a) {
+        s_min = std::min<long long>(s_min, s[a]);
+        size_t i = 0;
+        while (i < svals.size() && svals[i] != s[a]) ++i;
+        if (i == svals.size()) svals.push_back(s[a]);
+        sc_of[a] = (int)i;
+        for (int b = 0; b < k; ++b)
+            if (a != b) cls_of(B[a * k + b]);
+    }
+    const int ncw = (int)wvals.size(), nsc = (int)svals.size();
+    const u128 rt_max = ((u128)g->max_c * (u128)S + (u128)s_min - 1) / (u128)s_min;
+    if (ncw > RING_CLS_MAX || rt_max >= ((u128)1 << 31)) return TFPS_OK;
+    auto ceil_div = [](long long a, long long S_, long long d) {
+        if (a <= (LIMIT62 / S_)) return (a * S_ + d - 1) / d;
+        return (long long)(((u128)a * (u128)S_ + (u128)d - 1) / (u128)d);
+    };
+    const int KP = k <= 16 ? 16 : 64;
+    const int ebytes = 8 + 8 * ncw, rtrow = 4 * nsc;
+    const int wide_min = std::max(1, env_int("TFPS_RING_WIDE", 6));      // more edges than this: four lane pairs per vertex
+    const int wide2_min = std::max(wide_min, env_int("TFPS_RING_WIDE2", 24));   // more than this: all sixteen
+    const int rec_v = std::max(4, std::min(1024, env_int("TFPS_RING_REC_V", 128)));
+    const int rec_bytes = std::max(1024, env_int("TFPS_RING_REC_BYTES", 11000));
+    std::vector<int> pos_of((size_t)n);
+    for (int i = 0; i < n; ++i) pos_of[order[i]] = i;
+    // both adjacencies by level position: the other direction's degrees tell sinks and sources
+    std::vector<int> epd[2];
+    for (int dir = 0; dir < 2; ++dir) {
+        epd[dir].resize((size_t)n + 1);
+        CUDA_TRY(cudaMemcpyAsync(epd[dir].data(), dir == 0 ? g->f_eptr.p : g->b_eptr.p, sizeof(int) * ((size_t)n + 1), cudaMemcpyDeviceToHost, st));
+    }
+    CUDA_TRY(cudaStreamSynchronize(st));
+    for (int dir = 0; dir < 2; ++dir) {
+        tfps_graph::Ring& L = g->ring[dir];
+        const std::vector<int>& ep = epd[dir];
+        const std::vector<int>& ep_other = epd[1 - dir];
+        std::vector<int> nb((size_t)m);
+        std::vector<long long> tt((size_t)m);
+        if (m > 0) {
+            CUDA_TRY(cudaMemcpyAsync(nb.data(), dir == 0 ? g->f_nbr.p : g->b_nbr.p, sizeof(int) * (size_t)m, cudaMemcpyDeviceToHost, st));
+            CUDA_TRY(cudaMemcpyAsync(tt.data(), dir == 0 ? g->f_t.p : g->b_t.p, sizeof(long long) * (size_t)m, cudaMemcpyDeviceToHost, st));
+        }
+        CUDA_TRY(cudaStreamSynchronize(st));
+        // candidate processing orders: seq = level positions in processing order, sp = step pointers into seq
+        std::vector<int> seq_best, sp_best, qof_best;
+        long long R_best = -1;
+        for (int mode = 0; mode < 2; ++mode) {   // 0: topological levels, 1: the caller's numbering
+            if (mode == 1 && (!g->id_topo || env_int("TFPS_STEP_ORDER", 0) == 1)) continue;
+            std::vector<int> seq((size_t)n), sp;
+            if (mode == 0) {
+                for (int li = 0; li <= g->num_levels; ++li) sp.push_back((int)g->h_level_ptr[li]);
+                if (dir == 0) for (int i = 0; i < n; ++i) seq[(size_t)i] = i;
+                else {   // levels from the last to the first
+                    std::vector<int> sp2;
+                    int q = 0;
+                    sp2.push_back(0);
+                    for (int li = g->num_levels - 1; li >= 0; --li) {
+                        for (int p = sp[(size_t)li]; p < sp[(size_t)li + 1]; ++p) seq[(size_t)q++] = p;
+                        sp2.push_back(q);
+                    }
+                    sp.swap(sp2);
+                }
+            } else {
+                int lo = dir == 0 ? 0 : n - 1;   // first vertex of the running step
+                sp.push_back(0);
+                for (int stp = 0; stp < n; ++stp) {
+                    const int v = dir == 0 ? stp : n - 1 - stp;
+                    const int p = pos_of[v];
+                    bool indep = true;
+                    for (int e = ep[p]; e < ep[p + 1] && indep; ++e) indep = dir == 0 ? nb[e] < lo : nb[e] > lo;
+                    if (!indep) { sp.push_back(stp); lo = v; }
+                    seq[(size_t)stp] = p;
+                }
+                sp.push_back(n);
+            }
+            std::vector<int> qof((size_t)n);   // processing index of every vertex
+            for (int q = 0; q < n; ++q) qof[(size_t)order[seq[(size_t)q]]] = q;
+            long long R = 1;
+            for (size_t si = 0; si + 1 < sp.size(); ++si) {
+                int oldest = sp[si];
+                for (int q = sp[si]; q < sp[si + 1]; ++q) {
+                    const int p = seq[(size_t)q];
+                    for (int e = ep[p]; e < ep[p + 1]; ++e) oldest = std::min(oldest, qof[(size_t)nb[e]]);
+                }
+                R = std::max<long long>(R, (long long)sp[si + 1] - oldest);
+            }
+            if (R_best < 0 || R < R_best || env_int("TFPS_STEP_ORDER", 0) == 2) {
+                R_best = R; seq_best.swap(seq); sp_best.swap(sp); qof_best.swap(qof);
+            }
+        }
+        const std::vector<int>&seq = seq_best, &sp = sp_best, &qof = qof_best;
+        const int R = (int)R_best;
+        if (R_best > 65535) continue;
+        // rounds step by step, records of consecutive rounds.  A round has 16 items (one per lane pair); a vertex takes
+        // 1, 4 or 16 of them (kind 0, 1, 2) according to its degree, each with a share of its edges.
+        struct Item { int p, e0, e1; bool helper, skip; };   // level position, edge range within the vertex
+        struct Round { Item it[16]; int kind, cost; };
+        std::vector<unsigned char> raw, blob;   // records without and with their trailers
+        std::vector<int> desc, vlist, rec_raw, rec_nv, rec_vfirst, rec_first;
+        std::vector<size_t> rec_base;
+        int rec_max = 16, max_v = 2, nrecords = 0;
+        std::vector<int> idx;
+        std::vector<Round> rounds;
+        bool fits = true;
+        for (size_t si = 0; si + 1 < sp.size() && fits; ++si) {
+            idx.assign(seq.begin() + sp[si], seq.begin() + sp[si + 1]);
+            std::stable_sort(idx.begin(), idx.end(), [&](int x, int y) { return ep[x + 1] - ep[x] > ep[y + 1] - ep[y]; });
+            rounds.clear();
+            size_t i = 0;
+            auto deg = [&](size_t q) { return ep[idx[q] + 1] - ep[idx[q]]; };
+            for (int kind = 2; kind >= 0; --kind) {
+                const int gsz = kind == 2 ? 16 : kind == 1 ? 4 : 1, per = 16 / gsz;   // pairs per vertex, vertices per round
+                const int lower = kind == 2 ? wide2_min : kind == 1 ? wide_min : -1;  // degrees above this take this kind
+                while (i < idx.size() && deg(i) > lower) {
+                    Round r;
+                    r.kind = kind;
+                    r.cost = (deg(i) + gsz - 1) / gsz + 2 * kind;
+                    for (int q = 0; q < per; ++q) {
+                        const bool have = i < idx.size() && deg(i) > lower;
+                        const int p = have ? idx[i] : idx[0], d = have ? ep[p + 1] - ep[p] : 0, share = (d + gsz - 1) / gsz;
+                        for (int h = 0; h < gsz; ++h)
+                            r.it[q * gsz + h] = Item{p, std::min(d, h * share), std::min(d, (h + 1) * share), h > 0, !have};
+                        if (have) ++i;
+                    }
+                    rounds.push_back(r);
+                }
+            }
+            // dearest rounds first (the warps take the rounds of a step in turn)
+            std::vector<int> ro(rounds.size());
+            for (size_t q = 0; q < ro.size(); ++q) ro[q] = (int)q;
+            std::stable_sort(ro.begin(), ro.end(), [&](int x, int y) { return rounds[(size_t)x].cost > rounds[(size_t)y].cost; });
+            size_t r0 = 0;
+            bool first = true;
+            while (r0 < ro.size()) {
+                // rounds r0..r1-1 form a record: at most rec_v vertices and about rec_bytes bytes, at least one round
+                size_t r1 = r0;
+                int nv = 0, ne = 0;
+                while (r1 < ro.size()) {
+                    const Round& r = rounds[(size_t)ro[r1]];
+                    int dv = 0, de = 0;
+                    for (const Item& it : r.it) if (!it.skip && !it.helper) { ++dv; de += ep[it.p + 1] - ep[it.p]; }
+                    const long long bytes = 32 + 256LL * (long long)(r1 - r0 + 1) + 4LL * rec_v +
+                                            (((long long)(nv + dv) * rtrow + 7) & ~7LL) + (long long)(ne + de) * ebytes;
+                    if (r1 > r0 && (nv + dv > rec_v || bytes > rec_bytes)) break;
+                    nv += dv; ne += de; ++r1;
+                }
+                const int nr = (int)(r1 - r0);
+                const int rtoff = 32 + 256 * nr, eoff = rtoff + ((nv * rtrow + 7) & ~7);
+                const long long bytes_ll = (long long)eoff + (long long)ne * ebytes;   // without the trailer
+                if (bytes_ll > 60000 || nv > 4096) { fits = false; break; }   // edge offsets and one stage slot stay far below 64 KB
+                const int bytes = (int)bytes_ll;
+                const size_t base = raw.size();
+                raw.resize(base + (size_t)bytes, 0);
+                unsigned char* rec = raw.data() + base;
+                int hdr[4] = {nr, rtoff, rtrow, bytes};
+                memcpy(rec, hdr, 16);
+                const int vfirst = (int)vlist.size();
+                int vi = 0, ecur = eoff;
+                for (int rr = 0; rr < nr; ++rr) {
+                    const Round& r = rounds[(size_t)ro[r0 + (size_t)rr]];
+                    int my_eb = 0;
+                    for (int q = 0; q < 16; ++q) {
+                        const Item& it = r.it[q];
+                        int out[4] = {0, 0, 0, 0};
+                        if (it.skip) { out[0] = (1 << 29) | (r.kind << 27); }
+                        else {
+                            const int p = it.p, v = order[p], d = ep[p + 1] - ep[p];
+                            if (!it.helper) {
+                                // the vertex' runtimes, id row and edges enter the record once
+                                for (int c = 0; c < nsc; ++c) {
+                                    const int rtv = (int)ceil_div(g->h_c[v], S, svals[(size_t)c]);
+                                    memcpy(rec + rtoff + vi * rtrow + 4 * c, &rtv, 4);
+                                }
+                                vlist.push_back(v);
+                                for (int e = 0; e < d; ++e) {
+                                    unsigned char* er = rec + ecur + e * ebytes;
+                                    const int u = nb[(size_t)ep[p] + e];
+                                    const int us = qof[(size_t)u] % R;
+                                    memcpy(er, &us, 4);
+                                    for (int w = 1; w <= ncw; ++w) {
+                                        const long long tr = ceil_div(tt[(size_t)ep[p] + e], S, wvals[(size_t)w - 1]);
+                                        memcpy(er + 8 * w, &tr, 8);
+                                    }
+                                }
+                                my_eb = ecur;
+                                ecur += d * ebytes;
+                                ++vi;
+                            }
+                            const bool cpflag = ep_other[p + 1] == ep_other[p];   // forward: sink; backward: source
+                            out[0] = v | (r.kind << 27) | (it.helper ? 1 << 30 : 0) | (cpflag ? (int)0x80000000u : 0);
+                            out[1] = (qof[(size_t)v] % R) | ((vi - 1) << 16);
+                            out[2] = my_eb + it.e0 * ebytes;
+                            out[3] = my_eb + it.e1 * ebytes;
+                        }
+                        memcpy(rec + 32 + 256 * rr + 16 * q, out, 16);
+                    }
+                }
+                rec_base.push_back(base); rec_raw.push_back(bytes); rec_nv.push_back(nv); rec_vfirst.push_back(vfirst);
+                rec_first.push_back(first ? 1 : 0);
+                first = false;
+                max_v = std::max(max_v, (nv + 1) & ~1);
+                ++nrecords;
+                r0 = r1;
+            }
+        }
+        if (!fits || raw.size() / 8 >= ((size_t)1 << 31)) continue;
+        // Record i carries, as its trailer, the descriptor and the vertex list of record i + depth (the record that takes
+        // over its stage slot).  Stage slots: as many as fit beside the ring, at least three.
+        int depth = 0;
+        size_t smem = 0;
+        for (int d = RING_DEPTH_MAX; d >= 3 && depth == 0; --d) {
+            int rmax = 16;
+            for (int i = 0; i < nrecords; ++i)
+                rmax = std::max(rmax, (rec_raw[(size_t)i] + (i + d < nrecords ? 4 * rec_nv[(size_t)i + d] : 0) + 15) & ~15);
+            const size_t need = ring_smem_bytes(R, rmax, max_v, d, KP);
+            if (need + 1024 <= (size_t)g->smem_optin) { depth = d; smem = need; rec_max = rmax; }
+        }
+        if (depth == 0) continue;
+        std::vector<size_t> off((size_t)nrecords + 1, 0);
+        for (int i = 0; i < nrecords; ++i)
+            off[(size_t)i + 1] = off[(size_t)i] + (size_t)((rec_raw[(size_t)i] + (i + depth < nrecords ? 4 * rec_nv[(size_t)i + depth] : 0) + 15) & ~15);
+        if (off[(size_t)nrecords] / 16 >= ((size_t)1 << 31)) continue;
+        blob.assign(off[(size_t)nrecords], 0);
+        desc.assign(4 * ((size_t)nrecords + 1), 0);   // one zero descriptor past the end
+        for (int i = 0; i < nrecords; ++i) {
+            desc[4 * (size_t)i] = (int)(off[(size_t)i] / 16);
+            desc[4 * (size_t)i + 1] = (int)(off[(size_t)i + 1] - off[(size_t)i]);
+            desc[4 * (size_t)i + 2] = rec_nv[(size_t)i] | (rec_first[(size_t)i] ? (int)0x80000000u : 0);
+            desc[4 * (size_t)i + 3] = rec_vfirst[(size_t)i];
+        }
+        for (int i = 0; i < nrecords; ++i) {
+            unsigned char* rec = blob.data() + off[(size_t)i];
+            memcpy(rec, raw.data() + rec_base[(size_t)i], (size_t)rec_raw[(size_t)i]);
+            if (i + 1 < nrecords && rec_first[(size_t)i + 1]) {   // the next record opens a step
+                int nr;
+                memcpy(&nr, rec, 4);
+                nr |= (int)0x80000000u;
+                memcpy(rec, &nr, 4);
+            }
+            if (i + depth < nrecords) {
+                memcpy(rec + 16, &desc[4 * ((size_t)i + depth)], 16);
+                memcpy(rec + rec_raw[(size_t)i], &vlist[(size_t)rec_vfirst[(size_t)i + depth]], 4 * (size_t)rec_nv[(size_t)i + depth]);
+            }
+        }
+        raw.clear(); raw.shrink_to_fit();
+        std::vector<unsigned char> cls((size_t)KP * KP, 0), scv((size_t)KP, 0);
+        for (int pv = 0; pv < k; ++pv) {
+            scv[(size_t)pv] = (unsigned char)(4 * sc_of[pv]);
+            for (int pu = 0; pu < k; ++pu)   // forward: the edge runs from the neighbour to the vertex; backward the other way
+                cls[(size_t)pv * KP + pu] = (unsigned char)(pu == pv ? 0 : 8 * (cls_of(dir == 0 ? B[pu * k + pv] : B[pv * k + pu]) + 1));
+        }
+        TFPS_TRY(upload(L.blob, blob, st));
+        TFPS_TRY(upload(L.desc, desc, st));
+        TFPS_TRY(upload(L.vlist, vlist, st));
+        TFPS_TRY(upload(L.cls, cls, st));
+        TFPS_TRY(upload(L.sc, scv, st));
+        CUDA_TRY(cudaStreamSynchronize(st));
+        L.args = RingArgs{};
+        L.args.blob = L.blob.as<unsigned char>();
+        L.args.desc = L.desc.as<int4>();
+        L.args.vlist = L.vlist.as<int>();
+        L.args.cls = L.cls.as<unsigned char>();
+        L.args.sc = L.sc.as<unsigned char>();
+        L.args.num_records = nrecords;
+        L.args.kp = KP;
+        L.args.R = R;
+        L.args.rec_max = rec_max;
+        L.args.max_v = max_v;
+        L.args.ebytes = ebytes;
+        L.args.depth = depth;
+        L.smem = smem;
+        L.ok = true;
+    }
+    return TFPS_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -1206,6 +1508,7 @@ int tfps_devices_set(tfps_graph* g, int k, const int32_t* s, const int64_t* C, c
         g->fits32 = worst < (1LL << 31) - 1;
         TFPS_TRY(build_lean(g, k, s, B, scale, order, st));
         TFPS_TRY(build_levrec(g, k, s, B, scale, order, st));
+        TFPS_TRY(build_ring(g, k, s, B, scale, order, st));
     }
     CUDA_TRY(cudaStreamSynchronize(st));
     if (!g->aux_stream) {
@@ -1445,6 +1748,12 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
         // any P (1,590 levels of 660: 12.8 against 76.6 ms forward at P = 64), narrower ones only with enough candidates
         if (avg_width * P >= (1LL << 18) || avg_width >= 128) { sliced = false; lean_f.ok = false; lean_b.ok = false; }
     }
+    // Ring pass: where no lean pass applies, the ring fits and there are enough blocks of eight candidates for the machine
+    // (TFPS_RING = 2: whenever it fits; 0: never).
+    const bool use_ring = !(flags & (TFPS_EVAL_SLICED | TFPS_EVAL_LEVEL_SYNC)) && env_int("TFPS_RING", 1) != 0 &&
+                          !((!need_fwd || lean_f.ok) && (!need_bwd || lean_b.ok)) && g->ring[0].ok && g->ring[1].ok &&
+                          ldp < (1LL << 28) && ((P + RING_SLICE - 1) / RING_SLICE >= g->sm_count || env_int("TFPS_RING", 1) == 2);
+    if (use_ring) { lean_f.ok = false; lean_b.ok = false; }
     // The lean passes cannot leave their tables on a bad id (ids are masked), so the id check need not come first:
     // the loads kernel then runs on a low-priority stream beside them and fills the SMs the passes' last wave leaves idle.
     const bool overlap = (load || ml) && (need_fwd || need_bwd) && (!need_fwd || lean_f.ok) && (!need_bwd || lean_b.ok) &&
@@ -1488,6 +1797,20 @@ int tfps_eval_batch(tfps_graph* g, int64_t P, int64_t ldp, const uint8_t* part, 
                 }
                 continue;
             }
+        }
+        if (use_ring) {   // wide graph with a long window and enough candidates: blocks of eight candidates with a ring in shared memory
+            tfps_graph::Ring& L = g->ring[fwd ? 0 : 1];
+            RingArgs ra = L.args;
+            ra.part = part;
+            ra.lev = lev;
+            ra.cp = cp_here;
+            ra.status = status;
+            ra.P = P;
+            ra.ldp = ldp;
+            ra.wait_limit = std::max(0, env_int("TFPS_WAIT_LIMIT", 1 << 20));
+            g->last_kernel = "pass_ring_kernel";
+            CUDA_TRY(launch_pass_ring(ra, fwd, std::max(1, std::min(31, env_int("TFPS_RING_WARPS", 16))), L.smem, st));
+            continue;
         }
         if (sliced) {
             SlicedPlan plan;

@@ -196,6 +196,45 @@ cudaError_t launch_pass_stepchain(const LevRecArgs& a, bool fwd, const std::vect
 bool flow_applies(const LevRecArgs& a);   // the dataflow form covers k <= 16, items of at most eight edges of at most 64 bytes, P <= 4096
 cudaError_t launch_pass_flow(const LevRecArgs& a, bool fwd, int sm_count, cudaStream_t st);
 
+// Ring pass (ring.cu): candidate-sliced pass for wide graphs whose window is long.  A block owns RING_SLICE
+// candidates and keeps the finish times (forward) or bottom levels (backward) and the ids of the last R vertices in
+// processing order in shared memory.  The host packs records (never across a step boundary; a step = vertices that do
+// not depend on one another) in processing order:
+//   header  16 bytes: int4 {rounds, byte offset of the runtime table, bytes of a runtime row, 0}
+//   rounds  64 bytes each: four items int4 {v | skip << 29 | wide << 30 | cp << 31, ring slot | index within the
+//           record << 16, first edge byte, end edge byte}; one warp takes a round, eight lanes an item; the four items
+//           of a wide round are quarters of the edges of one vertex and meet through shuffles
+//   runtime [4 * nsc bytes per vertex of the record]  rt[c] = ceil(c_v * S / speed of class c)
+//   edge    [8 + 8 * ncls bytes each]  {ring slot of the neighbour, pad, W[1..ncls]}, W[c] = ceil(t_e * S / b_c)
+// desc[i] = {offset / 16, bytes, vertices | new step << 31, first index into vlist}; vlist names the vertices whose id
+// rows go with the record.  cls[pv * kp + pu] = 8 * class of the link between the neighbour's device pu and the
+// vertex's device pv (0 = same device); sc[d] = 4 * speed class of device d.
+constexpr int RING_SLICE = 8;
+constexpr int RING_DEPTH_MAX = 8;
+constexpr int RING_CLS_MAX = 30;
+struct RingArgs {
+    const uint8_t* part;
+    long long* lev;
+    long long* cp;
+    int* status;
+    long long P, ldp;
+    const unsigned char* blob;
+    const int4* desc;            // [num_records + 1], zero past the end
+    const int* vlist;
+    const unsigned char* cls;    // [kp * kp]
+    const unsigned char* sc;     // [kp]
+    int num_records;
+    int kp;                      // 16 or 64
+    int R;                       // ring length in vertices
+    int rec_max;                 // bytes of the largest record (multiple of 16)
+    int max_v;                   // most vertices in one record
+    int ebytes;                  // bytes of an edge entry
+    int depth;                   // stage slots
+    int wait_limit;
+};
+size_t ring_smem_bytes(int R, int rec_max, int max_v, int depth, int kp);
+cudaError_t launch_pass_ring(const RingArgs& a, bool fwd, int warps, size_t smem, cudaStream_t st);
+
 size_t lean_smem_bytes(const LeanPlan& plan, int slice, int warps, int depth, unsigned* slot_stride, unsigned* stage_bytes);
 cudaError_t launch_pass_lean(const LeanArgs& a, bool fwd, int slice, int cpt, int warps, size_t smem, cudaStream_t st);
 cudaError_t launch_pass_lean64(const LeanArgs& a, bool fwd, int slice, int warps, size_t smem, cudaStream_t st);

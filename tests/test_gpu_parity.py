@@ -712,7 +712,42 @@ def test_randomized_shapes_all_variants():
             run_and_compare(w.graph, dev, part, flags, pad_fill=255)
 
 
-@pytest.mark.parametrize("family", ["lean", "lean64", "steprec", "flow"])
+@pytest.mark.parametrize("warps,wide,rec_v", [(16, 8, 64), (1, 4, 4), (5, 8, 16), (31, 6, 64)])
+def test_ring_pass(warps, wide, rec_v, monkeypatch):
+    """The ring pass (blocks of eight candidates, finish times of the last R vertices in shared memory): ragged and
+    single slices, records of a few vertices (every stage slot is reused many times), wide rounds for vertices with many
+    edges next to vertices without any, a hub of hundreds of in-edges, a chain (one vertex per step), more than 16
+    devices, a relabelled graph (steps are the topological levels) and a caller's order (steps cut from the numbering)."""
+    from paper_1711_01912_b200 import tfps
+    monkeypatch.setenv("TFPS_RING", "2")
+    monkeypatch.setenv("TFPS_LEAN", "0")
+    monkeypatch.setenv("TFPS_RING_WARPS", str(warps))
+    monkeypatch.setenv("TFPS_RING_WIDE", str(wide))
+    monkeypatch.setenv("TFPS_RING_REC_V", str(rec_v))
+    rng = np.random.default_rng(977 + warps)
+    for P in (300, 8, 13, 1000):
+        w = I.config5(layers=14, width=64, P=P)
+        run_and_compare(w.graph, w.devices, w.part_full(), 0, pad_fill=255)
+    G = gpu_graph(w.graph, w.devices)
+    dpart, P, ldp = padded(w.part_full())
+    G.eval_batch(dpart, P, flags=0)
+    assert tfps.tfps_last_pass_kernel(G.handle) == "pass_ring_kernel"
+    G.close()
+    n = 700
+    edges = [(u, n - 1, int(rng.integers(0, 10 ** 6))) for u in range(n - 1)] + [(0, u, 5) for u in range(1, 60)]
+    gh = graph_from_edges(n, edges, rng.integers(0, 100, size=n))
+    run_and_compare(gh, _grouped_devices(4, rng), rng.integers(0, 4, size=(n, 270), dtype=np.uint8), 0, pad_fill=255)
+    n = 3000
+    chain = graph_from_edges(n, [(u, u + 1, int(rng.integers(0, 10 ** 5))) for u in range(n - 1)], rng.integers(0, 100, size=n))
+    run_and_compare(chain, _grouped_devices(4, rng), rng.integers(0, 4, size=(n, 40), dtype=np.uint8), 0, pad_fill=255)
+    w = I.small_random(5151 + warps, 500, 3000, 17, 40)
+    run_and_compare(w.graph, w.devices, w.part_full(), 0, pad_fill=255)
+    w = I.config5(layers=14, width=64, P=24)
+    g2, _ = I.relabel(w.graph, 5)
+    run_and_compare(g2, w.devices, w.part_full(), 0, pad_fill=255)
+
+
+@pytest.mark.parametrize("family", ["lean", "lean64", "steprec", "flow", "ring"])
 def test_bounded_waits_run_out(family, monkeypatch):
     """The bounded device-side waits, made to run out on the host's terms: with a limit of zero polls every wait of
     the windowed kernels (for a staged record) and of the persistent record pass (for the other blocks' signal) gives
@@ -724,6 +759,11 @@ def test_bounded_waits_run_out(family, monkeypatch):
         w = I.config5(layers=14, width=64, P=300)
         flags = tfps.EVAL_LEVEL_SYNC
         monkeypatch.setenv("TFPS_STEP_PERSISTENT" if family == "steprec" else "TFPS_STEP_FLOW", "1")
+    elif family == "ring":
+        w = I.config5(layers=14, width=64, P=300)
+        flags = tfps.EVAL_AUTO
+        monkeypatch.setenv("TFPS_RING", "2")
+        monkeypatch.setenv("TFPS_LEAN", "0")
     else:
         w = I.config2()
         w.P = 200
@@ -736,10 +776,10 @@ def test_bounded_waits_run_out(family, monkeypatch):
     out = G.eval_batch(dpart, P, flags=flags, check=False)
     kernel = tfps.tfps_last_pass_kernel(G.handle)
     assert kernel == {"lean": "pass_lean_kernel", "lean64": "pass_lean64_kernel", "steprec": "pass_steprec_kernel",
-                      "flow": "pass_flow_kernel"}[family]
+                      "flow": "pass_flow_kernel", "ring": "pass_ring_kernel"}[family]
     with pytest.raises(tfps.TfpsError) as ei:
         G.status()
     assert ei.value.code == tfps.ERR_TIMEOUT
     monkeypatch.delenv("TFPS_WAIT_LIMIT")
     G.close()
-    run_and_compare(w.graph, w.devices, w.part_full()[:, :w.P], 2 if family in ("lean", "lean64") else 1, pad_fill=255)
+    run_and_compare(w.graph, w.devices, w.part_full()[:, :w.P], {"lean": 2, "lean64": 2, "ring": 0}.get(family, 1), pad_fill=255)
